@@ -1,0 +1,183 @@
+/*
+ * camera.h — C ABI of the B200 (sm_100a) CAMERA micro-expert analysis library.
+ *
+ * The library computes, for one Mixture-of-Experts layer and a batch of
+ * calibration tokens, the per-micro-expert energy of the CAMERA paper and the
+ * two structured selections driven by it.  A micro-expert is intermediate
+ * channel i of an expert: row i of W_gate and W_up plus column i of W_down
+ * (paper Eq. 3).  Experts are ordered routed[0..n_routed) then
+ * shared[0..n_shared); the global micro-expert index is off[e] + i with off the
+ * prefix sum of d_ff (Algorithm 1 line 4, generalised to unequal d_ff).
+ *
+ * General rules
+ *  - "DEVICE" pointers are CUDA device memory of the current device, "HOST"
+ *    pointers ordinary host memory.  The caller owns every buffer.  The
+ *    library allocates no device memory: scratch comes from the caller's
+ *    workspace (query the *_workspace_bytes function first; 256-byte aligned).
+ *  - Calls enqueue work on `cuda_stream` (a cudaStream_t, NULL = default
+ *    stream) and return without synchronising unless stated otherwise.
+ *    HOST arrays passed in are consumed before the call returns.
+ *  - Return value: CAMERA_OK or a negative camera_status_t.  Argument errors
+ *    are reported before anything is launched.  Device-side trouble (a bounded
+ *    wait inside a kernel that ran out) never traps: it is recorded in the
+ *    workspace's status word, see camera_read_status.
+ *  - No call is re-entrant on the same workspace: calls that share a workspace
+ *    and overlap on the GPU race.
+ */
+#ifndef CAMERA_B200_H
+#define CAMERA_B200_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+  CAMERA_OK = 0,
+  CAMERA_ERR_INVALID_ARG = -1,
+  CAMERA_ERR_UNSUPPORTED_SHAPE = -2,
+  CAMERA_ERR_WORKSPACE = -3,
+  CAMERA_ERR_ARCH = -4,
+  CAMERA_ERR_CUDA = -5,
+  CAMERA_ERR_DEVICE_TIMEOUT = -6
+} camera_status_t;
+
+typedef enum { CAMERA_F32 = 0, CAMERA_BF16 = 1 } camera_dtype_t;
+
+/* Storage of one expert's W_down: CAMERA_DOWN_HF is the paper's [d_model, d_ff]
+ * (micro-expert i = column i); CAMERA_DOWN_ME_MAJOR is [d_ff, d_model] (row i). */
+typedef enum { CAMERA_DOWN_HF = 0, CAMERA_DOWN_ME_MAJOR = 1 } camera_down_layout_t;
+
+/* camera_layer_t.flags */
+enum {
+  CAMERA_ROUTER_NORM_TOPK = 1u,    /* divide the k kept probabilities by their sum ("Top&Norm") */
+  CAMERA_SHARED_GATE_SIGMOID = 2u  /* shared expert s gets coefficient sigmoid(x . w_shared_gate[s]) instead of 1 */
+};
+
+/* camera_score_aux_t.flags */
+enum {
+  CAMERA_SCORE_FORCE_SIMT = 1u     /* run the fp32-FMA scoring kernel even where the tensor-core kernel applies */
+};
+
+/* Stages of camera_score_layer, for the optional timing events. */
+enum {
+  CAMERA_STAGE_ROUTER = 0, CAMERA_STAGE_PERMUTE = 1, CAMERA_STAGE_ROWNORM = 2,
+  CAMERA_STAGE_SCORE = 3, CAMERA_STAGE_COMBINE = 4, CAMERA_N_STAGES = 5
+};
+
+/* One MoE layer (paper Algorithm 1 inputs: expert weights and router R). */
+typedef struct {
+  int32_t d_model;              /* multiple of 8 */
+  int32_t n_routed;             /* 0..256 routed experts */
+  int32_t top_k;                /* 1..min(n_routed,16); ignored when n_routed == 0 */
+  int32_t n_shared;             /* experts every token visits */
+  const int32_t* d_ff;          /* HOST [n_routed+n_shared], each > 0 */
+  int32_t dtype;                /* camera_dtype_t of x and of every weight */
+  uint32_t flags;
+  int32_t down_layout;          /* camera_down_layout_t */
+  const void* w_router;         /* DEVICE [n_routed, d_model] row-major */
+  const float* router_bias;     /* DEVICE [n_routed] fp32 added to the logits, or NULL */
+  const void* w_shared_gate;    /* DEVICE [n_shared, d_model]; required iff CAMERA_SHARED_GATE_SIGMOID */
+  const void* const* w_gate;    /* HOST array of DEVICE pointers, each [d_ff[e], d_model] row-major */
+  const void* const* w_up;      /* same */
+  const void* const* w_down;    /* each per down_layout */
+} camera_layer_t;
+
+/* Optional inputs/outputs of camera_score_layer; any pointer may be NULL. All DEVICE. */
+typedef struct {
+  float* phi2;                  /* [N_e]  ||Phi_i||_2^2       (Alg. 1 line 7) */
+  float* phi_inf_sq;            /* [N_e]  ||Phi_i||_inf^2     (Alg. 1 line 8) */
+  float* omega2;                /* [N_e]  ||w_i||_2^2         (Alg. 1 line 5) */
+  int32_t* topk_idx;            /* [T, top_k] chosen experts, by decreasing probability */
+  float* topk_w;                /* [T, top_k] their coefficients A */
+  const int32_t* topk_idx_in;   /* if both *_in are set the router is skipped and this routing is used */
+  const float* topk_w_in;
+  float* shared_w;              /* [n_shared, T] coefficients of the shared experts */
+  int32_t* expert_token_counts; /* [n_routed+n_shared] tokens each expert saw */
+  uint32_t flags;               /* CAMERA_SCORE_* */
+  void* stage_events[2 * CAMERA_N_STAGES]; /* cudaEvent_t pairs (begin,end) recorded around each stage, or NULL */
+} camera_score_aux_t;
+
+const char* camera_strerror(int status);
+int camera_version(void);
+
+/* Scratch needed by camera_score_layer for this layer shape and token count (0 on invalid arguments). */
+size_t camera_score_workspace_bytes(const camera_layer_t* layer, int64_t n_tokens);
+
+/*
+ * Algorithm 1 of the paper (micro-expert ranking) up to and including line 10:
+ *   A      <- Top&Norm(softmax(R x))                               line 2
+ *   omega2 <- ColumnSum(W_down * W_down)                           line 5
+ *   Lambda <- A[:,e] * SiLU(W_gate X) * (W_up X)                   line 6  (never stored)
+ *   phi2   <- ColumnSum(Lambda*Lambda), phi_inf <- ColumnMax|Lambda|^2   lines 7-8
+ *   energy <- [(1-alpha) phi2 + alpha phi_inf] * omega2            line 10, Eq. 11
+ * x: DEVICE [n_tokens, d_model] row-major, dtype layer->dtype.  energy: DEVICE [N_e] fp32.
+ * Arithmetic: inputs as stored, products and sums in fp32 (bf16: tensor cores with fp32
+ * accumulators), the final blend in fp64.  Routing ties go to the lower expert index.
+ * An expert no token reaches gets energy 0.  0 <= alpha <= 1.  n_tokens >= 0.
+ * The bf16 tensor-core path needs d_model % 64 == 0 and every d_ff % 64 == 0; other shapes
+ * (and fp32) run the fp32-FMA kernel.
+ */
+int camera_score_layer(const camera_layer_t* layer, const void* x, int64_t n_tokens, float alpha,
+                       float* energy, const camera_score_aux_t* aux,
+                       void* workspace, size_t workspace_bytes, void* cuda_stream);
+
+/* Synchronises the stream, reads the workspace's status word (0 = fine, else a
+ * camera_status_t recorded by a kernel) into *status_out and clears nothing. */
+int camera_read_status(const void* workspace, void* cuda_stream, int32_t* status_out);
+
+/* Scratch for camera_select_prune / camera_alloc_bits (n_levels = 2 for pruning). */
+size_t camera_select_workspace_bytes(int64_t n_total, int32_t n_segments, int32_t n_levels);
+
+/*
+ * CAMERA-P selection (Algorithm 2 line 9, S <- TopSelect(R, 1 - lambda)), for one or many
+ * layers at once.  energy: DEVICE [n_total] fp32, non-negative.  seg_offsets: HOST
+ * [n_segments+1] increasing, seg_offsets[0] = 0, last = n_total; one segment = one layer.  In
+ * every segment of n elements the floor(prune_ratio * n + 1e-9) lowest-energy micro-experts get
+ * keep_mask = 0, all others 1; among equal energies the lower index is pruned first.
+ * 0 <= prune_ratio < 1.  Optional: expert_offsets DEVICE int64 [n_experts_total+1] (global
+ * micro-expert offsets) with kept_per_expert DEVICE [n_experts_total]; thresholds DEVICE
+ * [n_segments] receives the energy of the lowest retained micro-expert.
+ */
+int camera_select_prune(const float* energy, const int64_t* seg_offsets, int32_t n_segments,
+                        double prune_ratio, const int64_t* expert_offsets, int32_t n_experts_total,
+                        uint8_t* keep_mask, int32_t* kept_per_expert, float* thresholds,
+                        void* workspace, size_t workspace_bytes, void* cuda_stream);
+
+/*
+ * CAMERA-Q class split (Algorithm 3 lines 5-8: ListSplitByRatio + GetSubIndex).  ratios: HOST
+ * [n_levels] (2..8 levels), most important class first, summing to 1; bits: HOST [n_levels]
+ * bit-widths 0..255.  Within a segment of n elements ranked from highest to lowest energy
+ * (equal energies: higher index first), class j takes ranks [c_{j-1}, c_j) with
+ * c_j = floor((r_1+..+r_j) n + 1e-9) and c_L = n.  bits_out: DEVICE [n_total] uint8;
+ * class_counts (optional, with expert_offsets): DEVICE [n_experts_total, n_levels].
+ */
+int camera_alloc_bits(const float* energy, const int64_t* seg_offsets, int32_t n_segments,
+                      const double* ratios, const int32_t* bits, int32_t n_levels,
+                      const int64_t* expert_offsets, int32_t n_experts_total,
+                      uint8_t* bits_out, int32_t* class_counts,
+                      void* workspace, size_t workspace_bytes, void* cuda_stream);
+
+/* Scratch for camera_analyze_layer_host: score + select scratch + staging of x and results. */
+size_t camera_analyze_workspace_bytes(const camera_layer_t* layer, int64_t n_tokens, int32_t n_levels);
+
+/*
+ * One whole analysis step with HOST token and result buffers: copies x_host (pinned or
+ * pageable, [n_tokens, d_model]) to the device, runs camera_score_layer, camera_select_prune
+ * at prune_ratio and camera_alloc_bits, and copies energy [N_e] fp32, keep_mask [N_e] and
+ * bits_out [N_e] back to the given HOST buffers (any may be NULL).  The layer's weights stay
+ * DEVICE resident.  Synchronises the stream before returning, and returns the workspace's
+ * status word if a kernel recorded one.
+ */
+int camera_analyze_layer_host(const camera_layer_t* layer, const void* x_host, int64_t n_tokens,
+                              float alpha, double prune_ratio,
+                              const double* ratios, const int32_t* bits, int32_t n_levels,
+                              float* energy_host, uint8_t* keep_host, uint8_t* bits_host,
+                              void* workspace, size_t workspace_bytes, void* cuda_stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* CAMERA_B200_H */

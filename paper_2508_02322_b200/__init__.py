@@ -1,0 +1,10 @@
+"""B200 (sm_100a) implementation of the CAMERA micro-expert analysis hot path.
+
+`binding` wraps the C ABI of libcamera_b200.so (include/camera.h); `workloads` draws the seeded
+synthetic layers and calibration tokens the tests and the benchmark run on.
+"""
+from . import workloads  # noqa: F401
+from .binding import (  # noqa: F401
+    CameraError, Layer, alloc_workspace, camera_alloc_bits, camera_analyze_layer_host,
+    camera_analyze_workspace_bytes, camera_read_status, camera_score_layer, camera_score_workspace_bytes,
+    camera_select_prune, camera_select_workspace_bytes, lib)

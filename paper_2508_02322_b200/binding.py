@@ -1,0 +1,296 @@
+"""ctypes binding of libcamera_b200.so: argument marshalling only.
+
+Every function here has the name of the C entry point it calls (include/camera.h).  PyTorch is
+used for device memory and streams; all arithmetic happens in the CUDA library.  There is no
+fallback: if the shared library cannot be built or loaded, importing this module fails.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+from typing import Dict, List, Optional, Sequence
+
+import torch
+
+from . import build as _build
+
+CAMERA_OK = 0
+CAMERA_F32, CAMERA_BF16 = 0, 1
+CAMERA_DOWN_HF, CAMERA_DOWN_ME_MAJOR = 0, 1
+CAMERA_ROUTER_NORM_TOPK, CAMERA_SHARED_GATE_SIGMOID = 1, 2
+CAMERA_SCORE_FORCE_SIMT = 1
+STAGES = ("router", "permute", "rownorm", "score", "combine")
+
+
+class camera_layer_t(C.Structure):
+    _fields_ = [("d_model", C.c_int32), ("n_routed", C.c_int32), ("top_k", C.c_int32), ("n_shared", C.c_int32),
+                ("d_ff", C.POINTER(C.c_int32)), ("dtype", C.c_int32), ("flags", C.c_uint32),
+                ("down_layout", C.c_int32), ("w_router", C.c_void_p), ("router_bias", C.c_void_p),
+                ("w_shared_gate", C.c_void_p), ("w_gate", C.POINTER(C.c_void_p)),
+                ("w_up", C.POINTER(C.c_void_p)), ("w_down", C.POINTER(C.c_void_p))]
+
+
+class camera_score_aux_t(C.Structure):
+    _fields_ = [("phi2", C.c_void_p), ("phi_inf_sq", C.c_void_p), ("omega2", C.c_void_p),
+                ("topk_idx", C.c_void_p), ("topk_w", C.c_void_p), ("topk_idx_in", C.c_void_p),
+                ("topk_w_in", C.c_void_p), ("shared_w", C.c_void_p), ("expert_token_counts", C.c_void_p),
+                ("flags", C.c_uint32), ("stage_events", C.c_void_p * 10)]
+
+
+def _load() -> C.CDLL:
+    path = _build.LIB
+    if _build.needs_build():
+        _build.build()
+    if not os.path.exists(path):
+        raise ImportError("libcamera_b200.so is missing and could not be built; there is no fallback path")
+    lib = C.CDLL(path)
+    lib.camera_strerror.restype = C.c_char_p
+    lib.camera_strerror.argtypes = [C.c_int]
+    lib.camera_version.restype = C.c_int
+    lib.camera_score_workspace_bytes.restype = C.c_size_t
+    lib.camera_score_workspace_bytes.argtypes = [C.POINTER(camera_layer_t), C.c_int64]
+    lib.camera_score_layer.restype = C.c_int
+    lib.camera_score_layer.argtypes = [C.POINTER(camera_layer_t), C.c_void_p, C.c_int64, C.c_float, C.c_void_p,
+                                       C.POINTER(camera_score_aux_t), C.c_void_p, C.c_size_t, C.c_void_p]
+    lib.camera_read_status.restype = C.c_int
+    lib.camera_read_status.argtypes = [C.c_void_p, C.c_void_p, C.POINTER(C.c_int32)]
+    lib.camera_select_workspace_bytes.restype = C.c_size_t
+    lib.camera_select_workspace_bytes.argtypes = [C.c_int64, C.c_int32, C.c_int32]
+    lib.camera_select_prune.restype = C.c_int
+    lib.camera_select_prune.argtypes = [C.c_void_p, C.POINTER(C.c_int64), C.c_int32, C.c_double, C.c_void_p,
+                                        C.c_int32, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_size_t,
+                                        C.c_void_p]
+    lib.camera_alloc_bits.restype = C.c_int
+    lib.camera_alloc_bits.argtypes = [C.c_void_p, C.POINTER(C.c_int64), C.c_int32, C.POINTER(C.c_double),
+                                      C.POINTER(C.c_int32), C.c_int32, C.c_void_p, C.c_int32, C.c_void_p,
+                                      C.c_void_p, C.c_void_p, C.c_size_t, C.c_void_p]
+    lib.camera_analyze_workspace_bytes.restype = C.c_size_t
+    lib.camera_analyze_workspace_bytes.argtypes = [C.POINTER(camera_layer_t), C.c_int64, C.c_int32]
+    lib.camera_analyze_layer_host.restype = C.c_int
+    lib.camera_analyze_layer_host.argtypes = [C.POINTER(camera_layer_t), C.c_void_p, C.c_int64, C.c_float,
+                                              C.c_double, C.POINTER(C.c_double), C.POINTER(C.c_int32), C.c_int32,
+                                              C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_size_t,
+                                              C.c_void_p]
+    return lib
+
+
+lib = _load()
+
+
+class CameraError(RuntimeError):
+    def __init__(self, status: int, where: str):
+        self.status = status
+        super().__init__(f"{where}: {lib.camera_strerror(status).decode()} ({status})")
+
+
+def _check(status: int, where: str) -> None:
+    if status != CAMERA_OK:
+        raise CameraError(status, where)
+
+
+def _ptr(t: Optional[torch.Tensor]) -> Optional[int]:
+    return None if t is None else t.data_ptr()
+
+
+def _stream_ptr(stream: Optional[torch.cuda.Stream]) -> Optional[int]:
+    s = torch.cuda.current_stream() if stream is None else stream
+    return s.cuda_stream or None
+
+
+class Layer:
+    """Holds the tensors of one MoE layer and the camera_layer_t that points at them.
+
+    w_gate / w_up: lists of [d_ff_e, d_model]; w_down: list of [d_model, d_ff_e] (down_layout "hf")
+    or [d_ff_e, d_model] ("me_major"); experts ordered routed first, then shared.
+    """
+
+    def __init__(self, w_router, w_gate: Sequence[torch.Tensor], w_up, w_down, top_k: int, n_shared: int = 0,
+                 router_bias=None, w_shared_gate=None, norm_topk: bool = True, down_layout: str = "hf"):
+        self.tensors = dict(w_router=w_router, router_bias=router_bias, w_shared_gate=w_shared_gate,
+                            w_gate=list(w_gate), w_up=list(w_up), w_down=list(w_down))
+        ref = w_gate[0]
+        for t in list(w_gate) + list(w_up) + list(w_down) + [t for t in (w_router, w_shared_gate) if t is not None]:
+            if not (t.is_contiguous() and t.dtype == ref.dtype and t.device == ref.device):
+                raise ValueError("layer tensors must be contiguous and share dtype and device")
+        if router_bias is not None and router_bias.dtype != torch.float32:
+            raise ValueError("router_bias must be float32")
+        self.dtype = ref.dtype
+        self.device = ref.device
+        n = len(w_gate)
+        self.n_experts = n
+        self.d_model = int(ref.shape[1])
+        self.d_ff = [int(w.shape[0]) for w in w_gate]
+        self.n_me = sum(self.d_ff)
+        self.n_routed = n - n_shared
+        self._d_ff = (C.c_int32 * n)(*self.d_ff)
+        self._wg = (C.c_void_p * n)(*[w.data_ptr() for w in w_gate])
+        self._wu = (C.c_void_p * n)(*[w.data_ptr() for w in w_up])
+        self._wd = (C.c_void_p * n)(*[w.data_ptr() for w in w_down])
+        flags = (CAMERA_ROUTER_NORM_TOPK if norm_topk else 0) | \
+                (CAMERA_SHARED_GATE_SIGMOID if w_shared_gate is not None else 0)
+        self.c = camera_layer_t(
+            self.d_model, self.n_routed, top_k, n_shared, self._d_ff,
+            CAMERA_BF16 if self.dtype == torch.bfloat16 else CAMERA_F32, flags,
+            CAMERA_DOWN_HF if down_layout == "hf" else CAMERA_DOWN_ME_MAJOR,
+            _ptr(w_router), _ptr(router_bias), _ptr(w_shared_gate), self._wg, self._wu, self._wd)
+        self.top_k = top_k
+        self.n_shared = n_shared
+
+    @classmethod
+    def from_workload(cls, L: Dict[str, object]) -> "Layer":
+        """From the dict paper_2508_02322_b200.workloads.make_layer returns."""
+        cfg = L["cfg"]
+        return cls(L["w_router"], L["w_gate"], L["w_up"], L["w_down"], cfg.top_k, cfg.n_shared, L["router_bias"],
+                   L["w_shared_gate"], cfg.norm_topk, L["down_layout"])
+
+
+def camera_score_workspace_bytes(layer: Layer, n_tokens: int) -> int:
+    return int(lib.camera_score_workspace_bytes(C.byref(layer.c), n_tokens))
+
+
+def camera_select_workspace_bytes(n_total: int, n_segments: int, n_levels: int) -> int:
+    return int(lib.camera_select_workspace_bytes(n_total, n_segments, n_levels))
+
+
+def camera_analyze_workspace_bytes(layer: Layer, n_tokens: int, n_levels: int) -> int:
+    return int(lib.camera_analyze_workspace_bytes(C.byref(layer.c), n_tokens, n_levels))
+
+
+def alloc_workspace(nbytes: int, device) -> torch.Tensor:
+    """A 256-byte aligned scratch buffer (torch's caching allocator aligns to 512 bytes)."""
+    return torch.empty(max(int(nbytes), 256), dtype=torch.uint8, device=device)
+
+
+def camera_score_layer(layer: Layer, x: torch.Tensor, alpha: float, *, energy: Optional[torch.Tensor] = None,
+                       workspace: Optional[torch.Tensor] = None, details: bool = False,
+                       routing_in=None, force_simt: bool = False, stage_events=None,
+                       stream: Optional[torch.cuda.Stream] = None, check_status: bool = False):
+    """Algorithm 1 up to the energies.  Returns energy [N_e] fp32, or with details=True a dict that
+    also holds phi2, phi_inf_sq, omega2, topk_idx, topk_w, shared_w and expert_token_counts.
+    routing_in = (topk_idx int32 [T,k], topk_w fp32 [T,k]) prescribes the routing.
+    stage_events = {stage: (torch.cuda.Event, torch.cuda.Event)} records per-stage timing events."""
+    if not (x.is_contiguous() and x.dtype == layer.dtype and x.dim() == 2 and x.shape[1] == layer.d_model):
+        raise ValueError("x must be a contiguous [T, d_model] tensor of the layer's dtype")
+    T = int(x.shape[0])
+    dev = x.device
+    if energy is None:
+        energy = torch.empty(layer.n_me, dtype=torch.float32, device=dev)
+    if workspace is None:
+        workspace = alloc_workspace(camera_score_workspace_bytes(layer, T), dev)
+    aux = camera_score_aux_t()
+    out = {"energy": energy}
+    keep_alive = []
+    if details:
+        k = layer.top_k if layer.n_routed else 0
+        out["phi2"] = torch.empty(layer.n_me, dtype=torch.float32, device=dev)
+        out["phi_inf_sq"] = torch.empty(layer.n_me, dtype=torch.float32, device=dev)
+        out["omega2"] = torch.empty(layer.n_me, dtype=torch.float32, device=dev)
+        out["topk_idx"] = torch.empty((T, k), dtype=torch.int32, device=dev)
+        out["topk_w"] = torch.empty((T, k), dtype=torch.float32, device=dev)
+        out["shared_w"] = torch.empty((layer.n_shared, T), dtype=torch.float32, device=dev)
+        out["expert_token_counts"] = torch.empty(layer.n_experts, dtype=torch.int32, device=dev)
+        for name in ("phi2", "phi_inf_sq", "omega2", "topk_idx", "topk_w", "shared_w", "expert_token_counts"):
+            setattr(aux, name, out[name].data_ptr())
+    if routing_in is not None:
+        idx, w = routing_in
+        idx = idx.to(device=dev, dtype=torch.int32).contiguous()
+        w = w.to(device=dev, dtype=torch.float32).contiguous()
+        keep_alive += [idx, w]
+        aux.topk_idx_in, aux.topk_w_in = idx.data_ptr(), w.data_ptr()
+    if force_simt:
+        aux.flags = CAMERA_SCORE_FORCE_SIMT
+    if stage_events:
+        for name, (e0, e1) in stage_events.items():
+            i = STAGES.index(name)
+            aux.stage_events[2 * i] = e0.cuda_event
+            aux.stage_events[2 * i + 1] = e1.cuda_event
+    sp = _stream_ptr(stream)
+    _check(lib.camera_score_layer(C.byref(layer.c), x.data_ptr(), T, float(alpha), energy.data_ptr(),
+                                  C.byref(aux), workspace.data_ptr(), workspace.numel(), sp), "camera_score_layer")
+    if check_status:
+        _check(camera_read_status(workspace, stream), "camera_score_layer (device status)")
+    return out if details else energy
+
+
+def camera_read_status(workspace: torch.Tensor, stream: Optional[torch.cuda.Stream] = None) -> int:
+    st = C.c_int32(0)
+    _check(lib.camera_read_status(workspace.data_ptr(), _stream_ptr(stream), C.byref(st)), "camera_read_status")
+    return int(st.value)
+
+
+def _segments(n_total: int, seg_offsets):
+    seg = [0, n_total] if seg_offsets is None else [int(v) for v in seg_offsets]
+    return (C.c_int64 * len(seg))(*seg), len(seg) - 1
+
+
+def camera_select_prune(energy: torch.Tensor, prune_ratio: float, *, seg_offsets=None,
+                        expert_offsets: Optional[torch.Tensor] = None, workspace: Optional[torch.Tensor] = None,
+                        keep_mask: Optional[torch.Tensor] = None, want_threshold: bool = False,
+                        stream: Optional[torch.cuda.Stream] = None):
+    """CAMERA-P mask.  Returns keep_mask uint8 [N]; with expert_offsets (int64, device) also the
+    retained count per expert; with want_threshold the per-segment threshold energies."""
+    n = energy.numel()
+    dev = energy.device
+    seg, n_seg = _segments(n, seg_offsets)
+    if keep_mask is None:
+        keep_mask = torch.empty(n, dtype=torch.uint8, device=dev)
+    if workspace is None:
+        workspace = alloc_workspace(camera_select_workspace_bytes(n, n_seg, 2), dev)
+    kept = thr = None
+    n_exp = 0
+    if expert_offsets is not None:
+        n_exp = expert_offsets.numel() - 1
+        kept = torch.empty(n_exp, dtype=torch.int32, device=dev)
+    if want_threshold:
+        thr = torch.empty(n_seg, dtype=torch.float32, device=dev)
+    _check(lib.camera_select_prune(energy.data_ptr(), seg, n_seg, float(prune_ratio), _ptr(expert_offsets), n_exp,
+                                   keep_mask.data_ptr(), _ptr(kept), _ptr(thr), workspace.data_ptr(),
+                                   workspace.numel(), _stream_ptr(stream)), "camera_select_prune")
+    res = [keep_mask]
+    if kept is not None:
+        res.append(kept)
+    if thr is not None:
+        res.append(thr)
+    return res[0] if len(res) == 1 else tuple(res)
+
+
+def camera_alloc_bits(energy: torch.Tensor, ratios: Sequence[float], bits: Sequence[int], *, seg_offsets=None,
+                      expert_offsets: Optional[torch.Tensor] = None, workspace: Optional[torch.Tensor] = None,
+                      bits_out: Optional[torch.Tensor] = None, stream: Optional[torch.cuda.Stream] = None):
+    """CAMERA-Q bit-width per micro-expert.  Returns bits_out uint8 [N]; with expert_offsets also
+    class_counts int32 [n_experts, n_levels]."""
+    n = energy.numel()
+    dev = energy.device
+    L = len(ratios)
+    seg, n_seg = _segments(n, seg_offsets)
+    if bits_out is None:
+        bits_out = torch.empty(n, dtype=torch.uint8, device=dev)
+    if workspace is None:
+        workspace = alloc_workspace(camera_select_workspace_bytes(n, n_seg, L), dev)
+    counts = None
+    n_exp = 0
+    if expert_offsets is not None:
+        n_exp = expert_offsets.numel() - 1
+        counts = torch.empty((n_exp, L), dtype=torch.int32, device=dev)
+    r = (C.c_double * L)(*[float(v) for v in ratios])
+    b = (C.c_int32 * L)(*[int(v) for v in bits])
+    _check(lib.camera_alloc_bits(energy.data_ptr(), seg, n_seg, r, b, L, _ptr(expert_offsets), n_exp,
+                                 bits_out.data_ptr(), _ptr(counts), workspace.data_ptr(), workspace.numel(),
+                                 _stream_ptr(stream)), "camera_alloc_bits")
+    return bits_out if counts is None else (bits_out, counts)
+
+
+def camera_analyze_layer_host(layer: Layer, x_host: torch.Tensor, alpha: float, prune_ratio: float,
+                              ratios: Sequence[float], bits: Sequence[int], *, energy_host: torch.Tensor,
+                              keep_host: torch.Tensor, bits_host: torch.Tensor, workspace: torch.Tensor,
+                              stream: Optional[torch.cuda.Stream] = None) -> None:
+    """One analysis step with host token/result buffers (see camera.h); blocks until done."""
+    if x_host.is_cuda or not x_host.is_contiguous() or x_host.dtype != layer.dtype:
+        raise ValueError("x_host must be a contiguous host tensor of the layer's dtype")
+    L = len(ratios)
+    r = (C.c_double * L)(*[float(v) for v in ratios])
+    b = (C.c_int32 * L)(*[int(v) for v in bits])
+    _check(lib.camera_analyze_layer_host(C.byref(layer.c), x_host.data_ptr(), int(x_host.shape[0]), float(alpha),
+                                         float(prune_ratio), r, b, L, _ptr(energy_host), _ptr(keep_host),
+                                         _ptr(bits_host), workspace.data_ptr(), workspace.numel(),
+                                         _stream_ptr(stream)), "camera_analyze_layer_host")

@@ -1,0 +1,347 @@
+// C ABI entry points of camera_score_layer and camera_analyze_layer_host: argument checks,
+// workspace carving, and the launch sequence.  No device memory is allocated here.
+#include <string.h>
+
+#include <vector>
+
+#include "common.cuh"
+
+namespace camera {
+
+int rownorm_blocks(int down_layout, int dtype, int f);
+
+namespace {
+
+constexpr int PLAN_SMS = 148;   // used only to size work units; the result is valid on any device
+
+size_t up256(size_t v) { return (v + 255) & ~(size_t)255; }
+
+struct ScoreLayout {
+  size_t totals, est, edyn, me_prefix, unit_prefix, counts, block_hist, local_rank, topk_idx, topk_w, shared_w,
+      perm_w, x_perm, part_sum, part_max, phi2, phi_inf_sq, omega2, tensor_maps, total;
+  int n_experts, n_me, n_blocks, chunk_tokens, max_rows_perm;
+  long long max_part;
+};
+
+int validate_layer(const camera_layer_t* L, int64_t T) {
+  if (L == nullptr || L->d_ff == nullptr || L->w_gate == nullptr || L->w_up == nullptr || L->w_down == nullptr)
+    return CAMERA_ERR_INVALID_ARG;
+  if (L->dtype != CAMERA_F32 && L->dtype != CAMERA_BF16) return CAMERA_ERR_INVALID_ARG;
+  if (L->down_layout != CAMERA_DOWN_HF && L->down_layout != CAMERA_DOWN_ME_MAJOR) return CAMERA_ERR_INVALID_ARG;
+  if (L->n_routed < 0 || L->n_shared < 0 || L->n_routed + L->n_shared < 1 || T < 0) return CAMERA_ERR_INVALID_ARG;
+  if (L->n_routed > MAX_ROUTED || L->n_shared > 64) return CAMERA_ERR_UNSUPPORTED_SHAPE;
+  if (L->n_routed > 0) {
+    if (L->top_k < 1 || L->top_k > L->n_routed) return CAMERA_ERR_INVALID_ARG;
+    if (L->top_k > MAX_TOPK) return CAMERA_ERR_UNSUPPORTED_SHAPE;
+    if (L->w_router == nullptr) return CAMERA_ERR_INVALID_ARG;
+  }
+  if (L->d_model < 8 || L->d_model % 8 != 0) return CAMERA_ERR_UNSUPPORTED_SHAPE;
+  if ((L->flags & CAMERA_SHARED_GATE_SIGMOID) && L->n_shared > 0 && L->w_shared_gate == nullptr)
+    return CAMERA_ERR_INVALID_ARG;
+  long long n_me = 0;
+  for (int e = 0; e < L->n_routed + L->n_shared; ++e) {
+    if (L->d_ff[e] < 8 || L->d_ff[e] % 8 != 0) return CAMERA_ERR_UNSUPPORTED_SHAPE;
+    if (L->w_gate[e] == nullptr || L->w_up[e] == nullptr || L->w_down[e] == nullptr) return CAMERA_ERR_INVALID_ARG;
+    n_me += L->d_ff[e];
+  }
+  if (n_me >= (1ll << 31)) return CAMERA_ERR_UNSUPPORTED_SHAPE;
+  const long long k = L->n_routed > 0 ? L->top_k : 0;
+  if (T * (k > 1 ? k : 1) + (long long)ROW_ALIGN * L->n_routed >= (1ll << 31)) return CAMERA_ERR_UNSUPPORTED_SHAPE;
+  return CAMERA_OK;
+}
+
+ScoreLayout score_layout(const camera_layer_t* L, int64_t T) {
+  ScoreLayout s;
+  memset(&s, 0, sizeof(s));
+  const int E = L->n_routed + L->n_shared;
+  const int k = L->n_routed > 0 ? L->top_k : 0;
+  const size_t esz = L->dtype == CAMERA_BF16 ? 2 : 4;
+  s.n_experts = E;
+  s.n_blocks = (int)((T + ROUTER_TOK - 1) / ROUTER_TOK);
+  long long n_me = 0;
+  double tiles = 0.0;
+  int f_routed_max = 0;
+  for (int e = 0; e < E; ++e) {
+    n_me += L->d_ff[e];
+    const double ct = (double)((L->d_ff[e] + CH_TILE - 1) / CH_TILE);
+    if (e < L->n_routed) {
+      f_routed_max = L->d_ff[e] > f_routed_max ? L->d_ff[e] : f_routed_max;
+    } else {
+      tiles += ct * (double)((T + UMMA_TOK - 1) / UMMA_TOK);
+    }
+  }
+  if (L->n_routed > 0) {
+    double avg_ct = 0.0;
+    for (int e = 0; e < L->n_routed; ++e) avg_ct += (double)((L->d_ff[e] + CH_TILE - 1) / CH_TILE);
+    avg_ct /= L->n_routed;
+    tiles += avg_ct * (double)(T * k) / UMMA_TOK;
+  }
+  s.n_me = (int)n_me;
+  // tokens per work unit: a power-of-two number of tiles, about 64 units per SM, 1..16 tiles
+  int chunk_tiles = 1;
+  while (chunk_tiles < 16 && tiles / (2.0 * chunk_tiles) >= 64.0 * PLAN_SMS) chunk_tiles *= 2;
+  s.chunk_tokens = chunk_tiles * UMMA_TOK;
+  s.max_rows_perm = (int)(T * k + (long long)ROW_ALIGN * L->n_routed);
+  long long part = 0;
+  if (L->n_routed > 0) part += (long long)f_routed_max * ((T * k) / s.chunk_tokens + L->n_routed);
+  for (int e = L->n_routed; e < E; ++e) part += (long long)L->d_ff[e] * ((T + s.chunk_tokens - 1) / s.chunk_tokens);
+  s.max_part = part > 0 ? part : 1;
+
+  size_t o = 0;
+  auto take = [&](size_t bytes) { size_t at = o; o = up256(o + bytes); return at; };
+  s.totals = take(sizeof(PlanTotals));
+  s.est = take(sizeof(ExpertStatic) * E);
+  s.edyn = take(sizeof(ExpertDyn) * E);
+  s.me_prefix = take(sizeof(int32_t) * (E + 1));
+  s.unit_prefix = take(sizeof(int32_t) * (E + 1));
+  s.counts = take(sizeof(int32_t) * E);
+  s.block_hist = take(sizeof(int32_t) * (size_t)s.n_blocks * L->n_routed);
+  s.local_rank = take(sizeof(int32_t) * (size_t)T * k);
+  s.topk_idx = take(sizeof(int32_t) * (size_t)T * k);
+  s.topk_w = take(sizeof(float) * (size_t)T * k);
+  s.shared_w = take(sizeof(float) * (size_t)T * L->n_shared);
+  s.perm_w = take(sizeof(float) * (size_t)s.max_rows_perm);
+  s.x_perm = take(esz * (size_t)s.max_rows_perm * L->d_model);
+  s.part_sum = take(sizeof(float) * (size_t)s.max_part);
+  s.part_max = take(sizeof(float) * (size_t)s.max_part);
+  s.phi2 = take(sizeof(float) * (size_t)n_me);
+  s.phi_inf_sq = take(sizeof(float) * (size_t)n_me);
+  s.omega2 = take(sizeof(float) * (size_t)n_me);
+  s.tensor_maps = take((size_t)128 * (2 * E + 2));
+  s.total = o;
+  return s;
+}
+
+#define CK(expr)                                   \
+  do {                                             \
+    if ((expr) != cudaSuccess) {                   \
+      cudaGetLastError();                          \
+      return CAMERA_ERR_CUDA;                      \
+    }                                              \
+  } while (0)
+
+struct StageTimer {
+  const camera_score_aux_t* aux;
+  cudaStream_t st;
+  void begin(int stage) const {
+    if (aux && aux->stage_events[2 * stage]) cudaEventRecord(static_cast<cudaEvent_t>(aux->stage_events[2 * stage]), st);
+  }
+  void end(int stage) const {
+    if (aux && aux->stage_events[2 * stage + 1])
+      cudaEventRecord(static_cast<cudaEvent_t>(aux->stage_events[2 * stage + 1]), st);
+  }
+};
+
+}  // namespace
+}  // namespace camera
+
+using namespace camera;
+
+extern "C" const char* camera_strerror(int status) {
+  switch (status) {
+    case CAMERA_OK: return "ok";
+    case CAMERA_ERR_INVALID_ARG: return "invalid argument";
+    case CAMERA_ERR_UNSUPPORTED_SHAPE: return "unsupported shape";
+    case CAMERA_ERR_WORKSPACE: return "workspace missing or too small";
+    case CAMERA_ERR_ARCH: return "device is not sm_100";
+    case CAMERA_ERR_CUDA: return "CUDA runtime error";
+    case CAMERA_ERR_DEVICE_TIMEOUT: return "a bounded wait inside a kernel ran out";
+    default: return "unknown status";
+  }
+}
+
+extern "C" int camera_version(void) { return 100; }
+
+extern "C" size_t camera_score_workspace_bytes(const camera_layer_t* layer, int64_t n_tokens) {
+  if (validate_layer(layer, n_tokens) != CAMERA_OK) return 0;
+  return score_layout(layer, n_tokens).total;
+}
+
+extern "C" int camera_score_layer(const camera_layer_t* L, const void* x, int64_t T, float alpha, float* energy,
+                                  const camera_score_aux_t* aux, void* workspace, size_t workspace_bytes,
+                                  void* cuda_stream) {
+  int rc = validate_layer(L, T);
+  if (rc != CAMERA_OK) return rc;
+  if (!(alpha >= 0.f && alpha <= 1.f) || energy == nullptr || (T > 0 && x == nullptr)) return CAMERA_ERR_INVALID_ARG;
+  if (aux && ((aux->topk_idx_in == nullptr) != (aux->topk_w_in == nullptr))) return CAMERA_ERR_INVALID_ARG;
+  {  // every matrix is read with 16-byte vector loads
+    uintptr_t bits = reinterpret_cast<uintptr_t>(x) | reinterpret_cast<uintptr_t>(L->w_router) |
+                     reinterpret_cast<uintptr_t>(L->w_shared_gate);
+    for (int e = 0; e < L->n_routed + L->n_shared; ++e)
+      bits |= reinterpret_cast<uintptr_t>(L->w_gate[e]) | reinterpret_cast<uintptr_t>(L->w_up[e]) |
+              reinterpret_cast<uintptr_t>(L->w_down[e]);
+    if (bits & 15) return CAMERA_ERR_INVALID_ARG;
+  }
+  const ScoreLayout lay = score_layout(L, T);
+  if (workspace == nullptr || workspace_bytes < lay.total || (reinterpret_cast<uintptr_t>(workspace) & 255))
+    return CAMERA_ERR_WORKSPACE;
+  int dev = 0, major = 0;
+  CK(cudaGetDevice(&dev));
+  CK(cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev));
+  if (major != 10) return CAMERA_ERR_ARCH;
+  cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+  char* ws = static_cast<char*>(workspace);
+  const int E = lay.n_experts;
+
+  ScoreCtx c;
+  memset(&c, 0, sizeof(c));
+  c.d_model = L->d_model; c.n_routed = L->n_routed; c.top_k = L->n_routed > 0 ? L->top_k : 0;
+  c.n_shared = L->n_shared; c.n_experts = E; c.n_me = lay.n_me;
+  c.dtype = L->dtype; c.down_layout = L->down_layout; c.flags = L->flags;
+  c.n_tokens = (int)T; c.n_blocks = lay.n_blocks; c.chunk_tokens = lay.chunk_tokens;
+  c.max_rows_perm = lay.max_rows_perm; c.max_part = lay.max_part; c.alpha = alpha;
+  c.x = x; c.w_router = L->w_router; c.router_bias = L->router_bias; c.w_shared_gate = L->w_shared_gate;
+  c.totals = reinterpret_cast<PlanTotals*>(ws + lay.totals);
+  c.est = reinterpret_cast<ExpertStatic*>(ws + lay.est);
+  c.edyn = reinterpret_cast<ExpertDyn*>(ws + lay.edyn);
+  c.me_prefix = reinterpret_cast<int32_t*>(ws + lay.me_prefix);
+  c.unit_prefix = reinterpret_cast<int32_t*>(ws + lay.unit_prefix);
+  c.counts = (aux && aux->expert_token_counts) ? aux->expert_token_counts : reinterpret_cast<int32_t*>(ws + lay.counts);
+  c.block_hist = reinterpret_cast<int32_t*>(ws + lay.block_hist);
+  c.local_rank = reinterpret_cast<int32_t*>(ws + lay.local_rank);
+  c.topk_idx = (aux && aux->topk_idx) ? aux->topk_idx : reinterpret_cast<int32_t*>(ws + lay.topk_idx);
+  c.topk_w = (aux && aux->topk_w) ? aux->topk_w : reinterpret_cast<float*>(ws + lay.topk_w);
+  c.shared_w = (aux && aux->shared_w) ? aux->shared_w : reinterpret_cast<float*>(ws + lay.shared_w);
+  c.perm_w = reinterpret_cast<float*>(ws + lay.perm_w);
+  c.x_perm = ws + lay.x_perm;
+  c.part_sum = reinterpret_cast<float*>(ws + lay.part_sum);
+  c.part_max = reinterpret_cast<float*>(ws + lay.part_max);
+  c.phi2 = (aux && aux->phi2) ? aux->phi2 : reinterpret_cast<float*>(ws + lay.phi2);
+  c.phi_inf_sq = (aux && aux->phi_inf_sq) ? aux->phi_inf_sq : reinterpret_cast<float*>(ws + lay.phi_inf_sq);
+  c.omega2 = (aux && aux->omega2) ? aux->omega2 : reinterpret_cast<float*>(ws + lay.omega2);
+  c.energy = energy;
+  c.tensor_maps = ws + lay.tensor_maps;
+
+  // host-known tables
+  std::vector<ExpertStatic> est(E);
+  std::vector<int32_t> me_prefix(E + 1);
+  int me = 0, norm_blocks = 0;
+  for (int e = 0; e < E; ++e) {
+    est[e].w_gate = L->w_gate[e]; est[e].w_up = L->w_up[e]; est[e].w_down = L->w_down[e];
+    est[e].d_ff = L->d_ff[e]; est[e].me_off = me;
+    est[e].shared_idx = e < L->n_routed ? -1 : e - L->n_routed;
+    est[e].norm_blk_begin = norm_blocks;
+    me_prefix[e] = me;
+    me += L->d_ff[e];
+    norm_blocks += rownorm_blocks(L->down_layout, L->dtype, L->d_ff[e]);
+  }
+  me_prefix[E] = me;
+
+  const bool use_umma = umma_shape_ok(L) && !(aux && (aux->flags & CAMERA_SCORE_FORCE_SIMT)) &&
+                        (reinterpret_cast<uintptr_t>(x) & 15) == 0;
+  std::vector<char> maps;
+  if (use_umma) {
+    maps.resize((size_t)128 * (2 * E + 2));
+    rc = encode_tensor_maps(L, c, maps.data());
+    if (rc != CAMERA_OK) return rc;
+  }
+
+  CK(cudaMemsetAsync(c.totals, 0, sizeof(PlanTotals), st));
+  CK(cudaMemsetAsync(c.counts, 0, sizeof(int32_t) * E, st));
+  CK(cudaMemcpyAsync(c.est, est.data(), sizeof(ExpertStatic) * E, cudaMemcpyHostToDevice, st));
+  CK(cudaMemcpyAsync(c.me_prefix, me_prefix.data(), sizeof(int32_t) * (E + 1), cudaMemcpyHostToDevice, st));
+  if (use_umma) CK(cudaMemcpyAsync(c.tensor_maps, maps.data(), maps.size(), cudaMemcpyHostToDevice, st));
+
+  const StageTimer tm{aux, st};
+  tm.begin(CAMERA_STAGE_ROUTER);
+  if (aux && aux->topk_idx_in) CK(launch_routing_from_input(c, aux->topk_idx_in, aux->topk_w_in, st));
+  else CK(launch_router(c, st));
+  tm.end(CAMERA_STAGE_ROUTER);
+
+  tm.begin(CAMERA_STAGE_PERMUTE);
+  CK(launch_plan(c, st));
+  CK(launch_permute(c, st));
+  tm.end(CAMERA_STAGE_PERMUTE);
+
+  tm.begin(CAMERA_STAGE_ROWNORM);
+  CK(launch_rownorm(c, norm_blocks, st));
+  tm.end(CAMERA_STAGE_ROWNORM);
+
+  tm.begin(CAMERA_STAGE_SCORE);
+  if (T > 0) {
+    if (use_umma) CK(launch_score_umma(c, st));
+    else CK(launch_score_simt(c, st));
+  }
+  tm.end(CAMERA_STAGE_SCORE);
+
+  tm.begin(CAMERA_STAGE_COMBINE);
+  CK(launch_combine(c, st));
+  tm.end(CAMERA_STAGE_COMBINE);
+  return CAMERA_OK;
+}
+
+extern "C" int camera_read_status(const void* workspace, void* cuda_stream, int32_t* status_out) {
+  if (workspace == nullptr || status_out == nullptr) return CAMERA_ERR_INVALID_ARG;
+  PlanTotals t;
+  cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+  CK(cudaMemcpyAsync(&t, workspace, sizeof(t), cudaMemcpyDeviceToHost, st));
+  CK(cudaStreamSynchronize(st));
+  *status_out = t.status;
+  return CAMERA_OK;
+}
+
+namespace {
+struct AnalyzeLayout {
+  size_t score, select, x, energy, keep, bits, total;
+  size_t score_bytes, select_bytes;
+};
+AnalyzeLayout analyze_layout(const camera_layer_t* L, int64_t T, int n_levels) {
+  AnalyzeLayout a;
+  const ScoreLayout s = score_layout(L, T);
+  const size_t esz = L->dtype == CAMERA_BF16 ? 2 : 4;
+  a.score_bytes = s.total;
+  a.select_bytes = camera_select_workspace_bytes(s.n_me, 1, n_levels < 2 ? 2 : n_levels);
+  size_t o = 0;
+  auto take = [&](size_t bytes) { size_t at = o; o = up256(o + bytes); return at; };
+  a.score = take(a.score_bytes);
+  a.select = take(a.select_bytes);
+  a.x = take(esz * (size_t)T * L->d_model);
+  a.energy = take(sizeof(float) * (size_t)s.n_me);
+  a.keep = take((size_t)s.n_me);
+  a.bits = take((size_t)s.n_me);
+  a.total = o;
+  return a;
+}
+}  // namespace
+
+extern "C" size_t camera_analyze_workspace_bytes(const camera_layer_t* layer, int64_t n_tokens, int32_t n_levels) {
+  if (validate_layer(layer, n_tokens) != CAMERA_OK || n_levels < 2 || n_levels > MAX_LEVELS) return 0;
+  return analyze_layout(layer, n_tokens, n_levels).total;
+}
+
+extern "C" int camera_analyze_layer_host(const camera_layer_t* L, const void* x_host, int64_t T, float alpha,
+                                         double prune_ratio, const double* ratios, const int32_t* bits,
+                                         int32_t n_levels, float* energy_host, uint8_t* keep_host, uint8_t* bits_host,
+                                         void* workspace, size_t workspace_bytes, void* cuda_stream) {
+  int rc = validate_layer(L, T);
+  if (rc != CAMERA_OK) return rc;
+  if (n_levels < 2 || n_levels > MAX_LEVELS || ratios == nullptr || bits == nullptr || (T > 0 && x_host == nullptr))
+    return CAMERA_ERR_INVALID_ARG;
+  const AnalyzeLayout a = analyze_layout(L, T, n_levels);
+  if (workspace == nullptr || workspace_bytes < a.total || (reinterpret_cast<uintptr_t>(workspace) & 255))
+    return CAMERA_ERR_WORKSPACE;
+  cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+  char* ws = static_cast<char*>(workspace);
+  const size_t esz = L->dtype == CAMERA_BF16 ? 2 : 4;
+  const ScoreLayout s = score_layout(L, T);
+  float* d_energy = reinterpret_cast<float*>(ws + a.energy);
+  uint8_t* d_keep = reinterpret_cast<uint8_t*>(ws + a.keep);
+  uint8_t* d_bits = reinterpret_cast<uint8_t*>(ws + a.bits);
+  if (T > 0) CK(cudaMemcpyAsync(ws + a.x, x_host, esz * (size_t)T * L->d_model, cudaMemcpyHostToDevice, st));
+  rc = camera_score_layer(L, ws + a.x, T, alpha, d_energy, nullptr, ws + a.score, a.score_bytes, cuda_stream);
+  if (rc != CAMERA_OK) return rc;
+  const int64_t seg[2] = {0, s.n_me};
+  rc = camera_select_prune(d_energy, seg, 1, prune_ratio, nullptr, 0, d_keep, nullptr, nullptr, ws + a.select,
+                           a.select_bytes, cuda_stream);
+  if (rc != CAMERA_OK) return rc;
+  if (keep_host) CK(cudaMemcpyAsync(keep_host, d_keep, (size_t)s.n_me, cudaMemcpyDeviceToHost, st));
+  rc = camera_alloc_bits(d_energy, seg, 1, ratios, bits, n_levels, nullptr, 0, d_bits, nullptr, ws + a.select,
+                         a.select_bytes, cuda_stream);
+  if (rc != CAMERA_OK) return rc;
+  if (energy_host) CK(cudaMemcpyAsync(energy_host, d_energy, sizeof(float) * (size_t)s.n_me, cudaMemcpyDeviceToHost, st));
+  if (bits_host) CK(cudaMemcpyAsync(bits_host, d_bits, (size_t)s.n_me, cudaMemcpyDeviceToHost, st));
+  int32_t status = 0;
+  rc = camera_read_status(ws + a.score, cuda_stream, &status);
+  if (rc != CAMERA_OK) return rc;
+  return status;
+}

@@ -1,0 +1,135 @@
+// Shared declarations of the CAMERA sm_100a library: plan tables, launch prototypes, small helpers.
+#pragma once
+
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "camera.h"
+
+namespace camera {
+
+// ---- tiling constants shared by the host planner and the kernels -----------------------------
+constexpr int ROUTER_TOK = 64;       // tokens per router CTA (also the unit of the stable counting sort)
+constexpr int ROW_ALIGN = 16;        // every expert's token list is padded to this many rows
+constexpr int CH_TILE = 64;          // micro-experts (channels) per scoring work unit
+constexpr int UMMA_TOK = 256;        // tokens per tensor-core tile (the MMA's N)
+constexpr int MAX_ROUTED = 256;
+constexpr int MAX_TOPK = 16;
+constexpr int MAX_LEVELS = 8;
+
+// Host-known facts about one expert; copied to the device on every call.
+struct ExpertStatic {
+  const void* w_gate;
+  const void* w_up;
+  const void* w_down;
+  int32_t d_ff;
+  int32_t me_off;        // global micro-expert offset
+  int32_t shared_idx;    // -1 for routed experts, else index among the shared ones
+  int32_t norm_blk_begin;  // first CTA of the row-norm grid that belongs to this expert
+};
+
+// Facts only the device knows (they depend on the routing); written by k_plan.
+struct ExpertDyn {
+  int32_t row_base;      // first row of this expert's token list (in x_perm for routed, in x for shared)
+  int32_t rows;          // tokens the expert sees
+  int32_t n_chunks;      // ceil(rows / chunk_tokens)
+  int32_t unit_begin;    // exclusive prefix over experts of n_chunks * (d_ff / CH_TILE)
+  int64_t part_begin;    // exclusive prefix over experts of n_chunks * d_ff (offset into the partials)
+};
+
+struct PlanTotals {
+  int32_t total_units;
+  int32_t total_rows;    // rows of x_perm in use (padded)
+  int32_t status;        // device status word (0 = fine)
+  int32_t pad;
+};
+
+// Everything the kernels of one camera_score_layer call need.
+struct ScoreCtx {
+  int32_t d_model, n_routed, top_k, n_shared, n_experts, n_me;
+  int32_t dtype, down_layout;
+  uint32_t flags;
+  int32_t n_tokens, n_blocks;       // n_blocks = ceil(T / ROUTER_TOK)
+  int32_t chunk_tokens;             // tokens per scoring work unit (multiple of UMMA_TOK)
+  int32_t max_rows_perm;            // capacity of x_perm in rows
+  int64_t max_part;                 // capacity of the partial arrays in floats
+  float alpha;
+  const void* x;
+  const void* w_router;
+  const float* router_bias;
+  const void* w_shared_gate;
+  // workspace
+  PlanTotals* totals;
+  ExpertStatic* est;
+  ExpertDyn* edyn;
+  int32_t* me_prefix;    // [n_experts+1] global micro-expert offsets (host-known)
+  int32_t* unit_prefix;  // [n_experts+1] exclusive prefix of scoring work units (device-known)
+  int32_t* block_hist;   // [n_blocks, n_routed] counts, then (in place) exclusive offsets over blocks
+  int32_t* counts;       // [n_experts]
+  int32_t* local_rank;   // [T, top_k] rank of the pair among the same expert's pairs in its block
+  int32_t* topk_idx;     // [T, top_k]
+  float* topk_w;         // [T, top_k]
+  float* shared_w;       // [n_shared, T]
+  float* perm_w;         // [max_rows_perm]
+  void* x_perm;          // [max_rows_perm, d_model]
+  float* part_sum;       // [max_part]
+  float* part_max;       // [max_part]
+  float* phi2;           // [n_me]
+  float* phi_inf_sq;     // [n_me]
+  float* omega2;         // [n_me]
+  float* energy;         // [n_me]
+  void* tensor_maps;     // CUtensorMap[2 * n_experts + 2]
+};
+
+// ---- launches (each enqueues on `st`, returns the launch's cudaError_t) ------------------------
+cudaError_t launch_router(const ScoreCtx& c, cudaStream_t st);
+cudaError_t launch_routing_from_input(const ScoreCtx& c, const int32_t* idx_in, const float* w_in, cudaStream_t st);
+cudaError_t launch_plan(const ScoreCtx& c, cudaStream_t st);
+cudaError_t launch_permute(const ScoreCtx& c, cudaStream_t st);
+cudaError_t launch_rownorm(const ScoreCtx& c, int n_norm_blocks, cudaStream_t st);
+cudaError_t launch_score_simt(const ScoreCtx& c, cudaStream_t st);
+cudaError_t launch_score_umma(const ScoreCtx& c, cudaStream_t st);
+cudaError_t launch_combine(const ScoreCtx& c, cudaStream_t st);
+bool umma_shape_ok(const camera_layer_t* L);
+int encode_tensor_maps(const camera_layer_t* L, const ScoreCtx& c, void* host_maps /* 128 B each */);
+
+// ---- device helpers ------------------------------------------------------------------------------
+template <typename T> __device__ __forceinline__ float to_f32(T v);
+template <> __device__ __forceinline__ float to_f32<float>(float v) { return v; }
+template <> __device__ __forceinline__ float to_f32<__nv_bfloat16>(__nv_bfloat16 v) { return __bfloat162float(v); }
+
+// Unpacks a 16-byte vector of elements into floats: 4 for fp32, 8 for bf16.
+template <typename T> struct Vec16;
+template <> struct Vec16<float> {
+  static constexpr int N = 4;
+  __device__ __forceinline__ static void load(const float* p, float* out) {
+    float4 v = *reinterpret_cast<const float4*>(p);
+    out[0] = v.x; out[1] = v.y; out[2] = v.z; out[3] = v.w;
+  }
+};
+template <> struct Vec16<__nv_bfloat16> {
+  static constexpr int N = 8;
+  __device__ __forceinline__ static void load(const __nv_bfloat16* p, float* out) {
+    uint4 v = *reinterpret_cast<const uint4*>(p);
+    const uint32_t w[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+      out[2 * i] = __uint_as_float(w[i] << 16);
+      out[2 * i + 1] = __uint_as_float(w[i] & 0xffff0000u);
+    }
+  }
+};
+
+// Largest e with prefix[e] <= v, for a non-decreasing prefix[0..n] (prefix[0] <= v < prefix[n]).
+template <typename P>
+__device__ __forceinline__ int upper_segment(const P* prefix, int n, P v) {
+  int lo = 0, hi = n;
+  while (hi - lo > 1) {
+    int mid = (lo + hi) >> 1;
+    if (prefix[mid] <= v) lo = mid; else hi = mid;
+  }
+  return lo;
+}
+
+}  // namespace camera

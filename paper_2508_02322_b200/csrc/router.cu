@@ -1,0 +1,340 @@
+// Router (Algorithm 1 line 2: A <- Top&Norm(R X)), the stable counting sort of (token, expert)
+// pairs by expert, and the token permutation that lays every expert's tokens out contiguously.
+#include "common.cuh"
+
+namespace camera {
+
+namespace {
+
+constexpr int RT_THREADS = 256;
+constexpr int RT_KC = 32;            // k-chunk of the logit GEMM
+constexpr int RT_COLS = 64;          // logit columns per pass
+constexpr int RT_LD = ROUTER_TOK + 4;
+
+__device__ __forceinline__ float warp_max(float v) {
+#pragma unroll
+  for (int o = 16; o; o >>= 1) v = fmaxf(v, __shfl_xor_sync(0xffffffffu, v, o));
+  return v;
+}
+__device__ __forceinline__ float warp_sum(float v) {
+#pragma unroll
+  for (int o = 16; o; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+  return v;
+}
+
+// One CTA = ROUTER_TOK consecutive tokens.  Logits z = x . w (+bias) in fp32 FMA over all routed
+// experts and the sigmoid-gated shared experts; softmax over the routed ones; the top_k largest
+// logits are kept (equal logits: lower expert first); weights are the softmax probabilities,
+// divided by their sum under CAMERA_ROUTER_NORM_TOPK.  Also emits, for the counting sort, each
+// pair's rank among the same expert's pairs of this block and the block's per-expert histogram.
+template <typename T>
+__global__ void __launch_bounds__(RT_THREADS) k_router(ScoreCtx c, const int32_t* idx_in, const float* w_in) {
+  extern __shared__ float smem[];
+  const int n_gated = (c.flags & CAMERA_SHARED_GATE_SIGMOID) ? c.n_shared : 0;
+  const int nc = c.n_routed + n_gated;
+  const int nc_pad = ((nc + RT_COLS - 1) / RT_COLS) * RT_COLS;
+  const int ldl = nc_pad + 1;
+  float* Xs = smem;                              // [RT_KC][RT_LD]
+  float* Ws = Xs + RT_KC * RT_LD;                // [RT_KC][RT_LD]
+  float* logits = Ws + RT_KC * RT_LD;            // [ROUTER_TOK][ldl]
+  int* sel_e = reinterpret_cast<int*>(logits + ROUTER_TOK * ldl);  // [ROUTER_TOK * top_k]
+
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int tx = tid & 15, ty = tid >> 4;
+  const int blk = blockIdx.x;
+  const int tok0 = blk * ROUTER_TOK;
+  const int d = c.d_model;
+  const T* X = static_cast<const T*>(c.x);
+  constexpr int VN = Vec16<T>::N;
+  constexpr int VPR = RT_KC / VN;                // vectors per row of a k-chunk
+
+  for (int col0 = 0; col0 < nc_pad; col0 += RT_COLS) {
+    float acc[4][4];
+#pragma unroll
+    for (int i = 0; i < 4; ++i)
+#pragma unroll
+      for (int j = 0; j < 4; ++j) acc[i][j] = 0.f;
+
+    for (int k0 = 0; k0 < d; k0 += RT_KC) {
+      __syncthreads();
+      for (int v = tid; v < ROUTER_TOK * VPR; v += RT_THREADS) {
+        const int row = v / VPR, kv = (v % VPR) * VN;
+        float f[VN];
+#pragma unroll
+        for (int i = 0; i < VN; ++i) f[i] = 0.f;
+        const int t = tok0 + row;
+        if (t < c.n_tokens && k0 + kv < d) Vec16<T>::load(X + (size_t)t * d + k0 + kv, f);
+#pragma unroll
+        for (int i = 0; i < VN; ++i) Xs[(kv + i) * RT_LD + row] = f[i];
+      }
+      for (int v = tid; v < RT_COLS * VPR; v += RT_THREADS) {
+        const int row = v / VPR, kv = (v % VPR) * VN;
+        float f[VN];
+#pragma unroll
+        for (int i = 0; i < VN; ++i) f[i] = 0.f;
+        const int col = col0 + row;
+        if (col < nc && k0 + kv < d) {
+          const T* wrow = col < c.n_routed
+              ? static_cast<const T*>(c.w_router) + (size_t)col * d
+              : static_cast<const T*>(c.w_shared_gate) + (size_t)(col - c.n_routed) * d;
+          Vec16<T>::load(wrow + k0 + kv, f);
+        }
+#pragma unroll
+        for (int i = 0; i < VN; ++i) Ws[(kv + i) * RT_LD + row] = f[i];
+      }
+      __syncthreads();
+#pragma unroll 8
+      for (int k = 0; k < RT_KC; ++k) {
+        const float4 a = *reinterpret_cast<const float4*>(Xs + k * RT_LD + ty * 4);
+        const float4 b = *reinterpret_cast<const float4*>(Ws + k * RT_LD + tx * 4);
+        const float av[4] = {a.x, a.y, a.z, a.w}, bv[4] = {b.x, b.y, b.z, b.w};
+#pragma unroll
+        for (int i = 0; i < 4; ++i)
+#pragma unroll
+          for (int j = 0; j < 4; ++j) acc[i][j] = fmaf(av[i], bv[j], acc[i][j]);
+      }
+    }
+#pragma unroll
+    for (int i = 0; i < 4; ++i)
+#pragma unroll
+      for (int j = 0; j < 4; ++j) logits[(ty * 4 + i) * ldl + col0 + tx * 4 + j] = acc[i][j];
+  }
+  __syncthreads();
+
+  // coefficients of the shared experts: 1, or sigmoid of their gate logit
+  for (int i = tid; i < ROUTER_TOK * c.n_shared; i += RT_THREADS) {
+    const int s = i / ROUTER_TOK, tl = i % ROUTER_TOK, t = tok0 + tl;
+    if (t < c.n_tokens) {
+      float a = 1.f;
+      if (n_gated) a = 1.f / (1.f + expf(-logits[tl * ldl + c.n_routed + s]));
+      c.shared_w[(size_t)s * c.n_tokens + t] = a;
+    }
+  }
+
+  const int k = c.top_k;
+  if (c.n_routed > 0) {
+    for (int tl = warp; tl < ROUTER_TOK; tl += RT_THREADS / 32) {
+      const int t = tok0 + tl;
+      if (t >= c.n_tokens) {
+        if (lane < k) sel_e[tl * k + lane] = -1;
+        continue;
+      }
+      int my_e = 0;
+      float my_p = 0.f;
+      if (idx_in != nullptr) {
+        if (lane < k) {
+          my_e = idx_in[(size_t)t * k + lane];
+          my_p = w_in[(size_t)t * k + lane];
+          if (my_e < 0 || my_e >= c.n_routed) {
+            atomicExch(&c.totals->status, (int)CAMERA_ERR_INVALID_ARG);
+            my_e = 0; my_p = 0.f;
+          }
+        }
+      } else {
+        float v[MAX_ROUTED / 32];
+#pragma unroll
+        for (int i = 0; i < MAX_ROUTED / 32; ++i) {
+          const int col = lane + 32 * i;
+          v[i] = -INFINITY;
+          if (col < c.n_routed) v[i] = logits[tl * ldl + col] + (c.router_bias ? c.router_bias[col] : 0.f);
+        }
+        float zmax = -INFINITY;
+#pragma unroll
+        for (int i = 0; i < MAX_ROUTED / 32; ++i) zmax = fmaxf(zmax, v[i]);
+        zmax = warp_max(zmax);
+        float den = 0.f;
+#pragma unroll
+        for (int i = 0; i < MAX_ROUTED / 32; ++i) den += (lane + 32 * i < c.n_routed) ? expf(v[i] - zmax) : 0.f;
+        den = warp_sum(den);
+        float chosen = 0.f;
+        for (int s = 0; s < k; ++s) {
+          float best = -INFINITY;
+          int bi = 0x7fffffff;
+#pragma unroll
+          for (int i = 0; i < MAX_ROUTED / 32; ++i)
+            if (v[i] > best) { best = v[i]; bi = lane + 32 * i; }
+#pragma unroll
+          for (int o = 16; o; o >>= 1) {
+            const float ov = __shfl_xor_sync(0xffffffffu, best, o);
+            const int oi = __shfl_xor_sync(0xffffffffu, bi, o);
+            if (ov > best || (ov == best && oi < bi)) { best = ov; bi = oi; }
+          }
+          const float p = expf(best - zmax) / den;
+#pragma unroll
+          for (int i = 0; i < MAX_ROUTED / 32; ++i)
+            if (lane + 32 * i == bi) v[i] = -INFINITY;
+          if (lane == s) { my_e = bi; my_p = p; }
+          chosen += p;
+        }
+        if (c.flags & CAMERA_ROUTER_NORM_TOPK) my_p /= chosen;
+      }
+      if (lane < k) {
+        c.topk_idx[(size_t)t * k + lane] = my_e;
+        c.topk_w[(size_t)t * k + lane] = my_p;
+        sel_e[tl * k + lane] = my_e;
+      }
+    }
+    __syncthreads();
+    // rank of each pair among the pairs of the same expert in this block, in (token, slot) order
+    const int npairs = ROUTER_TOK * k;
+    for (int e = warp; e < c.n_routed; e += RT_THREADS / 32) {
+      int run = 0;
+      for (int base = 0; base < npairs; base += 32) {
+        const int p = base + lane;
+        const bool m = (p < npairs) && (sel_e[p] == e);
+        const unsigned b = __ballot_sync(0xffffffffu, m);
+        if (m) c.local_rank[(size_t)tok0 * k + p] = run + __popc(b & ((1u << lane) - 1u));
+        run += __popc(b);
+      }
+      if (lane == 0) c.block_hist[(size_t)blk * c.n_routed + e] = run;
+    }
+  }
+}
+
+// One CTA per routed expert: exclusive scan of its per-block counts over the blocks (in place).
+__global__ void __launch_bounds__(256) k_block_scan(ScoreCtx c) {
+  __shared__ int wsum[8];
+  __shared__ int chunk_total;
+  const int e = blockIdx.x, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  int run = 0;
+  for (int base = 0; base < c.n_blocks; base += 256) {
+    const int b = base + tid;
+    const int v = b < c.n_blocks ? c.block_hist[(size_t)b * c.n_routed + e] : 0;
+    int incl = v;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+      const int n = __shfl_up_sync(0xffffffffu, incl, o);
+      if (lane >= o) incl += n;
+    }
+    if (lane == 31) wsum[warp] = incl;
+    __syncthreads();
+    int woff = 0;
+    for (int w = 0; w < warp; ++w) woff += wsum[w];
+    if (tid == 255) chunk_total = woff + incl;
+    if (b < c.n_blocks) c.block_hist[(size_t)b * c.n_routed + e] = run + woff + incl - v;
+    __syncthreads();
+    run += chunk_total;
+  }
+  if (tid == 0) c.counts[e] = run;
+}
+
+// Single thread: lays the experts' token lists out back to back (each padded to ROW_ALIGN rows)
+// and numbers the scoring work units and partial slots.
+__global__ void k_plan(ScoreCtx c) {
+  if (threadIdx.x != 0 || blockIdx.x != 0) return;
+  int row = 0, units = 0;
+  long long part = 0;
+  for (int e = 0; e < c.n_experts; ++e) {
+    ExpertDyn dy;
+    if (e < c.n_routed) {
+      dy.rows = c.counts[e];
+      dy.row_base = row;
+      row += (dy.rows + ROW_ALIGN - 1) / ROW_ALIGN * ROW_ALIGN;
+    } else {
+      dy.rows = c.n_tokens;
+      dy.row_base = 0;
+      c.counts[e] = c.n_tokens;
+    }
+    const int f = c.est[e].d_ff;
+    dy.n_chunks = (dy.rows + c.chunk_tokens - 1) / c.chunk_tokens;
+    dy.unit_begin = units;
+    dy.part_begin = part;
+    c.edyn[e] = dy;
+    c.unit_prefix[e] = units;
+    units += dy.n_chunks * ((f + CH_TILE - 1) / CH_TILE);
+    part += (long long)dy.n_chunks * f;
+  }
+  if (row > c.max_rows_perm || part > c.max_part) {
+    atomicExch(&c.totals->status, (int)CAMERA_ERR_WORKSPACE);
+    units = 0;
+    for (int e = 0; e <= c.n_experts; ++e) c.unit_prefix[e] = 0;
+    for (int e = 0; e < c.n_experts; ++e) { c.edyn[e].n_chunks = 0; c.edyn[e].rows = 0; }
+  }
+  c.unit_prefix[c.n_experts] = units;
+  c.totals->total_units = units;
+  c.totals->total_rows = row;
+}
+
+// One warp per token: copies the token's hidden state to its row in every chosen expert's list.
+__global__ void __launch_bounds__(256) k_permute(ScoreCtx c, int row_bytes) {
+  const int lane = threadIdx.x & 31;
+  const int t = blockIdx.x * 8 + (threadIdx.x >> 5);
+  if (t >= c.n_tokens) return;
+  const int k = c.top_k;
+  int pos_l = 0;
+  if (lane < k) {
+    const int e = c.topk_idx[(size_t)t * k + lane];
+    pos_l = c.edyn[e].row_base + c.block_hist[(size_t)(t / ROUTER_TOK) * c.n_routed + e] +
+            c.local_rank[(size_t)t * k + lane];
+    c.perm_w[pos_l] = c.topk_w[(size_t)t * k + lane];
+  }
+  int pos[MAX_TOPK];
+#pragma unroll
+  for (int s = 0; s < MAX_TOPK; ++s) pos[s] = __shfl_sync(0xffffffffu, pos_l, s);
+  const uint4* src = reinterpret_cast<const uint4*>(static_cast<const char*>(c.x) + (size_t)t * row_bytes);
+  const int nvec = row_bytes / 16;
+  for (int v = lane; v < nvec; v += 32) {
+    const uint4 val = __ldg(src + v);
+#pragma unroll
+    for (int s = 0; s < MAX_TOPK; ++s)
+      if (s < k)
+        reinterpret_cast<uint4*>(static_cast<char*>(c.x_perm) + (size_t)pos[s] * row_bytes)[v] = val;
+  }
+}
+
+// One CTA per routed expert: zero rows and zero weights for the padding behind its token list.
+__global__ void __launch_bounds__(128) k_pad_rows(ScoreCtx c, int row_bytes) {
+  const ExpertDyn dy = c.edyn[blockIdx.x];
+  const int end = (dy.rows + ROW_ALIGN - 1) / ROW_ALIGN * ROW_ALIGN;
+  const int nvec = row_bytes / 16;
+  for (int r = dy.rows; r < end; ++r) {
+    const size_t row = (size_t)dy.row_base + r;
+    uint4* dst = reinterpret_cast<uint4*>(static_cast<char*>(c.x_perm) + row * row_bytes);
+    for (int v = threadIdx.x; v < nvec; v += blockDim.x) dst[v] = make_uint4(0, 0, 0, 0);
+    if (threadIdx.x == 0) c.perm_w[row] = 0.f;
+  }
+}
+
+size_t router_smem_bytes(const ScoreCtx& c) {
+  const int n_gated = (c.flags & CAMERA_SHARED_GATE_SIGMOID) ? c.n_shared : 0;
+  const int nc = c.n_routed + n_gated;
+  const int nc_pad = ((nc + RT_COLS - 1) / RT_COLS) * RT_COLS;
+  return sizeof(float) * (2 * RT_KC * RT_LD + ROUTER_TOK * (nc_pad + 1)) + sizeof(int) * ROUTER_TOK * MAX_TOPK;
+}
+
+}  // namespace
+
+cudaError_t launch_routing_from_input(const ScoreCtx& c, const int32_t* idx_in, const float* w_in, cudaStream_t st) {
+  if (c.n_blocks == 0) return cudaSuccess;
+  const size_t smem = router_smem_bytes(c);
+  if (c.dtype == CAMERA_BF16) {
+    cudaError_t e = cudaFuncSetAttribute(k_router<__nv_bfloat16>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    if (e != cudaSuccess) return e;
+    k_router<__nv_bfloat16><<<c.n_blocks, RT_THREADS, smem, st>>>(c, idx_in, w_in);
+  } else {
+    cudaError_t e = cudaFuncSetAttribute(k_router<float>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    if (e != cudaSuccess) return e;
+    k_router<float><<<c.n_blocks, RT_THREADS, smem, st>>>(c, idx_in, w_in);
+  }
+  return cudaGetLastError();
+}
+
+cudaError_t launch_router(const ScoreCtx& c, cudaStream_t st) {
+  return launch_routing_from_input(c, nullptr, nullptr, st);
+}
+
+cudaError_t launch_plan(const ScoreCtx& c, cudaStream_t st) {
+  if (c.n_routed > 0 && c.n_blocks > 0) k_block_scan<<<c.n_routed, 256, 0, st>>>(c);
+  k_plan<<<1, 32, 0, st>>>(c);
+  return cudaGetLastError();
+}
+
+cudaError_t launch_permute(const ScoreCtx& c, cudaStream_t st) {
+  if (c.n_routed == 0 || c.n_tokens == 0) return cudaSuccess;
+  const int row_bytes = c.d_model * (c.dtype == CAMERA_BF16 ? 2 : 4);
+  k_permute<<<(c.n_tokens + 7) / 8, 256, 0, st>>>(c, row_bytes);
+  k_pad_rows<<<c.n_routed, 128, 0, st>>>(c, row_bytes);
+  return cudaGetLastError();
+}
+
+}  // namespace camera

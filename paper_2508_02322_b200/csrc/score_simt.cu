@@ -1,0 +1,162 @@
+// fp32-FMA scoring kernel (Algorithm 1 lines 6-8 with Lambda kept in registers) and the final
+// combine (line 10, Eq. 11).  This kernel serves fp32 layers and shapes the tensor-core kernel
+// does not take; it uses the same work units and partial layout as the tensor-core kernel.
+#include "common.cuh"
+
+namespace camera {
+
+namespace {
+
+constexpr int SS_THREADS = 256;
+constexpr int SS_TOK = 64;
+constexpr int SS_KC = 16;
+constexpr int SS_LD = 68;
+
+// Work unit = (expert, tile of CH_TILE channels, chunk of chunk_tokens tokens).  For every
+// token tile the CTA forms g = W_gate x and u = W_up x for 64 tokens x 64 channels in fp32,
+// then lambda = a_t * SiLU(g) * u and folds lambda^2 / |lambda| into per-channel running sum / max.
+// One partial (sum, max) per channel and chunk goes to the workspace; chunks are added later in
+// a fixed order, so results do not depend on scheduling.
+template <typename T>
+__global__ void __launch_bounds__(SS_THREADS) k_score_simt(ScoreCtx c) {
+  __shared__ __align__(16) float Xs[SS_KC][SS_LD];
+  __shared__ __align__(16) float Gs[SS_KC][SS_LD];
+  __shared__ __align__(16) float Us[SS_KC][SS_LD];
+  __shared__ float red_s[16][CH_TILE];
+  __shared__ float red_m[16][CH_TILE];
+  constexpr int VN = Vec16<T>::N;
+  constexpr int VPR = SS_KC / VN;
+  const int tid = threadIdx.x, tx = tid & 15, ty = tid >> 4;
+  const int d = c.d_model;
+  const int total_units = c.totals->total_units;
+
+  for (int unit = blockIdx.x; unit < total_units; unit += gridDim.x) {
+    const int e = upper_segment(c.unit_prefix, c.n_experts, unit);
+    const ExpertStatic es = c.est[e];
+    const ExpertDyn dy = c.edyn[e];
+    const int f = es.d_ff;
+    const int n_ct = (f + CH_TILE - 1) / CH_TILE;
+    const int rem = unit - c.unit_prefix[e];
+    const int chunk = rem / n_ct, ct = rem % n_ct;
+    const int ch0 = ct * CH_TILE;
+    const int row_begin = chunk * c.chunk_tokens;
+    const int rows = min(c.chunk_tokens, dy.rows - row_begin);
+    const T* Xsrc = (es.shared_idx < 0 ? static_cast<const T*>(c.x_perm) : static_cast<const T*>(c.x)) +
+                    (size_t)(dy.row_base + row_begin) * d;
+    const float* wsrc = (es.shared_idx < 0 ? c.perm_w + dy.row_base
+                                           : c.shared_w + (size_t)es.shared_idx * c.n_tokens) + row_begin;
+    const T* Wg = static_cast<const T*>(es.w_gate);
+    const T* Wu = static_cast<const T*>(es.w_up);
+
+    float s[4] = {0.f, 0.f, 0.f, 0.f}, m[4] = {0.f, 0.f, 0.f, 0.f};
+    for (int r0 = 0; r0 < rows; r0 += SS_TOK) {
+      float ag[4][4], au[4][4];
+#pragma unroll
+      for (int i = 0; i < 4; ++i)
+#pragma unroll
+        for (int j = 0; j < 4; ++j) { ag[i][j] = 0.f; au[i][j] = 0.f; }
+      for (int k0 = 0; k0 < d; k0 += SS_KC) {
+        __syncthreads();
+        for (int v = tid; v < 3 * SS_TOK * VPR; v += SS_THREADS) {
+          const int which = v / (SS_TOK * VPR), w = v % (SS_TOK * VPR);
+          const int row = w / VPR, kv = (w % VPR) * VN;
+          float fv[VN];
+#pragma unroll
+          for (int i = 0; i < VN; ++i) fv[i] = 0.f;
+          if (k0 + kv < d) {
+            if (which == 0) {
+              if (r0 + row < rows) Vec16<T>::load(Xsrc + (size_t)(r0 + row) * d + k0 + kv, fv);
+            } else if (ch0 + row < f) {
+              Vec16<T>::load((which == 1 ? Wg : Wu) + (size_t)(ch0 + row) * d + k0 + kv, fv);
+            }
+          }
+          float* dst = which == 0 ? &Xs[0][0] : (which == 1 ? &Gs[0][0] : &Us[0][0]);
+#pragma unroll
+          for (int i = 0; i < VN; ++i) dst[(kv + i) * SS_LD + row] = fv[i];
+        }
+        __syncthreads();
+#pragma unroll
+        for (int k = 0; k < SS_KC; ++k) {
+          const float4 a = *reinterpret_cast<const float4*>(&Xs[k][ty * 4]);
+          const float4 g = *reinterpret_cast<const float4*>(&Gs[k][tx * 4]);
+          const float4 u = *reinterpret_cast<const float4*>(&Us[k][tx * 4]);
+          const float av[4] = {a.x, a.y, a.z, a.w}, gv[4] = {g.x, g.y, g.z, g.w}, uv[4] = {u.x, u.y, u.z, u.w};
+#pragma unroll
+          for (int i = 0; i < 4; ++i)
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+              ag[i][j] = fmaf(av[i], gv[j], ag[i][j]);
+              au[i][j] = fmaf(av[i], uv[j], au[i][j]);
+            }
+        }
+      }
+#pragma unroll
+      for (int i = 0; i < 4; ++i) {
+        const int row = r0 + ty * 4 + i;
+        const float a_t = row < rows ? wsrc[row] : 0.f;
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+          const float g = ag[i][j];
+          const float lam = a_t * (g / (1.f + expf(-g))) * au[i][j];
+          s[j] = fmaf(lam, lam, s[j]);
+          m[j] = fmaxf(m[j], fabsf(lam));
+        }
+      }
+    }
+    __syncthreads();
+#pragma unroll
+    for (int j = 0; j < 4; ++j) { red_s[ty][tx * 4 + j] = s[j]; red_m[ty][tx * 4 + j] = m[j]; }
+    __syncthreads();
+    if (tid < CH_TILE && ch0 + tid < f) {
+      float ts = 0.f, tm = 0.f;
+#pragma unroll
+      for (int y = 0; y < 16; ++y) { ts += red_s[y][tid]; tm = fmaxf(tm, red_m[y][tid]); }
+      const size_t slot = (size_t)dy.part_begin + (size_t)chunk * f + ch0 + tid;
+      c.part_sum[slot] = ts;
+      c.part_max[slot] = tm;
+    }
+  }
+}
+
+// Adds the chunk partials of every micro-expert in chunk order (fp64), squares the max and
+// blends: E_i = [(1-alpha) phi2_i + alpha phi_inf_i] * omega2_i   (Eq. 11).
+__global__ void __launch_bounds__(256) k_combine(ScoreCtx c) {
+  const int i = blockIdx.x * blockDim.x + threadIdx.x;
+  if (i >= c.n_me) return;
+  const int e = upper_segment(c.me_prefix, c.n_experts, i);
+  const int ch = i - c.me_prefix[e];
+  const ExpertDyn dy = c.edyn[e];
+  const int f = c.est[e].d_ff;
+  double s = 0.0;
+  float m = 0.f;
+  for (int j = 0; j < dy.n_chunks; ++j) {
+    const size_t slot = (size_t)dy.part_begin + (size_t)j * f + ch;
+    s += (double)c.part_sum[slot];
+    m = fmaxf(m, c.part_max[slot]);
+  }
+  const double m2 = (double)m * (double)m;
+  const double a = (double)c.alpha;
+  c.phi2[i] = (float)s;
+  c.phi_inf_sq[i] = (float)m2;
+  c.energy[i] = (float)(((1.0 - a) * s + a * m2) * (double)c.omega2[i]);
+}
+
+}  // namespace
+
+cudaError_t launch_score_simt(const ScoreCtx& c, cudaStream_t st) {
+  int dev = 0, sms = 148;
+  cudaGetDevice(&dev);
+  cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+  const int grid = sms * 4;
+  if (c.dtype == CAMERA_BF16) k_score_simt<__nv_bfloat16><<<grid, SS_THREADS, 0, st>>>(c);
+  else k_score_simt<float><<<grid, SS_THREADS, 0, st>>>(c);
+  return cudaGetLastError();
+}
+
+cudaError_t launch_combine(const ScoreCtx& c, cudaStream_t st) {
+  if (c.n_me == 0) return cudaSuccess;
+  k_combine<<<(c.n_me + 255) / 256, 256, 0, st>>>(c);
+  return cudaGetLastError();
+}
+
+}  // namespace camera

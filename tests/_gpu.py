@@ -1,0 +1,111 @@
+"""Shared pieces of the GPU parity tests: run the CUDA path through the C ABI binding, run the
+float64 oracle on the same stored values, and compare under the stated tolerances."""
+import numpy as np
+import torch
+
+import oracle as O
+from _util import to_oracle_layer, f64
+
+REL_TOL = 1e-3          # scores: fp32 accumulation of bf16/fp32 products against float64
+TIE_TOL = 1e-5          # routing: relative gap of the k-th and (k+1)-th probability below which either is right
+
+
+def assert_close(name, got, ref, rel=REL_TOL):
+    got = np.asarray(got, dtype=np.float64)
+    ref = np.asarray(ref, dtype=np.float64)
+    scale = np.maximum(np.abs(ref), 1e-30)
+    err = np.abs(got - ref) / scale
+    # values that are exactly zero in the oracle must be exactly zero on the GPU
+    zero = ref == 0
+    assert (got[zero] == 0).all(), f"{name}: non-zero where the oracle is exactly zero"
+    bad = err[~zero] > rel
+    assert not bad.any(), f"{name}: {bad.sum()} of {bad.size} beyond {rel}, worst {err[~zero].max():.3e}"
+
+
+def check_routing(olayer, Xd, topk_idx, topk_w):
+    """GPU routing against the oracle's.  Returns the number of near-tie tokens whose expert set differs."""
+    if olayer.n_routed == 0:
+        return 0
+    p = O.router_probs(olayer, Xd)
+    idx_o, w_o = O.top_and_norm(p, olayer.top_k, olayer.norm_topk)
+    gi = topk_idx.cpu().numpy().astype(np.int64)
+    gw = topk_w.cpu().numpy().astype(np.float64)
+    same = (np.sort(gi, axis=1) == np.sort(idx_o, axis=1)).all(axis=1)
+    k = olayer.top_k
+    if not same.all():
+        ps = -np.sort(-p, axis=1)
+        if k < p.shape[1]:
+            gap = (ps[:, k - 1] - ps[:, k]) / ps[:, k - 1]
+            assert (gap[~same] < TIE_TOL).all(), "expert sets differ on tokens that are not near-ties"
+        else:
+            raise AssertionError("expert sets differ with k == n_routed")
+    # weights of the tokens that agree, matched by expert
+    order_g, order_o = np.argsort(gi, axis=1), np.argsort(idx_o, axis=1)
+    wg = np.take_along_axis(gw, order_g, axis=1)[same]
+    wo = np.take_along_axis(w_o, order_o, axis=1)[same]
+    assert np.abs(wg - wo).max() <= 2e-5 * max(1.0, np.abs(wo).max()), "router weights differ"
+    # order of the exported slots: decreasing probability
+    assert (np.diff(gw, axis=1) <= 1e-6).all()
+    return int((~same).sum())
+
+
+def run_and_compare(P, L, X, alpha=0.95, channels=None, force_simt=False, check_dense=False):
+    """Scores one layer on the GPU (own routing, then the oracle's routing injected) and checks
+    every component against the oracle.  `channels` restricts the oracle to sampled micro-experts."""
+    layer = P.Layer.from_workload(L)
+    olayer = to_oracle_layer(L)
+    Xd = f64(X)
+    ws = P.alloc_workspace(P.camera_score_workspace_bytes(layer, X.shape[0]), X.device)
+    out = P.camera_score_layer(layer, X, alpha, details=True, workspace=ws, force_simt=force_simt)
+    assert P.camera_read_status(ws) == 0
+    flips = check_routing(olayer, Xd, out["topk_idx"], out["topk_w"])
+
+    # (1) scoring under the GPU's own routing: the oracle is given that routing
+    routing = None
+    if olayer.n_routed:
+        routing = (out["topk_idx"].cpu().numpy().astype(np.int64), out["topk_w"].cpu().numpy().astype(np.float64))
+    shared_w = out["shared_w"].cpu().numpy().astype(np.float64).T
+    if olayer.n_shared:
+        assert_close("shared_w", shared_w, O.shared_coeff(olayer, Xd), rel=2e-5)
+    phi2, phi_inf, omega2 = O.camera_components(olayer, Xd, channels=channels, routing=routing)
+    sel = ~np.isnan(phi2)
+    assert_close("omega2", out["omega2"].cpu().numpy(), omega2)
+    assert_close("phi2", out["phi2"].cpu().numpy()[sel], phi2[sel])
+    assert_close("phi_inf_sq", out["phi_inf_sq"].cpu().numpy()[sel], phi_inf[sel])
+    E = O.energy(phi2, phi_inf, omega2, float(np.float32(alpha)))
+    assert_close("energy", out["energy"].cpu().numpy()[sel], E[sel])
+    counts = out["expert_token_counts"].cpu().numpy()
+    if olayer.n_routed:
+        assert np.array_equal(counts[:olayer.n_routed], np.bincount(routing[0].reshape(-1), minlength=olayer.n_routed))
+    assert (counts[olayer.n_routed:] == X.shape[0]).all()
+
+    # (2) the oracle's routing injected into the GPU path: no token is excluded
+    if olayer.n_routed:
+        idx_o, w_o = O.top_and_norm(O.router_probs(olayer, Xd), olayer.top_k, olayer.norm_topk)
+        w32 = w_o.astype(np.float32)
+        out2 = P.camera_score_layer(layer, X, alpha, details=True, workspace=ws, force_simt=force_simt,
+                                    routing_in=(torch.from_numpy(idx_o.astype(np.int32)), torch.from_numpy(w32)))
+        assert P.camera_read_status(ws) == 0
+        p2, pi, w2 = O.camera_components(olayer, Xd, channels=channels, routing=(idx_o, w32.astype(np.float64)))
+        assert_close("phi2 (oracle routing)", out2["phi2"].cpu().numpy()[sel], p2[sel])
+        assert_close("phi_inf_sq (oracle routing)", out2["phi_inf_sq"].cpu().numpy()[sel], pi[sel])
+        assert_close("energy (oracle routing)", out2["energy"].cpu().numpy()[sel],
+                     O.energy(p2, pi, w2, float(np.float32(alpha)))[sel])
+    if check_dense:
+        d2, dinf, dw = O.camera_components_dense(olayer, Xd)
+        if flips == 0:
+            assert_close("phi2 vs literal Algorithm 1", out["phi2"].cpu().numpy(), d2)
+            assert_close("phi_inf_sq vs literal Algorithm 1", out["phi_inf_sq"].cpu().numpy(), dinf)
+    return out, flips
+
+
+def sample_channels(d_ff, per_expert, seed=0):
+    """A seeded sample of micro-experts per expert that always holds the first and last channel
+    and a channel on either side of a 64-channel tile edge."""
+    r = np.random.default_rng(seed)
+    ch = {}
+    for e, f in enumerate(d_ff):
+        must = {0, f - 1, min(63, f - 1), min(64, f - 1)}
+        extra = set(r.choice(f, size=min(per_expert, f), replace=False).tolist())
+        ch[e] = sorted(must | extra)
+    return ch

@@ -1,0 +1,78 @@
+"""Host-only checks of the C ABI: the library loads, exports what include/camera.h declares, and
+rejects bad arguments before anything touches a GPU."""
+import ctypes as C
+import os
+import re
+
+import pytest
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+@pytest.fixture(scope="module")
+def P():
+    import paper_2508_02322_b200 as pkg
+    return pkg
+
+
+def declared_functions():
+    text = open(os.path.join(ROOT, "include", "camera.h")).read()
+    text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
+    return sorted(set(re.findall(r"\b(camera_[a-z_]+)\s*\(", text)))
+
+
+def test_library_exports_every_declared_symbol(P):
+    names = declared_functions()
+    assert {"camera_score_layer", "camera_select_prune", "camera_alloc_bits"} <= set(names)
+    for n in names:
+        assert hasattr(P.lib, n), n
+    assert P.lib.camera_version() >= 100
+    assert P.lib.camera_strerror(0) == b"ok" and b"workspace" in P.lib.camera_strerror(-3)
+
+
+def _layer_struct(P, d_model=64, n_routed=4, top_k=2, d_ff=(64, 64, 64, 64), n_shared=0, dtype=1, flags=1):
+    from paper_2508_02322_b200.binding import camera_layer_t
+    n = len(d_ff)
+    dff = (C.c_int32 * n)(*d_ff)
+    ptrs = (C.c_void_p * n)(*[4096] * n)
+    s = camera_layer_t(d_model, n_routed, top_k, n_shared, dff, dtype, flags, 0, 4096, None, None, ptrs, ptrs, ptrs)
+    s._keep = (dff, ptrs)
+    return s
+
+
+def test_workspace_query_validates_shapes(P):
+    ok = _layer_struct(P)
+    assert P.lib.camera_score_workspace_bytes(C.byref(ok), 1000) > 0
+    assert P.lib.camera_score_workspace_bytes(C.byref(ok), 0) > 0
+    assert P.lib.camera_score_workspace_bytes(C.byref(ok), -1) == 0
+    assert P.lib.camera_score_workspace_bytes(C.byref(_layer_struct(P, top_k=5)), 10) == 0      # k > n_routed
+    assert P.lib.camera_score_workspace_bytes(C.byref(_layer_struct(P, d_model=60)), 10) == 0   # d_model % 8
+    assert P.lib.camera_score_workspace_bytes(C.byref(_layer_struct(P, d_ff=(64, 64, 64, 60))), 10) == 0
+    assert P.lib.camera_score_workspace_bytes(C.byref(_layer_struct(P, dtype=7)), 10) == 0
+    assert P.lib.camera_score_workspace_bytes(None, 10) == 0
+    # more tokens never need less scratch
+    a = P.lib.camera_score_workspace_bytes(C.byref(ok), 1000)
+    b = P.lib.camera_score_workspace_bytes(C.byref(ok), 100000)
+    assert b > a
+    assert P.lib.camera_select_workspace_bytes(1000, 1, 2) > 0
+    assert P.lib.camera_select_workspace_bytes(1000, 1, 9) == 0
+    assert P.lib.camera_analyze_workspace_bytes(C.byref(ok), 1000, 3) > P.lib.camera_score_workspace_bytes(C.byref(ok), 1000)
+
+
+def test_argument_errors_return_before_any_launch(P):
+    ok = _layer_struct(P)
+    # alpha outside [0,1], null energy: rejected on the host (pointers here are fake and never dereferenced)
+    assert P.lib.camera_score_layer(C.byref(ok), 4096, 10, C.c_float(1.5), 4096, None, 4096, 1 << 30, None) == -1
+    assert P.lib.camera_score_layer(C.byref(ok), 4096, 10, C.c_float(0.5), None, None, 4096, 1 << 30, None) == -1
+    assert P.lib.camera_score_layer(C.byref(ok), 4096, 10, C.c_float(0.5), 4096, None, None, 0, None) == -3
+    seg = (C.c_int64 * 2)(0, 10)
+    bad = (C.c_int64 * 2)(1, 10)
+    assert P.lib.camera_select_prune(4096, seg, 1, C.c_double(1.0), None, 0, 4096, None, None, 4096, 1 << 20, None) == -1
+    assert P.lib.camera_select_prune(4096, bad, 1, C.c_double(0.5), None, 0, 4096, None, None, 4096, 1 << 20, None) == -1
+    assert P.lib.camera_select_prune(4096, seg, 1, C.c_double(0.5), None, 0, 4096, None, None, 4096, 16, None) == -3
+    r = (C.c_double * 3)(0.2, 0.5, 0.2)
+    b = (C.c_int32 * 3)(3, 2, 1)
+    assert P.lib.camera_alloc_bits(4096, seg, 1, r, b, 3, None, 0, 4096, None, 4096, 1 << 20, None) == -1   # ratios sum
+    r = (C.c_double * 3)(0.2, 0.6, 0.2)
+    b = (C.c_int32 * 3)(3, 2, 300)
+    assert P.lib.camera_alloc_bits(4096, seg, 1, r, b, 3, None, 0, 4096, None, 4096, 1 << 20, None) == -1   # bit-width

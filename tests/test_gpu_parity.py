@@ -1,0 +1,255 @@
+"""GPU parity: the CUDA path, called through the C ABI binding, against the float64 oracle on the
+same seeded inputs.  Scores within 1e-3 relative (fp32 accumulation), routing / masks / bit-widths
+bit-exact (routing: except near-ties, which are reported)."""
+import numpy as np
+import pytest
+import torch
+
+import oracle as O
+from _gpu import REL_TOL, assert_close, run_and_compare, sample_channels
+from _util import f64, to_oracle_layer
+
+pytestmark = pytest.mark.gpu
+
+DEV = "cuda:0"
+
+
+@pytest.fixture(scope="module")
+def P():
+    import paper_2508_02322_b200 as pkg
+    return pkg
+
+
+def W():
+    from paper_2508_02322_b200 import workloads
+    return workloads
+
+
+def small_cfg(**kw):
+    base = dict(name="small", d_model=256, n_routed=6, top_k=2, d_ff_routed=128, d_ff_shared=(192,),
+                shared_gate_sigmoid=True, n_tokens=700, dtype="bf16", x_dist="normal_rms1", router_bias_std=0.3)
+    base.update(kw)
+    return W().LayerConfig(**base)
+
+
+# ------------------------------------------------------------------ config 1: tiny fp32, everything
+def test_tiny_fp32_full(P):
+    cfg = W().CONFIGS["tiny_fp32"]
+    L = W().make_layer(cfg, seed=0, device=DEV)
+    X = W().make_tokens(cfg, seed=0, device=DEV)
+    out, flips = run_and_compare(P, L, X, alpha=0.95, check_dense=True)
+    E = out["energy"]
+    E_np = E.cpu().numpy()
+    keep = P.camera_select_prune(E, 0.40)
+    assert np.array_equal(keep.cpu().numpy(), O.select_prune(E_np, 0.40))
+    assert int((keep == 0).sum()) == int(0.4 * 4096)
+    bits = P.camera_alloc_bits(E, [0.2, 0.6, 0.2], [4, 3, 2])
+    assert np.array_equal(bits.cpu().numpy(), O.alloc_bits(E_np, [0.2, 0.6, 0.2], [4, 3, 2])[0])
+    # mask from GPU scores against mask from oracle scores: may differ only inside the tolerance band
+    olayer = to_oracle_layer(L)
+    Eo = O.energy(*O.camera_components(olayer, f64(X)), float(np.float32(0.95)))
+    keep_o = O.select_prune(Eo, 0.40)
+    diff = np.nonzero(keep.cpu().numpy() != keep_o)[0]
+    tau = np.sort(Eo)[int(0.4 * 4096)]
+    assert (np.abs(Eo[diff] - tau) <= REL_TOL * tau).all()
+    assert int(keep.sum()) == int(keep_o.sum())
+
+
+@pytest.mark.parametrize("alpha", [0.0, 0.5, 1.0])
+def test_tiny_fp32_alpha_sweep(P, alpha):
+    cfg = W().scaled(W().CONFIGS["tiny_fp32"], n_tokens=200)
+    L = W().make_layer(cfg, seed=1, device=DEV)
+    X = W().make_tokens(cfg, seed=1, device=DEV)
+    run_and_compare(P, L, X, alpha=alpha)
+
+
+# ------------------------------------------------------------------ bf16: tensor-core kernel and the FMA kernel
+@pytest.mark.parametrize("force_simt", [False, True])
+@pytest.mark.parametrize("down_layout", ["hf", "me_major"])
+def test_small_bf16(P, force_simt, down_layout):
+    cfg = small_cfg()
+    L = W().make_layer(cfg, seed=2, device=DEV, down_layout=down_layout)
+    X = W().make_tokens(cfg, seed=2, device=DEV)
+    run_and_compare(P, L, X, alpha=0.95, force_simt=force_simt, check_dense=True)
+
+
+@pytest.mark.parametrize("T", [1, 15, 16, 17, 255, 256, 257, 1030])
+def test_ragged_token_counts(P, T):
+    cfg = small_cfg(n_tokens=T, n_routed=4, d_ff_routed=64, d_ff_shared=(64,))
+    L = W().make_layer(cfg, seed=3, device=DEV)
+    X = W().make_tokens(cfg, seed=3, device=DEV)
+    run_and_compare(P, L, X, alpha=0.5)
+
+
+def test_zero_tokens(P):
+    cfg = small_cfg(n_tokens=0)
+    L = W().make_layer(cfg, seed=4, device=DEV)
+    X = W().make_tokens(cfg, seed=4, device=DEV)
+    layer = P.Layer.from_workload(L)
+    out = P.camera_score_layer(layer, X, 0.95, details=True)
+    assert (out["energy"] == 0).all() and (out["phi2"] == 0).all()
+    assert_close("omega2", out["omega2"].cpu().numpy(), O.camera_components(to_oracle_layer(L), f64(X))[2])
+
+
+def test_starved_and_flooded_experts(P):
+    """One expert no token reaches, one expert that takes a slot of every token."""
+    cfg = small_cfg(n_tokens=600, n_routed=5, top_k=2, d_ff_shared=())
+    L = W().make_layer(cfg, seed=5, device=DEV)
+    L["router_bias"] = torch.tensor([0.0, -50.0, 0.0, 50.0, 0.0], device=DEV)
+    X = W().make_tokens(cfg, seed=5, device=DEV)
+    out, _ = run_and_compare(P, L, X, alpha=0.95)
+    counts = out["expert_token_counts"].cpu().numpy()
+    assert counts[1] == 0 and counts[3] == 600
+    assert (out["energy"][128:256] == 0).all()
+
+
+def test_dense_model_as_single_expert(P):
+    """N_E = 1: the paper's dense-model case, as one routed expert and as one shared expert."""
+    for n_routed, shared in ((1, ()), (0, (128,))):
+        cfg = small_cfg(n_tokens=300, n_routed=n_routed, top_k=1, d_ff_routed=128, d_ff_shared=shared,
+                        shared_gate_sigmoid=False, router_bias_std=0.0)
+        L = W().make_layer(cfg, seed=6, device=DEV)
+        X = W().make_tokens(cfg, seed=6, device=DEV)
+        out, _ = run_and_compare(P, L, X, alpha=0.95)
+        if n_routed:
+            assert (out["topk_w"] == 1).all()
+
+
+def test_unnormalised_router_and_many_experts(P):
+    cfg = small_cfg(n_tokens=500, n_routed=70, top_k=6, d_ff_routed=64, d_ff_shared=(64, 64),
+                    shared_gate_sigmoid=False, norm_topk=False)
+    L = W().make_layer(cfg, seed=7, device=DEV)
+    X = W().make_tokens(cfg, seed=7, device=DEV)
+    run_and_compare(P, L, X, alpha=0.95)
+
+
+def test_fma_kernel_takes_odd_shapes(P):
+    """bf16 shapes the tensor-core kernel does not take (d_model, d_ff not multiples of 64)."""
+    cfg = small_cfg(d_model=136, d_ff_routed=72, d_ff_shared=(40,), n_tokens=333)
+    L = W().make_layer(cfg, seed=8, device=DEV)
+    X = W().make_tokens(cfg, seed=8, device=DEV)
+    run_and_compare(P, L, X, alpha=0.95)
+
+
+def test_heavy_tailed_inputs(P):
+    cfg = small_cfg(x_dist="student_t4_outliers", n_tokens=900, shared_gate_sigmoid=False)
+    L = W().make_layer(cfg, seed=9, device=DEV)
+    X = W().make_tokens(cfg, seed=9, device=DEV)
+    run_and_compare(P, L, X, alpha=1.0)
+
+
+def test_bit_reproducible(P):
+    cfg = small_cfg(n_tokens=2000)
+    L = W().make_layer(cfg, seed=10, device=DEV)
+    X = W().make_tokens(cfg, seed=10, device=DEV)
+    layer = P.Layer.from_workload(L)
+    a = P.camera_score_layer(layer, X, 0.95).clone()
+    b = P.camera_score_layer(layer, X, 0.95)
+    assert torch.equal(a, b)
+
+
+def test_multi_chunk_units(P):
+    """Enough tokens per expert that a work unit spans several token tiles and chunks."""
+    cfg = small_cfg(n_tokens=6000, n_routed=2, top_k=1, d_ff_routed=64, d_ff_shared=(64,))
+    L = W().make_layer(cfg, seed=11, device=DEV)
+    X = W().make_tokens(cfg, seed=11, device=DEV)
+    run_and_compare(P, L, X, alpha=0.95)
+
+
+# ------------------------------------------------------------------ argument checks need no kernel to run
+def test_argument_errors(P):
+    cfg = small_cfg(n_tokens=64)
+    L = W().make_layer(cfg, seed=12, device=DEV)
+    X = W().make_tokens(cfg, seed=12, device=DEV)
+    layer = P.Layer.from_workload(L)
+    with pytest.raises(P.CameraError) as e:
+        P.camera_score_layer(layer, X, 1.5)
+    assert e.value.status == -1
+    with pytest.raises(P.CameraError) as e:
+        P.camera_score_layer(layer, X, 0.5, workspace=P.alloc_workspace(1024, DEV))
+    assert e.value.status == -3
+    with pytest.raises(P.CameraError):
+        P.camera_select_prune(torch.zeros(10, device=DEV), 1.0)
+    with pytest.raises(P.CameraError):
+        P.camera_alloc_bits(torch.zeros(10, device=DEV), [0.5, 0.4], [2, 1])
+
+
+# ------------------------------------------------------------------ selection kernels on their own
+def _energies(n, seed, ties=True):
+    g = torch.Generator(device="cpu").manual_seed(seed)
+    E = torch.rand(n, generator=g) ** 4
+    if ties and n > 50:
+        E[n // 10: n // 10 + n // 20] = 0.0
+        E[n // 2: n // 2 + 7] = E[n // 2]
+        E[-3:] = E[0]
+    return E
+
+
+@pytest.mark.parametrize("n", [1, 2, 37, 1000, 4096, 184320])
+@pytest.mark.parametrize("ratio", [0.0, 0.2, 0.4, 0.6, 0.97])
+def test_select_prune_bit_exact(P, n, ratio):
+    E = _energies(n, n)
+    keep, thr = P.camera_select_prune(E.to(DEV), ratio, want_threshold=True)
+    ref = O.select_prune(E.numpy(), ratio)
+    assert np.array_equal(keep.cpu().numpy(), ref)
+    assert float(thr[0]) == E.numpy()[ref == 1].min()
+
+
+def test_select_prune_all_equal(P):
+    E = torch.full((5000,), 0.125)
+    keep = P.camera_select_prune(E.to(DEV), 0.3)
+    assert np.array_equal(keep.cpu().numpy(), O.select_prune(E.numpy(), 0.3))
+    assert (keep[:1500] == 0).all() and (keep[1500:] == 1).all()
+
+
+def test_select_segments_and_expert_counts(P):
+    sizes = [4096, 1000, 0, 7777, 3]
+    seg = np.concatenate([[0], np.cumsum(sizes)])
+    E = _energies(int(seg[-1]), 99)
+    exp_off = np.unique(np.concatenate([seg, np.arange(0, seg[-1], 512)]))
+    keep, kept = P.camera_select_prune(E.to(DEV), 0.4, seg_offsets=seg.tolist(),
+                                       expert_offsets=torch.from_numpy(exp_off).to(DEV))
+    ref = np.concatenate([O.select_prune(E.numpy()[seg[s]:seg[s + 1]], 0.4) for s in range(len(sizes))])
+    assert np.array_equal(keep.cpu().numpy(), ref)
+    assert np.array_equal(kept.cpu().numpy(), [ref[exp_off[i]:exp_off[i + 1]].sum() for i in range(len(exp_off) - 1)])
+
+
+@pytest.mark.parametrize("n", [5, 1003, 92928])
+@pytest.mark.parametrize("scheme", [([0.2, 0.6, 0.2], [3, 2, 1]), ([0.1, 0.8, 0.1], [4, 3, 2]),
+                                    ([0.5, 0.0, 0.5], [3, 2, 1]), ([0.25, 0.25, 0.25, 0.25], [8, 4, 3, 2]),
+                                    ([1.0, 0.0], [4, 2]), ([0.0, 1.0], [4, 2])])
+def test_alloc_bits_bit_exact(P, n, scheme):
+    ratios, bits = scheme
+    E = _energies(n, 7 * n)
+    off = np.unique(np.concatenate([[0, n], np.arange(0, n, 1408)]))
+    out, counts = P.camera_alloc_bits(E.to(DEV), ratios, bits, expert_offsets=torch.from_numpy(off).to(DEV))
+    ref_bits, ref_cls = O.alloc_bits(E.numpy(), ratios, bits)
+    assert np.array_equal(out.cpu().numpy(), ref_bits)
+    assert np.array_equal(counts.cpu().numpy(), O.sub_index(ref_cls, off, len(ratios)))
+
+
+def test_bit_budget_on_gpu(P):
+    """The appendix' worked example realised by the allocation: [3,2,1] x [0.1,0.8,0.1] averages 2 bits."""
+    E = _energies(12800, 5, ties=False)
+    out = P.camera_alloc_bits(E.to(DEV), [0.1, 0.8, 0.1], [3, 2, 1])
+    assert float(out.float().mean()) == 2.0
+    assert abs(O.average_bits([3, 2, 1], [0.1, 0.8, 0.1], 128, 32) - 2.25) < 1e-12
+
+
+# ------------------------------------------------------------------ the host-buffer entry point
+def test_analyze_layer_host(P):
+    cfg = small_cfg(n_tokens=900)
+    L = W().make_layer(cfg, seed=13, device=DEV)
+    X = W().make_tokens(cfg, seed=13, device=DEV)
+    layer = P.Layer.from_workload(L)
+    E = P.camera_score_layer(layer, X, 0.95)
+    keep = P.camera_select_prune(E, 0.4)
+    bits = P.camera_alloc_bits(E, [0.2, 0.6, 0.2], [3, 2, 1])
+    xh = X.cpu().pin_memory()
+    eh = torch.empty(layer.n_me, dtype=torch.float32).pin_memory()
+    kh = torch.empty(layer.n_me, dtype=torch.uint8).pin_memory()
+    bh = torch.empty(layer.n_me, dtype=torch.uint8).pin_memory()
+    ws = P.alloc_workspace(P.camera_analyze_workspace_bytes(layer, 900, 3), DEV)
+    P.camera_analyze_layer_host(layer, xh, 0.95, 0.4, [0.2, 0.6, 0.2], [3, 2, 1], energy_host=eh, keep_host=kh,
+                                bits_host=bh, workspace=ws)
+    assert torch.equal(eh, E.cpu()) and torch.equal(kh, keep.cpu()) and torch.equal(bh, bits.cpu())
