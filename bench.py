@@ -1,0 +1,334 @@
+#!/usr/bin/env python
+"""Benchmark of the CAMERA analysis hot path on B200.
+
+One step = one MoE layer analysed end to end: camera_score_layer (router, permutation, W_down
+norms, fused gate/up scoring, energy), camera_select_prune at 20/40/60 % and camera_alloc_bits for a
+2.25-bit budget, on synthetic calibration tokens of the Qwen2-57B-A14B layer shape.
+
+    python bench.py --gpus N --steps K --warmup W            (N > 1: launched by torch.distributed.run)
+    python bench.py --impl reference ...                      (the float64 CPU oracle on a bounded sample)
+
+Prints one JSON line.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+METRIC = "micro-expert scoring tokens/s per MoE layer"
+UNIT = "tokens/s"
+PRUNE_RATIOS = (0.2, 0.4, 0.6)
+BIT_RATIOS, BIT_LEVELS = (0.2, 0.6, 0.2), (3, 2, 1)     # average 2 bits + 0.25 group overhead
+ALPHA = 0.95
+PAPER_CONTEXT = "paper: <5 min for the full Qwen2-57B-A14B analysis on one A100-40GB (incl. model forwards)"
+# kernels launched by one step: score = router, block scan, plan, permute, pad, norms, scoring, combine;
+# every selection = 8 histogram passes + mark
+LAUNCHES_PER_STEP = 8 + 9 * (len(PRUNE_RATIOS) + 1)
+# DRAM bytes per launch of the scoring kernel from the committed ncu capture, scaled per unit of work
+# (bytes per gate/up flop measured on the profiled case); None until a capture exists.
+SCORE_KERNEL_DRAM_BYTES_PER_FLOP = None
+
+
+def shard_layers(n_layers: int, world: int, rank: int):
+    """Layers of the model a rank analyses when the layers are spread over `world` ranks."""
+    return list(range(rank, n_layers, world))
+
+
+def max_over_ranks(ms: float, dist=None, device="cpu") -> float:
+    """Largest per-rank time; a collective only when a process group exists."""
+    if dist is None or not dist.is_initialized() or dist.get_world_size() == 1:
+        return ms
+    import torch
+    t = torch.tensor([ms], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def load_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        p = json.load(open(path))
+        return {"source": "measured", "hbm_gbs": p["hbm_gbs"], "bf16_tflops": p["bf16_tflops"],
+                "bf16_tflops_sustained": p.get("bf16_tflops_sustained", p["bf16_tflops"])}
+    return {"source": "fallback", "hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
+
+
+class ClockSampler:
+    """Samples SM clocks and throttle reasons with nvidia-smi while the timed region runs."""
+    QUERY = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+             "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+             "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.index = index
+        self.proc = None
+        self.lines = []
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", f"--id={self.index}", f"--query-gpu={self.QUERY}", "--format=csv,noheader,nounits",
+                 "-lms", "100"], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            self.thread = threading.Thread(target=self._read, daemon=True)
+            self.thread.start()
+        except OSError:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.lines.append(line.strip())
+
+    def stop(self):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except subprocess.TimeoutExpired:
+            self.proc.kill()
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for l in self.lines:
+            f = [x.strip() for x in l.split(",")]
+            if len(f) < 7:
+                continue
+            try:
+                sm.append(float(f[0])); mx.append(float(f[1]))
+            except ValueError:
+                continue
+            for n, v in zip(names, f[3:7]):
+                if v.lower().startswith("active"):
+                    reasons.add(n)
+        return {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": max(mx) if mx else None,
+                "samples": len(sm), "reasons": sorted(reasons)}
+
+
+def blas_threads() -> int:
+    """Threads the oracle's numpy BLAS runs on."""
+    try:
+        from threadpoolctl import threadpool_info
+        n = [p.get("num_threads", 0) for p in threadpool_info() if p.get("user_api") == "blas"]
+        if n:
+            return int(max(n))
+    except Exception:
+        pass
+    return len(os.sched_getaffinity(0))
+
+
+def oracle_prepare(L, X):
+    """Widens the stored weights and tokens to float64 for the oracle (not timed)."""
+    sys.path.insert(0, os.path.join(ROOT, "tests"))
+    from _util import f64, to_oracle_layer
+    return to_oracle_layer(L), f64(X)
+
+
+def oracle_step(ol, Xd):
+    """One step of the CPU oracle, as it stands: scores, three prune masks, one bit allocation.  Returns seconds."""
+    import oracle as O
+    t0 = time.perf_counter()
+    E = O.energy(*O.camera_components(ol, Xd), ALPHA)
+    for r in PRUNE_RATIOS:
+        O.select_prune(E, r)
+    O.alloc_bits(E, BIT_RATIOS, BIT_LEVELS)
+    return time.perf_counter() - t0
+
+
+def run_reference(args):
+    """--impl reference: the float64 oracle on host cores, bounded sample per step."""
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    from paper_2508_02322_b200 import workloads as W
+    cfg = W.CONFIGS[args.config]
+    n_sample = args.oracle_tokens or 512
+    L = W.make_layer(cfg, seed=0, layer_id=0, device="cpu")
+    X = W.make_tokens(W.scaled(cfg, n_tokens=n_sample), seed=0, layer_id=0, device="cpu")
+    ol, Xd = oracle_prepare(L, X)
+    for _ in range(args.warmup):
+        oracle_step(ol, Xd)
+    dt = sum(oracle_step(ol, Xd) for _ in range(args.steps))
+    value = n_sample * args.steps / dt
+    cores = blas_threads()
+    sample = f"first {n_sample} tokens of one {cfg.name} layer, all {cfg.n_micro_experts} micro-experts, per step"
+    print(json.dumps({
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": 1e3 * dt / args.steps, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": f"{cfg.name} layer (sample)", "n_tokens": n_sample},
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0}))
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=28)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--config", default="qwen2_57b_a14b")
+    ap.add_argument("--tokens", type=int, default=0, help="override the tokens per layer (profiling small cases)")
+    ap.add_argument("--oracle-tokens", type=int, default=0, help="tokens of the CPU-oracle sample (default 512 for --impl reference, 2048 for the cpu_baseline leg)")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-e2e", action="store_true")
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
+    if args.impl == "reference":
+        return run_reference(args)
+
+    import torch
+    import torch.distributed as dist
+    import paper_2508_02322_b200 as P
+    from paper_2508_02322_b200 import workloads as W
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    torch.cuda.set_device(local)
+    dev = torch.device("cuda", local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=dev)
+
+    cfg = W.CONFIGS[args.config]
+    if args.tokens:
+        cfg = W.scaled(cfg, n_tokens=args.tokens)
+    T = cfg.n_tokens
+    # every rank analyses its own layer (weights and tokens seeded by the layer id): no data-path collective
+    L = W.make_layer(cfg, seed=0, layer_id=rank, device=dev)
+    layer = P.Layer.from_workload(L)
+    Xs = [W.make_tokens(cfg, seed=0, layer_id=rank + world * i, device=dev) for i in range(2)]
+    n_me = layer.n_me
+    ws_score = P.alloc_workspace(P.camera_score_workspace_bytes(layer, T), dev)
+    ws_sel = P.alloc_workspace(P.camera_select_workspace_bytes(n_me, 1, len(BIT_LEVELS)), dev)
+    energy = torch.empty(n_me, dtype=torch.float32, device=dev)
+    keep = torch.empty((len(PRUNE_RATIOS), n_me), dtype=torch.uint8, device=dev)
+    bits = torch.empty(n_me, dtype=torch.uint8, device=dev)
+    stream = torch.cuda.current_stream()
+
+    def step(i, events=None):
+        P.camera_score_layer(layer, Xs[i % 2], ALPHA, energy=energy, workspace=ws_score, stage_events=events)
+        for j, r in enumerate(PRUNE_RATIOS):
+            P.camera_select_prune(energy, r, workspace=ws_sel, keep_mask=keep[j])
+        P.camera_alloc_bits(energy, BIT_RATIOS, BIT_LEVELS, workspace=ws_sel, bits_out=bits)
+
+    def sync_all():
+        torch.cuda.synchronize()
+        if world > 1:
+            dist.barrier()
+            torch.cuda.synchronize()
+
+    for i in range(args.warmup):
+        step(i)
+    torch.cuda.synchronize()
+    status = P.camera_read_status(ws_score)
+    if status != 0:
+        raise RuntimeError(f"device status {status} after warm-up")
+
+    stage_ev = [{s: (torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for s in P.binding.STAGES}
+                for _ in range(args.steps)]
+    for evs in stage_ev:            # events must exist before their handles are passed down
+        for e0, e1 in evs.values():
+            e0.record(stream); e1.record(stream)
+    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    sampler = ClockSampler(local)
+    sync_all()
+    sampler.start()
+    ev0.record(stream)
+    for i in range(args.steps):
+        step(i, stage_ev[i])
+    ev1.record(stream)
+    sync_all()
+    clocks = sampler.stop()
+    ms_local = ev0.elapsed_time(ev1)
+    ms = max_over_ranks(ms_local, dist if world > 1 else None, dev)
+    stage_ms = {s: statistics.mean(e[s][0].elapsed_time(e[s][1]) for e in stage_ev) for s in P.binding.STAGES}
+    status = P.camera_read_status(ws_score)
+    if status != 0:
+        raise RuntimeError(f"device status {status} in the timed region")
+
+    value = world * T * args.steps / (ms * 1e-3)
+    ms_per_step = ms / args.steps
+
+    # ---- end to end through the host-buffer entry point: H2D of the tokens, D2H of the results, every step
+    e2e = None
+    if not args.no_e2e:
+        del ws_score
+        torch.cuda.empty_cache()
+        ws_an = P.alloc_workspace(P.camera_analyze_workspace_bytes(layer, T, len(BIT_LEVELS)), dev)
+        xh = [x.cpu().pin_memory() for x in Xs]
+        eh = torch.empty(n_me, dtype=torch.float32).pin_memory()
+        kh = torch.empty((len(PRUNE_RATIOS), n_me), dtype=torch.uint8).pin_memory()
+        bh = torch.empty(n_me, dtype=torch.uint8).pin_memory()
+        n_e2e = max(2, min(args.steps, 4))
+        for i in range(2):
+            P.camera_analyze_layer_host(layer, xh[i % 2], ALPHA, PRUNE_RATIOS, BIT_RATIOS, BIT_LEVELS, energy_host=eh,
+                                        keep_host=kh, bits_host=bh, workspace=ws_an)
+        sync_all()
+        a0, a1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a0.record(stream)
+        for i in range(n_e2e):
+            P.camera_analyze_layer_host(layer, xh[i % 2], ALPHA, PRUNE_RATIOS, BIT_RATIOS, BIT_LEVELS, energy_host=eh,
+                                        keep_host=kh, bits_host=bh, workspace=ws_an)
+        a1.record(stream)
+        sync_all()
+        e2e_ms = max_over_ranks(a0.elapsed_time(a1), dist if world > 1 else None, dev)
+        e2e = {"value": world * T * n_e2e / (e2e_ms * 1e-3), "unit": UNIT,
+               "h2d_bytes_per_step": xh[0].numel() * xh[0].element_size(),
+               "d2h_bytes_per_step": eh.numel() * 4 + kh.numel() + bh.numel(), "steps": n_e2e,
+               "ms_per_step": e2e_ms / n_e2e}
+
+    if rank != 0:
+        if world > 1:
+            dist.destroy_process_group()
+        return
+
+    peaks = load_peaks()
+    flop = cfg.gate_up_flop
+    score_ms = stage_ms["score"]
+    achieved = flop / (score_ms * 1e-3) / 1e12
+    roofline = {"kernel": "k_score_umma", "bound": "tensor", "achieved": achieved,
+                "peak": peaks["bf16_tflops_sustained"], "unit": "TFLOP/s", "frac": achieved / peaks["bf16_tflops_sustained"],
+                "frac_of_burst_peak": achieved / peaks["bf16_tflops"], "peak_source": peaks["source"] + " (sustained bf16)",
+                "flop_per_launch": flop, "ms_per_launch": score_ms,
+                "traffic": None if SCORE_KERNEL_DRAM_BYTES_PER_FLOP is None else SCORE_KERNEL_DRAM_BYTES_PER_FLOP * flop}
+
+    cpu = None
+    if not args.no_cpu_baseline:
+        n_s = min(args.oracle_tokens or 2048, T)
+        Lc = {k: ([t.cpu() for t in v] if isinstance(v, list) else (v.cpu() if hasattr(v, "cpu") else v)) for k, v in L.items()}
+        ol, Xd = oracle_prepare(Lc, Xs[0][:n_s].cpu())
+        secs = oracle_step(ol, Xd)
+        tps = n_s / secs
+        cpu = {"value": tps, "unit": UNIT, "cores": blas_threads(), "kind": "oracle",
+               "sample": f"first {n_s} tokens of the same layer, all {n_me} micro-experts, {secs:.1f} s"}
+
+    out = {
+        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
+        "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": "bf16" if cfg.dtype == "bf16" else "f32", "data": "synthetic",
+        "config": {"workload": f"{cfg.name} layer: d_model {cfg.d_model}, {cfg.n_routed}x{cfg.d_ff_routed} top-{cfg.top_k}"
+                               f" + shared {list(cfg.d_ff_shared)}, {T} tokens", "tokens_per_layer": T,
+                   "micro_experts": n_me, "alpha": ALPHA, "prune_ratios": list(PRUNE_RATIOS),
+                   "bit_levels": list(BIT_LEVELS), "bit_ratios": list(BIT_RATIOS), "l2": "inputs larger than L2",
+                   "parallelism": f"layers x{world}" if world > 1 else "single GPU"},
+        "model_seconds": cfg.n_layers * ms_per_step * 1e-3 / world,
+        "stage_ms": stage_ms, "clocks": clocks, "e2e": e2e, "gpu_launches": LAUNCHES_PER_STEP * args.steps,
+        "roofline": roofline, "cpu_baseline": cpu, "context": PAPER_CONTEXT,
+    }
+    print(json.dumps(out))
+    if world > 1:
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

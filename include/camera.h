@@ -166,13 +166,13 @@ size_t camera_analyze_workspace_bytes(const camera_layer_t* layer, int64_t n_tok
 /*
  * One whole analysis step with HOST token and result buffers: copies x_host (pinned or
  * pageable, [n_tokens, d_model]) to the device, runs camera_score_layer, camera_select_prune
- * at prune_ratio and camera_alloc_bits, and copies energy [N_e] fp32, keep_mask [N_e] and
- * bits_out [N_e] back to the given HOST buffers (any may be NULL).  The layer's weights stay
- * DEVICE resident.  Synchronises the stream before returning, and returns the workspace's
- * status word if a kernel recorded one.
+ * once per entry of prune_ratios (HOST [n_prune], may be empty) and camera_alloc_bits, and copies
+ * energy [N_e] fp32, keep masks [n_prune, N_e] and bits_out [N_e] back to the given HOST buffers
+ * (any may be NULL).  The layer's weights stay DEVICE resident.  Synchronises the stream before
+ * returning, and returns the workspace's status word if a kernel recorded one.
  */
 int camera_analyze_layer_host(const camera_layer_t* layer, const void* x_host, int64_t n_tokens,
-                              float alpha, double prune_ratio,
+                              float alpha, const double* prune_ratios, int32_t n_prune,
                               const double* ratios, const int32_t* bits, int32_t n_levels,
                               float* energy_host, uint8_t* keep_host, uint8_t* bits_host,
                               void* workspace, size_t workspace_bytes, void* cuda_stream);

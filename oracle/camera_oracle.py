@@ -238,7 +238,9 @@ def camera_components(layer: OracleLayer, X: np.ndarray,
             phi2[off[e] + ch] = 0.0
             phi_inf[off[e] + ch] = 0.0
             continue
-        Lam = a[:, None] * expert_hidden(X[tok], layer.w_gate[e][ch], layer.w_up[e][ch])
+        w_gate = layer.w_gate[e] if channels is None else layer.w_gate[e][ch]
+        w_up = layer.w_up[e] if channels is None else layer.w_up[e][ch]
+        Lam = a[:, None] * expert_hidden(X[tok], w_gate, w_up)
         phi2[off[e] + ch] = (Lam * Lam).sum(axis=0)
         phi_inf[off[e] + ch] = np.abs(Lam).max(axis=0) ** 2
     return phi2, phi_inf, omega2

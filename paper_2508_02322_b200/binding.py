@@ -68,7 +68,8 @@ def _load() -> C.CDLL:
     lib.camera_analyze_workspace_bytes.argtypes = [C.POINTER(camera_layer_t), C.c_int64, C.c_int32]
     lib.camera_analyze_layer_host.restype = C.c_int
     lib.camera_analyze_layer_host.argtypes = [C.POINTER(camera_layer_t), C.c_void_p, C.c_int64, C.c_float,
-                                              C.c_double, C.POINTER(C.c_double), C.POINTER(C.c_int32), C.c_int32,
+                                              C.POINTER(C.c_double), C.c_int32,
+                                              C.POINTER(C.c_double), C.POINTER(C.c_int32), C.c_int32,
                                               C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_size_t,
                                               C.c_void_p]
     return lib
@@ -280,17 +281,20 @@ def camera_alloc_bits(energy: torch.Tensor, ratios: Sequence[float], bits: Seque
     return bits_out if counts is None else (bits_out, counts)
 
 
-def camera_analyze_layer_host(layer: Layer, x_host: torch.Tensor, alpha: float, prune_ratio: float,
+def camera_analyze_layer_host(layer: Layer, x_host: torch.Tensor, alpha: float, prune_ratios: Sequence[float],
                               ratios: Sequence[float], bits: Sequence[int], *, energy_host: torch.Tensor,
                               keep_host: torch.Tensor, bits_host: torch.Tensor, workspace: torch.Tensor,
                               stream: Optional[torch.cuda.Stream] = None) -> None:
-    """One analysis step with host token/result buffers (see camera.h); blocks until done."""
+    """One analysis step with host token/result buffers (see camera.h); blocks until done.
+    keep_host is [len(prune_ratios), N_e] uint8."""
     if x_host.is_cuda or not x_host.is_contiguous() or x_host.dtype != layer.dtype:
         raise ValueError("x_host must be a contiguous host tensor of the layer's dtype")
     L = len(ratios)
     r = (C.c_double * L)(*[float(v) for v in ratios])
     b = (C.c_int32 * L)(*[int(v) for v in bits])
+    n_prune = len(prune_ratios)
+    pr = (C.c_double * max(n_prune, 1))(*[float(v) for v in prune_ratios])
     _check(lib.camera_analyze_layer_host(C.byref(layer.c), x_host.data_ptr(), int(x_host.shape[0]), float(alpha),
-                                         float(prune_ratio), r, b, L, _ptr(energy_host), _ptr(keep_host),
+                                         pr, n_prune, r, b, L, _ptr(energy_host), _ptr(keep_host),
                                          _ptr(bits_host), workspace.data_ptr(), workspace.numel(),
                                          _stream_ptr(stream)), "camera_analyze_layer_host")

@@ -310,12 +310,14 @@ extern "C" size_t camera_analyze_workspace_bytes(const camera_layer_t* layer, in
 }
 
 extern "C" int camera_analyze_layer_host(const camera_layer_t* L, const void* x_host, int64_t T, float alpha,
-                                         double prune_ratio, const double* ratios, const int32_t* bits,
-                                         int32_t n_levels, float* energy_host, uint8_t* keep_host, uint8_t* bits_host,
-                                         void* workspace, size_t workspace_bytes, void* cuda_stream) {
+                                         const double* prune_ratios, int32_t n_prune, const double* ratios,
+                                         const int32_t* bits, int32_t n_levels, float* energy_host,
+                                         uint8_t* keep_host, uint8_t* bits_host, void* workspace,
+                                         size_t workspace_bytes, void* cuda_stream) {
   int rc = validate_layer(L, T);
   if (rc != CAMERA_OK) return rc;
-  if (n_levels < 2 || n_levels > MAX_LEVELS || ratios == nullptr || bits == nullptr || (T > 0 && x_host == nullptr))
+  if (n_levels < 2 || n_levels > MAX_LEVELS || ratios == nullptr || bits == nullptr || (T > 0 && x_host == nullptr) ||
+      n_prune < 0 || (n_prune > 0 && prune_ratios == nullptr))
     return CAMERA_ERR_INVALID_ARG;
   const AnalyzeLayout a = analyze_layout(L, T, n_levels);
   if (workspace == nullptr || workspace_bytes < a.total || (reinterpret_cast<uintptr_t>(workspace) & 255))
@@ -330,15 +332,18 @@ extern "C" int camera_analyze_layer_host(const camera_layer_t* L, const void* x_
   if (T > 0) CK(cudaMemcpyAsync(ws + a.x, x_host, esz * (size_t)T * L->d_model, cudaMemcpyHostToDevice, st));
   rc = camera_score_layer(L, ws + a.x, T, alpha, d_energy, nullptr, ws + a.score, a.score_bytes, cuda_stream);
   if (rc != CAMERA_OK) return rc;
+  if (energy_host) CK(cudaMemcpyAsync(energy_host, d_energy, sizeof(float) * (size_t)s.n_me, cudaMemcpyDeviceToHost, st));
   const int64_t seg[2] = {0, s.n_me};
-  rc = camera_select_prune(d_energy, seg, 1, prune_ratio, nullptr, 0, d_keep, nullptr, nullptr, ws + a.select,
-                           a.select_bytes, cuda_stream);
-  if (rc != CAMERA_OK) return rc;
-  if (keep_host) CK(cudaMemcpyAsync(keep_host, d_keep, (size_t)s.n_me, cudaMemcpyDeviceToHost, st));
+  for (int p = 0; p < n_prune; ++p) {
+    rc = camera_select_prune(d_energy, seg, 1, prune_ratios[p], nullptr, 0, d_keep, nullptr, nullptr, ws + a.select,
+                             a.select_bytes, cuda_stream);
+    if (rc != CAMERA_OK) return rc;
+    if (keep_host)
+      CK(cudaMemcpyAsync(keep_host + (size_t)p * s.n_me, d_keep, (size_t)s.n_me, cudaMemcpyDeviceToHost, st));
+  }
   rc = camera_alloc_bits(d_energy, seg, 1, ratios, bits, n_levels, nullptr, 0, d_bits, nullptr, ws + a.select,
                          a.select_bytes, cuda_stream);
   if (rc != CAMERA_OK) return rc;
-  if (energy_host) CK(cudaMemcpyAsync(energy_host, d_energy, sizeof(float) * (size_t)s.n_me, cudaMemcpyDeviceToHost, st));
   if (bits_host) CK(cudaMemcpyAsync(bits_host, d_bits, (size_t)s.n_me, cudaMemcpyDeviceToHost, st));
   int32_t status = 0;
   rc = camera_read_status(ws + a.score, cuda_stream, &status);

@@ -243,13 +243,13 @@ def test_analyze_layer_host(P):
     X = W().make_tokens(cfg, seed=13, device=DEV)
     layer = P.Layer.from_workload(L)
     E = P.camera_score_layer(layer, X, 0.95)
-    keep = P.camera_select_prune(E, 0.4)
+    keep = torch.stack([P.camera_select_prune(E, r) for r in (0.2, 0.6)])
     bits = P.camera_alloc_bits(E, [0.2, 0.6, 0.2], [3, 2, 1])
     xh = X.cpu().pin_memory()
     eh = torch.empty(layer.n_me, dtype=torch.float32).pin_memory()
-    kh = torch.empty(layer.n_me, dtype=torch.uint8).pin_memory()
+    kh = torch.empty((2, layer.n_me), dtype=torch.uint8).pin_memory()
     bh = torch.empty(layer.n_me, dtype=torch.uint8).pin_memory()
     ws = P.alloc_workspace(P.camera_analyze_workspace_bytes(layer, 900, 3), DEV)
-    P.camera_analyze_layer_host(layer, xh, 0.95, 0.4, [0.2, 0.6, 0.2], [3, 2, 1], energy_host=eh, keep_host=kh,
+    P.camera_analyze_layer_host(layer, xh, 0.95, [0.2, 0.6], [0.2, 0.6, 0.2], [3, 2, 1], energy_host=eh, keep_host=kh,
                                 bits_host=bh, workspace=ws)
     assert torch.equal(eh, E.cpu()) and torch.equal(kh, keep.cpu()) and torch.equal(bh, bits.cpu())
