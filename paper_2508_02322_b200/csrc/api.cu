@@ -1,5 +1,6 @@
 // C ABI entry points of camera_score_layer and camera_analyze_layer_host: argument checks,
 // workspace carving, and the launch sequence.  No device memory is allocated here.
+#include <stdlib.h>
 #include <string.h>
 
 #include <vector>
@@ -15,6 +16,18 @@ namespace {
 constexpr int PLAN_SMS = 148;   // used only to size work units; the result is valid on any device
 
 size_t up256(size_t v) { return (v + 255) & ~(size_t)255; }
+
+// Channel tiles per scheduling group.  20 tiles = 1280 micro-experts: 18 MB of gate+up rows at
+// d_model 3584, small enough to stay in one L2 partition next to the token tiles in flight.
+// CAMERA_CT_GROUP overrides it (tuning aid).
+int score_ct_group() {
+  const char* env = getenv("CAMERA_CT_GROUP");
+  if (env != nullptr) {
+    const int v = atoi(env);
+    if (v >= 1 && v <= 4096) return v;
+  }
+  return 20;
+}
 
 struct ScoreLayout {
   size_t totals, est, edyn, me_prefix, unit_prefix, counts, block_hist, local_rank, topk_idx, topk_w, shared_w,
@@ -188,7 +201,7 @@ extern "C" int camera_score_layer(const camera_layer_t* L, const void* x, int64_
   c.d_model = L->d_model; c.n_routed = L->n_routed; c.top_k = L->n_routed > 0 ? L->top_k : 0;
   c.n_shared = L->n_shared; c.n_experts = E; c.n_me = lay.n_me;
   c.dtype = L->dtype; c.down_layout = L->down_layout; c.flags = L->flags;
-  c.n_tokens = (int)T; c.n_blocks = lay.n_blocks; c.chunk_tokens = lay.chunk_tokens;
+  c.n_tokens = (int)T; c.n_blocks = lay.n_blocks; c.chunk_tokens = lay.chunk_tokens; c.ct_group = score_ct_group();
   c.max_rows_perm = lay.max_rows_perm; c.max_part = lay.max_part; c.alpha = alpha;
   c.x = x; c.w_router = L->w_router; c.router_bias = L->router_bias; c.w_shared_gate = L->w_shared_gate;
   c.totals = reinterpret_cast<PlanTotals*>(ws + lay.totals);

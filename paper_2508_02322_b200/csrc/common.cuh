@@ -52,6 +52,7 @@ struct ScoreCtx {
   uint32_t flags;
   int32_t n_tokens, n_blocks;       // n_blocks = ceil(T / ROUTER_TOK)
   int32_t chunk_tokens;             // tokens per scoring work unit (multiple of UMMA_TOK)
+  int32_t ct_group;                 // channel tiles per scheduling group (see decode_unit)
   int32_t max_rows_perm;            // capacity of x_perm in rows
   int64_t max_part;                 // capacity of the partial arrays in floats
   float alpha;
@@ -130,6 +131,37 @@ __device__ __forceinline__ int upper_segment(const P* prefix, int n, P v) {
     if (prefix[mid] <= v) lo = mid; else hi = mid;
   }
   return lo;
+}
+
+// One scoring work unit: CH_TILE channels of one expert against one chunk of its token list.
+struct UnitInfo {
+  int e, chunk, ch0, f, rows, row0, shared_idx;
+  long long part_slot;       // part_begin + chunk * f + ch0
+};
+
+// Units of an expert are numbered channel-group by channel-group: inside a group of `ct_group`
+// channel tiles the order is (chunk, channel tile).  CTAs that run at the same time take
+// consecutive units, so together they touch at most ct_group weight tiles (which stay in L2 while
+// the group walks down the expert's whole token list) and a handful of token tiles.
+__device__ __forceinline__ UnitInfo decode_unit(const ScoreCtx& c, int unit) {
+  UnitInfo u;
+  u.e = upper_segment(c.unit_prefix, c.n_experts, unit);
+  const ExpertDyn dy = c.edyn[u.e];
+  u.f = c.est[u.e].d_ff;
+  u.shared_idx = c.est[u.e].shared_idx;
+  const int n_ct = (u.f + CH_TILE - 1) / CH_TILE;
+  int rem = unit - c.unit_prefix[u.e];
+  const int per_full_group = dy.n_chunks * c.ct_group;
+  const int g = min(rem / per_full_group, (n_ct - 1) / c.ct_group);
+  rem -= g * per_full_group;
+  const int in_group = min(c.ct_group, n_ct - g * c.ct_group);
+  u.chunk = rem / in_group;
+  u.ch0 = (g * c.ct_group + rem % in_group) * CH_TILE;
+  const int row_begin = u.chunk * c.chunk_tokens;
+  u.rows = min(c.chunk_tokens, dy.rows - row_begin);
+  u.row0 = dy.row_base + row_begin;
+  u.part_slot = dy.part_begin + (long long)u.chunk * u.f + u.ch0;
+  return u;
 }
 
 }  // namespace camera

@@ -31,20 +31,12 @@ __global__ void __launch_bounds__(SS_THREADS) k_score_simt(ScoreCtx c) {
   const int total_units = c.totals->total_units;
 
   for (int unit = blockIdx.x; unit < total_units; unit += gridDim.x) {
-    const int e = upper_segment(c.unit_prefix, c.n_experts, unit);
-    const ExpertStatic es = c.est[e];
-    const ExpertDyn dy = c.edyn[e];
-    const int f = es.d_ff;
-    const int n_ct = (f + CH_TILE - 1) / CH_TILE;
-    const int rem = unit - c.unit_prefix[e];
-    const int chunk = rem / n_ct, ct = rem % n_ct;
-    const int ch0 = ct * CH_TILE;
-    const int row_begin = chunk * c.chunk_tokens;
-    const int rows = min(c.chunk_tokens, dy.rows - row_begin);
+    const UnitInfo u = decode_unit(c, unit);
+    const ExpertStatic es = c.est[u.e];
+    const int f = u.f, ch0 = u.ch0, rows = u.rows;
     const T* Xsrc = (es.shared_idx < 0 ? static_cast<const T*>(c.x_perm) : static_cast<const T*>(c.x)) +
-                    (size_t)(dy.row_base + row_begin) * d;
-    const float* wsrc = (es.shared_idx < 0 ? c.perm_w + dy.row_base
-                                           : c.shared_w + (size_t)es.shared_idx * c.n_tokens) + row_begin;
+                    (size_t)u.row0 * d;
+    const float* wsrc = (es.shared_idx < 0 ? c.perm_w : c.shared_w + (size_t)es.shared_idx * c.n_tokens) + u.row0;
     const T* Wg = static_cast<const T*>(es.w_gate);
     const T* Wu = static_cast<const T*>(es.w_up);
 
@@ -111,7 +103,7 @@ __global__ void __launch_bounds__(SS_THREADS) k_score_simt(ScoreCtx c) {
       float ts = 0.f, tm = 0.f;
 #pragma unroll
       for (int y = 0; y < 16; ++y) { ts += red_s[y][tid]; tm = fmaxf(tm, red_m[y][tid]); }
-      const size_t slot = (size_t)dy.part_begin + (size_t)chunk * f + ch0 + tid;
+      const size_t slot = (size_t)u.part_slot + tid;
       c.part_sum[slot] = ts;
       c.part_max[slot] = tm;
     }

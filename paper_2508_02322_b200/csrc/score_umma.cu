@@ -140,29 +140,6 @@ __device__ __forceinline__ void tmem_ld16(uint32_t taddr, uint32_t* v) {
 }
 __device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
 
-struct UnitInfo {
-  int e, chunk, ch0, f, rows, row0, n_tiles, shared_idx;
-  long long part_slot;       // part_begin + chunk * f + ch0
-};
-
-__device__ __forceinline__ UnitInfo decode_unit(const ScoreCtx& c, int unit) {
-  UnitInfo u;
-  u.e = upper_segment(c.unit_prefix, c.n_experts, unit);
-  const ExpertDyn dy = c.edyn[u.e];
-  u.f = c.est[u.e].d_ff;
-  u.shared_idx = c.est[u.e].shared_idx;
-  const int n_ct = u.f / CH_TILE;
-  const int rem = unit - c.unit_prefix[u.e];
-  u.chunk = rem / n_ct;
-  u.ch0 = (rem % n_ct) * CH_TILE;
-  const int row_begin = u.chunk * c.chunk_tokens;
-  u.rows = min(c.chunk_tokens, dy.rows - row_begin);
-  u.row0 = dy.row_base + row_begin;
-  u.n_tiles = (u.rows + UMMA_TOK - 1) / UMMA_TOK;
-  u.part_slot = dy.part_begin + (long long)u.chunk * u.f + u.ch0;
-  return u;
-}
-
 __global__ void __launch_bounds__(U_THREADS, 1) k_score_umma(const ScoreCtx c) {
   extern __shared__ uint8_t smem_raw[];
   const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
@@ -209,13 +186,14 @@ __global__ void __launch_bounds__(U_THREADS, 1) k_score_umma(const ScoreCtx c) {
       const char* maps = static_cast<const char*>(c.tensor_maps);
       for (int unit = blockIdx.x; ok && unit < total_units; unit += gridDim.x) {
         const UnitInfo u = decode_unit(c, unit);
+        const int n_tiles = (u.rows + UMMA_TOK - 1) / UMMA_TOK;
         const void* map_g = maps + (size_t)128 * (2 * u.e);
         const void* map_u = maps + (size_t)128 * (2 * u.e + 1);
         const void* map_x = maps + (size_t)128 * (2 * c.n_experts + (u.shared_idx < 0 ? 0 : 1));
         tensormap_acquire(map_g);
         tensormap_acquire(map_u);
         tensormap_acquire(map_x);
-        for (int tt = 0; ok && tt < u.n_tiles; ++tt) {
+        for (int tt = 0; ok && tt < n_tiles; ++tt) {
           const int row = u.row0 + tt * UMMA_TOK;
           for (int kb = 0; kb < n_kb; ++kb) {
             if (!mbar_wait(empty_bar(stage), phase ^ 1u, abort_flag)) { ok = false; break; }
@@ -246,7 +224,8 @@ __global__ void __launch_bounds__(U_THREADS, 1) k_score_umma(const ScoreCtx c) {
       bool ok = true;
       for (int unit = blockIdx.x; ok && unit < total_units; unit += gridDim.x) {
         const UnitInfo u = decode_unit(c, unit);
-        for (int tt = 0; ok && tt < u.n_tiles; ++tt) {
+        const int n_tiles = (u.rows + UMMA_TOK - 1) / UMMA_TOK;
+        for (int tt = 0; ok && tt < n_tiles; ++tt) {
           const int nv = (min(UMMA_TOK, u.rows - tt * UMMA_TOK) + 15) & ~15;
           const uint32_t idesc = make_idesc(nv);
           if (!mbar_wait(tempty_bar(acc), acc_phase ^ 1u, abort_flag)) { ok = false; break; }
@@ -278,9 +257,10 @@ __global__ void __launch_bounds__(U_THREADS, 1) k_score_umma(const ScoreCtx c) {
     const bool lo = lane < 16;
     for (int unit = blockIdx.x; ok && unit < total_units; unit += gridDim.x) {
       const UnitInfo u = decode_unit(c, unit);
+      const int n_tiles = (u.rows + UMMA_TOK - 1) / UMMA_TOK;
       const float* wsrc = u.shared_idx < 0 ? c.perm_w + u.row0 : c.shared_w + (size_t)u.shared_idx * c.n_tokens + u.row0;
       float s = 0.f, m = 0.f;
-      for (int tt = 0; ok && tt < u.n_tiles; ++tt) {
+      for (int tt = 0; ok && tt < n_tiles; ++tt) {
         const int valid = min(UMMA_TOK, u.rows - tt * UMMA_TOK);
         const int nv = (valid + 15) & ~15;
         // each warp stages the tile's router weights for itself, so the four warps never wait on
