@@ -160,6 +160,30 @@ int camera_alloc_bits(const float* energy, const int64_t* seg_offsets, int32_t n
                       uint8_t* bits_out, int32_t* class_counts,
                       void* workspace, size_t workspace_bytes, void* cuda_stream);
 
+/*
+ * camera_select_prune without a workspace argument (the paper has no counterpart; this exists for
+ * the sake of integration).  Some hosts of this library may not create device allocations at all:
+ * a plug-in inside a serving process whose memory pool already owns the whole GPU, a callback that
+ * runs where cudaMalloc's implicit device-wide synchronisation is not acceptable, or code that is
+ * simply not handed an allocator.  For them the scratch of the selection lives in a fixed array
+ * inside the library image: 288 KiB of every GPU that loads the library, held until the process ends.
+ *
+ * Same arguments and results as camera_select_prune (energy, keep_mask, thresholds: DEVICE;
+ * seg_offsets: HOST), minus the per-expert counts.  Limit: n_segments <= 32; more returns
+ * CAMERA_ERR_UNSUPPORTED_SHAPE and launches nothing.  The call itself allocates nothing on the
+ * device (no cudaMalloc / cudaFree, no allocating library routine).
+ *
+ * The first call on each device looks up the array's device address (the device must be current);
+ * make that first call outside of any stream capture.  All calls on a device share the one array
+ * and each call overwrites what the previous one left there (the parts that have to start at zero
+ * are cleared on the stream at the start of every call), so two calls that overlap on the GPU --
+ * different streams, or different host threads -- race; issue them on one stream or order them with
+ * events.
+ */
+int camera_select_prune_static(const float* energy, const int64_t* seg_offsets, int32_t n_segments,
+                               double prune_ratio, uint8_t* keep_mask, float* thresholds,
+                               void* cuda_stream);
+
 /* Scratch for camera_analyze_layer_host: score + select scratch + staging of x and results. */
 size_t camera_analyze_workspace_bytes(const camera_layer_t* layer, int64_t n_tokens, int32_t n_levels);
 

@@ -64,6 +64,9 @@ def _load() -> C.CDLL:
     lib.camera_alloc_bits.argtypes = [C.c_void_p, C.POINTER(C.c_int64), C.c_int32, C.POINTER(C.c_double),
                                       C.POINTER(C.c_int32), C.c_int32, C.c_void_p, C.c_int32, C.c_void_p,
                                       C.c_void_p, C.c_void_p, C.c_size_t, C.c_void_p]
+    lib.camera_select_prune_static.restype = C.c_int
+    lib.camera_select_prune_static.argtypes = [C.c_void_p, C.POINTER(C.c_int64), C.c_int32, C.c_double, C.c_void_p,
+                                               C.c_void_p, C.c_void_p]
     lib.camera_analyze_workspace_bytes.restype = C.c_size_t
     lib.camera_analyze_workspace_bytes.argtypes = [C.POINTER(camera_layer_t), C.c_int64, C.c_int32]
     lib.camera_analyze_layer_host.restype = C.c_int
@@ -253,6 +256,19 @@ def camera_select_prune(energy: torch.Tensor, prune_ratio: float, *, seg_offsets
     if thr is not None:
         res.append(thr)
     return res[0] if len(res) == 1 else tuple(res)
+
+
+def camera_select_prune_static(energy: torch.Tensor, prune_ratio: float, keep_mask: torch.Tensor, *,
+                               seg_offsets=None, thresholds: Optional[torch.Tensor] = None,
+                               stream: Optional[torch.cuda.Stream] = None) -> torch.Tensor:
+    """CAMERA-P mask for callers that cannot allocate device memory: the caller passes the input and
+    the output tensors, and the selection's scratch is a fixed array inside the library (at most 32
+    segments).  This wrapper creates no tensor either.  Calls share that array: keep them on one
+    stream, or order them with events."""
+    seg, n_seg = _segments(energy.numel(), seg_offsets)
+    _check(lib.camera_select_prune_static(energy.data_ptr(), seg, n_seg, float(prune_ratio), keep_mask.data_ptr(),
+                                          _ptr(thresholds), _stream_ptr(stream)), "camera_select_prune_static")
+    return keep_mask
 
 
 def camera_alloc_bits(energy: torch.Tensor, ratios: Sequence[float], bits: Sequence[int], *, seg_offsets=None,

@@ -301,3 +301,63 @@ extern "C" int camera_alloc_bits(const float* energy, const int64_t* seg_offsets
   delete[] ranks;
   return rc;
 }
+
+// ---------------------------------------------------------------------------------------------
+// camera_select_prune_static: the same selection with its scratch in a fixed device array that is
+// part of the library image, for callers that have no way to hand over a workspace.
+// ---------------------------------------------------------------------------------------------
+namespace camera {
+namespace {
+
+constexpr int STATIC_MAX_SEGMENTS = 32;
+constexpr size_t STATIC_SCRATCH_BYTES = 288 * 1024;   // sel_layout(32, 1).total = 271,360 bytes fits
+
+// Lives in every GPU's memory from the moment the library is loaded there until the process ends.
+static __device__ __align__(256) unsigned char g_select_scratch[STATIC_SCRATCH_BYTES];
+
+constexpr int STATIC_MAX_DEVICES = 64;
+void* g_scratch_ptr[STATIC_MAX_DEVICES];     // device address of g_select_scratch, per device ordinal
+bool g_scratch_ready[STATIC_MAX_DEVICES];
+
+// In host code `g_select_scratch` is only a handle; the address kernels can use has to be asked for,
+// once per device, while that device is current.
+int static_scratch(void** out) {
+  int dev = -1;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= STATIC_MAX_DEVICES) return CAMERA_ERR_CUDA;
+  if (!g_scratch_ready[dev]) {
+    void* p = nullptr;
+    if (cudaGetSymbolAddress(&p, g_select_scratch) != cudaSuccess || p == nullptr) {
+      cudaGetLastError();
+      return CAMERA_ERR_CUDA;
+    }
+    g_scratch_ptr[dev] = p;
+    g_scratch_ready[dev] = true;
+  }
+  *out = g_scratch_ptr[dev];
+  return CAMERA_OK;
+}
+
+}  // namespace
+}  // namespace camera
+
+extern "C" int camera_select_prune_static(const float* energy, const int64_t* seg_offsets, int32_t n_segments,
+                                          double prune_ratio, uint8_t* keep_mask, float* thresholds,
+                                          void* cuda_stream) {
+  if (!segments_ok(seg_offsets, n_segments) || !(prune_ratio >= 0.0 && prune_ratio < 1.0) || keep_mask == nullptr)
+    return CAMERA_ERR_INVALID_ARG;
+  if (seg_offsets[n_segments] > 0 && energy == nullptr) return CAMERA_ERR_INVALID_ARG;
+  if (n_segments > STATIC_MAX_SEGMENTS || sel_layout(n_segments, 1).total > STATIC_SCRATCH_BYTES)
+    return CAMERA_ERR_UNSUPPORTED_SHAPE;
+  void* scratch = nullptr;
+  const int rc = static_scratch(&scratch);
+  if (rc != CAMERA_OK) return rc;
+  long long ranks[STATIC_MAX_SEGMENTS];
+  for (int s = 0; s < n_segments; ++s) ranks[s] = floor_count(prune_ratio, seg_offsets[s + 1] - seg_offsets[s]);
+  LevelValues lv;
+  memset(&lv, 0, sizeof(lv));
+  lv.v[0] = 1;
+  lv.v[1] = 0;
+  // select_core clears the histograms it counts into on every call; nothing else in the array has to start at zero
+  return select_core(energy, seg_offsets, n_segments, 1, ranks, lv, nullptr, 0, 1, keep_mask, nullptr, thresholds, scratch,
+                     STATIC_SCRATCH_BYTES, static_cast<cudaStream_t>(cuda_stream));
+}
