@@ -178,6 +178,8 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--config", default="qwen2_57b_a14b")
     ap.add_argument("--tokens", type=int, default=0, help="override the tokens per layer (profiling small cases)")
+    ap.add_argument("--routed", type=int, default=0, help="override the number of routed experts (profiling slices)")
+    ap.add_argument("--topk", type=int, default=0, help="override top-k (with --routed and --tokens: a slice that keeps the full layer's tokens per expert)")
     ap.add_argument("--oracle-tokens", type=int, default=0, help="tokens of the CPU-oracle sample (default 512 for --impl reference, 2048 for the cpu_baseline leg)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
@@ -202,6 +204,10 @@ def main():
     cfg = W.CONFIGS[args.config]
     if args.tokens:
         cfg = W.scaled(cfg, n_tokens=args.tokens)
+    if args.routed:
+        cfg = W.scaled(cfg, n_routed=args.routed, top_k=min(args.topk or cfg.top_k, args.routed))
+    elif args.topk:
+        cfg = W.scaled(cfg, top_k=args.topk)
     T = cfg.n_tokens
     # every rank analyses its own layer (weights and tokens seeded by the layer id): no data-path collective
     L = W.make_layer(cfg, seed=0, layer_id=rank, device=dev)
