@@ -117,8 +117,8 @@ size_t camera_score_workspace_bytes(const camera_layer_t* layer, int64_t n_token
  * Arithmetic: inputs as stored, products and sums in fp32 (bf16: tensor cores with fp32
  * accumulators), the final blend in fp64.  Routing ties go to the lower expert index.
  * An expert no token reaches gets energy 0.  0 <= alpha <= 1.  n_tokens >= 0.
- * The bf16 tensor-core path needs d_model % 64 == 0 and every d_ff % 64 == 0; other shapes
- * (and fp32) run the fp32-FMA kernel.
+ * The bf16 tensor-core path needs d_model % 64 == 0; other shapes (and fp32) run the fp32-FMA
+ * kernel.
  */
 int camera_score_layer(const camera_layer_t* layer, const void* x, int64_t n_tokens, float alpha,
                        float* energy, const camera_score_aux_t* aux,

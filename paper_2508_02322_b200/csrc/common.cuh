@@ -12,7 +12,7 @@ namespace camera {
 // ---- tiling constants shared by the host planner and the kernels -----------------------------
 constexpr int ROUTER_TOK = 64;       // tokens per router CTA (also the unit of the stable counting sort)
 constexpr int ROW_ALIGN = 16;        // every expert's token list is padded to this many rows
-constexpr int CH_TILE = 64;          // micro-experts (channels) per scoring work unit
+constexpr int CH_TILE = 128;         // micro-experts (channels) per scoring work unit
 constexpr int UMMA_TOK = 256;        // tokens per tensor-core tile (the MMA's N)
 constexpr int MAX_ROUTED = 256;
 constexpr int MAX_TOPK = 16;

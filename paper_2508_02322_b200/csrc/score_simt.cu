@@ -11,9 +11,11 @@ constexpr int SS_THREADS = 256;
 constexpr int SS_TOK = 64;
 constexpr int SS_KC = 16;
 constexpr int SS_LD = 68;
+constexpr int SS_CH = 64;           // channels per pass
 
-// Work unit = (expert, tile of CH_TILE channels, chunk of chunk_tokens tokens).  For every
-// token tile the CTA forms g = W_gate x and u = W_up x for 64 tokens x 64 channels in fp32,
+// Work unit = (expert, tile of CH_TILE channels, chunk of chunk_tokens tokens), handled as
+// CH_TILE / 64 passes of 64 channels.  For every token tile the CTA forms g = W_gate x and
+// u = W_up x for 64 tokens x 64 channels in fp32,
 // then lambda = a_t * SiLU(g) * u and folds lambda^2 / |lambda| into per-channel running sum / max.
 // One partial (sum, max) per channel and chunk goes to the workspace; chunks are added later in
 // a fixed order, so results do not depend on scheduling.
@@ -22,18 +24,20 @@ __global__ void __launch_bounds__(SS_THREADS) k_score_simt(ScoreCtx c) {
   __shared__ __align__(16) float Xs[SS_KC][SS_LD];
   __shared__ __align__(16) float Gs[SS_KC][SS_LD];
   __shared__ __align__(16) float Us[SS_KC][SS_LD];
-  __shared__ float red_s[16][CH_TILE];
-  __shared__ float red_m[16][CH_TILE];
+  __shared__ float red_s[16][SS_CH];
+  __shared__ float red_m[16][SS_CH];
   constexpr int VN = Vec16<T>::N;
   constexpr int VPR = SS_KC / VN;
   const int tid = threadIdx.x, tx = tid & 15, ty = tid >> 4;
   const int d = c.d_model;
   const int total_units = c.totals->total_units;
 
-  for (int unit = blockIdx.x; unit < total_units; unit += gridDim.x) {
-    const UnitInfo u = decode_unit(c, unit);
+  for (int work = blockIdx.x; work < total_units * (CH_TILE / SS_CH); work += gridDim.x) {
+    const UnitInfo u = decode_unit(c, work / (CH_TILE / SS_CH));
     const ExpertStatic es = c.est[u.e];
-    const int f = u.f, ch0 = u.ch0, rows = u.rows;
+    const int pass_off = (work % (CH_TILE / SS_CH)) * SS_CH;
+    const int f = u.f, ch0 = u.ch0 + pass_off, rows = u.rows;
+    if (ch0 >= f) continue;
     const T* Xsrc = (es.shared_idx < 0 ? static_cast<const T*>(c.x_perm) : static_cast<const T*>(c.x)) +
                     (size_t)u.row0 * d;
     const float* wsrc = (es.shared_idx < 0 ? c.perm_w : c.shared_w + (size_t)es.shared_idx * c.n_tokens) + u.row0;
@@ -99,11 +103,11 @@ __global__ void __launch_bounds__(SS_THREADS) k_score_simt(ScoreCtx c) {
 #pragma unroll
     for (int j = 0; j < 4; ++j) { red_s[ty][tx * 4 + j] = s[j]; red_m[ty][tx * 4 + j] = m[j]; }
     __syncthreads();
-    if (tid < CH_TILE && ch0 + tid < f) {
+    if (tid < SS_CH && ch0 + tid < f) {
       float ts = 0.f, tm = 0.f;
 #pragma unroll
       for (int y = 0; y < 16; ++y) { ts += red_s[y][tid]; tm = fmaxf(tm, red_m[y][tid]); }
-      const size_t slot = (size_t)u.part_slot + tid;
+      const size_t slot = (size_t)u.part_slot + pass_off + tid;
       c.part_sum[slot] = ts;
       c.part_max[slot] = tm;
     }

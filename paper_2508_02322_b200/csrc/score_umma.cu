@@ -3,16 +3,16 @@
 //   to per-micro-expert sum(Lambda^2) and max|Lambda| in the epilogue; it never reaches HBM.
 //
 // One persistent CTA per SM, 6 warps:
-//   warps 0-3  epilogue: tcgen05.ld the accumulator, SiLU * up * router weight, running sum / max
-//   warp  4    producer: TMA loads of the weight tile (A operand) and the token tile (B operand)
+//   warps 0-3  epilogue: tcgen05.ld both accumulators, SiLU * up * router weight, running sum / max
+//   warp  4    producer: TMA loads of the two weight tiles (A operands) and the token tile (B operand)
 //   warp  5    tensor-memory allocation and the single thread that issues tcgen05.mma
 //
-// Operand orientation: the MMA's M dimension (128 TMEM lanes) holds 64 micro-experts as
-// interleaved groups [16 gate rows | 16 up rows] x 4, its N dimension (up to 256 columns) holds
-// tokens.  Every epilogue thread therefore owns one weight row for all tokens of the tile: the
-// per-channel reduction over tokens runs down its own registers, and gate/up of a channel sit 16
-// lanes apart in the same warp, one shuffle away.  Two 256-column accumulators alternate, so the
-// epilogue of one token tile overlaps the MMAs of the next.
+// Operand orientation: the MMA's M dimension (128 TMEM lanes) holds 128 micro-experts, its N
+// dimension (up to 256 columns) holds tokens.  Two accumulators share every token tile: columns
+// 0-255 take W_gate x, columns 256-511 take W_up x of the same 128 micro-experts, so one pass over
+// K pulls 64 KB from L2 for 8.4 Mflop.  Every epilogue thread owns one micro-expert for all tokens of
+// the tile: gate and up of a (micro-expert, token) pair arrive in the same thread, and the reduction
+// over tokens runs down its own registers.
 //
 // Every wait on an mbarrier is bounded: when a wait runs out the CTA records
 // CAMERA_ERR_DEVICE_TIMEOUT in the status word, lets its copies land, frees its tensor memory and
@@ -27,15 +27,16 @@ namespace camera {
 namespace {
 
 constexpr int U_THREADS = 192;
-constexpr int U_STAGES = 4;
+constexpr int U_STAGES = 3;
 constexpr int U_BK = 64;                         // bf16 elements per k-block = one 128-byte swizzle row
-constexpr int U_A_BYTES = 128 * 128;             // 128 weight rows x 128 B
+constexpr int U_A_BYTES = CH_TILE * 128;         // 128 weight rows x 128 B (one of gate / up)
 constexpr int U_B_BYTES = UMMA_TOK * 128;        // 256 token rows x 128 B
-constexpr int U_STAGE_BYTES = U_A_BYTES + U_B_BYTES;
+constexpr int U_STAGE_BYTES = 2 * U_A_BYTES + U_B_BYTES;
 constexpr int U_TMEM_COLS = 512;
-constexpr int U_WBUF_BYTES = 4 * 2 * UMMA_TOK * 4;    // router weights of a token tile: per epilogue warp, double-buffered
+constexpr int U_WBUF_BYTES = 4 * UMMA_TOK * 4;   // router weights of a token tile, one copy per epilogue warp
 constexpr int U_SMEM_BYTES = U_STAGES * U_STAGE_BYTES + U_WBUF_BYTES + 256 + 1024;
 constexpr unsigned long long U_WAIT_LIMIT_NS = 4000000000ull;
+static_assert(CH_TILE == 128, "one micro-expert per TMEM lane");
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
 
@@ -130,6 +131,8 @@ __device__ __forceinline__ void umma_commit(uint32_t bar) {
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
 
+// 16 consecutive accumulator columns of this thread's TMEM lane.  The registers hold the values only
+// after tmem_ld_wait, which names them so that no use can be scheduled ahead of it.
 __device__ __forceinline__ void tmem_ld16(uint32_t taddr, uint32_t* v) {
   asm volatile(
       "tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15}, [%16];"
@@ -138,20 +141,46 @@ __device__ __forceinline__ void tmem_ld16(uint32_t taddr, uint32_t* v) {
       : "r"(taddr)
       : "memory");
 }
-__device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
+__device__ __forceinline__ void tmem_ld_wait(uint32_t* a, uint32_t* b) {
+  asm volatile("tcgen05.wait::ld.sync.aligned;"
+               : "+r"(a[0]), "+r"(a[1]), "+r"(a[2]), "+r"(a[3]), "+r"(a[4]), "+r"(a[5]), "+r"(a[6]), "+r"(a[7]),
+                 "+r"(a[8]), "+r"(a[9]), "+r"(a[10]), "+r"(a[11]), "+r"(a[12]), "+r"(a[13]), "+r"(a[14]), "+r"(a[15]),
+                 "+r"(b[0]), "+r"(b[1]), "+r"(b[2]), "+r"(b[3]), "+r"(b[4]), "+r"(b[5]), "+r"(b[6]), "+r"(b[7]),
+                 "+r"(b[8]), "+r"(b[9]), "+r"(b[10]), "+r"(b[11]), "+r"(b[12]), "+r"(b[13]), "+r"(b[14]), "+r"(b[15])
+               :
+               : "memory");
+}
+
+// lambda = a_t * SiLU(g) * u for 16 tokens of this thread's micro-expert; folds lambda^2 and |lambda|.
+__device__ __forceinline__ void fold16(const uint32_t* vg, const uint32_t* vu, const float* wb, float& s, float& m) {
+  float a[16];
+#pragma unroll
+  for (int q = 0; q < 4; ++q) {
+    const float4 w4 = *reinterpret_cast<const float4*>(wb + 4 * q);
+    a[4 * q] = w4.x; a[4 * q + 1] = w4.y; a[4 * q + 2] = w4.z; a[4 * q + 3] = w4.w;
+  }
+#pragma unroll
+  for (int j = 0; j < 16; ++j) {
+    const float g = __uint_as_float(vg[j]), up = __uint_as_float(vu[j]);
+    const float sig = __fdividef(1.f, 1.f + __expf(-g));
+    const float lam = (a[j] * up) * (g * sig);
+    s = fmaf(lam, lam, s);
+    m = fmaxf(m, fabsf(lam));
+  }
+}
 
 __global__ void __launch_bounds__(U_THREADS, 1) k_score_umma(const ScoreCtx c) {
   extern __shared__ uint8_t smem_raw[];
   const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
   uint8_t* const base_ptr = smem_raw + (base - smem_u32(smem_raw));
-  // [stages: A | B] [wbuf 4 warps x 2 x 256 floats] [barriers] [tmem slot] [abort flag]
+  // [stages: A_gate | A_up | B] [wbuf 4 warps x 256 floats] [barriers] [tmem slot] [abort flag]
   float* const wbuf = reinterpret_cast<float*>(base_ptr + U_STAGES * U_STAGE_BYTES);
   const uint32_t bars = base + U_STAGES * U_STAGE_BYTES + U_WBUF_BYTES;
   auto full_bar = [&](int s) { return bars + 8u * s; };
   auto empty_bar = [&](int s) { return bars + 8u * (U_STAGES + s); };
-  auto tfull_bar = [&](int a) { return bars + 8u * (2 * U_STAGES + a); };
-  auto tempty_bar = [&](int a) { return bars + 8u * (2 * U_STAGES + 2 + a); };
-  uint8_t* const tail = base_ptr + U_STAGES * U_STAGE_BYTES + U_WBUF_BYTES + 8 * (2 * U_STAGES + 4);
+  const uint32_t tfull_bar = bars + 8u * (2 * U_STAGES);
+  const uint32_t tempty_bar = bars + 8u * (2 * U_STAGES + 1);
+  uint8_t* const tail = base_ptr + U_STAGES * U_STAGE_BYTES + U_WBUF_BYTES + 8 * (2 * U_STAGES + 2);
   volatile uint32_t* const tmem_slot = reinterpret_cast<volatile uint32_t*>(tail);
   volatile int* const abort_flag = reinterpret_cast<volatile int*>(tail + 8);
 
@@ -161,7 +190,8 @@ __global__ void __launch_bounds__(U_THREADS, 1) k_score_umma(const ScoreCtx c) {
 
   if (tid == 0) {
     for (int s = 0; s < U_STAGES; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
-    for (int a = 0; a < 2; ++a) { mbar_init(tfull_bar(a), 1); mbar_init(tempty_bar(a), 128); }
+    mbar_init(tfull_bar, 1);
+    mbar_init(tempty_bar, 128);
     *abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
@@ -198,14 +228,11 @@ __global__ void __launch_bounds__(U_THREADS, 1) k_score_umma(const ScoreCtx c) {
           for (int kb = 0; kb < n_kb; ++kb) {
             if (!mbar_wait(empty_bar(stage), phase ^ 1u, abort_flag)) { ok = false; break; }
             const uint32_t a_dst = base + stage * U_STAGE_BYTES;
-            const uint32_t b_dst = a_dst + U_A_BYTES;
             mbar_expect_tx(full_bar(stage), U_STAGE_BYTES);
-#pragma unroll
-            for (int q = 0; q < 4; ++q) {
-              tma_load_2d(a_dst + q * 4096, map_g, full_bar(stage), kb * U_BK, u.ch0 + q * 16);
-              tma_load_2d(a_dst + q * 4096 + 2048, map_u, full_bar(stage), kb * U_BK, u.ch0 + q * 16);
-            }
-            tma_load_2d(b_dst, map_x, full_bar(stage), kb * U_BK, row);
+            // weight rows past d_ff and token rows past the tensor are filled with zeros
+            tma_load_2d(a_dst, map_g, full_bar(stage), kb * U_BK, u.ch0);
+            tma_load_2d(a_dst + U_A_BYTES, map_u, full_bar(stage), kb * U_BK, u.ch0);
+            tma_load_2d(a_dst + 2 * U_A_BYTES, map_x, full_bar(stage), kb * U_BK, row);
             if (++stage == U_STAGES) { stage = 0; phase ^= 1u; }
           }
         }
@@ -219,8 +246,8 @@ __global__ void __launch_bounds__(U_THREADS, 1) k_score_umma(const ScoreCtx c) {
   } else if (warp == 5) {
     // ------------------------------------------------------------------ MMA issuer
     if (lane == 0) {
-      int stage = 0, acc = 0;
-      uint32_t phase = 0, acc_phase = 0;
+      int stage = 0;
+      uint32_t phase = 0, tile_phase = 0;
       bool ok = true;
       for (int unit = blockIdx.x; ok && unit < total_units; unit += gridDim.x) {
         const UnitInfo u = decode_unit(c, unit);
@@ -228,33 +255,38 @@ __global__ void __launch_bounds__(U_THREADS, 1) k_score_umma(const ScoreCtx c) {
         for (int tt = 0; ok && tt < n_tiles; ++tt) {
           const int nv = (min(UMMA_TOK, u.rows - tt * UMMA_TOK) + 15) & ~15;
           const uint32_t idesc = make_idesc(nv);
-          if (!mbar_wait(tempty_bar(acc), acc_phase ^ 1u, abort_flag)) { ok = false; break; }
+          // both accumulators are free again once the epilogue has read the previous tile out
+          if (!mbar_wait(tempty_bar, tile_phase ^ 1u, abort_flag)) { ok = false; break; }
           tc_fence_after();
-          const uint32_t d_tmem = tmem_base + (uint32_t)(acc * UMMA_TOK);
           for (int kb = 0; kb < n_kb; ++kb) {
             if (!mbar_wait(full_bar(stage), phase, abort_flag)) { ok = false; break; }
             tc_fence_after();
             const uint32_t a_addr = base + stage * U_STAGE_BYTES;
-            const unsigned long long a_desc = make_smem_desc(a_addr);
-            const unsigned long long b_desc = make_smem_desc(a_addr + U_A_BYTES);
+            const unsigned long long g_desc = make_smem_desc(a_addr);
+            const unsigned long long u_desc = make_smem_desc(a_addr + U_A_BYTES);
+            const unsigned long long b_desc = make_smem_desc(a_addr + 2 * U_A_BYTES);
 #pragma unroll
-            for (int k = 0; k < U_BK / 16; ++k)   // 16 bf16 = 32 bytes per MMA along K: +2 in 16-byte units
-              umma_bf16(d_tmem, a_desc + 2 * k, b_desc + 2 * k, idesc, (uint32_t)((kb | k) != 0));
+            for (int k = 0; k < U_BK / 16; ++k) {   // 16 bf16 = 32 bytes per MMA along K: +2 in 16-byte units
+              const uint32_t acc = (uint32_t)((kb | k) != 0);
+              umma_bf16(tmem_base, g_desc + 2 * k, b_desc + 2 * k, idesc, acc);
+              umma_bf16(tmem_base + UMMA_TOK, u_desc + 2 * k, b_desc + 2 * k, idesc, acc);
+            }
             umma_commit(empty_bar(stage));
             if (++stage == U_STAGES) { stage = 0; phase ^= 1u; }
           }
           if (!ok) break;
-          umma_commit(tfull_bar(acc));
-          if (++acc == 2) { acc = 0; acc_phase ^= 1u; }
+          umma_commit(tfull_bar);
+          tile_phase ^= 1u;
         }
       }
     }
   } else {
     // ------------------------------------------------------------------ epilogue (warps 0-3)
-    int acc = 0;
-    uint32_t acc_phase = 0;
+    uint32_t tile_phase = 0;
     bool ok = true;
-    const bool lo = lane < 16;
+    float* const wb = wbuf + warp * UMMA_TOK;
+    const uint32_t t_gate = tmem_base + ((uint32_t)(warp * 32) << 16);
+    const uint32_t t_up = t_gate + UMMA_TOK;
     for (int unit = blockIdx.x; ok && unit < total_units; unit += gridDim.x) {
       const UnitInfo u = decode_unit(c, unit);
       const int n_tiles = (u.rows + UMMA_TOK - 1) / UMMA_TOK;
@@ -263,44 +295,37 @@ __global__ void __launch_bounds__(U_THREADS, 1) k_score_umma(const ScoreCtx c) {
       for (int tt = 0; ok && tt < n_tiles; ++tt) {
         const int valid = min(UMMA_TOK, u.rows - tt * UMMA_TOK);
         const int nv = (valid + 15) & ~15;
-        // each warp stages the tile's router weights for itself, so the four warps never wait on
-        // one another and a wait that runs out can be left warp by warp
-        float* wb = wbuf + (warp * 2 + acc) * UMMA_TOK;
+        // each warp stages the tile's router weights for itself (while the MMAs of the tile run), so
+        // the four warps never wait on one another and a wait that runs out can be left warp by warp
+        __syncwarp();
         for (int i = lane; i < UMMA_TOK; i += 32) wb[i] = i < valid ? wsrc[tt * UMMA_TOK + i] : 0.f;
         __syncwarp();
-        ok = __all_sync(0xffffffffu, mbar_wait(tfull_bar(acc), acc_phase, abort_flag));
+        ok = __all_sync(0xffffffffu, mbar_wait(tfull_bar, tile_phase, abort_flag));
         if (!ok) break;
         tc_fence_after();
-        const uint32_t taddr = tmem_base + ((uint32_t)(warp * 32) << 16) + (uint32_t)(acc * UMMA_TOK);
-        for (int c0 = 0; c0 < nv; c0 += 16) {
-          uint32_t v[16];
-          tmem_ld16(taddr + c0, v);
-          tmem_ld_wait();
-#pragma unroll
-          for (int j = 0; j < 8; ++j) {
-            const float even = __uint_as_float(v[2 * j]), odd = __uint_as_float(v[2 * j + 1]);
-            const float recv = __shfl_xor_sync(0xffffffffu, lo ? odd : even, 16);
-            const float g = lo ? even : recv;
-            const float up = lo ? recv : odd;
-            const float a = wb[c0 + 2 * j + (lo ? 0 : 1)];
-            const float sig = __fdividef(1.f, 1.f + __expf(-g));
-            const float lam = a * (g * sig) * up;
-            s = fmaf(lam, lam, s);
-            m = fmaxf(m, fabsf(lam));
+        // two register sets alternate: the loads of the next 16 columns fly while these are folded
+        uint32_t g0[16], u0[16], g1[16], u1[16];
+        tmem_ld16(t_gate, g0);
+        tmem_ld16(t_up, u0);
+        for (int c0 = 0; c0 < nv; c0 += 32) {
+          tmem_ld_wait(g0, u0);
+          if (c0 + 16 < nv) { tmem_ld16(t_gate + c0 + 16, g1); tmem_ld16(t_up + c0 + 16, u1); }
+          fold16(g0, u0, wb + c0, s, m);
+          if (c0 + 16 < nv) {
+            tmem_ld_wait(g1, u1);
+            if (c0 + 32 < nv) { tmem_ld16(t_gate + c0 + 32, g0); tmem_ld16(t_up + c0 + 32, u0); }
+            fold16(g1, u1, wb + c0 + 16, s, m);
           }
         }
         tc_fence_before();
-        mbar_arrive(tempty_bar(acc));
-        if (++acc == 2) { acc = 0; acc_phase ^= 1u; }
+        mbar_arrive(tempty_bar);
+        tile_phase ^= 1u;
       }
-      if (ok) {
-        s += __shfl_xor_sync(0xffffffffu, s, 16);
-        m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, 16));
-        if (lo) {
-          const size_t slot = (size_t)u.part_slot + warp * 16 + lane;
-          c.part_sum[slot] = s;
-          c.part_max[slot] = m;
-        }
+      const int ch = u.ch0 + warp * 32 + lane;
+      if (ok && ch < u.f) {
+        const size_t slot = (size_t)u.part_slot + warp * 32 + lane;
+        c.part_sum[slot] = s;
+        c.part_max[slot] = m;
       }
     }
   }
@@ -351,7 +376,6 @@ bool encode_2d(EncodeTiledFn fn, void* out, const void* ptr, uint64_t rows, uint
 bool umma_shape_ok(const camera_layer_t* L) {
   if (L->dtype != CAMERA_BF16 || L->d_model % U_BK != 0) return false;
   for (int e = 0; e < L->n_routed + L->n_shared; ++e) {
-    if (L->d_ff[e] % CH_TILE != 0) return false;
     if ((reinterpret_cast<uintptr_t>(L->w_gate[e]) & 15) || (reinterpret_cast<uintptr_t>(L->w_up[e]) & 15)) return false;
   }
   return true;
@@ -364,8 +388,8 @@ int encode_tensor_maps(const camera_layer_t* L, const ScoreCtx& c, void* host_ma
   char* out = static_cast<char*>(host_maps);
   const int E = c.n_experts;
   for (int e = 0; e < E; ++e) {
-    if (!encode_2d(fn, out + (size_t)128 * (2 * e), L->w_gate[e], (uint64_t)L->d_ff[e], (uint64_t)c.d_model, 16) ||
-        !encode_2d(fn, out + (size_t)128 * (2 * e + 1), L->w_up[e], (uint64_t)L->d_ff[e], (uint64_t)c.d_model, 16))
+    if (!encode_2d(fn, out + (size_t)128 * (2 * e), L->w_gate[e], (uint64_t)L->d_ff[e], (uint64_t)c.d_model, CH_TILE) ||
+        !encode_2d(fn, out + (size_t)128 * (2 * e + 1), L->w_up[e], (uint64_t)L->d_ff[e], (uint64_t)c.d_model, CH_TILE))
       return CAMERA_ERR_CUDA;
   }
   if (!encode_2d(fn, out + (size_t)128 * (2 * E), c.x_perm, (uint64_t)(c.max_rows_perm > 0 ? c.max_rows_perm : 1),
