@@ -121,7 +121,7 @@ ScoreLayout score_layout(const camera_layer_t* L, int64_t T) {
   s.phi2 = take(sizeof(float) * (size_t)n_me);
   s.phi_inf_sq = take(sizeof(float) * (size_t)n_me);
   s.omega2 = take(sizeof(float) * (size_t)n_me);
-  s.tensor_maps = take((size_t)128 * (2 * E + 2));
+  s.tensor_maps = take((size_t)128 * (2 * E + N_EXTRA_MAPS));
   s.total = o;
   return s;
 }
@@ -243,10 +243,12 @@ extern "C" int camera_score_layer(const camera_layer_t* L, const void* x, int64_
 
   const bool use_umma = umma_shape_ok(L) && !(aux && (aux->flags & CAMERA_SCORE_FORCE_SIMT)) &&
                         (reinterpret_cast<uintptr_t>(x) & 15) == 0;
+  const bool use_router_umma = use_umma && router_umma_ok(c);
   std::vector<char> maps;
   if (use_umma) {
-    maps.resize((size_t)128 * (2 * E + 2));
+    maps.resize((size_t)128 * (2 * E + N_EXTRA_MAPS));
     rc = encode_tensor_maps(L, c, maps.data());
+    if (rc == CAMERA_OK && use_router_umma) rc = encode_router_maps(c, maps.data());
     if (rc != CAMERA_OK) return rc;
   }
 
@@ -258,8 +260,13 @@ extern "C" int camera_score_layer(const camera_layer_t* L, const void* x, int64_
 
   const StageTimer tm{aux, st};
   tm.begin(CAMERA_STAGE_ROUTER);
-  if (aux && aux->topk_idx_in) CK(launch_routing_from_input(c, aux->topk_idx_in, aux->topk_w_in, st));
-  else CK(launch_router(c, st));
+  {
+    const int32_t* idx_in = aux ? aux->topk_idx_in : nullptr;
+    const float* w_in = aux ? aux->topk_w_in : nullptr;
+    if (use_router_umma) CK(launch_router_umma(c, idx_in, w_in, st));
+    else if (idx_in) CK(launch_routing_from_input(c, idx_in, w_in, st));
+    else CK(launch_router(c, st));
+  }
   tm.end(CAMERA_STAGE_ROUTER);
 
   tm.begin(CAMERA_STAGE_PERMUTE);

@@ -10,13 +10,14 @@
 namespace camera {
 
 // ---- tiling constants shared by the host planner and the kernels -----------------------------
-constexpr int ROUTER_TOK = 64;       // tokens per router CTA (also the unit of the stable counting sort)
+constexpr int ROUTER_TOK = 32;       // tokens per block of the stable counting sort
 constexpr int ROW_ALIGN = 16;        // every expert's token list is padded to this many rows
 constexpr int CH_TILE = 128;         // micro-experts (channels) per scoring work unit
 constexpr int UMMA_TOK = 256;        // tokens per tensor-core tile (the MMA's N)
 constexpr int MAX_ROUTED = 256;
 constexpr int MAX_TOPK = 16;
 constexpr int MAX_LEVELS = 8;
+constexpr int N_EXTRA_MAPS = 5;
 
 // Host-known facts about one expert; copied to the device on every call.
 struct ExpertStatic {
@@ -80,7 +81,8 @@ struct ScoreCtx {
   float* phi_inf_sq;     // [n_me]
   float* omega2;         // [n_me]
   float* energy;         // [n_me]
-  void* tensor_maps;     // CUtensorMap[2 * n_experts + 2]
+  void* tensor_maps;     // CUtensorMap[2 * n_experts + N_EXTRA_MAPS]: gate, up per expert; x_perm, x (scoring);
+                         // x, w_router, w_shared_gate (router)
 };
 
 // ---- launches (each enqueues on `st`, returns the launch's cudaError_t) ------------------------
@@ -92,8 +94,14 @@ cudaError_t launch_rownorm(const ScoreCtx& c, int n_norm_blocks, cudaStream_t st
 cudaError_t launch_score_simt(const ScoreCtx& c, cudaStream_t st);
 cudaError_t launch_score_umma(const ScoreCtx& c, cudaStream_t st);
 cudaError_t launch_combine(const ScoreCtx& c, cudaStream_t st);
+cudaError_t launch_router_umma(const ScoreCtx& c, const int32_t* idx_in, const float* w_in, cudaStream_t st);
 bool umma_shape_ok(const camera_layer_t* L);
+bool router_umma_ok(const ScoreCtx& c);
 int encode_tensor_maps(const camera_layer_t* L, const ScoreCtx& c, void* host_maps /* 128 B each */);
+int encode_router_maps(const ScoreCtx& c, void* host_maps);
+// Tensor map of a bf16 row-major [rows, d] matrix in boxes of 64 columns x box_rows rows with the
+// 128-byte swizzle (a null matrix gives an all-zero map that must not be used).
+bool encode_bf16_2d(void* out, const void* ptr, uint64_t rows, uint64_t d, uint32_t box_rows);
 
 // ---- device helpers ------------------------------------------------------------------------------
 template <typename T> __device__ __forceinline__ float to_f32(T v);

@@ -7,9 +7,10 @@ namespace camera {
 namespace {
 
 constexpr int RT_THREADS = 256;
+constexpr int RT_TOK = 64;           // tokens per CTA = RT_TOK / ROUTER_TOK blocks of the counting sort
 constexpr int RT_KC = 32;            // k-chunk of the logit GEMM
 constexpr int RT_COLS = 64;          // logit columns per pass
-constexpr int RT_LD = ROUTER_TOK + 4;
+constexpr int RT_LD = RT_TOK + 4;
 
 __device__ __forceinline__ float warp_max(float v) {
 #pragma unroll
@@ -22,7 +23,7 @@ __device__ __forceinline__ float warp_sum(float v) {
   return v;
 }
 
-// One CTA = ROUTER_TOK consecutive tokens.  Logits z = x . w (+bias) in fp32 FMA over all routed
+// One CTA = RT_TOK consecutive tokens.  Logits z = x . w (+bias) in fp32 FMA over all routed
 // experts and the sigmoid-gated shared experts; softmax over the routed ones; the top_k largest
 // logits are kept (equal logits: lower expert first); weights are the softmax probabilities,
 // divided by their sum under CAMERA_ROUTER_NORM_TOPK.  Also emits, for the counting sort, each
@@ -36,13 +37,12 @@ __global__ void __launch_bounds__(RT_THREADS) k_router(ScoreCtx c, const int32_t
   const int ldl = nc_pad + 1;
   float* Xs = smem;                              // [RT_KC][RT_LD]
   float* Ws = Xs + RT_KC * RT_LD;                // [RT_KC][RT_LD]
-  float* logits = Ws + RT_KC * RT_LD;            // [ROUTER_TOK][ldl]
-  int* sel_e = reinterpret_cast<int*>(logits + ROUTER_TOK * ldl);  // [ROUTER_TOK * top_k]
+  float* logits = Ws + RT_KC * RT_LD;            // [RT_TOK][ldl]
+  int* sel_e = reinterpret_cast<int*>(logits + RT_TOK * ldl);  // [RT_TOK * top_k]
 
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int tx = tid & 15, ty = tid >> 4;
-  const int blk = blockIdx.x;
-  const int tok0 = blk * ROUTER_TOK;
+  const int tok0 = blockIdx.x * RT_TOK;
   const int d = c.d_model;
   const T* X = static_cast<const T*>(c.x);
   constexpr int VN = Vec16<T>::N;
@@ -57,7 +57,7 @@ __global__ void __launch_bounds__(RT_THREADS) k_router(ScoreCtx c, const int32_t
 
     for (int k0 = 0; k0 < d; k0 += RT_KC) {
       __syncthreads();
-      for (int v = tid; v < ROUTER_TOK * VPR; v += RT_THREADS) {
+      for (int v = tid; v < RT_TOK * VPR; v += RT_THREADS) {
         const int row = v / VPR, kv = (v % VPR) * VN;
         float f[VN];
 #pragma unroll
@@ -102,8 +102,8 @@ __global__ void __launch_bounds__(RT_THREADS) k_router(ScoreCtx c, const int32_t
   __syncthreads();
 
   // coefficients of the shared experts: 1, or sigmoid of their gate logit
-  for (int i = tid; i < ROUTER_TOK * c.n_shared; i += RT_THREADS) {
-    const int s = i / ROUTER_TOK, tl = i % ROUTER_TOK, t = tok0 + tl;
+  for (int i = tid; i < RT_TOK * c.n_shared; i += RT_THREADS) {
+    const int s = i / RT_TOK, tl = i % RT_TOK, t = tok0 + tl;
     if (t < c.n_tokens) {
       float a = 1.f;
       if (n_gated) a = 1.f / (1.f + expf(-logits[tl * ldl + c.n_routed + s]));
@@ -113,7 +113,7 @@ __global__ void __launch_bounds__(RT_THREADS) k_router(ScoreCtx c, const int32_t
 
   const int k = c.top_k;
   if (c.n_routed > 0) {
-    for (int tl = warp; tl < ROUTER_TOK; tl += RT_THREADS / 32) {
+    for (int tl = warp; tl < RT_TOK; tl += RT_THREADS / 32) {
       const int t = tok0 + tl;
       if (t >= c.n_tokens) {
         if (lane < k) sel_e[tl * k + lane] = -1;
@@ -177,16 +177,22 @@ __global__ void __launch_bounds__(RT_THREADS) k_router(ScoreCtx c, const int32_t
     __syncthreads();
     // rank of each pair among the pairs of the same expert in this block, in (token, slot) order
     const int npairs = ROUTER_TOK * k;
-    for (int e = warp; e < c.n_routed; e += RT_THREADS / 32) {
-      int run = 0;
-      for (int base = 0; base < npairs; base += 32) {
-        const int p = base + lane;
-        const bool m = (p < npairs) && (sel_e[p] == e);
-        const unsigned b = __ballot_sync(0xffffffffu, m);
-        if (m) c.local_rank[(size_t)tok0 * k + p] = run + __popc(b & ((1u << lane) - 1u));
-        run += __popc(b);
+    for (int sb = 0; sb < RT_TOK / ROUTER_TOK; ++sb) {
+      const int blk = blockIdx.x * (RT_TOK / ROUTER_TOK) + sb;
+      if (blk >= c.n_blocks) break;
+      const int* sel_b = sel_e + sb * npairs;
+      int32_t* rank_b = c.local_rank + (size_t)(tok0 + sb * ROUTER_TOK) * k;
+      for (int e = warp; e < c.n_routed; e += RT_THREADS / 32) {
+        int run = 0;
+        for (int base = 0; base < npairs; base += 32) {
+          const int p = base + lane;
+          const bool m = (p < npairs) && (sel_b[p] == e);
+          const unsigned b = __ballot_sync(0xffffffffu, m);
+          if (m) rank_b[p] = run + __popc(b & ((1u << lane) - 1u));
+          run += __popc(b);
+        }
+        if (lane == 0) c.block_hist[(size_t)blk * c.n_routed + e] = run;
       }
-      if (lane == 0) c.block_hist[(size_t)blk * c.n_routed + e] = run;
     }
   }
 }
@@ -299,7 +305,7 @@ size_t router_smem_bytes(const ScoreCtx& c) {
   const int n_gated = (c.flags & CAMERA_SHARED_GATE_SIGMOID) ? c.n_shared : 0;
   const int nc = c.n_routed + n_gated;
   const int nc_pad = ((nc + RT_COLS - 1) / RT_COLS) * RT_COLS;
-  return sizeof(float) * (2 * RT_KC * RT_LD + ROUTER_TOK * (nc_pad + 1)) + sizeof(int) * ROUTER_TOK * MAX_TOPK;
+  return sizeof(float) * (2 * RT_KC * RT_LD + RT_TOK * (nc_pad + 1)) + sizeof(int) * RT_TOK * MAX_TOPK;
 }
 
 }  // namespace
@@ -307,14 +313,15 @@ size_t router_smem_bytes(const ScoreCtx& c) {
 cudaError_t launch_routing_from_input(const ScoreCtx& c, const int32_t* idx_in, const float* w_in, cudaStream_t st) {
   if (c.n_blocks == 0) return cudaSuccess;
   const size_t smem = router_smem_bytes(c);
+  const int grid = (c.n_tokens + RT_TOK - 1) / RT_TOK;
   if (c.dtype == CAMERA_BF16) {
     cudaError_t e = cudaFuncSetAttribute(k_router<__nv_bfloat16>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;
-    k_router<__nv_bfloat16><<<c.n_blocks, RT_THREADS, smem, st>>>(c, idx_in, w_in);
+    k_router<__nv_bfloat16><<<grid, RT_THREADS, smem, st>>>(c, idx_in, w_in);
   } else {
     cudaError_t e = cudaFuncSetAttribute(k_router<float>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;
-    k_router<float><<<c.n_blocks, RT_THREADS, smem, st>>>(c, idx_in, w_in);
+    k_router<float><<<grid, RT_THREADS, smem, st>>>(c, idx_in, w_in);
   }
   return cudaGetLastError();
 }
