@@ -10,6 +10,9 @@ REL_TOL = 1e-3          # scores: fp32 accumulation of bf16/fp32 products agains
 FLOOR = 1e-6            # ... relative to max(|ref_i|, FLOOR * max|ref|): a micro-expert a million times below the
                         # layer's largest score is dominated by the absolute rounding error of its fp32 dot products
 TIE_TOL = 1e-5          # routing: relative gap of the k-th and (k+1)-th probability below which either is right
+W_TOL = 1e-4            # router / shared-gate coefficients: a logit is an fp32 sum of d_model products of size ~1
+                        # (absolute error up to ~d_model * 2^-24 = 2e-4 at d_model 3584, observed 3e-5), and softmax and
+                        # sigmoid pass an absolute logit error on as a relative error of at most the same size
 
 
 def assert_close(name, got, ref, rel=REL_TOL):
@@ -45,7 +48,7 @@ def check_routing(olayer, Xd, topk_idx, topk_w):
     order_g, order_o = np.argsort(gi, axis=1), np.argsort(idx_o, axis=1)
     wg = np.take_along_axis(gw, order_g, axis=1)[same]
     wo = np.take_along_axis(w_o, order_o, axis=1)[same]
-    assert np.abs(wg - wo).max() <= 2e-5 * max(1.0, np.abs(wo).max()), "router weights differ"
+    assert np.abs(wg - wo).max() <= W_TOL * max(1.0, np.abs(wo).max()), "router weights differ"
     # order of the exported slots: decreasing probability
     assert (np.diff(gw, axis=1) <= 1e-6).all()
     return int((~same).sum())
@@ -68,7 +71,7 @@ def run_and_compare(P, L, X, alpha=0.95, channels=None, force_simt=False, check_
         routing = (out["topk_idx"].cpu().numpy().astype(np.int64), out["topk_w"].cpu().numpy().astype(np.float64))
     shared_w = out["shared_w"].cpu().numpy().astype(np.float64).T
     if olayer.n_shared:
-        assert_close("shared_w", shared_w, O.shared_coeff(olayer, Xd), rel=2e-5)
+        assert_close("shared_w", shared_w, O.shared_coeff(olayer, Xd), rel=W_TOL)
     phi2, phi_inf, omega2 = O.camera_components(olayer, Xd, channels=channels, routing=routing)
     sel = ~np.isnan(phi2)
     assert_close("omega2", out["omega2"].cpu().numpy(), omega2)
