@@ -181,6 +181,7 @@ def main():
     ap.add_argument("--routed", type=int, default=0, help="override the number of routed experts (profiling slices)")
     ap.add_argument("--topk", type=int, default=0, help="override top-k (with --routed and --tokens: a slice that keeps the full layer's tokens per expert)")
     ap.add_argument("--oracle-tokens", type=int, default=0, help="tokens of the CPU-oracle sample (default 512 for --impl reference, 2048 for the cpu_baseline leg)")
+    ap.add_argument("--cta-pair", action="store_true", help="score on CTA pairs (tcgen05 cta_group::2) instead of single CTAs")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     args = ap.parse_args()
@@ -222,7 +223,8 @@ def main():
     stream = torch.cuda.current_stream()
 
     def step(i, events=None):
-        P.camera_score_layer(layer, Xs[i % 2], ALPHA, energy=energy, workspace=ws_score, stage_events=events)
+        P.camera_score_layer(layer, Xs[i % 2], ALPHA, energy=energy, workspace=ws_score, stage_events=events,
+                             cta_pair=args.cta_pair)
         for j, r in enumerate(PRUNE_RATIOS):
             P.camera_select_prune(energy, r, workspace=ws_sel, keep_mask=keep[j])
         P.camera_alloc_bits(energy, BIT_RATIOS, BIT_LEVELS, workspace=ws_sel, bits_out=bits)

@@ -58,7 +58,9 @@ enum {
 
 /* camera_score_aux_t.flags */
 enum {
-  CAMERA_SCORE_FORCE_SIMT = 1u     /* run the fp32-FMA scoring kernel even where the tensor-core kernel applies */
+  CAMERA_SCORE_FORCE_SIMT = 1u,    /* run the fp32-FMA kernels even where the tensor-core kernels apply */
+  CAMERA_SCORE_CTA_PAIR = 2u       /* tensor-core scoring on CTA pairs (tcgen05 cta_group::2): less L2 and shared-memory
+                                      traffic per flop, but measured slower under the power cap; off by default */
 };
 
 /* Stages of camera_score_layer, for the optional timing events. */

@@ -19,6 +19,7 @@ CAMERA_F32, CAMERA_BF16 = 0, 1
 CAMERA_DOWN_HF, CAMERA_DOWN_ME_MAJOR = 0, 1
 CAMERA_ROUTER_NORM_TOPK, CAMERA_SHARED_GATE_SIGMOID = 1, 2
 CAMERA_SCORE_FORCE_SIMT = 1
+CAMERA_SCORE_CTA_PAIR = 2
 STAGES = ("router", "permute", "rownorm", "score", "combine")
 
 
@@ -167,7 +168,7 @@ def alloc_workspace(nbytes: int, device) -> torch.Tensor:
 
 def camera_score_layer(layer: Layer, x: torch.Tensor, alpha: float, *, energy: Optional[torch.Tensor] = None,
                        workspace: Optional[torch.Tensor] = None, details: bool = False,
-                       routing_in=None, force_simt: bool = False, stage_events=None,
+                       routing_in=None, force_simt: bool = False, cta_pair: bool = False, stage_events=None,
                        stream: Optional[torch.cuda.Stream] = None, check_status: bool = False):
     """Algorithm 1 up to the energies.  Returns energy [N_e] fp32, or with details=True a dict that
     also holds phi2, phi_inf_sq, omega2, topk_idx, topk_w, shared_w and expert_token_counts.
@@ -201,8 +202,7 @@ def camera_score_layer(layer: Layer, x: torch.Tensor, alpha: float, *, energy: O
         w = w.to(device=dev, dtype=torch.float32).contiguous()
         keep_alive += [idx, w]
         aux.topk_idx_in, aux.topk_w_in = idx.data_ptr(), w.data_ptr()
-    if force_simt:
-        aux.flags = CAMERA_SCORE_FORCE_SIMT
+    aux.flags = (CAMERA_SCORE_FORCE_SIMT if force_simt else 0) | (CAMERA_SCORE_CTA_PAIR if cta_pair else 0)
     if stage_events:
         for name, (e0, e1) in stage_events.items():
             i = STAGES.index(name)

@@ -17,17 +17,17 @@ constexpr int PLAN_SMS = 148;   // used only to size work units; the result is v
 
 size_t up256(size_t v) { return (v + 255) & ~(size_t)255; }
 
-// Channel tiles per scheduling group.  20 tiles = 2560 micro-experts: 37 MB of gate+up rows at
-// d_model 3584, which stay in L2 while the concurrent CTAs walk down the expert's token list
-// (measured on the Qwen2-shaped layer: 5 / 10 / 20 / 40 tiles -> 862 / 991 / 1111 / 1083 TFLOP/s).
-// CAMERA_CT_GROUP overrides it (tuning aid).
-int score_ct_group() {
-  const char* env = getenv("CAMERA_CT_GROUP");
+// Micro-experts per scheduling group.  2560 of them are 37 MB of gate+up rows at d_model 3584,
+// which stay in L2 while the concurrent CTAs walk down the expert's token list (measured on the
+// Qwen2-shaped layer: 640 / 1280 / 2560 / 5120 -> 862 / 991 / 1111 / 1083 TFLOP/s).
+// CAMERA_GROUP_CHANNELS overrides it (tuning aid).
+int score_group_channels() {
+  const char* env = getenv("CAMERA_GROUP_CHANNELS");
   if (env != nullptr) {
     const int v = atoi(env);
-    if (v >= 1 && v <= 4096) return v;
+    if (v >= 256 && v <= (1 << 20)) return v;
   }
-  return 20;
+  return 2560;
 }
 
 struct ScoreLayout {
@@ -202,7 +202,7 @@ extern "C" int camera_score_layer(const camera_layer_t* L, const void* x, int64_
   c.d_model = L->d_model; c.n_routed = L->n_routed; c.top_k = L->n_routed > 0 ? L->top_k : 0;
   c.n_shared = L->n_shared; c.n_experts = E; c.n_me = lay.n_me;
   c.dtype = L->dtype; c.down_layout = L->down_layout; c.flags = L->flags;
-  c.n_tokens = (int)T; c.n_blocks = lay.n_blocks; c.chunk_tokens = lay.chunk_tokens; c.ct_group = score_ct_group();
+  c.n_tokens = (int)T; c.n_blocks = lay.n_blocks; c.chunk_tokens = lay.chunk_tokens;
   c.max_rows_perm = lay.max_rows_perm; c.max_part = lay.max_part; c.alpha = alpha;
   c.x = x; c.w_router = L->w_router; c.router_bias = L->router_bias; c.w_shared_gate = L->w_shared_gate;
   c.totals = reinterpret_cast<PlanTotals*>(ws + lay.totals);
@@ -243,6 +243,9 @@ extern "C" int camera_score_layer(const camera_layer_t* L, const void* x, int64_
 
   const bool use_umma = umma_shape_ok(L) && !(aux && (aux->flags & CAMERA_SCORE_FORCE_SIMT)) &&
                         (reinterpret_cast<uintptr_t>(x) & 15) == 0;
+  const bool use_pair = use_umma && aux && (aux->flags & CAMERA_SCORE_CTA_PAIR);
+  c.ch_tile = use_pair ? 2 * CH_TILE : CH_TILE;
+  c.ct_group = score_group_channels() / c.ch_tile;
   const bool use_router_umma = use_umma && router_umma_ok(c);
   std::vector<char> maps;
   if (use_umma) {
@@ -280,7 +283,8 @@ extern "C" int camera_score_layer(const camera_layer_t* L, const void* x, int64_
 
   tm.begin(CAMERA_STAGE_SCORE);
   if (T > 0) {
-    if (use_umma) CK(launch_score_umma(c, st));
+    if (use_pair) CK(launch_score_umma_pair(c, st));
+    else if (use_umma) CK(launch_score_umma(c, st));
     else CK(launch_score_simt(c, st));
   }
   tm.end(CAMERA_STAGE_SCORE);

@@ -12,12 +12,12 @@ namespace camera {
 // ---- tiling constants shared by the host planner and the kernels -----------------------------
 constexpr int ROUTER_TOK = 32;       // tokens per block of the stable counting sort
 constexpr int ROW_ALIGN = 16;        // every expert's token list is padded to this many rows
-constexpr int CH_TILE = 128;         // micro-experts (channels) per scoring work unit
+constexpr int CH_TILE = 128;         // micro-experts (channels) per scoring work unit; CTA pairs take 2 * CH_TILE
 constexpr int UMMA_TOK = 256;        // tokens per tensor-core tile (the MMA's N)
 constexpr int MAX_ROUTED = 256;
 constexpr int MAX_TOPK = 16;
 constexpr int MAX_LEVELS = 8;
-constexpr int N_EXTRA_MAPS = 5;
+constexpr int N_EXTRA_MAPS = 6;
 
 // Host-known facts about one expert; copied to the device on every call.
 struct ExpertStatic {
@@ -35,7 +35,7 @@ struct ExpertDyn {
   int32_t row_base;      // first row of this expert's token list (in x_perm for routed, in x for shared)
   int32_t rows;          // tokens the expert sees
   int32_t n_chunks;      // ceil(rows / chunk_tokens)
-  int32_t unit_begin;    // exclusive prefix over experts of n_chunks * (d_ff / CH_TILE)
+  int32_t unit_begin;    // exclusive prefix over experts of n_chunks * ceil(d_ff / ch_tile)
   int64_t part_begin;    // exclusive prefix over experts of n_chunks * d_ff (offset into the partials)
 };
 
@@ -53,6 +53,7 @@ struct ScoreCtx {
   uint32_t flags;
   int32_t n_tokens, n_blocks;       // n_blocks = ceil(T / ROUTER_TOK)
   int32_t chunk_tokens;             // tokens per scoring work unit (multiple of UMMA_TOK)
+  int32_t ch_tile;                  // micro-experts per scoring work unit: CH_TILE, or 2 * CH_TILE for CTA pairs
   int32_t ct_group;                 // channel tiles per scheduling group (see decode_unit)
   int32_t max_rows_perm;            // capacity of x_perm in rows
   int64_t max_part;                 // capacity of the partial arrays in floats
@@ -82,7 +83,7 @@ struct ScoreCtx {
   float* omega2;         // [n_me]
   float* energy;         // [n_me]
   void* tensor_maps;     // CUtensorMap[2 * n_experts + N_EXTRA_MAPS]: gate, up per expert; x_perm, x (scoring);
-                         // x, w_router, w_shared_gate (router)
+                         // x, w_router, w_shared_gate (router); x_perm in boxes of 128 rows (CTA pairs)
 };
 
 // ---- launches (each enqueues on `st`, returns the launch's cudaError_t) ------------------------
@@ -93,6 +94,7 @@ cudaError_t launch_permute(const ScoreCtx& c, cudaStream_t st);
 cudaError_t launch_rownorm(const ScoreCtx& c, int n_norm_blocks, cudaStream_t st);
 cudaError_t launch_score_simt(const ScoreCtx& c, cudaStream_t st);
 cudaError_t launch_score_umma(const ScoreCtx& c, cudaStream_t st);
+cudaError_t launch_score_umma_pair(const ScoreCtx& c, cudaStream_t st);
 cudaError_t launch_combine(const ScoreCtx& c, cudaStream_t st);
 cudaError_t launch_router_umma(const ScoreCtx& c, const int32_t* idx_in, const float* w_in, cudaStream_t st);
 bool umma_shape_ok(const camera_layer_t* L);
@@ -141,7 +143,7 @@ __device__ __forceinline__ int upper_segment(const P* prefix, int n, P v) {
   return lo;
 }
 
-// One scoring work unit: CH_TILE channels of one expert against one chunk of its token list.
+// One scoring work unit: ch_tile channels of one expert against one chunk of its token list.
 struct UnitInfo {
   int e, chunk, ch0, f, rows, row0, shared_idx;
   long long part_slot;       // part_begin + chunk * f + ch0
@@ -157,14 +159,14 @@ __device__ __forceinline__ UnitInfo decode_unit(const ScoreCtx& c, int unit) {
   const ExpertDyn dy = c.edyn[u.e];
   u.f = c.est[u.e].d_ff;
   u.shared_idx = c.est[u.e].shared_idx;
-  const int n_ct = (u.f + CH_TILE - 1) / CH_TILE;
+  const int n_ct = (u.f + c.ch_tile - 1) / c.ch_tile;
   int rem = unit - c.unit_prefix[u.e];
   const int per_full_group = dy.n_chunks * c.ct_group;
   const int g = min(rem / per_full_group, (n_ct - 1) / c.ct_group);
   rem -= g * per_full_group;
   const int in_group = min(c.ct_group, n_ct - g * c.ct_group);
   u.chunk = rem / in_group;
-  u.ch0 = (g * c.ct_group + rem % in_group) * CH_TILE;
+  u.ch0 = (g * c.ct_group + rem % in_group) * c.ch_tile;
   const int row_begin = u.chunk * c.chunk_tokens;
   u.rows = min(c.chunk_tokens, dy.rows - row_begin);
   u.row0 = dy.row_base + row_begin;

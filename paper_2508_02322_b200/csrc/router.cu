@@ -247,7 +247,7 @@ __global__ void k_plan(ScoreCtx c) {
     dy.part_begin = part;
     c.edyn[e] = dy;
     c.unit_prefix[e] = units;
-    units += dy.n_chunks * ((f + CH_TILE - 1) / CH_TILE);
+    units += dy.n_chunks * ((f + c.ch_tile - 1) / c.ch_tile);
     part += (long long)dy.n_chunks * f;
   }
   if (row > c.max_rows_perm || part > c.max_part) {

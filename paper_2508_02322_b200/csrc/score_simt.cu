@@ -13,8 +13,8 @@ constexpr int SS_KC = 16;
 constexpr int SS_LD = 68;
 constexpr int SS_CH = 64;           // channels per pass
 
-// Work unit = (expert, tile of CH_TILE channels, chunk of chunk_tokens tokens), handled as
-// CH_TILE / 64 passes of 64 channels.  For every token tile the CTA forms g = W_gate x and
+// Work unit = (expert, tile of ch_tile channels, chunk of chunk_tokens tokens), handled as
+// ch_tile / 64 passes of 64 channels.  For every token tile the CTA forms g = W_gate x and
 // u = W_up x for 64 tokens x 64 channels in fp32,
 // then lambda = a_t * SiLU(g) * u and folds lambda^2 / |lambda| into per-channel running sum / max.
 // One partial (sum, max) per channel and chunk goes to the workspace; chunks are added later in
@@ -32,10 +32,11 @@ __global__ void __launch_bounds__(SS_THREADS) k_score_simt(ScoreCtx c) {
   const int d = c.d_model;
   const int total_units = c.totals->total_units;
 
-  for (int work = blockIdx.x; work < total_units * (CH_TILE / SS_CH); work += gridDim.x) {
-    const UnitInfo u = decode_unit(c, work / (CH_TILE / SS_CH));
+  const int passes = c.ch_tile / SS_CH;
+  for (int work = blockIdx.x; work < total_units * passes; work += gridDim.x) {
+    const UnitInfo u = decode_unit(c, work / passes);
     const ExpertStatic es = c.est[u.e];
-    const int pass_off = (work % (CH_TILE / SS_CH)) * SS_CH;
+    const int pass_off = (work % passes) * SS_CH;
     const int f = u.f, ch0 = u.ch0 + pass_off, rows = u.rows;
     if (ch0 >= f) continue;
     const T* Xsrc = (es.shared_idx < 0 ? static_cast<const T*>(c.x_perm) : static_cast<const T*>(c.x)) +

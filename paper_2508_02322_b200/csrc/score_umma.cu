@@ -291,6 +291,12 @@ int encode_tensor_maps(const camera_layer_t* L, const ScoreCtx& c, void* host_ma
   if (!encode_2d(fn, out + (size_t)128 * (2 * E + 1), c.n_tokens > 0 ? c.x : c.x_perm,
                  (uint64_t)(c.n_tokens > 0 ? c.n_tokens : 1), (uint64_t)c.d_model, UMMA_TOK))
     return CAMERA_ERR_CUDA;
+  // the same two matrices in boxes of 128 rows: each CTA of a pair loads half a token tile
+  if (!encode_2d(fn, out + (size_t)128 * (2 * E + 2), c.n_tokens > 0 ? c.x : c.x_perm,
+                 (uint64_t)(c.n_tokens > 0 ? c.n_tokens : 1), (uint64_t)c.d_model, UMMA_TOK / 2) ||
+      !encode_2d(fn, out + (size_t)128 * (2 * E + 5), c.x_perm, (uint64_t)(c.max_rows_perm > 0 ? c.max_rows_perm : 1),
+                 (uint64_t)c.d_model, UMMA_TOK / 2))
+    return CAMERA_ERR_CUDA;
   return CAMERA_OK;
 }
 

@@ -1,0 +1,283 @@
+// Tensor-core scoring kernel for bf16 layers on CTA pairs (Algorithm 1 lines 6-8).
+//
+// Same computation and the same epilogue as k_score_umma, but two CTAs on neighbouring SMs share one
+// MMA (tcgen05 cta_group::2): the pair handles 256 micro-experts x 256 tokens, each CTA keeps the
+// W_gate / W_up rows of its own 128 micro-experts and only half of the token tile in shared memory,
+// and the tensor cores of both SMs read both halves.  Per k-block a CTA pulls 48 KB from L2 for
+// 8.4 Mflop (64 KB without pairing) and reads a third less operand data from shared memory.
+//
+// Roles per CTA (6 warps): warps 0-3 epilogue, warp 4 lane 0 TMA producer, warp 5 tensor-memory
+// allocation; lane 0 of warp 5 of the pair's first CTA issues the MMAs for both.  Barriers:
+//   full[s]   (first CTA)  bytes of both CTAs' loads of stage s have landed
+//   empty[s]  (each CTA)   the MMAs that read stage s are done           (tcgen05.commit to both CTAs)
+//   tfull     (each CTA)   both accumulators of the tile are complete     (tcgen05.commit to both CTAs)
+//   tempty    (first CTA)  the epilogue threads of both CTAs have read the accumulators out
+// Every wait is bounded, as in k_score_umma.
+#include <string.h>
+
+#include "common.cuh"
+#include "umma.cuh"
+
+namespace camera {
+
+namespace {
+
+constexpr int P_THREADS = 192;
+constexpr int P_STAGES = 4;
+constexpr int P_A_BYTES = 128 * 128;             // 128 weight rows x 128 B (one of gate / up)
+constexpr int P_B_BYTES = 128 * 128;             // this CTA's half of the token tile
+constexpr int P_STAGE_BYTES = 2 * P_A_BYTES + P_B_BYTES;
+constexpr int P_TMEM_COLS = 512;
+constexpr int P_WBUF_BYTES = 4 * UMMA_TOK * 4;
+constexpr int P_SMEM_BYTES = P_STAGES * P_STAGE_BYTES + P_WBUF_BYTES + 256 + 1024;
+
+__device__ __forceinline__ uint32_t cluster_ctarank() {
+  uint32_t r;
+  asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
+  return r;
+}
+__device__ __forceinline__ void cluster_sync_all() {
+  asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
+  asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+// Address of the same shared-memory location in CTA `rank` of the cluster.
+__device__ __forceinline__ uint32_t map_to_cta(uint32_t addr, uint32_t rank) {
+  uint32_t r;
+  asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(addr), "r"(rank));
+  return r;
+}
+__device__ __forceinline__ void mbar_arrive_cluster(uint32_t cluster_addr) {
+  asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
+}
+// TMA tile load into this CTA's shared memory whose completion bytes go to a barrier of the pair.
+__device__ __forceinline__ void tma_load_2d_pair(uint32_t dst, const void* tmap, uint32_t bar_cluster_addr, int x, int y) {
+  asm volatile(
+      "cp.async.bulk.tensor.2d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
+      ::"r"(dst), "l"(tmap), "r"(bar_cluster_addr), "r"(x), "r"(y)
+      : "memory");
+}
+// Instruction descriptor for the pair: bf16 x bf16 -> fp32, K-major operands, M = 256 (128 per CTA), N = n.
+__device__ __forceinline__ uint32_t make_idesc_pair(int n) {
+  return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(n >> 3) << 17) | ((256u >> 4) << 24);
+}
+__device__ __forceinline__ void umma_bf16_pair(uint32_t d_tmem, unsigned long long a, unsigned long long b, uint32_t idesc,
+                                               uint32_t accumulate) {
+  asm volatile(
+      "{\n"
+      ".reg .pred p;\n"
+      "setp.ne.b32 p, %4, 0;\n"
+      "tcgen05.mma.cta_group::2.kind::f16 [%0], %1, %2, %3, p;\n"
+      "}\n"
+      ::"r"(d_tmem), "l"(a), "l"(b), "r"(idesc), "r"(accumulate)
+      : "memory");
+}
+// Arrives on the barrier at this shared-memory offset in both CTAs once the MMAs issued so far are done.
+__device__ __forceinline__ void umma_commit_pair(uint32_t bar) {
+  const uint16_t mask = 3;
+  asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;"
+               ::"r"(bar), "h"(mask)
+               : "memory");
+}
+
+__device__ __forceinline__ void fold16_pair(const uint32_t* vg, const uint32_t* vu, const float* wb, float& s, float& m) {
+  float a[16];
+#pragma unroll
+  for (int q = 0; q < 4; ++q) {
+    const float4 w4 = *reinterpret_cast<const float4*>(wb + 4 * q);
+    a[4 * q] = w4.x; a[4 * q + 1] = w4.y; a[4 * q + 2] = w4.z; a[4 * q + 3] = w4.w;
+  }
+#pragma unroll
+  for (int j = 0; j < 16; ++j) {
+    const float g = __uint_as_float(vg[j]), up = __uint_as_float(vu[j]);
+    const float sig = __fdividef(1.f, 1.f + __expf(-g));
+    const float lam = (a[j] * up) * (g * sig);
+    s = fmaf(lam, lam, s);
+    m = fmaxf(m, fabsf(lam));
+  }
+}
+
+__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(P_THREADS, 1) k_score_umma_pair(const ScoreCtx c) {
+  extern __shared__ uint8_t smem_raw[];
+  const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+  uint8_t* const base_ptr = smem_raw + (base - smem_u32(smem_raw));
+  // [stages: A_gate | A_up | B half] [wbuf 4 warps x 256 floats] [barriers] [tmem slot] [abort flag]
+  float* const wbuf = reinterpret_cast<float*>(base_ptr + P_STAGES * P_STAGE_BYTES);
+  const uint32_t bars = base + P_STAGES * P_STAGE_BYTES + P_WBUF_BYTES;
+  auto full_bar = [&](int s) { return bars + 8u * s; };
+  auto empty_bar = [&](int s) { return bars + 8u * (P_STAGES + s); };
+  const uint32_t tfull_bar = bars + 8u * (2 * P_STAGES);
+  const uint32_t tempty_bar = bars + 8u * (2 * P_STAGES + 1);
+  uint8_t* const tail = base_ptr + P_STAGES * P_STAGE_BYTES + P_WBUF_BYTES + 8 * (2 * P_STAGES + 2);
+  volatile uint32_t* const tmem_slot = reinterpret_cast<volatile uint32_t*>(tail);
+  volatile int* const abort_flag = reinterpret_cast<volatile int*>(tail + 8);
+
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const uint32_t rank = cluster_ctarank();
+  const int pair = blockIdx.x >> 1, n_pairs = gridDim.x >> 1;
+  const int total_units = c.totals->total_units;
+  const int n_kb = c.d_model / UMMA_BK;
+
+  if (tid == 0) {
+    for (int s = 0; s < P_STAGES; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
+    mbar_init(tfull_bar, 1);
+    mbar_init(tempty_bar, 256);
+    *abort_flag = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+  }
+  if (warp == 5) {   // one warp of each CTA of the pair takes part in the allocation; both get the same address
+    asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32((const void*)tmem_slot)),
+                 "r"(P_TMEM_COLS)
+                 : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
+  }
+  tc_fence_before();
+  __syncthreads();
+  cluster_sync_all();     // the other CTA's barriers are initialised before anything arrives on them
+  tc_fence_after();
+  const uint32_t tmem_base = *tmem_slot;
+
+  if (warp == 4) {
+    // ------------------------------------------------------------------ TMA producer (each CTA loads its own share)
+    if (lane == 0) {
+      int stage = 0;
+      uint32_t phase = 0;
+      bool ok = true;
+      const char* maps = static_cast<const char*>(c.tensor_maps);
+      for (int unit = pair; ok && unit < total_units; unit += n_pairs) {
+        const UnitInfo u = decode_unit(c, unit);
+        const int n_tiles = (u.rows + UMMA_TOK - 1) / UMMA_TOK;
+        const void* map_g = maps + (size_t)128 * (2 * u.e);
+        const void* map_u = maps + (size_t)128 * (2 * u.e + 1);
+        const void* map_x = maps + (size_t)128 * (2 * c.n_experts + (u.shared_idx < 0 ? 5 : 2));
+        tensormap_acquire(map_g);
+        tensormap_acquire(map_u);
+        tensormap_acquire(map_x);
+        const int ch = u.ch0 + 128 * (int)rank;     // past d_ff for the second CTA of an odd last tile: reads zeros
+        for (int tt = 0; ok && tt < n_tiles; ++tt) {
+          const int nv = (min(UMMA_TOK, u.rows - tt * UMMA_TOK) + 15) & ~15;
+          const int row = u.row0 + tt * UMMA_TOK + (int)rank * (nv >> 1);   // this CTA holds tokens [rank * nv/2, +nv/2)
+          for (int kb = 0; kb < n_kb; ++kb) {
+            if (!mbar_wait(empty_bar(stage), phase ^ 1u, abort_flag)) { ok = false; break; }
+            const uint32_t a_dst = base + stage * P_STAGE_BYTES;
+            const uint32_t full0 = map_to_cta(full_bar(stage), 0);
+            if (rank == 0) mbar_expect_tx(full_bar(stage), 2 * P_STAGE_BYTES);
+            tma_load_2d_pair(a_dst, map_g, full0, kb * UMMA_BK, ch);
+            tma_load_2d_pair(a_dst + P_A_BYTES, map_u, full0, kb * UMMA_BK, ch);
+            tma_load_2d_pair(a_dst + 2 * P_A_BYTES, map_x, full0, kb * UMMA_BK, row);
+            if (++stage == P_STAGES) { stage = 0; phase ^= 1u; }
+          }
+        }
+      }
+      if (!ok) {
+        const unsigned long long t0 = globaltimer_ns();
+        while (globaltimer_ns() - t0 < 2000000ull) __nanosleep(1000);
+      }
+    }
+  } else if (warp == 5) {
+    // ------------------------------------------------------------------ MMA issuer (first CTA of the pair only)
+    if (lane == 0 && rank == 0) {
+      int stage = 0;
+      uint32_t phase = 0, tile_phase = 0;
+      bool ok = true;
+      for (int unit = pair; ok && unit < total_units; unit += n_pairs) {
+        const UnitInfo u = decode_unit(c, unit);
+        const int n_tiles = (u.rows + UMMA_TOK - 1) / UMMA_TOK;
+        for (int tt = 0; ok && tt < n_tiles; ++tt) {
+          const int nv = (min(UMMA_TOK, u.rows - tt * UMMA_TOK) + 15) & ~15;
+          const uint32_t idesc = make_idesc_pair(nv);
+          if (!mbar_wait(tempty_bar, tile_phase ^ 1u, abort_flag)) { ok = false; break; }
+          tc_fence_after();
+          for (int kb = 0; kb < n_kb; ++kb) {
+            if (!mbar_wait(full_bar(stage), phase, abort_flag)) { ok = false; break; }
+            tc_fence_after();
+            const uint32_t a_addr = base + stage * P_STAGE_BYTES;
+            const unsigned long long g_desc = make_smem_desc(a_addr);
+            const unsigned long long u_desc = make_smem_desc(a_addr + P_A_BYTES);
+            const unsigned long long b_desc = make_smem_desc(a_addr + 2 * P_A_BYTES);
+#pragma unroll
+            for (int k = 0; k < UMMA_BK / 16; ++k) {
+              const uint32_t acc = (uint32_t)((kb | k) != 0);
+              umma_bf16_pair(tmem_base, g_desc + 2 * k, b_desc + 2 * k, idesc, acc);
+              umma_bf16_pair(tmem_base + UMMA_TOK, u_desc + 2 * k, b_desc + 2 * k, idesc, acc);
+            }
+            umma_commit_pair(empty_bar(stage));
+            if (++stage == P_STAGES) { stage = 0; phase ^= 1u; }
+          }
+          if (!ok) break;
+          umma_commit_pair(tfull_bar);
+          tile_phase ^= 1u;
+        }
+      }
+    }
+  } else {
+    // ------------------------------------------------------------------ epilogue (warps 0-3 of both CTAs)
+    uint32_t tile_phase = 0;
+    bool ok = true;
+    float* const wb = wbuf + warp * UMMA_TOK;
+    const uint32_t t_gate = tmem_base + ((uint32_t)(warp * 32) << 16);
+    const uint32_t t_up = t_gate + UMMA_TOK;
+    const uint32_t tempty0 = map_to_cta(tempty_bar, 0);
+    for (int unit = pair; ok && unit < total_units; unit += n_pairs) {
+      const UnitInfo u = decode_unit(c, unit);
+      const int n_tiles = (u.rows + UMMA_TOK - 1) / UMMA_TOK;
+      const float* wsrc = u.shared_idx < 0 ? c.perm_w + u.row0 : c.shared_w + (size_t)u.shared_idx * c.n_tokens + u.row0;
+      float s = 0.f, m = 0.f;
+      for (int tt = 0; ok && tt < n_tiles; ++tt) {
+        const int valid = min(UMMA_TOK, u.rows - tt * UMMA_TOK);
+        const int nv = (valid + 15) & ~15;
+        __syncwarp();
+        for (int i = lane; i < UMMA_TOK; i += 32) wb[i] = i < valid ? wsrc[tt * UMMA_TOK + i] : 0.f;
+        __syncwarp();
+        ok = __all_sync(0xffffffffu, mbar_wait(tfull_bar, tile_phase, abort_flag));
+        if (!ok) break;
+        tc_fence_after();
+        uint32_t g0[16], u0[16], g1[16], u1[16];
+        tmem_ld16(t_gate, g0);
+        tmem_ld16(t_up, u0);
+        for (int c0 = 0; c0 < nv; c0 += 32) {
+          tmem_ld_wait(g0, u0);
+          if (c0 + 16 < nv) { tmem_ld16(t_gate + c0 + 16, g1); tmem_ld16(t_up + c0 + 16, u1); }
+          fold16_pair(g0, u0, wb + c0, s, m);
+          if (c0 + 16 < nv) {
+            tmem_ld_wait(g1, u1);
+            if (c0 + 32 < nv) { tmem_ld16(t_gate + c0 + 32, g0); tmem_ld16(t_up + c0 + 32, u0); }
+            fold16_pair(g1, u1, wb + c0 + 16, s, m);
+          }
+        }
+        tc_fence_before();
+        mbar_arrive_cluster(tempty0);
+        tile_phase ^= 1u;
+      }
+      const int ch = u.ch0 + 128 * (int)rank + warp * 32 + lane;
+      if (ok && ch < u.f) {
+        const size_t slot = (size_t)u.part_slot + 128 * rank + warp * 32 + lane;
+        c.part_sum[slot] = s;
+        c.part_max[slot] = m;
+      }
+    }
+  }
+
+  tc_fence_before();
+  __syncthreads();
+  if (*abort_flag && tid == 0) atomicExch(&c.totals->status, (int)CAMERA_ERR_DEVICE_TIMEOUT);
+  cluster_sync_all();     // neither CTA leaves while the other may still read its shared or tensor memory
+  if (warp == 5) {
+    tc_fence_after();
+    asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(P_TMEM_COLS) : "memory");
+  }
+}
+
+}  // namespace
+
+cudaError_t launch_score_umma_pair(const ScoreCtx& c, cudaStream_t st) {
+  int dev = 0, sms = 148;
+  cudaGetDevice(&dev);
+  cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+  cudaError_t e = cudaFuncSetAttribute(k_score_umma_pair, cudaFuncAttributeMaxDynamicSharedMemorySize, P_SMEM_BYTES);
+  if (e != cudaSuccess) return e;
+  k_score_umma_pair<<<sms & ~1, P_THREADS, P_SMEM_BYTES, st>>>(c);
+  return cudaGetLastError();
+}
+
+}  // namespace camera

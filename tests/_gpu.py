@@ -54,14 +54,14 @@ def check_routing(olayer, Xd, topk_idx, topk_w):
     return int((~same).sum())
 
 
-def run_and_compare(P, L, X, alpha=0.95, channels=None, force_simt=False, check_dense=False):
+def run_and_compare(P, L, X, alpha=0.95, channels=None, force_simt=False, check_dense=False, cta_pair=False):
     """Scores one layer on the GPU (own routing, then the oracle's routing injected) and checks
     every component against the oracle.  `channels` restricts the oracle to sampled micro-experts."""
     layer = P.Layer.from_workload(L)
     olayer = to_oracle_layer(L)
     Xd = f64(X)
     ws = P.alloc_workspace(P.camera_score_workspace_bytes(layer, X.shape[0]), X.device)
-    out = P.camera_score_layer(layer, X, alpha, details=True, workspace=ws, force_simt=force_simt)
+    out = P.camera_score_layer(layer, X, alpha, details=True, workspace=ws, force_simt=force_simt, cta_pair=cta_pair)
     assert P.camera_read_status(ws) == 0
     flips = check_routing(olayer, Xd, out["topk_idx"], out["topk_w"])
 
@@ -88,7 +88,7 @@ def run_and_compare(P, L, X, alpha=0.95, channels=None, force_simt=False, check_
     if olayer.n_routed:
         idx_o, w_o = O.top_and_norm(O.router_probs(olayer, Xd), olayer.top_k, olayer.norm_topk)
         w32 = w_o.astype(np.float32)
-        out2 = P.camera_score_layer(layer, X, alpha, details=True, workspace=ws, force_simt=force_simt,
+        out2 = P.camera_score_layer(layer, X, alpha, details=True, workspace=ws, force_simt=force_simt, cta_pair=cta_pair,
                                     routing_in=(torch.from_numpy(idx_o.astype(np.int32)), torch.from_numpy(w32)))
         assert P.camera_read_status(ws) == 0
         p2, pi, w2 = O.camera_components(olayer, Xd, channels=channels, routing=(idx_o, w32.astype(np.float64)))

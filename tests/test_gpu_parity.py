@@ -64,21 +64,22 @@ def test_tiny_fp32_alpha_sweep(P, alpha):
 
 
 # ------------------------------------------------------------------ bf16: tensor-core kernel and the FMA kernel
-@pytest.mark.parametrize("force_simt", [False, True])
+@pytest.mark.parametrize("kernel", ["umma", "umma_pair", "simt"])
 @pytest.mark.parametrize("down_layout", ["hf", "me_major"])
-def test_small_bf16(P, force_simt, down_layout):
+def test_small_bf16(P, kernel, down_layout):
     cfg = small_cfg()
     L = W().make_layer(cfg, seed=2, device=DEV, down_layout=down_layout)
     X = W().make_tokens(cfg, seed=2, device=DEV)
-    run_and_compare(P, L, X, alpha=0.95, force_simt=force_simt, check_dense=True)
+    run_and_compare(P, L, X, alpha=0.95, force_simt=kernel == "simt", cta_pair=kernel == "umma_pair", check_dense=True)
 
 
+@pytest.mark.parametrize("cta_pair", [False, True])
 @pytest.mark.parametrize("T", [1, 15, 16, 17, 255, 256, 257, 1030])
-def test_ragged_token_counts(P, T):
+def test_ragged_token_counts(P, T, cta_pair):
     cfg = small_cfg(n_tokens=T, n_routed=4, d_ff_routed=64, d_ff_shared=(64,))
     L = W().make_layer(cfg, seed=3, device=DEV)
     X = W().make_tokens(cfg, seed=3, device=DEV)
-    run_and_compare(P, L, X, alpha=0.5)
+    run_and_compare(P, L, X, alpha=0.5, cta_pair=cta_pair)
 
 
 def test_zero_tokens(P):
@@ -148,12 +149,14 @@ def test_bit_reproducible(P):
     assert torch.equal(a, b)
 
 
-def test_multi_chunk_units(P):
-    """Enough tokens per expert that a work unit spans several token tiles and chunks."""
-    cfg = small_cfg(n_tokens=6000, n_routed=2, top_k=1, d_ff_routed=64, d_ff_shared=(64,))
+@pytest.mark.parametrize("cta_pair", [False, True])
+def test_multi_chunk_units(P, cta_pair):
+    """Enough tokens per expert that a work unit spans several token tiles and chunks; d_ff values that
+    leave a channel tile partly (320 = 2 * 128 + 64) or, for the second CTA of a pair, wholly empty."""
+    cfg = small_cfg(n_tokens=6000, n_routed=2, top_k=1, d_ff_routed=320, d_ff_shared=(64,))
     L = W().make_layer(cfg, seed=11, device=DEV)
     X = W().make_tokens(cfg, seed=11, device=DEV)
-    run_and_compare(P, L, X, alpha=0.95)
+    run_and_compare(P, L, X, alpha=0.95, cta_pair=cta_pair)
 
 
 # ------------------------------------------------------------------ argument checks need no kernel to run
