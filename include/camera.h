@@ -59,8 +59,14 @@ enum {
 /* camera_score_aux_t.flags */
 enum {
   CAMERA_SCORE_FORCE_SIMT = 1u,    /* run the fp32-FMA kernels even where the tensor-core kernels apply */
-  CAMERA_SCORE_CTA_PAIR = 2u       /* tensor-core scoring on CTA pairs (tcgen05 cta_group::2): less L2 and shared-memory
+  CAMERA_SCORE_CTA_PAIR = 2u,      /* tensor-core scoring on CTA pairs (tcgen05 cta_group::2): less L2 and shared-memory
                                       traffic per flop, but measured slower under the power cap; off by default */
+  CAMERA_SCORE_ACCUMULATE = 4u     /* phi2 and phi_inf_sq (both required) already hold the result of earlier batches of
+                                      calibration tokens of this layer; this call folds its batch in (the column sums of
+                                      Alg. 1 line 7 add up over batches, the column maxima of line 8 take the maximum)
+                                      and writes the energy of all batches so far; the workspace's status word is
+                                      not cleared by such a call, so one camera_read_status after the last batch
+                                      reports trouble in any of them (use the same workspace for all batches) */
 };
 
 /* Stages of camera_score_layer, for the optional timing events. */
@@ -116,6 +122,7 @@ size_t camera_score_workspace_bytes(const camera_layer_t* layer, int64_t n_token
  *   phi2   <- ColumnSum(Lambda*Lambda), phi_inf <- ColumnMax|Lambda|^2   lines 7-8
  *   energy <- [(1-alpha) phi2 + alpha phi_inf] * omega2            line 10, Eq. 11
  * x: DEVICE [n_tokens, d_model] row-major, dtype layer->dtype.  energy: DEVICE [N_e] fp32.
+ * The calibration set may be fed in several calls (batches of tokens) with CAMERA_SCORE_ACCUMULATE.
  * Arithmetic: inputs as stored, products and sums in fp32 (bf16: tensor cores with fp32
  * accumulators), the final blend in fp64.  Routing ties go to the lower expert index.
  * An expert no token reaches gets energy 0.  0 <= alpha <= 1.  n_tokens >= 0.
@@ -186,12 +193,15 @@ int camera_select_prune_static(const float* energy, const int64_t* seg_offsets, 
                                double prune_ratio, uint8_t* keep_mask, float* thresholds,
                                void* cuda_stream);
 
-/* Scratch for camera_analyze_layer_host: score + select scratch + staging of x and results. */
+/* Scratch for camera_analyze_layer_host: score + select scratch for one batch of tokens, two staging
+ * buffers for batches of x, and the results. */
 size_t camera_analyze_workspace_bytes(const camera_layer_t* layer, int64_t n_tokens, int32_t n_levels);
 
 /*
  * One whole analysis step with HOST token and result buffers: copies x_host (pinned or
- * pageable, [n_tokens, d_model]) to the device, runs camera_score_layer, camera_select_prune
+ * pageable, [n_tokens, d_model]) to the device in batches of 65536 tokens on a copy stream of its
+ * own, scoring batch b (camera_score_layer, accumulating) while batch b+1 is on its way; then runs
+ * camera_select_prune
  * once per entry of prune_ratios (HOST [n_prune], may be empty) and camera_alloc_bits, and copies
  * energy [N_e] fp32, keep masks [n_prune, N_e] and bits_out [N_e] back to the given HOST buffers
  * (any may be NULL).  The layer's weights stay DEVICE resident.  Synchronises the stream before

@@ -20,6 +20,7 @@ CAMERA_DOWN_HF, CAMERA_DOWN_ME_MAJOR = 0, 1
 CAMERA_ROUTER_NORM_TOPK, CAMERA_SHARED_GATE_SIGMOID = 1, 2
 CAMERA_SCORE_FORCE_SIMT = 1
 CAMERA_SCORE_CTA_PAIR = 2
+CAMERA_SCORE_ACCUMULATE = 4
 STAGES = ("router", "permute", "rownorm", "score", "combine")
 
 
@@ -169,11 +170,15 @@ def alloc_workspace(nbytes: int, device) -> torch.Tensor:
 def camera_score_layer(layer: Layer, x: torch.Tensor, alpha: float, *, energy: Optional[torch.Tensor] = None,
                        workspace: Optional[torch.Tensor] = None, details: bool = False,
                        routing_in=None, force_simt: bool = False, cta_pair: bool = False, stage_events=None,
+                       phi2: Optional[torch.Tensor] = None, phi_inf_sq: Optional[torch.Tensor] = None,
+                       accumulate: bool = False,
                        stream: Optional[torch.cuda.Stream] = None, check_status: bool = False):
     """Algorithm 1 up to the energies.  Returns energy [N_e] fp32, or with details=True a dict that
     also holds phi2, phi_inf_sq, omega2, topk_idx, topk_w, shared_w and expert_token_counts.
     routing_in = (topk_idx int32 [T,k], topk_w fp32 [T,k]) prescribes the routing.
-    stage_events = {stage: (torch.cuda.Event, torch.cuda.Event)} records per-stage timing events."""
+    stage_events = {stage: (torch.cuda.Event, torch.cuda.Event)} records per-stage timing events.
+    phi2 / phi_inf_sq name the tensors that receive those components; with accumulate=True they must
+    hold the result of earlier batches of tokens, and this batch is folded into them."""
     if not (x.is_contiguous() and x.dtype == layer.dtype and x.dim() == 2 and x.shape[1] == layer.d_model):
         raise ValueError("x must be a contiguous [T, d_model] tensor of the layer's dtype")
     T = int(x.shape[0])
@@ -202,7 +207,14 @@ def camera_score_layer(layer: Layer, x: torch.Tensor, alpha: float, *, energy: O
         w = w.to(device=dev, dtype=torch.float32).contiguous()
         keep_alive += [idx, w]
         aux.topk_idx_in, aux.topk_w_in = idx.data_ptr(), w.data_ptr()
-    aux.flags = (CAMERA_SCORE_FORCE_SIMT if force_simt else 0) | (CAMERA_SCORE_CTA_PAIR if cta_pair else 0)
+    for name, t in (("phi2", phi2), ("phi_inf_sq", phi_inf_sq)):
+        if t is not None:
+            if not (t.is_contiguous() and t.dtype == torch.float32 and t.numel() == layer.n_me and t.device == dev):
+                raise ValueError(f"{name} must be a contiguous fp32 [N_e] tensor on the device of x")
+            out[name] = t
+            setattr(aux, name, t.data_ptr())
+    aux.flags = ((CAMERA_SCORE_FORCE_SIMT if force_simt else 0) | (CAMERA_SCORE_CTA_PAIR if cta_pair else 0) |
+                 (CAMERA_SCORE_ACCUMULATE if accumulate else 0))
     if stage_events:
         for name, (e0, e1) in stage_events.items():
             i = STAGES.index(name)

@@ -178,6 +178,8 @@ extern "C" int camera_score_layer(const camera_layer_t* L, const void* x, int64_
   if (rc != CAMERA_OK) return rc;
   if (!(alpha >= 0.f && alpha <= 1.f) || energy == nullptr || (T > 0 && x == nullptr)) return CAMERA_ERR_INVALID_ARG;
   if (aux && ((aux->topk_idx_in == nullptr) != (aux->topk_w_in == nullptr))) return CAMERA_ERR_INVALID_ARG;
+  const bool accumulate = aux && (aux->flags & CAMERA_SCORE_ACCUMULATE);
+  if (accumulate && (aux->phi2 == nullptr || aux->phi_inf_sq == nullptr)) return CAMERA_ERR_INVALID_ARG;
   {  // every matrix is read with 16-byte vector loads
     uintptr_t bits = reinterpret_cast<uintptr_t>(x) | reinterpret_cast<uintptr_t>(L->w_router) |
                      reinterpret_cast<uintptr_t>(L->w_shared_gate);
@@ -204,6 +206,7 @@ extern "C" int camera_score_layer(const camera_layer_t* L, const void* x, int64_
   c.dtype = L->dtype; c.down_layout = L->down_layout; c.flags = L->flags;
   c.n_tokens = (int)T; c.n_blocks = lay.n_blocks; c.chunk_tokens = lay.chunk_tokens;
   c.max_rows_perm = lay.max_rows_perm; c.max_part = lay.max_part; c.alpha = alpha;
+  c.accumulate = accumulate ? 1 : 0;
   c.x = x; c.w_router = L->w_router; c.router_bias = L->router_bias; c.w_shared_gate = L->w_shared_gate;
   c.totals = reinterpret_cast<PlanTotals*>(ws + lay.totals);
   c.est = reinterpret_cast<ExpertStatic*>(ws + lay.est);
@@ -255,7 +258,9 @@ extern "C" int camera_score_layer(const camera_layer_t* L, const void* x, int64_
     if (rc != CAMERA_OK) return rc;
   }
 
-  CK(cudaMemsetAsync(c.totals, 0, sizeof(PlanTotals), st));
+  // the plan kernel rewrites the totals on every call; the status word is sticky across the calls of one
+  // accumulation, so that one read after the last batch sees trouble in any of them
+  if (!accumulate) CK(cudaMemsetAsync(c.totals, 0, sizeof(PlanTotals), st));
   CK(cudaMemsetAsync(c.counts, 0, sizeof(int32_t) * E, st));
   CK(cudaMemcpyAsync(c.est, est.data(), sizeof(ExpertStatic) * E, cudaMemcpyHostToDevice, st));
   CK(cudaMemcpyAsync(c.me_prefix, me_prefix.data(), sizeof(int32_t) * (E + 1), cudaMemcpyHostToDevice, st));
@@ -306,13 +311,17 @@ extern "C" int camera_read_status(const void* workspace, void* cuda_stream, int3
 }
 
 namespace {
+constexpr int64_t ANALYZE_BATCH_TOKENS = 65536;   // tokens per host-to-device batch of camera_analyze_layer_host
+
 struct AnalyzeLayout {
-  size_t score, select, x, energy, keep, bits, total;
+  size_t score, select, x[2], energy, phi2, phi_inf, keep, bits, total;
   size_t score_bytes, select_bytes;
+  int64_t batch;
 };
 AnalyzeLayout analyze_layout(const camera_layer_t* L, int64_t T, int n_levels) {
   AnalyzeLayout a;
-  const ScoreLayout s = score_layout(L, T);
+  a.batch = T < ANALYZE_BATCH_TOKENS ? T : ANALYZE_BATCH_TOKENS;
+  const ScoreLayout s = score_layout(L, a.batch);
   const size_t esz = L->dtype == CAMERA_BF16 ? 2 : 4;
   a.score_bytes = s.total;
   a.select_bytes = camera_select_workspace_bytes(s.n_me, 1, n_levels < 2 ? 2 : n_levels);
@@ -320,13 +329,37 @@ AnalyzeLayout analyze_layout(const camera_layer_t* L, int64_t T, int n_levels) {
   auto take = [&](size_t bytes) { size_t at = o; o = up256(o + bytes); return at; };
   a.score = take(a.score_bytes);
   a.select = take(a.select_bytes);
-  a.x = take(esz * (size_t)T * L->d_model);
+  a.x[0] = take(esz * (size_t)a.batch * L->d_model);
+  a.x[1] = take(T > a.batch ? esz * (size_t)a.batch * L->d_model : 0);
   a.energy = take(sizeof(float) * (size_t)s.n_me);
+  a.phi2 = take(sizeof(float) * (size_t)s.n_me);
+  a.phi_inf = take(sizeof(float) * (size_t)s.n_me);
   a.keep = take((size_t)s.n_me);
   a.bits = take((size_t)s.n_me);
   a.total = o;
   return a;
 }
+
+// The copy stream and the events that order it against the caller's stream; destroyed when the call returns.
+struct CopyPipe {
+  cudaStream_t copy = nullptr;
+  cudaEvent_t copied[2] = {nullptr, nullptr}, consumed[2] = {nullptr, nullptr};
+  bool create() {
+    if (cudaStreamCreateWithFlags(&copy, cudaStreamNonBlocking) != cudaSuccess) return false;
+    for (int i = 0; i < 2; ++i)
+      if (cudaEventCreateWithFlags(&copied[i], cudaEventDisableTiming) != cudaSuccess ||
+          cudaEventCreateWithFlags(&consumed[i], cudaEventDisableTiming) != cudaSuccess)
+        return false;
+    return true;
+  }
+  ~CopyPipe() {
+    for (int i = 0; i < 2; ++i) {
+      if (copied[i]) cudaEventDestroy(copied[i]);
+      if (consumed[i]) cudaEventDestroy(consumed[i]);
+    }
+    if (copy) cudaStreamDestroy(copy);
+  }
+};
 }  // namespace
 
 extern "C" size_t camera_analyze_workspace_bytes(const camera_layer_t* layer, int64_t n_tokens, int32_t n_levels) {
@@ -350,27 +383,53 @@ extern "C" int camera_analyze_layer_host(const camera_layer_t* L, const void* x_
   cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
   char* ws = static_cast<char*>(workspace);
   const size_t esz = L->dtype == CAMERA_BF16 ? 2 : 4;
-  const ScoreLayout s = score_layout(L, T);
+  const size_t row_bytes = esz * (size_t)L->d_model;
+  int n_me = 0;
+  for (int e = 0; e < L->n_routed + L->n_shared; ++e) n_me += L->d_ff[e];
   float* d_energy = reinterpret_cast<float*>(ws + a.energy);
   uint8_t* d_keep = reinterpret_cast<uint8_t*>(ws + a.keep);
   uint8_t* d_bits = reinterpret_cast<uint8_t*>(ws + a.bits);
-  if (T > 0) CK(cudaMemcpyAsync(ws + a.x, x_host, esz * (size_t)T * L->d_model, cudaMemcpyHostToDevice, st));
-  rc = camera_score_layer(L, ws + a.x, T, alpha, d_energy, nullptr, ws + a.score, a.score_bytes, cuda_stream);
-  if (rc != CAMERA_OK) return rc;
-  if (energy_host) CK(cudaMemcpyAsync(energy_host, d_energy, sizeof(float) * (size_t)s.n_me, cudaMemcpyDeviceToHost, st));
-  const int64_t seg[2] = {0, s.n_me};
+  camera_score_aux_t aux;
+  memset(&aux, 0, sizeof(aux));
+  aux.phi2 = reinterpret_cast<float*>(ws + a.phi2);
+  aux.phi_inf_sq = reinterpret_cast<float*>(ws + a.phi_inf);
+
+  const int64_t n_batches = T > 0 ? (T + a.batch - 1) / a.batch : 1;
+  CopyPipe pipe;
+  if (n_batches > 1 && !pipe.create()) { cudaGetLastError(); return CAMERA_ERR_CUDA; }
+  for (int64_t b = 0; b < n_batches; ++b) {
+    const int buf = (int)(b & 1);
+    const int64_t t0 = b * a.batch;
+    const int64_t n = T - t0 < a.batch ? T - t0 : a.batch;
+    const char* src = static_cast<const char*>(x_host) + (size_t)t0 * row_bytes;
+    if (n_batches == 1) {
+      if (n > 0) CK(cudaMemcpyAsync(ws + a.x[0], src, (size_t)n * row_bytes, cudaMemcpyHostToDevice, st));
+    } else {
+      // batch b travels on the copy stream while batch b-1 is being scored on the caller's stream
+      if (b >= 2) CK(cudaStreamWaitEvent(pipe.copy, pipe.consumed[buf], 0));
+      CK(cudaMemcpyAsync(ws + a.x[buf], src, (size_t)n * row_bytes, cudaMemcpyHostToDevice, pipe.copy));
+      CK(cudaEventRecord(pipe.copied[buf], pipe.copy));
+      CK(cudaStreamWaitEvent(st, pipe.copied[buf], 0));
+    }
+    aux.flags = b > 0 ? CAMERA_SCORE_ACCUMULATE : 0u;
+    rc = camera_score_layer(L, ws + a.x[buf], n, alpha, d_energy, &aux, ws + a.score, a.score_bytes, cuda_stream);
+    if (rc != CAMERA_OK) return rc;
+    if (n_batches > 1) CK(cudaEventRecord(pipe.consumed[buf], st));
+  }
+  if (energy_host) CK(cudaMemcpyAsync(energy_host, d_energy, sizeof(float) * (size_t)n_me, cudaMemcpyDeviceToHost, st));
+  const int64_t seg[2] = {0, n_me};
   for (int p = 0; p < n_prune; ++p) {
     rc = camera_select_prune(d_energy, seg, 1, prune_ratios[p], nullptr, 0, d_keep, nullptr, nullptr, ws + a.select,
                              a.select_bytes, cuda_stream);
     if (rc != CAMERA_OK) return rc;
     if (keep_host)
-      CK(cudaMemcpyAsync(keep_host + (size_t)p * s.n_me, d_keep, (size_t)s.n_me, cudaMemcpyDeviceToHost, st));
+      CK(cudaMemcpyAsync(keep_host + (size_t)p * n_me, d_keep, (size_t)n_me, cudaMemcpyDeviceToHost, st));
   }
   rc = camera_alloc_bits(d_energy, seg, 1, ratios, bits, n_levels, nullptr, 0, d_bits, nullptr, ws + a.select,
                          a.select_bytes, cuda_stream);
   if (rc != CAMERA_OK) return rc;
-  if (bits_host) CK(cudaMemcpyAsync(bits_host, d_bits, (size_t)s.n_me, cudaMemcpyDeviceToHost, st));
-  int32_t status = 0;
+  if (bits_host) CK(cudaMemcpyAsync(bits_host, d_bits, (size_t)n_me, cudaMemcpyDeviceToHost, st));
+  int32_t status = 0;    // accumulating calls leave the status word alone: this covers every batch
   rc = camera_read_status(ws + a.score, cuda_stream, &status);
   if (rc != CAMERA_OK) return rc;
   return status;

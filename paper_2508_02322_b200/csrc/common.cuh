@@ -58,6 +58,7 @@ struct ScoreCtx {
   int32_t max_rows_perm;            // capacity of x_perm in rows
   int64_t max_part;                 // capacity of the partial arrays in floats
   float alpha;
+  int32_t accumulate;               // fold this call's tokens into the phi2 / phi_inf_sq already there
   const void* x;
   const void* w_router;
   const float* router_bias;

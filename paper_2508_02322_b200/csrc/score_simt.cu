@@ -131,7 +131,11 @@ __global__ void __launch_bounds__(256) k_combine(ScoreCtx c) {
     s += (double)c.part_sum[slot];
     m = fmaxf(m, c.part_max[slot]);
   }
-  const double m2 = (double)m * (double)m;
+  double m2 = (double)m * (double)m;
+  if (c.accumulate) {     // earlier batches of tokens: sums add, maxima take the maximum
+    s += (double)c.phi2[i];
+    m2 = fmax(m2, (double)c.phi_inf_sq[i]);
+  }
   const double a = (double)c.alpha;
   c.phi2[i] = (float)s;
   c.phi_inf_sq[i] = (float)m2;

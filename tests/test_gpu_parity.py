@@ -256,3 +256,56 @@ def test_analyze_layer_host(P):
     P.camera_analyze_layer_host(layer, xh, 0.95, [0.2, 0.6], [0.2, 0.6, 0.2], [3, 2, 1], energy_host=eh, keep_host=kh,
                                 bits_host=bh, workspace=ws)
     assert torch.equal(eh, E.cpu()) and torch.equal(kh, keep.cpu()) and torch.equal(bh, bits.cpu())
+
+
+# ------------------------------------------------------------------ the calibration set fed in batches
+@pytest.mark.parametrize("kernel", ["umma", "simt"])
+def test_accumulate_over_token_batches(P, kernel):
+    """Column sums add up and column maxima take the maximum over batches of tokens (Algorithm 1 lines 7-8):
+    three uneven batches must give the scores of the whole set."""
+    cfg = small_cfg(n_tokens=2500)
+    L = W().make_layer(cfg, seed=14, device=DEV)
+    X = W().make_tokens(cfg, seed=14, device=DEV)
+    layer = P.Layer.from_workload(L)
+    ws = P.alloc_workspace(P.camera_score_workspace_bytes(layer, 1499), DEV)
+    phi2 = torch.empty(layer.n_me, dtype=torch.float32, device=DEV)
+    phi_inf = torch.empty_like(phi2)
+    idx, w = [], []
+    out = None
+    for b, (t0, t1) in enumerate(((0, 1000), (1000, 1001), (1001, 2500))):
+        out = P.camera_score_layer(layer, X[t0:t1].contiguous(), 0.95, details=True, workspace=ws, phi2=phi2,
+                                   phi_inf_sq=phi_inf, accumulate=b > 0, force_simt=kernel == "simt")
+        idx.append(out["topk_idx"].cpu().numpy().astype(np.int64))
+        w.append(out["topk_w"].cpu().numpy().astype(np.float64))
+    assert P.camera_read_status(ws) == 0
+    p2, pinf, w2 = O.camera_components(to_oracle_layer(L), f64(X), routing=(np.concatenate(idx), np.concatenate(w)))
+    assert_close("phi2 over batches", phi2.cpu().numpy(), p2)
+    assert_close("phi_inf_sq over batches", phi_inf.cpu().numpy(), pinf)
+    assert_close("energy over batches", out["energy"].cpu().numpy(), O.energy(p2, pinf, w2, float(np.float32(0.95))))
+    whole = P.camera_score_layer(layer, X, 0.95, force_simt=kernel == "simt")
+    assert_close("batches vs one call", out["energy"].cpu().numpy(), whole.cpu().numpy(), rel=1e-5)
+    with pytest.raises(P.CameraError):      # accumulating needs the running components
+        P.camera_score_layer(layer, X[:10].contiguous(), 0.95, accumulate=True)
+
+
+def test_analyze_layer_host_in_batches(P):
+    """More tokens than one host-to-device batch (65536): batches are copied on a second stream while the
+    previous one is scored; the result must be that of one call over all tokens."""
+    cfg = small_cfg(n_tokens=150001, d_model=128, n_routed=4, d_ff_routed=128, d_ff_shared=(64,))
+    L = W().make_layer(cfg, seed=15, device=DEV)
+    X = W().make_tokens(cfg, seed=15, device=DEV)
+    layer = P.Layer.from_workload(L)
+    E = P.camera_score_layer(layer, X, 0.95)
+    xh = X.cpu().pin_memory()
+    eh = torch.empty(layer.n_me, dtype=torch.float32).pin_memory()
+    kh = torch.empty((2, layer.n_me), dtype=torch.uint8).pin_memory()
+    bh = torch.empty(layer.n_me, dtype=torch.uint8).pin_memory()
+    ws = P.alloc_workspace(P.camera_analyze_workspace_bytes(layer, cfg.n_tokens, 3), DEV)
+    for _ in range(2):      # the second call reuses the workspace the first one left behind
+        eh.zero_()
+        P.camera_analyze_layer_host(layer, xh, 0.95, [0.2, 0.6], [0.2, 0.6, 0.2], [3, 2, 1], energy_host=eh,
+                                    keep_host=kh, bits_host=bh, workspace=ws)
+        assert_close("energy in batches", eh.numpy(), E.cpu().numpy(), rel=1e-5)
+        for j, r in enumerate((0.2, 0.6)):
+            assert np.array_equal(kh[j].numpy(), O.select_prune(eh.numpy(), r))
+        assert np.array_equal(bh.numpy(), O.alloc_bits(eh.numpy(), [0.2, 0.6, 0.2], [3, 2, 1])[0])
