@@ -34,9 +34,9 @@ PAPER_CONTEXT = "paper: <5 min for the full Qwen2-57B-A14B analysis on one A100-
 # kernels launched by one step: score = router, block scan, plan, permute, pad, norms, scoring, combine;
 # every selection = 8 histogram passes + mark
 LAUNCHES_PER_STEP = 8 + 9 * (len(PRUNE_RATIOS) + 1)
-# DRAM bytes per launch of the scoring kernel from the committed ncu capture, scaled per unit of work
-# (bytes per gate/up flop measured on the profiled case); None until a capture exists.
-SCORE_KERNEL_DRAM_BYTES_PER_FLOP = None
+# DRAM bytes (read + write) per gate/up flop of the scoring kernel, from the committed ncu capture of a
+# 1/8 slice of the layer whose traffic grows in proportion to the flop (profiles/k_score_umma_qwen2_slice.md).
+SCORE_KERNEL_DRAM_BYTES_PER_FLOP = 10.49e9 / 1.924e13
 
 
 def shard_layers(n_layers: int, world: int, rank: int):
