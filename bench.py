@@ -308,7 +308,8 @@ def main():
                 "peak": peaks["bf16_tflops_sustained"], "unit": "TFLOP/s", "frac": achieved / peaks["bf16_tflops_sustained"],
                 "frac_of_burst_peak": achieved / peaks["bf16_tflops"], "peak_source": peaks["source"] + " (sustained bf16)",
                 "flop_per_launch": flop, "ms_per_launch": score_ms,
-                "traffic": None if SCORE_KERNEL_DRAM_BYTES_PER_FLOP is None else SCORE_KERNEL_DRAM_BYTES_PER_FLOP * flop}
+                "traffic": SCORE_KERNEL_DRAM_BYTES_PER_FLOP * flop
+                if (args.config == "qwen2_57b_a14b" and not args.cta_pair) else None}
 
     cpu = None
     if not args.no_cpu_baseline:
