@@ -199,7 +199,7 @@ size_t camera_analyze_workspace_bytes(const camera_layer_t* layer, int64_t n_tok
 
 /*
  * One whole analysis step with HOST token and result buffers: copies x_host (pinned or
- * pageable, [n_tokens, d_model]) to the device in batches of 65536 tokens on a copy stream of its
+ * pageable, [n_tokens, d_model]) to the device in batches of 65536 tokens (the first one 16384) on a copy stream of its
  * own, scoring batch b (camera_score_layer, accumulating) while batch b+1 is on its way; then runs
  * camera_select_prune
  * once per entry of prune_ratios (HOST [n_prune], may be empty) and camera_alloc_bits, and copies

@@ -41,7 +41,7 @@ __all__ = [
     "coefficients", "expert_hidden", "forward", "phi_matrix", "basis",
     "me_offsets", "camera_components_dense", "camera_components", "energy",
     "camera_rank", "n_pruned", "select_prune", "class_boundaries",
-    "alloc_bits", "sub_index", "decode_error", "best_subset_error",
+    "alloc_bits", "sub_index", "sub_index_lists", "slice_layer", "decode_error", "best_subset_error",
     "average_bits",
 ]
 
@@ -312,6 +312,42 @@ def sub_index(cls_or_mask: np.ndarray, offsets: np.ndarray, n_classes: int) -> n
         for j in range(n_classes):
             out[e, j] = int((seg == j).sum())
     return out
+
+
+def sub_index_lists(labels: np.ndarray, offsets: np.ndarray, order: Sequence[int]):
+    """GetSubIndex (Algorithm 3 line 8; the per-expert retained sets of Algorithm 2 lines 9-10).
+
+    For every expert, its micro-experts (channel numbers inside the expert)
+    listed label by label in the given `order` of label values, ascending
+    channel inside a label; micro-experts whose label is not in `order` are
+    left out.  Returns (lists, counts): lists[e] is an int64 array, counts is
+    [n_experts, len(order)].  With labels = keep mask and order = [1] this is
+    the retained set S of each expert; with labels = precision class and
+    order = all classes it is the reordering that colocates micro-experts of
+    equal precision (Section "CAMERA-Q")."""
+    lists, counts = [], np.zeros((len(offsets) - 1, len(order)), dtype=np.int64)
+    for e in range(len(offsets) - 1):
+        seg = np.asarray(labels[offsets[e]:offsets[e + 1]])
+        parts = []
+        for j, v in enumerate(order):
+            ch = np.nonzero(seg == v)[0]
+            counts[e, j] = ch.size
+            parts.append(ch)
+        lists.append(np.concatenate(parts).astype(np.int64) if parts else np.zeros(0, dtype=np.int64))
+    return lists, counts
+
+
+def slice_layer(layer: OracleLayer, lists: Sequence[np.ndarray]) -> OracleLayer:
+    """Algorithm 2 lines 11-13: W_up <- W_up[S,:], W_gate <- W_gate[S,:],
+    W_down <- W_down[:,S] for every expert, S given as channel lists (any
+    order; a permutation of all channels merely reorders the micro-experts)."""
+    return OracleLayer(
+        w_router=layer.w_router, top_k=layer.top_k,
+        w_gate=[w[np.asarray(ix, dtype=np.int64)] for w, ix in zip(layer.w_gate, lists)],
+        w_up=[w[np.asarray(ix, dtype=np.int64)] for w, ix in zip(layer.w_up, lists)],
+        w_down=[w[:, np.asarray(ix, dtype=np.int64)] for w, ix in zip(layer.w_down, lists)],
+        router_bias=layer.router_bias, norm_topk=layer.norm_topk, n_shared=layer.n_shared,
+        w_shared_gate=layer.w_shared_gate)
 
 
 # ----------------------------------------------------------------------------

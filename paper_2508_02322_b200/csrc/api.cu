@@ -394,13 +394,15 @@ extern "C" int camera_analyze_layer_host(const camera_layer_t* L, const void* x_
   aux.phi2 = reinterpret_cast<float*>(ws + a.phi2);
   aux.phi_inf_sq = reinterpret_cast<float*>(ws + a.phi_inf);
 
-  const int64_t n_batches = T > 0 ? (T + a.batch - 1) / a.batch : 1;
+  // the first batch is a quarter of the others: its copy is the only one nothing overlaps
+  const int64_t first = T > a.batch ? a.batch / 4 : T;
+  const int64_t n_batches = T > a.batch ? 1 + (T - first + a.batch - 1) / a.batch : 1;
   CopyPipe pipe;
   if (n_batches > 1 && !pipe.create()) { cudaGetLastError(); return CAMERA_ERR_CUDA; }
   for (int64_t b = 0; b < n_batches; ++b) {
     const int buf = (int)(b & 1);
-    const int64_t t0 = b * a.batch;
-    const int64_t n = T - t0 < a.batch ? T - t0 : a.batch;
+    const int64_t t0 = b == 0 ? 0 : first + (b - 1) * a.batch;
+    const int64_t n = b == 0 ? first : (T - t0 < a.batch ? T - t0 : a.batch);
     const char* src = static_cast<const char*>(x_host) + (size_t)t0 * row_bytes;
     if (n_batches == 1) {
       if (n > 0) CK(cudaMemcpyAsync(ws + a.x[0], src, (size_t)n * row_bytes, cudaMemcpyHostToDevice, st));

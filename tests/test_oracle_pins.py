@@ -372,3 +372,54 @@ def test_float32_rerun_within_tolerance():
                                                           Wu.astype(np.float64))
     s64, m64 = (lam64 * lam64).sum(axis=0), np.abs(lam64).max(axis=0) ** 2
     assert np.abs(s32 / s64 - 1).max() < 1e-4 and np.abs(m32 / m64 - 1).max() < 1e-4
+
+
+# ---------------------------------------------------------------- GetSubIndex and weight slicing (Alg. 2 lines 9-13, Alg. 3 line 8)
+def test_sliced_layer_decodes_like_the_retained_micro_experts():
+    """Slicing W_up[S,:], W_gate[S,:], W_down[:,S] (Alg. 2 lines 11-13) must give the layer whose output is
+    Phi[:,S] W[S,:], the Y-hat of Eq. 7 -- computed here from the full Phi and W, never from the slices."""
+    r = rng(40)
+    layer = random_layer(r, d=7, d_ff=(5, 4, 6, 3), n_shared=1, top_k=2, shared_gate=True, bias=True)
+    X = r.standard_normal((23, 7))
+    off = O.me_offsets(layer)
+    E = O.energy(*O.camera_components(layer, X), 0.5)
+    keep = O.select_prune(E, 0.4)
+    lists, counts = O.sub_index_lists(keep, off, [1])
+    assert counts.sum() == keep.sum() and [len(l) for l in lists] == counts[:, 0].tolist()
+    S = np.nonzero(keep)[0]
+    assert np.array_equal(np.concatenate([off[e] + lists[e] for e in range(4)]), S)       # ascending inside an expert
+    Y_hat = O.phi_matrix(layer, X)[:, S] @ O.basis(layer)[S, :]
+    assert np.allclose(O.forward(O.slice_layer(layer, lists), X), Y_hat, rtol=1e-12, atol=1e-12)
+    # and the error of that layer is the decoding error of the pruned set
+    err = ((O.forward(layer, X) - O.forward(O.slice_layer(layer, lists), X)) ** 2).sum()
+    assert abs(err - O.decode_error(O.phi_matrix(layer, X), O.basis(layer), np.nonzero(keep == 0)[0])) <= 1e-10 * max(err, 1)
+
+
+def test_reordering_by_class_keeps_the_layer_and_colocates_classes():
+    r = rng(41)
+    layer = random_layer(r, d=6, d_ff=(8, 5, 7), n_shared=0, top_k=2)
+    X = r.standard_normal((17, 6))
+    off = O.me_offsets(layer)
+    E = O.energy(*O.camera_components(layer, X), 0.95)
+    _, cls = O.alloc_bits(E, [0.25, 0.5, 0.25], [4, 3, 2])
+    lists, counts = O.sub_index_lists(cls, off, [0, 1, 2])
+    assert np.array_equal(counts, O.sub_index(cls, off, 3))
+    for e in range(3):
+        assert sorted(lists[e].tolist()) == list(range(layer.d_ff[e]))                     # a permutation
+        seg = cls[off[e]:off[e + 1]][lists[e]]
+        assert (np.diff(seg.astype(int)) >= 0).all()                                       # classes contiguous, in order
+        for j in range(3):                                                                 # stable inside a class
+            part = lists[e][seg == j]
+            assert (np.diff(part) > 0).all()
+    assert np.allclose(O.forward(O.slice_layer(layer, lists), X), O.forward(layer, X), rtol=1e-12, atol=1e-12)
+    # brute force: the same lists from a stable sort by (class, channel)
+    for e in range(3):
+        seg = cls[off[e]:off[e + 1]]
+        assert lists[e].tolist() == sorted(range(len(seg)), key=lambda i: (int(seg[i]), i))
+
+
+def test_sub_index_leaves_out_other_labels_and_handles_empty_experts():
+    labels = np.array([1, 0, 1, 1, 0, 0, 0, 1, 0], dtype=np.uint8)
+    lists, counts = O.sub_index_lists(labels, np.array([0, 4, 4, 7, 9]), [1])
+    assert [l.tolist() for l in lists] == [[0, 2, 3], [], [], [0]]
+    assert counts[:, 0].tolist() == [3, 0, 0, 1]
