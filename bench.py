@@ -184,6 +184,7 @@ def main():
     ap.add_argument("--cta-pair", action="store_true", help="score on CTA pairs (tcgen05 cta_group::2) instead of single CTAs")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--no-compact", action="store_true")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
     if args.impl == "reference":
@@ -267,6 +268,33 @@ def main():
     value = world * T * args.steps / (ms * 1e-3)
     ms_per_step = ms / args.steps
 
+    # ---- the selection applied to the weights (Algorithm 2 lines 9-13), timed on its own after the step loop
+    compact = None
+    if not args.no_compact:
+        off = P.expert_offsets_tensor(layer)
+        outw = {k: [torch.empty_like(w) for w in layer.tensors[k]] for k in ("w_gate", "w_up", "w_down")}
+        ws_c = P.alloc_workspace(4096 + 64 * layer.n_experts, dev)
+        c0, c1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        def apply_mask():
+            sub, counts = P.camera_sub_index(keep[1], off, [1])
+            P.camera_compact_weights(layer, sub, counts, 1, out=outw, workspace=ws_c)
+        for _ in range(3):
+            apply_mask()
+        sync_all()
+        c0.record(stream)
+        for _ in range(5):
+            apply_mask()
+        c1.record(stream)
+        sync_all()
+        c_ms = c0.elapsed_time(c1) / 5
+        kept = int(keep[1].sum().item())
+        esz = 2 if cfg.dtype == "bf16" else 4
+        c_bytes = 3 * 2 * kept * cfg.d_model * esz       # kept rows/columns of three matrices, read once and written once
+        compact = {"what": f"sub-index + gather of W_gate, W_up, W_down at prune ratio {PRUNE_RATIOS[1]}", "ms": c_ms,
+                   "algorithmic_gb": c_bytes / 1e9, "achieved_gbs": c_bytes / 1e9 / (c_ms * 1e-3),
+                   "frac_of_hbm_peak": c_bytes / 1e9 / (c_ms * 1e-3) / load_peaks()["hbm_gbs"]}
+        del outw
+
     # ---- end to end through the host-buffer entry point: H2D of the tokens, D2H of the results, every step
     e2e = None
     if not args.no_e2e:
@@ -332,7 +360,7 @@ def main():
                    "parallelism": f"layers x{world}" if world > 1 else "single GPU"},
         "model_seconds": cfg.n_layers * ms_per_step * 1e-3 / world,
         "stage_ms": stage_ms, "clocks": clocks, "e2e": e2e, "gpu_launches": LAUNCHES_PER_STEP * args.steps,
-        "roofline": roofline, "cpu_baseline": cpu, "context": PAPER_CONTEXT,
+        "roofline": roofline, "compact": compact, "cpu_baseline": cpu, "context": PAPER_CONTEXT,
     }
     print(json.dumps(out))
     if world > 1:

@@ -193,6 +193,41 @@ int camera_select_prune_static(const float* energy, const int64_t* seg_offsets, 
                                double prune_ratio, uint8_t* keep_mask, float* thresholds,
                                void* cuda_stream);
 
+/*
+ * GetSubIndex (Algorithm 3 line 8; the per-expert retained sets S of Algorithm 2 lines 9-10).
+ * labels: DEVICE [N_e] uint8, one per micro-expert -- a keep mask of camera_select_prune, or the
+ * bits_out of camera_alloc_bits.  expert_offsets: DEVICE int64 [n_experts+1], global micro-expert
+ * offsets.  label_order: HOST [n_labels] (1..8 distinct values 0..255).  For every expert e the
+ * channels (0 .. d_ff[e]-1) whose label is label_order[0] are written to
+ * sub_index[expert_offsets[e] ...] in ascending order, followed by those of label_order[1], and
+ * so on (a stable partition by label); micro-experts with any other label are left out and the
+ * tail of the expert's segment is not written.  counts: DEVICE [n_experts, n_labels], how many
+ * entries each label contributed.  With label_order = {1} on a keep mask the list is the retained
+ * set; with every bit-width in label_order it is the reordering that puts micro-experts of equal
+ * precision next to each other (Section "CAMERA-Q").
+ */
+int camera_sub_index(const uint8_t* labels, const int64_t* expert_offsets, int32_t n_experts,
+                     const int32_t* label_order, int32_t n_labels, int32_t* sub_index, int32_t* counts,
+                     void* cuda_stream);
+
+/* Scratch for camera_compact_weights. */
+size_t camera_compact_workspace_bytes(int32_t n_experts);
+
+/*
+ * Algorithm 2 lines 11-13: W_up <- W_up[S,:], W_gate <- W_gate[S,:], W_down <- W_down[:,S], with S
+ * the first m_e = counts[e,0] + .. + counts[e,n_take-1] entries of expert e's list in sub_index
+ * (both as written by camera_sub_index; DEVICE).  w_gate_out / w_up_out / w_down_out: HOST arrays
+ * of DEVICE pointers, one per expert, 16-byte aligned, with room for the worst case the caller
+ * allows (d_ff[e] rows is always enough): row r of w_gate_out[e] receives row sub_index[r] of
+ * w_gate[e], likewise w_up; W_down in CAMERA_DOWN_ME_MAJOR likewise; in CAMERA_DOWN_HF column j of
+ * w_down_out[e] (a [d_model, down_ld[e]] matrix; down_ld HOST, NULL = d_ff[e]) receives column
+ * sub_index[j].  Rows / columns from m_e on are not written.  Outputs must not overlap inputs.
+ */
+int camera_compact_weights(const camera_layer_t* layer, const int32_t* sub_index, const int32_t* counts,
+                           int32_t n_labels, int32_t n_take, void* const* w_gate_out, void* const* w_up_out,
+                           void* const* w_down_out, const int32_t* down_ld, void* workspace,
+                           size_t workspace_bytes, void* cuda_stream);
+
 /* Scratch for camera_analyze_layer_host: score + select scratch for one batch of tokens, two staging
  * buffers for batches of x, and the results. */
 size_t camera_analyze_workspace_bytes(const camera_layer_t* layer, int64_t n_tokens, int32_t n_levels);

@@ -77,6 +77,15 @@ def _load() -> C.CDLL:
                                               C.POINTER(C.c_double), C.POINTER(C.c_int32), C.c_int32,
                                               C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_size_t,
                                               C.c_void_p]
+    lib.camera_sub_index.restype = C.c_int
+    lib.camera_sub_index.argtypes = [C.c_void_p, C.c_void_p, C.c_int32, C.POINTER(C.c_int32), C.c_int32, C.c_void_p,
+                                     C.c_void_p, C.c_void_p]
+    lib.camera_compact_workspace_bytes.restype = C.c_size_t
+    lib.camera_compact_workspace_bytes.argtypes = [C.c_int32]
+    lib.camera_compact_weights.restype = C.c_int
+    lib.camera_compact_weights.argtypes = [C.POINTER(camera_layer_t), C.c_void_p, C.c_void_p, C.c_int32, C.c_int32,
+                                           C.POINTER(C.c_void_p), C.POINTER(C.c_void_p), C.POINTER(C.c_void_p),
+                                           C.POINTER(C.c_int32), C.c_void_p, C.c_size_t, C.c_void_p]
     return lib
 
 
@@ -326,3 +335,49 @@ def camera_analyze_layer_host(layer: Layer, x_host: torch.Tensor, alpha: float, 
                                          pr, n_prune, r, b, L, _ptr(energy_host), _ptr(keep_host),
                                          _ptr(bits_host), workspace.data_ptr(), workspace.numel(),
                                          _stream_ptr(stream)), "camera_analyze_layer_host")
+
+
+def expert_offsets_tensor(layer: Layer) -> torch.Tensor:
+    """Global micro-expert offsets of the layer's experts: int64 [n_experts + 1] on its device."""
+    off = [0]
+    for f in layer.d_ff:
+        off.append(off[-1] + f)
+    return torch.tensor(off, dtype=torch.int64, device=layer.device)
+
+
+def camera_sub_index(labels: torch.Tensor, expert_offsets: torch.Tensor, label_order: Sequence[int], *,
+                     stream: Optional[torch.cuda.Stream] = None):
+    """GetSubIndex.  labels uint8 [N_e] (keep mask or bit-widths), expert_offsets int64 [E+1] on the device.
+    Returns (sub_index int32 [N_e], counts int32 [E, len(label_order)])."""
+    if labels.dtype != torch.uint8 or not labels.is_contiguous():
+        raise ValueError("labels must be a contiguous uint8 tensor")
+    n_exp = expert_offsets.numel() - 1
+    order = (C.c_int32 * len(label_order))(*[int(v) for v in label_order])
+    sub = torch.empty(labels.numel(), dtype=torch.int32, device=labels.device)
+    counts = torch.empty((n_exp, len(label_order)), dtype=torch.int32, device=labels.device)
+    _check(lib.camera_sub_index(labels.data_ptr(), expert_offsets.data_ptr(), n_exp, order, len(label_order),
+                                sub.data_ptr(), counts.data_ptr(), _stream_ptr(stream)), "camera_sub_index")
+    return sub, counts
+
+
+def camera_compact_weights(layer: Layer, sub_index: torch.Tensor, counts: torch.Tensor, n_take: int, *,
+                           out: Optional[Dict[str, List[torch.Tensor]]] = None, down_ld: Optional[Sequence[int]] = None,
+                           workspace: Optional[torch.Tensor] = None, stream: Optional[torch.cuda.Stream] = None):
+    """Gathers W_gate[S,:], W_up[S,:], W_down[:,S] (Algorithm 2 lines 11-13) with S the entries of the first n_take
+    labels of every expert's list.  `out` = {"w_gate": [...], "w_up": [...], "w_down": [...]} (per expert, sized
+    like the sources unless down_ld says otherwise); allocated when missing.  Returns `out`; the rows / columns
+    actually written per expert are counts[:, :n_take].sum(1)."""
+    t = layer.tensors
+    if out is None:
+        out = {k: [torch.empty_like(w) for w in t[k]] for k in ("w_gate", "w_up", "w_down")}
+    n = layer.n_experts
+    pg = (C.c_void_p * n)(*[w.data_ptr() for w in out["w_gate"]])
+    pu = (C.c_void_p * n)(*[w.data_ptr() for w in out["w_up"]])
+    pd = (C.c_void_p * n)(*[w.data_ptr() for w in out["w_down"]])
+    ld = None if down_ld is None else (C.c_int32 * n)(*[int(v) for v in down_ld])
+    if workspace is None:
+        workspace = alloc_workspace(int(lib.camera_compact_workspace_bytes(n)), layer.device)
+    _check(lib.camera_compact_weights(C.byref(layer.c), sub_index.data_ptr(), counts.data_ptr(), int(counts.shape[1]),
+                                      int(n_take), pg, pu, pd, ld, workspace.data_ptr(), workspace.numel(),
+                                      _stream_ptr(stream)), "camera_compact_weights")
+    return out
