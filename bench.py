@@ -185,6 +185,7 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-compact", action="store_true")
+    ap.add_argument("--no-forward", action="store_true")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
     if args.impl == "reference":
@@ -269,7 +270,7 @@ def main():
     ms_per_step = ms / args.steps
 
     # ---- the selection applied to the weights (Algorithm 2 lines 9-13), timed on its own after the step loop
-    compact = None
+    compact = forward = None
     if not args.no_compact:
         off = P.expert_offsets_tensor(layer)
         outw = {k: [torch.empty_like(w) for w in layer.tensors[k]] for k in ("w_gate", "w_up", "w_down")}
@@ -278,6 +279,8 @@ def main():
         def apply_mask():
             sub, counts = P.camera_sub_index(keep[1], off, [1])
             P.camera_compact_weights(layer, sub, counts, 1, out=outw, workspace=ws_c)
+            return counts
+        counts = apply_mask()
         for _ in range(3):
             apply_mask()
         sync_all()
@@ -293,6 +296,33 @@ def main():
         compact = {"what": f"sub-index + gather of W_gate, W_up, W_down at prune ratio {PRUNE_RATIOS[1]}", "ms": c_ms,
                    "algorithmic_gb": c_bytes / 1e9, "achieved_gbs": c_bytes / 1e9 / (c_ms * 1e-3),
                    "frac_of_hbm_peak": c_bytes / 1e9 / (c_ms * 1e-3) / load_peaks()["hbm_gbs"]}
+        # ---- the output of the full and of the sliced layer on one batch of tokens, and their distance (Eq. 7)
+        if not args.no_forward and cfg.dtype == "bf16":
+            Tb = min(T, 65536)
+            xb = Xs[0][:Tb]
+            m = counts[:, 0].cpu().tolist()
+            sliced = P.Layer(L["w_router"], [outw["w_gate"][e][:m[e]] for e in range(layer.n_experts)],
+                             [outw["w_up"][e][:m[e]] for e in range(layer.n_experts)], outw["w_down"], cfg.top_k,
+                             cfg.n_shared, L["router_bias"], L["w_shared_gate"], cfg.norm_topk, "hf", down_ld=layer.d_ff)
+            ws_f = P.alloc_workspace(P.camera_forward_workspace_bytes(layer, Tb), dev)
+            yb = torch.empty((Tb, cfg.d_model), dtype=torch.float32, device=dev)
+            yh = torch.empty_like(yb)
+            def timed(fn, reps=3):
+                fn(); sync_all()
+                f0, f1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                f0.record(stream)
+                for _ in range(reps):
+                    fn()
+                f1.record(stream); sync_all()
+                return f0.elapsed_time(f1) / reps
+            full_ms = timed(lambda: P.camera_layer_forward(layer, xb, y=yb, workspace=ws_f))
+            sl_ms = timed(lambda: P.camera_layer_forward(sliced, xb, y=yh, workspace=ws_f))
+            err = P.camera_output_error(yb, yh).cpu().tolist()
+            flop_full = 1.5 * cfg.gate_up_flop * Tb / T
+            forward = {"tokens": Tb, "full_layer_ms": full_ms, "full_layer_tflops": flop_full / (full_ms * 1e-3) / 1e12,
+                       "sliced_layer_ms": sl_ms, "prune_ratio": PRUNE_RATIOS[1],
+                       "relative_output_error": err[0] / err[1] if err[1] > 0 else None, "mean_cosine": err[2]}
+            del ws_f, yb, yh
         del outw
 
     # ---- end to end through the host-buffer entry point: H2D of the tokens, D2H of the results, every step
@@ -360,7 +390,7 @@ def main():
                    "parallelism": f"layers x{world}" if world > 1 else "single GPU"},
         "model_seconds": cfg.n_layers * ms_per_step * 1e-3 / world,
         "stage_ms": stage_ms, "clocks": clocks, "e2e": e2e, "gpu_launches": LAUNCHES_PER_STEP * args.steps,
-        "roofline": roofline, "compact": compact, "cpu_baseline": cpu, "context": PAPER_CONTEXT,
+        "roofline": roofline, "compact": compact, "forward": forward, "cpu_baseline": cpu, "context": PAPER_CONTEXT,
     }
     print(json.dumps(out))
     if world > 1:

@@ -91,6 +91,9 @@ typedef struct {
   const void* const* w_gate;    /* HOST array of DEVICE pointers, each [d_ff[e], d_model] row-major */
   const void* const* w_up;      /* same */
   const void* const* w_down;    /* each per down_layout */
+  const int32_t* w_down_ld;     /* HOST [n_routed+n_shared] or NULL: leading dimension (elements) of each W_down in
+                                   CAMERA_DOWN_HF layout when its rows are longer than d_ff[e] (a sliced layer kept in
+                                   buffers of the original width); multiples of 8; NULL = d_ff[e] */
 } camera_layer_t;
 
 /* Optional inputs/outputs of camera_score_layer; any pointer may be NULL. All DEVICE. */
@@ -227,6 +230,35 @@ int camera_compact_weights(const camera_layer_t* layer, const int32_t* sub_index
                            int32_t n_labels, int32_t n_take, void* const* w_gate_out, void* const* w_up_out,
                            void* const* w_down_out, const int32_t* down_ld, void* workspace,
                            size_t workspace_bytes, void* cuda_stream);
+
+/* Scratch for camera_layer_forward (holds the token lists, h and the per-expert output rows). */
+size_t camera_forward_workspace_bytes(const camera_layer_t* layer, int64_t n_tokens);
+
+/*
+ * The layer's output, Eq. 1-2:  y_t = sum_e A_{t,e} W_down_e [ SiLU(W_gate_e x_t) * (W_up_e x_t) ],  with the
+ * router coefficients A of camera_score_layer (aux: topk_idx_in / topk_w_in prescribe them, topk_idx / topk_w /
+ * shared_w / expert_token_counts export them; other fields are ignored).  Applied to a layer sliced by
+ * camera_compact_weights it gives Y_hat = Phi[:,S] W[S,:], the retained micro-experts' output of Eq. 7.
+ * x: DEVICE [n_tokens, d_model] bf16;  y: DEVICE [n_tokens, d_model] fp32, 16-byte aligned.
+ * bf16 layers in CAMERA_DOWN_HF layout with d_model % 64 == 0 only (else CAMERA_ERR_UNSUPPORTED_SHAPE); d_ff[e] may
+ * be any value >= 0 (an expert that lost every micro-expert contributes nothing), provided W_down rows start on
+ * 16-byte boundaries: d_ff[e] % 8 == 0 or w_down_ld given.  Arithmetic: bf16 products with fp32 accumulation on
+ * tensor cores, h rounded to bf16 between the two GEMMs, a token's k + n_shared expert outputs added in fp32 in a
+ * fixed order.  Feed long calibration sets in batches: the workspace grows with n_tokens.
+ */
+int camera_layer_forward(const camera_layer_t* layer, const void* x, int64_t n_tokens, float* y,
+                         const camera_score_aux_t* aux, void* workspace, size_t workspace_bytes, void* cuda_stream);
+
+/* Scratch for camera_output_error. */
+size_t camera_output_error_workspace_bytes(int64_t n_tokens);
+
+/*
+ * Distance between two layer outputs (the metrics of the paper's table of hidden-state errors):
+ * out: DEVICE double[3] = { ||Y - Y_hat||_F^2 (the objective of Eq. 7), ||Y||_F^2, mean over tokens of the cosine
+ * similarity of y_t and y_hat_t }.  y, y_hat: DEVICE [n_tokens, d_model] fp32.  Sums in float64, fixed order.
+ */
+int camera_output_error(const float* y, const float* y_hat, int64_t n_tokens, int32_t d_model, double* out,
+                        void* workspace, size_t workspace_bytes, void* cuda_stream);
 
 /* Scratch for camera_analyze_layer_host: score + select scratch for one batch of tokens, two staging
  * buffers for batches of x, and the results. */

@@ -29,7 +29,8 @@ class camera_layer_t(C.Structure):
                 ("d_ff", C.POINTER(C.c_int32)), ("dtype", C.c_int32), ("flags", C.c_uint32),
                 ("down_layout", C.c_int32), ("w_router", C.c_void_p), ("router_bias", C.c_void_p),
                 ("w_shared_gate", C.c_void_p), ("w_gate", C.POINTER(C.c_void_p)),
-                ("w_up", C.POINTER(C.c_void_p)), ("w_down", C.POINTER(C.c_void_p))]
+                ("w_up", C.POINTER(C.c_void_p)), ("w_down", C.POINTER(C.c_void_p)),
+                ("w_down_ld", C.POINTER(C.c_int32))]
 
 
 class camera_score_aux_t(C.Structure):
@@ -77,6 +78,16 @@ def _load() -> C.CDLL:
                                               C.POINTER(C.c_double), C.POINTER(C.c_int32), C.c_int32,
                                               C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_size_t,
                                               C.c_void_p]
+    lib.camera_forward_workspace_bytes.restype = C.c_size_t
+    lib.camera_forward_workspace_bytes.argtypes = [C.POINTER(camera_layer_t), C.c_int64]
+    lib.camera_layer_forward.restype = C.c_int
+    lib.camera_layer_forward.argtypes = [C.POINTER(camera_layer_t), C.c_void_p, C.c_int64, C.c_void_p,
+                                         C.POINTER(camera_score_aux_t), C.c_void_p, C.c_size_t, C.c_void_p]
+    lib.camera_output_error_workspace_bytes.restype = C.c_size_t
+    lib.camera_output_error_workspace_bytes.argtypes = [C.c_int64]
+    lib.camera_output_error.restype = C.c_int
+    lib.camera_output_error.argtypes = [C.c_void_p, C.c_void_p, C.c_int64, C.c_int32, C.c_void_p, C.c_void_p, C.c_size_t,
+                                        C.c_void_p]
     lib.camera_sub_index.restype = C.c_int
     lib.camera_sub_index.argtypes = [C.c_void_p, C.c_void_p, C.c_int32, C.POINTER(C.c_int32), C.c_int32, C.c_void_p,
                                      C.c_void_p, C.c_void_p]
@@ -120,7 +131,8 @@ class Layer:
     """
 
     def __init__(self, w_router, w_gate: Sequence[torch.Tensor], w_up, w_down, top_k: int, n_shared: int = 0,
-                 router_bias=None, w_shared_gate=None, norm_topk: bool = True, down_layout: str = "hf"):
+                 router_bias=None, w_shared_gate=None, norm_topk: bool = True, down_layout: str = "hf",
+                 down_ld: Optional[Sequence[int]] = None):
         self.tensors = dict(w_router=w_router, router_bias=router_bias, w_shared_gate=w_shared_gate,
                             w_gate=list(w_gate), w_up=list(w_up), w_down=list(w_down))
         ref = w_gate[0]
@@ -147,7 +159,9 @@ class Layer:
             self.d_model, self.n_routed, top_k, n_shared, self._d_ff,
             CAMERA_BF16 if self.dtype == torch.bfloat16 else CAMERA_F32, flags,
             CAMERA_DOWN_HF if down_layout == "hf" else CAMERA_DOWN_ME_MAJOR,
-            _ptr(w_router), _ptr(router_bias), _ptr(w_shared_gate), self._wg, self._wu, self._wd)
+            _ptr(w_router), _ptr(router_bias), _ptr(w_shared_gate), self._wg, self._wu, self._wd,
+            None if down_ld is None else (C.c_int32 * n)(*[int(v) for v in down_ld]))
+        self._down_ld = self.c.w_down_ld      # keeps the array alive
         self.top_k = top_k
         self.n_shared = n_shared
 
@@ -380,4 +394,48 @@ def camera_compact_weights(layer: Layer, sub_index: torch.Tensor, counts: torch.
     _check(lib.camera_compact_weights(C.byref(layer.c), sub_index.data_ptr(), counts.data_ptr(), int(counts.shape[1]),
                                       int(n_take), pg, pu, pd, ld, workspace.data_ptr(), workspace.numel(),
                                       _stream_ptr(stream)), "camera_compact_weights")
+    return out
+
+
+def camera_forward_workspace_bytes(layer: Layer, n_tokens: int) -> int:
+    return int(lib.camera_forward_workspace_bytes(C.byref(layer.c), n_tokens))
+
+
+def camera_layer_forward(layer: Layer, x: torch.Tensor, *, y: Optional[torch.Tensor] = None, routing_in=None,
+                         workspace: Optional[torch.Tensor] = None, want_routing: bool = False,
+                         stream: Optional[torch.cuda.Stream] = None):
+    """The layer's output y [T, d_model] fp32 (Eq. 1-2).  routing_in = (topk_idx, topk_w) prescribes the routed
+    coefficients; want_routing also returns the (topk_idx, topk_w) the call used."""
+    T = int(x.shape[0])
+    dev = x.device
+    if y is None:
+        y = torch.empty((T, layer.d_model), dtype=torch.float32, device=dev)
+    if workspace is None:
+        workspace = alloc_workspace(camera_forward_workspace_bytes(layer, T), dev)
+    aux = camera_score_aux_t()
+    keep_alive = []
+    if routing_in is not None:
+        idx = routing_in[0].to(device=dev, dtype=torch.int32).contiguous()
+        w = routing_in[1].to(device=dev, dtype=torch.float32).contiguous()
+        keep_alive += [idx, w]
+        aux.topk_idx_in, aux.topk_w_in = idx.data_ptr(), w.data_ptr()
+    routing = None
+    if want_routing:
+        k = layer.top_k if layer.n_routed else 0
+        routing = (torch.empty((T, k), dtype=torch.int32, device=dev), torch.empty((T, k), dtype=torch.float32, device=dev))
+        aux.topk_idx, aux.topk_w = routing[0].data_ptr(), routing[1].data_ptr()
+    _check(lib.camera_layer_forward(C.byref(layer.c), x.data_ptr(), T, y.data_ptr(), C.byref(aux), workspace.data_ptr(),
+                                    workspace.numel(), _stream_ptr(stream)), "camera_layer_forward")
+    return (y, routing) if want_routing else y
+
+
+def camera_output_error(y: torch.Tensor, y_hat: torch.Tensor, *, stream: Optional[torch.cuda.Stream] = None) -> torch.Tensor:
+    """float64 [3] on the device: ||Y - Y_hat||_F^2, ||Y||_F^2, mean cosine similarity of the token outputs."""
+    if y.shape != y_hat.shape or y.dtype != torch.float32 or y_hat.dtype != torch.float32 or y.dim() != 2:
+        raise ValueError("y and y_hat must be fp32 [T, d_model] tensors of one shape")
+    T, d = int(y.shape[0]), int(y.shape[1])
+    out = torch.empty(3, dtype=torch.float64, device=y.device)
+    ws = alloc_workspace(int(lib.camera_output_error_workspace_bytes(T)), y.device)
+    _check(lib.camera_output_error(y.contiguous().data_ptr(), y_hat.contiguous().data_ptr(), T, d, out.data_ptr(),
+                                   ws.data_ptr(), ws.numel(), _stream_ptr(stream)), "camera_output_error")
     return out

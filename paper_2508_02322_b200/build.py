@@ -9,7 +9,7 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 ROOT = os.path.dirname(HERE)
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libcamera_b200.so")
-SOURCES = ["api.cu", "compact.cu", "router.cu", "router_umma.cu", "rownorm.cu", "score_simt.cu", "score_umma.cu", "score_umma2.cu", "select.cu"]
+SOURCES = ["api.cu", "compact.cu", "forward.cu", "router.cu", "router_umma.cu", "rownorm.cu", "score_simt.cu", "score_umma.cu", "score_umma2.cu", "select.cu"]
 
 
 def _nvcc() -> str:

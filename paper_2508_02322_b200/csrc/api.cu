@@ -37,7 +37,8 @@ struct ScoreLayout {
   long long max_part;
 };
 
-int validate_layer(const camera_layer_t* L, int64_t T) {
+// `forward`: the layer-forward entry point takes any d_ff >= 0 (a sliced layer), only in the paper's W_down layout.
+int validate_layer(const camera_layer_t* L, int64_t T, bool forward = false) {
   if (L == nullptr || L->d_ff == nullptr || L->w_gate == nullptr || L->w_up == nullptr || L->w_down == nullptr)
     return CAMERA_ERR_INVALID_ARG;
   if (L->dtype != CAMERA_F32 && L->dtype != CAMERA_BF16) return CAMERA_ERR_INVALID_ARG;
@@ -54,8 +55,13 @@ int validate_layer(const camera_layer_t* L, int64_t T) {
     return CAMERA_ERR_INVALID_ARG;
   long long n_me = 0;
   for (int e = 0; e < L->n_routed + L->n_shared; ++e) {
-    if (L->d_ff[e] < 8 || L->d_ff[e] % 8 != 0) return CAMERA_ERR_UNSUPPORTED_SHAPE;
-    if (L->w_gate[e] == nullptr || L->w_up[e] == nullptr || L->w_down[e] == nullptr) return CAMERA_ERR_INVALID_ARG;
+    if (forward ? L->d_ff[e] < 0 : (L->d_ff[e] < 8 || L->d_ff[e] % 8 != 0)) return CAMERA_ERR_UNSUPPORTED_SHAPE;
+    if ((L->w_gate[e] == nullptr || L->w_up[e] == nullptr || L->w_down[e] == nullptr) && L->d_ff[e] > 0)
+      return CAMERA_ERR_INVALID_ARG;     // an expert without micro-experts needs no matrices
+    if (L->w_down_ld != nullptr) {
+      if (L->down_layout != CAMERA_DOWN_HF || L->w_down_ld[e] < L->d_ff[e] || L->w_down_ld[e] < 8 || L->w_down_ld[e] % 8 != 0)
+        return CAMERA_ERR_INVALID_ARG;
+    }
     n_me += L->d_ff[e];
   }
   if (n_me >= (1ll << 31)) return CAMERA_ERR_UNSUPPORTED_SHAPE;
@@ -171,12 +177,23 @@ extern "C" size_t camera_score_workspace_bytes(const camera_layer_t* layer, int6
   return score_layout(layer, n_tokens).total;
 }
 
-extern "C" int camera_score_layer(const camera_layer_t* L, const void* x, int64_t T, float alpha, float* energy,
-                                  const camera_score_aux_t* aux, void* workspace, size_t workspace_bytes,
-                                  void* cuda_stream) {
-  int rc = validate_layer(L, T);
+namespace camera {
+
+size_t score_workspace_bytes_any(const camera_layer_t* L, int64_t T, bool forward) {
+  if (validate_layer(L, T, forward) != CAMERA_OK) return 0;
+  return score_layout(L, T).total;
+}
+
+// Everything of camera_score_layer up to the token lists: checks, workspace carving, tables and tensor
+// maps, router, plan, permutation.  `fwd` (layer forward) relaxes the shape rules and names, per expert,
+// where the intermediate h and the expert's output rows go.
+int score_front(const camera_layer_t* L, const void* x, int64_t T, float alpha, float* energy,
+                const camera_score_aux_t* aux, void* workspace, size_t workspace_bytes, cudaStream_t st,
+                const ForwardBuffers* fwd, ScoreFront* out) {
+  int rc = validate_layer(L, T, fwd != nullptr);
   if (rc != CAMERA_OK) return rc;
-  if (!(alpha >= 0.f && alpha <= 1.f) || energy == nullptr || (T > 0 && x == nullptr)) return CAMERA_ERR_INVALID_ARG;
+  if (!(alpha >= 0.f && alpha <= 1.f) || (energy == nullptr && fwd == nullptr) || (T > 0 && x == nullptr))
+    return CAMERA_ERR_INVALID_ARG;
   if (aux && ((aux->topk_idx_in == nullptr) != (aux->topk_w_in == nullptr))) return CAMERA_ERR_INVALID_ARG;
   const bool accumulate = aux && (aux->flags & CAMERA_SCORE_ACCUMULATE);
   if (accumulate && (aux->phi2 == nullptr || aux->phi_inf_sq == nullptr)) return CAMERA_ERR_INVALID_ARG;
@@ -195,11 +212,10 @@ extern "C" int camera_score_layer(const camera_layer_t* L, const void* x, int64_
   CK(cudaGetDevice(&dev));
   CK(cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev));
   if (major != 10) return CAMERA_ERR_ARCH;
-  cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
   char* ws = static_cast<char*>(workspace);
   const int E = lay.n_experts;
 
-  ScoreCtx c;
+  ScoreCtx& c = out->c;
   memset(&c, 0, sizeof(c));
   c.d_model = L->d_model; c.n_routed = L->n_routed; c.top_k = L->n_routed > 0 ? L->top_k : 0;
   c.n_shared = L->n_shared; c.n_experts = E; c.n_me = lay.n_me;
@@ -238,6 +254,10 @@ extern "C" int camera_score_layer(const camera_layer_t* L, const void* x, int64_
     est[e].d_ff = L->d_ff[e]; est[e].me_off = me;
     est[e].shared_idx = e < L->n_routed ? -1 : e - L->n_routed;
     est[e].norm_blk_begin = norm_blocks;
+    est[e].down_ld = L->w_down_ld ? L->w_down_ld[e] : L->d_ff[e];
+    est[e].h_ld = fwd ? fwd->h_ld[e] : 0;
+    est[e].h = fwd ? fwd->h[e] : nullptr;
+    est[e].y_part = fwd ? fwd->y_part[e] : nullptr;
     me_prefix[e] = me;
     me += L->d_ff[e];
     norm_blocks += rownorm_blocks(L->down_layout, L->dtype, L->d_ff[e]);
@@ -246,7 +266,7 @@ extern "C" int camera_score_layer(const camera_layer_t* L, const void* x, int64_
 
   const bool use_umma = umma_shape_ok(L) && !(aux && (aux->flags & CAMERA_SCORE_FORCE_SIMT)) &&
                         (reinterpret_cast<uintptr_t>(x) & 15) == 0;
-  const bool use_pair = use_umma && aux && (aux->flags & CAMERA_SCORE_CTA_PAIR);
+  const bool use_pair = use_umma && fwd == nullptr && aux && (aux->flags & CAMERA_SCORE_CTA_PAIR);
   c.ch_tile = use_pair ? 2 * CH_TILE : CH_TILE;
   c.ct_group = score_group_channels() / c.ch_tile;
   const bool use_router_umma = use_umma && router_umma_ok(c);
@@ -281,6 +301,26 @@ extern "C" int camera_score_layer(const camera_layer_t* L, const void* x, int64_
   CK(launch_plan(c, st));
   CK(launch_permute(c, st));
   tm.end(CAMERA_STAGE_PERMUTE);
+  out->norm_blocks = norm_blocks;
+  out->use_umma = use_umma;
+  out->use_pair = use_pair;
+  return CAMERA_OK;
+}
+
+}  // namespace camera
+
+extern "C" int camera_score_layer(const camera_layer_t* L, const void* x, int64_t T, float alpha, float* energy,
+                                  const camera_score_aux_t* aux, void* workspace, size_t workspace_bytes,
+                                  void* cuda_stream) {
+  if (energy == nullptr) return CAMERA_ERR_INVALID_ARG;
+  cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+  ScoreFront f;
+  const int rc = score_front(L, x, T, alpha, energy, aux, workspace, workspace_bytes, st, nullptr, &f);
+  if (rc != CAMERA_OK) return rc;
+  const ScoreCtx& c = f.c;
+  const bool use_umma = f.use_umma, use_pair = f.use_pair;
+  const int norm_blocks = f.norm_blocks;
+  const StageTimer tm{aux, st};
 
   tm.begin(CAMERA_STAGE_ROWNORM);
   CK(launch_rownorm(c, norm_blocks, st));

@@ -28,6 +28,11 @@ struct ExpertStatic {
   int32_t me_off;        // global micro-expert offset
   int32_t shared_idx;    // -1 for routed experts, else index among the shared ones
   int32_t norm_blk_begin;  // first CTA of the row-norm grid that belongs to this expert
+  int32_t down_ld;       // leading dimension of w_down in the [d_model, d_ff] layout
+  int32_t h_ld;          // layer forward only: leading dimension of h
+  void* h;               // layer forward only: this expert's intermediate A * SiLU(W_gate x) * (W_up x), bf16, one row
+                         // per row of its token list (routed: indexed like x_perm; shared: like x)
+  float* y_part;         // layer forward only: this expert's output rows [rows, d_model] fp32, indexed like h
 };
 
 // Facts only the device knows (they depend on the routing); written by k_plan.
@@ -37,13 +42,15 @@ struct ExpertDyn {
   int32_t n_chunks;      // ceil(rows / chunk_tokens)
   int32_t unit_begin;    // exclusive prefix over experts of n_chunks * ceil(d_ff / ch_tile)
   int64_t part_begin;    // exclusive prefix over experts of n_chunks * d_ff (offset into the partials)
+  int32_t chunk_begin;   // exclusive prefix over experts of n_chunks
+  int32_t pad;
 };
 
 struct PlanTotals {
   int32_t total_units;
   int32_t total_rows;    // rows of x_perm in use (padded)
   int32_t status;        // device status word (0 = fine)
-  int32_t pad;
+  int32_t total_chunks;  // sum over experts of n_chunks
 };
 
 // Everything the kernels of one camera_score_layer call need.
@@ -87,6 +94,22 @@ struct ScoreCtx {
                          // x, w_router, w_shared_gate (router); x_perm in boxes of 128 rows (CTA pairs)
 };
 
+// What camera_layer_forward hands to score_front: per expert (HOST arrays), where h and the output rows go.
+struct ForwardBuffers {
+  void* const* h;
+  const int32_t* h_ld;
+  float* const* y_part;
+};
+struct ScoreFront {
+  ScoreCtx c;
+  int norm_blocks;
+  bool use_umma, use_pair;
+};
+int score_front(const camera_layer_t* L, const void* x, int64_t T, float alpha, float* energy,
+                const camera_score_aux_t* aux, void* workspace, size_t workspace_bytes, cudaStream_t st,
+                const ForwardBuffers* fwd, ScoreFront* out);
+size_t score_workspace_bytes_any(const camera_layer_t* L, int64_t T, bool forward);
+
 // ---- launches (each enqueues on `st`, returns the launch's cudaError_t) ------------------------
 cudaError_t launch_router(const ScoreCtx& c, cudaStream_t st);
 cudaError_t launch_routing_from_input(const ScoreCtx& c, const int32_t* idx_in, const float* w_in, cudaStream_t st);
@@ -98,6 +121,7 @@ cudaError_t launch_score_umma(const ScoreCtx& c, cudaStream_t st);
 cudaError_t launch_score_umma_pair(const ScoreCtx& c, cudaStream_t st);
 cudaError_t launch_combine(const ScoreCtx& c, cudaStream_t st);
 cudaError_t launch_router_umma(const ScoreCtx& c, const int32_t* idx_in, const float* w_in, cudaStream_t st);
+cudaError_t launch_score_umma_write_h(const ScoreCtx& c, cudaStream_t st);
 bool umma_shape_ok(const camera_layer_t* L);
 bool router_umma_ok(const ScoreCtx& c);
 int encode_tensor_maps(const camera_layer_t* L, const ScoreCtx& c, void* host_maps /* 128 B each */);
@@ -105,6 +129,8 @@ int encode_router_maps(const ScoreCtx& c, void* host_maps);
 // Tensor map of a bf16 row-major [rows, d] matrix in boxes of 64 columns x box_rows rows with the
 // 128-byte swizzle (a null matrix gives an all-zero map that must not be used).
 bool encode_bf16_2d(void* out, const void* ptr, uint64_t rows, uint64_t d, uint32_t box_rows);
+// The same for rows of `cols` elements that lie `pitch` elements apart.
+bool encode_bf16_2d_pitch(void* out, const void* ptr, uint64_t rows, uint64_t cols, uint64_t pitch, uint32_t box_rows);
 
 // ---- device helpers ------------------------------------------------------------------------------
 template <typename T> __device__ __forceinline__ float to_f32(T v);

@@ -1,0 +1,409 @@
+// The layer's output (Eq. 1-2): y_t = sum_e A_{t,e} W_down_e [ SiLU(W_gate_e x_t) * (W_up_e x_t) ], on the routing and
+// token lists of the scoring path.  It exists to evaluate a selection: the output of the sliced layer is
+// Y_hat = Phi[:,S] W[S,:] of Eq. 7, and camera_output_error gives ||Y - Y_hat||_F^2 and the cosine similarity.
+//
+//   k_score_umma<WRITE_H>   h = A * SiLU(W_gate x) * (W_up x) per (token row, micro-expert), bf16      (score_umma.cu)
+//   k_down_umma             y_part[row, :] = W_down h[row, :] per expert, tcgen05, fp32 out
+//   k_unpermute_sum         y[t, :] = sum over the token's k routed rows and its shared-expert rows, fixed order
+#include <string.h>
+
+#include <vector>
+
+#include "common.cuh"
+#include "umma.cuh"
+
+namespace camera {
+
+namespace {
+
+constexpr int D_THREADS = 192;
+constexpr int D_STAGES = 4;
+constexpr int D_TILE = 128;                       // output channels (rows of W_down) per work unit = TMEM lanes
+constexpr int D_A_BYTES = D_TILE * 128;
+constexpr int D_B_BYTES = UMMA_TOK * 128;
+constexpr int D_STAGE_BYTES = D_A_BYTES + D_B_BYTES;
+constexpr int D_TMEM_COLS = 512;
+constexpr int D_SMEM_BYTES = D_STAGES * D_STAGE_BYTES + 256 + 1024;
+
+struct DownUnit {
+  int e, rows, row0, c0, n_kb, row_limit;
+  float* y;
+};
+
+// Work units are numbered (token chunk, output-channel tile) with the tile fastest: the CTAs running at one time
+// share a chunk of h through L2 while an expert's W_down stays resident.
+__device__ __forceinline__ DownUnit decode_down_unit(const ScoreCtx& c, int unit, int n_dt) {
+  DownUnit u;
+  const int chunk = unit / n_dt;
+  int lo = 0, hi = c.n_experts;
+  while (hi - lo > 1) {
+    const int mid = (lo + hi) >> 1;
+    if (c.edyn[mid].chunk_begin <= chunk) lo = mid; else hi = mid;
+  }
+  u.e = lo;
+  const ExpertDyn dy = c.edyn[lo];
+  const ExpertStatic es = c.est[lo];
+  const int ck = chunk - dy.chunk_begin;
+  u.rows = min(c.chunk_tokens, dy.rows - ck * c.chunk_tokens);
+  u.row0 = dy.row_base + ck * c.chunk_tokens;
+  u.c0 = (unit % n_dt) * D_TILE;
+  u.n_kb = (es.d_ff + UMMA_BK - 1) / UMMA_BK;
+  u.row_limit = (es.shared_idx < 0 ? c.max_rows_perm : c.n_tokens) - u.row0;
+  u.y = es.y_part;
+  return u;
+}
+
+__global__ void __launch_bounds__(D_THREADS, 1) k_down_umma(const ScoreCtx c, const void* maps_raw, int n_dt) {
+  extern __shared__ uint8_t smem_raw[];
+  const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+  uint8_t* const base_ptr = smem_raw + (base - smem_u32(smem_raw));
+  const uint32_t bars = base + D_STAGES * D_STAGE_BYTES;
+  auto full_bar = [&](int s) { return bars + 8u * s; };
+  auto empty_bar = [&](int s) { return bars + 8u * (D_STAGES + s); };
+  auto tfull_bar = [&](int a) { return bars + 8u * (2 * D_STAGES + a); };
+  auto tempty_bar = [&](int a) { return bars + 8u * (2 * D_STAGES + 2 + a); };
+  uint8_t* const tail = base_ptr + D_STAGES * D_STAGE_BYTES + 8 * (2 * D_STAGES + 4);
+  volatile uint32_t* const tmem_slot = reinterpret_cast<volatile uint32_t*>(tail);
+  volatile int* const abort_flag = reinterpret_cast<volatile int*>(tail + 8);
+
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const int total_units = c.totals->total_chunks * n_dt;
+
+  if (tid == 0) {
+    for (int s = 0; s < D_STAGES; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
+    for (int a = 0; a < 2; ++a) { mbar_init(tfull_bar(a), 1); mbar_init(tempty_bar(a), 128); }
+    *abort_flag = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+  }
+  if (warp == 5) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32((const void*)tmem_slot)),
+                 "r"(D_TMEM_COLS)
+                 : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = *tmem_slot;
+
+  if (warp == 4) {
+    // ------------------------------------------------------------------ TMA producer
+    if (lane == 0) {
+      int stage = 0;
+      uint32_t phase = 0;
+      bool ok = true;
+      const char* maps = static_cast<const char*>(maps_raw);
+      for (int unit = blockIdx.x; ok && unit < total_units; unit += gridDim.x) {
+        const DownUnit u = decode_down_unit(c, unit, n_dt);
+        if (u.n_kb == 0) continue;
+        const int n_tiles = (u.rows + UMMA_TOK - 1) / UMMA_TOK;
+        const void* map_w = maps + (size_t)128 * (2 * u.e);
+        const void* map_h = maps + (size_t)128 * (2 * u.e + 1);
+        tensormap_acquire(map_w);
+        tensormap_acquire(map_h);
+        for (int tt = 0; ok && tt < n_tiles; ++tt) {
+          const int row = u.row0 + tt * UMMA_TOK;
+          for (int kb = 0; kb < u.n_kb; ++kb) {
+            if (!mbar_wait(empty_bar(stage), phase ^ 1u, abort_flag)) { ok = false; break; }
+            const uint32_t a_dst = base + stage * D_STAGE_BYTES;
+            mbar_expect_tx(full_bar(stage), D_STAGE_BYTES);
+            // W_down columns past d_ff and rows past d_model, h rows past the buffer: filled with zeros
+            tma_load_2d(a_dst, map_w, full_bar(stage), kb * UMMA_BK, u.c0);
+            tma_load_2d(a_dst + D_A_BYTES, map_h, full_bar(stage), kb * UMMA_BK, row);
+            if (++stage == D_STAGES) { stage = 0; phase ^= 1u; }
+          }
+        }
+      }
+      if (!ok) {
+        const unsigned long long t0 = globaltimer_ns();
+        while (globaltimer_ns() - t0 < 2000000ull) __nanosleep(1000);
+      }
+    }
+  } else if (warp == 5) {
+    // ------------------------------------------------------------------ MMA issuer
+    if (lane == 0) {
+      int stage = 0, acc = 0;
+      uint32_t phase = 0, acc_phase = 0;
+      bool ok = true;
+      for (int unit = blockIdx.x; ok && unit < total_units; unit += gridDim.x) {
+        const DownUnit u = decode_down_unit(c, unit, n_dt);
+        if (u.n_kb == 0) continue;
+        const int n_tiles = (u.rows + UMMA_TOK - 1) / UMMA_TOK;
+        for (int tt = 0; ok && tt < n_tiles; ++tt) {
+          const int nv = (min(UMMA_TOK, u.rows - tt * UMMA_TOK) + 15) & ~15;
+          const uint32_t idesc = make_idesc(nv);
+          if (!mbar_wait(tempty_bar(acc), acc_phase ^ 1u, abort_flag)) { ok = false; break; }
+          tc_fence_after();
+          const uint32_t d_tmem = tmem_base + (uint32_t)(acc * UMMA_TOK);
+          for (int kb = 0; kb < u.n_kb; ++kb) {
+            if (!mbar_wait(full_bar(stage), phase, abort_flag)) { ok = false; break; }
+            tc_fence_after();
+            const uint32_t a_addr = base + stage * D_STAGE_BYTES;
+            const unsigned long long a_desc = make_smem_desc(a_addr);
+            const unsigned long long b_desc = make_smem_desc(a_addr + D_A_BYTES);
+#pragma unroll
+            for (int k = 0; k < UMMA_BK / 16; ++k)
+              umma_bf16(d_tmem, a_desc + 2 * k, b_desc + 2 * k, idesc, (uint32_t)((kb | k) != 0));
+            umma_commit(empty_bar(stage));
+            if (++stage == D_STAGES) { stage = 0; phase ^= 1u; }
+          }
+          if (!ok) break;
+          umma_commit(tfull_bar(acc));
+          if (++acc == 2) { acc = 0; acc_phase ^= 1u; }
+        }
+      }
+    }
+  } else {
+    // ------------------------------------------------------------------ epilogue (warps 0-3): lane = output channel
+    int acc = 0;
+    uint32_t acc_phase = 0;
+    bool ok = true;
+    for (int unit = blockIdx.x; ok && unit < total_units; unit += gridDim.x) {
+      const DownUnit u = decode_down_unit(c, unit, n_dt);
+      const int n_tiles = (u.rows + UMMA_TOK - 1) / UMMA_TOK;
+      const int ch = u.c0 + warp * 32 + lane;
+      float* const ycol = u.y + (size_t)u.row0 * c.d_model + ch;
+      for (int tt = 0; ok && tt < n_tiles; ++tt) {
+        const int nv = (min(UMMA_TOK, u.rows - tt * UMMA_TOK) + 15) & ~15;
+        const int n_store = min(nv, u.row_limit - tt * UMMA_TOK);
+        float* const ytile = ycol + (size_t)tt * UMMA_TOK * c.d_model;
+        if (u.n_kb == 0) {   // an expert without micro-experts contributes zeros
+          if (ch < c.d_model)
+            for (int j = 0; j < n_store; ++j) ytile[(size_t)j * c.d_model] = 0.f;
+          continue;
+        }
+        ok = __all_sync(0xffffffffu, mbar_wait(tfull_bar(acc), acc_phase, abort_flag));
+        if (!ok) break;
+        tc_fence_after();
+        const uint32_t taddr = tmem_base + ((uint32_t)(warp * 32) << 16) + (uint32_t)(acc * UMMA_TOK);
+        for (int c0 = 0; c0 < nv; c0 += 16) {
+          uint32_t v[16];
+          tmem_ld16(taddr + c0, v);
+          tmem_ld_wait(v);
+          if (ch < c.d_model) {
+#pragma unroll
+            for (int j = 0; j < 16; ++j)     // a warp writes 32 consecutive channels of one token row: 128 bytes
+              if (c0 + j < n_store) ytile[(size_t)(c0 + j) * c.d_model] = __uint_as_float(v[j]);
+          }
+        }
+        tc_fence_before();
+        mbar_arrive(tempty_bar(acc));
+        if (++acc == 2) { acc = 0; acc_phase ^= 1u; }
+      }
+    }
+  }
+
+  tc_fence_before();
+  __syncthreads();
+  if (*abort_flag && tid == 0) atomicExch(&c.totals->status, (int)CAMERA_ERR_DEVICE_TIMEOUT);
+  if (warp == 5) {
+    __syncwarp();
+    tc_fence_after();
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(D_TMEM_COLS) : "memory");
+  }
+}
+
+// One warp per token: y[t, :] = its k routed rows of y_perm (in slot order) plus its row of every shared expert.
+__global__ void __launch_bounds__(256) k_unpermute_sum(const ScoreCtx c, float* __restrict__ y) {
+  const int lane = threadIdx.x & 31;
+  const int t = blockIdx.x * 8 + (threadIdx.x >> 5);
+  if (t >= c.n_tokens) return;
+  const int k = c.top_k, d = c.d_model;
+  long long pos_l = 0;
+  if (lane < k) {
+    const int e = c.topk_idx[(size_t)t * k + lane];
+    pos_l = c.edyn[e].row_base + c.block_hist[(size_t)(t / ROUTER_TOK) * c.n_routed + e] + c.local_rank[(size_t)t * k + lane];
+  }
+  const float* routed = c.n_routed > 0 ? c.est[0].y_part : nullptr;
+  for (int v = lane * 4; v < d; v += 128) {
+    float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+    for (int s = 0; s < k; ++s) {
+      const long long pos = __shfl_sync(0xffffffffu, pos_l, s);
+      const float4 p = *reinterpret_cast<const float4*>(routed + (size_t)pos * d + v);
+      acc.x += p.x; acc.y += p.y; acc.z += p.z; acc.w += p.w;
+    }
+    for (int s = 0; s < c.n_shared; ++s) {
+      const float4 p = *reinterpret_cast<const float4*>(c.est[c.n_routed + s].y_part + (size_t)t * d + v);
+      acc.x += p.x; acc.y += p.y; acc.z += p.z; acc.w += p.w;
+    }
+    *reinterpret_cast<float4*>(y + (size_t)t * d + v) = acc;
+  }
+}
+
+// Per CTA of 8 tokens: sum (y - y_hat)^2, sum y^2, sum of the tokens' cosine similarities, in double.
+__global__ void __launch_bounds__(256) k_error_partials(const float* __restrict__ y, const float* __restrict__ yh,
+                                                        long long n_tokens, int d, double* __restrict__ part) {
+  __shared__ double red[8][3];
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  const long long t = (long long)blockIdx.x * 8 + warp;
+  double e2 = 0.0, n2 = 0.0, cs = 0.0;
+  if (t < n_tokens) {
+    double dot = 0.0, h2 = 0.0;
+    for (int v = lane; v < d; v += 32) {
+      const double a = y[(size_t)t * d + v], b = yh[(size_t)t * d + v];
+      e2 += (a - b) * (a - b); n2 += a * a; h2 += b * b; dot += a * b;
+    }
+#pragma unroll
+    for (int o = 16; o; o >>= 1) {
+      e2 += __shfl_xor_sync(0xffffffffu, e2, o); n2 += __shfl_xor_sync(0xffffffffu, n2, o);
+      h2 += __shfl_xor_sync(0xffffffffu, h2, o); dot += __shfl_xor_sync(0xffffffffu, dot, o);
+    }
+    cs = (n2 > 0.0 && h2 > 0.0) ? dot / sqrt(n2 * h2) : (n2 == h2 ? 1.0 : 0.0);
+  }
+  if (lane == 0) { red[warp][0] = e2; red[warp][1] = n2; red[warp][2] = cs; }
+  __syncthreads();
+  if (threadIdx.x < 3) {
+    double s = 0.0;
+    for (int w = 0; w < 8; ++w) s += red[w][threadIdx.x];
+    part[(size_t)blockIdx.x * 3 + threadIdx.x] = s;
+  }
+}
+
+// One CTA adds the partials in a fixed order.
+__global__ void __launch_bounds__(256) k_error_final(const double* __restrict__ part, long long n_part, long long n_tokens,
+                                                     double* __restrict__ out) {
+  __shared__ double red[256][3];
+  double s[3] = {0.0, 0.0, 0.0};
+  for (long long i = threadIdx.x; i < n_part; i += 256)
+    for (int j = 0; j < 3; ++j) s[j] += part[i * 3 + j];
+  for (int j = 0; j < 3; ++j) red[threadIdx.x][j] = s[j];
+  __syncthreads();
+  if (threadIdx.x < 3) {
+    double t = 0.0;
+    for (int i = 0; i < 256; ++i) t += red[i][threadIdx.x];
+    out[threadIdx.x] = threadIdx.x == 2 ? (n_tokens > 0 ? t / (double)n_tokens : 1.0) : t;
+  }
+}
+
+size_t up256(size_t v) { return (v + 255) & ~(size_t)255; }
+
+struct FwdLayout {
+  size_t score, maps, h_routed, y_perm, total, score_bytes;
+  std::vector<size_t> h_shared, y_shared;
+  int h_ld_routed, max_rows_perm;
+  std::vector<int> h_ld;
+};
+
+FwdLayout fwd_layout(const camera_layer_t* L, int64_t T) {
+  FwdLayout f;
+  const int E = L->n_routed + L->n_shared;
+  const int k = L->n_routed > 0 ? L->top_k : 0;
+  f.score_bytes = score_workspace_bytes_any(L, T, true);
+  f.max_rows_perm = (int)(T * k + (long long)ROW_ALIGN * L->n_routed);
+  int f_max = 0;
+  for (int e = 0; e < L->n_routed; ++e) f_max = L->d_ff[e] > f_max ? L->d_ff[e] : f_max;
+  f.h_ld_routed = ((f_max + CH_TILE - 1) / CH_TILE) * CH_TILE;
+  if (f.h_ld_routed == 0) f.h_ld_routed = CH_TILE;
+  f.h_ld.resize(E);
+  size_t o = 0;
+  auto take = [&](size_t bytes) { size_t at = o; o = up256(o + bytes); return at; };
+  f.score = take(f.score_bytes);
+  f.maps = take((size_t)128 * 2 * E);
+  f.h_routed = take(L->n_routed > 0 ? (size_t)2 * f.max_rows_perm * f.h_ld_routed : 0);
+  f.y_perm = take(L->n_routed > 0 ? sizeof(float) * (size_t)f.max_rows_perm * L->d_model : 0);
+  for (int e = 0; e < E; ++e) {
+    if (e < L->n_routed) { f.h_ld[e] = f.h_ld_routed; continue; }
+    f.h_ld[e] = ((L->d_ff[e] + CH_TILE - 1) / CH_TILE) * CH_TILE;
+    if (f.h_ld[e] == 0) f.h_ld[e] = CH_TILE;
+    f.h_shared.push_back(take((size_t)2 * T * f.h_ld[e]));
+    f.y_shared.push_back(take(sizeof(float) * (size_t)T * L->d_model));
+  }
+  f.total = o;
+  return f;
+}
+
+}  // namespace
+}  // namespace camera
+
+using namespace camera;
+
+extern "C" size_t camera_forward_workspace_bytes(const camera_layer_t* layer, int64_t n_tokens) {
+  if (score_workspace_bytes_any(layer, n_tokens, true) == 0) return 0;
+  return fwd_layout(layer, n_tokens).total;
+}
+
+extern "C" int camera_layer_forward(const camera_layer_t* L, const void* x, int64_t T, float* y,
+                                    const camera_score_aux_t* aux, void* workspace, size_t workspace_bytes,
+                                    void* cuda_stream) {
+  if (L == nullptr || y == nullptr || (reinterpret_cast<uintptr_t>(y) & 15)) return CAMERA_ERR_INVALID_ARG;
+  if (score_workspace_bytes_any(L, T, true) == 0) return CAMERA_ERR_INVALID_ARG;
+  if (L->dtype != CAMERA_BF16 || L->down_layout != CAMERA_DOWN_HF || L->d_model % UMMA_BK != 0 || !umma_shape_ok(L) ||
+      (reinterpret_cast<uintptr_t>(x) & 15))
+    return CAMERA_ERR_UNSUPPORTED_SHAPE;
+  const FwdLayout fl = fwd_layout(L, T);
+  if (workspace == nullptr || workspace_bytes < fl.total || (reinterpret_cast<uintptr_t>(workspace) & 255))
+    return CAMERA_ERR_WORKSPACE;
+  cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+  char* ws = static_cast<char*>(workspace);
+  const int E = L->n_routed + L->n_shared;
+  std::vector<void*> h(E);
+  std::vector<float*> yp(E);
+  for (int e = 0; e < E; ++e) {
+    if (e < L->n_routed) {
+      h[e] = ws + fl.h_routed;
+      yp[e] = reinterpret_cast<float*>(ws + fl.y_perm);
+    } else {
+      h[e] = ws + fl.h_shared[e - L->n_routed];
+      yp[e] = reinterpret_cast<float*>(ws + fl.y_shared[e - L->n_routed]);
+    }
+    if (L->w_down_ld == nullptr && L->d_ff[e] % 8 != 0) return CAMERA_ERR_UNSUPPORTED_SHAPE;   // TMA row pitch: 16 bytes
+  }
+  const ForwardBuffers fb{h.data(), fl.h_ld.data(), yp.data()};
+  camera_score_aux_t a2;
+  memset(&a2, 0, sizeof(a2));
+  if (aux) { a2 = *aux; a2.flags &= ~(uint32_t)(CAMERA_SCORE_FORCE_SIMT | CAMERA_SCORE_CTA_PAIR | CAMERA_SCORE_ACCUMULATE); }
+  ScoreFront f;
+  int rc = score_front(L, x, T, 0.f, nullptr, &a2, ws + fl.score, fl.score_bytes, st, &fb, &f);
+  if (rc != CAMERA_OK) return rc;
+  if (!f.use_umma) return CAMERA_ERR_UNSUPPORTED_SHAPE;
+  if (T == 0) return CAMERA_OK;
+  const ScoreCtx& c = f.c;
+
+  // tensor maps of the second GEMM: per expert W_down [d_model rows, d_ff] and h [rows, h_ld]
+  std::vector<char> maps((size_t)128 * 2 * E);
+  for (int e = 0; e < E; ++e) {
+    const int ld = L->w_down_ld ? L->w_down_ld[e] : L->d_ff[e];
+    const uint64_t rows_h = e < L->n_routed ? (uint64_t)(fl.max_rows_perm > 0 ? fl.max_rows_perm : 1) : (uint64_t)T;
+    if (!encode_bf16_2d_pitch(maps.data() + (size_t)128 * (2 * e), L->d_ff[e] > 0 ? L->w_down[e] : nullptr,
+                              (uint64_t)L->d_model, (uint64_t)L->d_ff[e], (uint64_t)ld, D_TILE) ||
+        !encode_bf16_2d_pitch(maps.data() + (size_t)128 * (2 * e + 1), h[e], rows_h, (uint64_t)fl.h_ld[e],
+                              (uint64_t)fl.h_ld[e], UMMA_TOK))
+      return CAMERA_ERR_CUDA;
+  }
+  if (cudaMemcpyAsync(ws + fl.maps, maps.data(), maps.size(), cudaMemcpyHostToDevice, st) != cudaSuccess) {
+    cudaGetLastError();
+    return CAMERA_ERR_CUDA;
+  }
+  if (launch_score_umma_write_h(c, st) != cudaSuccess) { cudaGetLastError(); return CAMERA_ERR_CUDA; }
+  int dev = 0, sms = 148;
+  cudaGetDevice(&dev);
+  cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+  if (cudaFuncSetAttribute(k_down_umma, cudaFuncAttributeMaxDynamicSharedMemorySize, D_SMEM_BYTES) != cudaSuccess) {
+    cudaGetLastError();
+    return CAMERA_ERR_CUDA;
+  }
+  const int n_dt = (L->d_model + D_TILE - 1) / D_TILE;
+  k_down_umma<<<sms, D_THREADS, D_SMEM_BYTES, st>>>(c, ws + fl.maps, n_dt);
+  k_unpermute_sum<<<(unsigned)((T + 7) / 8), 256, 0, st>>>(c, y);
+  return cudaGetLastError() == cudaSuccess ? CAMERA_OK : CAMERA_ERR_CUDA;
+}
+
+extern "C" size_t camera_output_error_workspace_bytes(int64_t n_tokens) {
+  return n_tokens < 0 ? 0 : up256(sizeof(double) * 3 * (size_t)((n_tokens + 7) / 8 + 1));
+}
+
+extern "C" int camera_output_error(const float* y, const float* y_hat, int64_t n_tokens, int32_t d_model, double* out,
+                                   void* workspace, size_t workspace_bytes, void* cuda_stream) {
+  if (n_tokens < 0 || d_model < 1 || out == nullptr || (n_tokens > 0 && (y == nullptr || y_hat == nullptr)))
+    return CAMERA_ERR_INVALID_ARG;
+  if (workspace == nullptr || workspace_bytes < camera_output_error_workspace_bytes(n_tokens) ||
+      (reinterpret_cast<uintptr_t>(workspace) & 255))
+    return CAMERA_ERR_WORKSPACE;
+  cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+  double* part = static_cast<double*>(workspace);
+  const long long n_part = (n_tokens + 7) / 8;
+  if (n_part > 0) k_error_partials<<<(unsigned)n_part, 256, 0, st>>>(y, y_hat, n_tokens, d_model, part);
+  k_error_final<<<1, 256, 0, st>>>(part, n_part, n_tokens, out);
+  return cudaGetLastError() == cudaSuccess ? CAMERA_OK : CAMERA_ERR_CUDA;
+}

@@ -228,7 +228,7 @@ __global__ void __launch_bounds__(256) k_block_scan(ScoreCtx c) {
 // and numbers the scoring work units and partial slots.
 __global__ void k_plan(ScoreCtx c) {
   if (threadIdx.x != 0 || blockIdx.x != 0) return;
-  int row = 0, units = 0;
+  int row = 0, units = 0, chunks = 0;
   long long part = 0;
   for (int e = 0; e < c.n_experts; ++e) {
     ExpertDyn dy;
@@ -245,6 +245,9 @@ __global__ void k_plan(ScoreCtx c) {
     dy.n_chunks = (dy.rows + c.chunk_tokens - 1) / c.chunk_tokens;
     dy.unit_begin = units;
     dy.part_begin = part;
+    dy.chunk_begin = chunks;
+    dy.pad = 0;
+    chunks += dy.n_chunks;
     c.edyn[e] = dy;
     c.unit_prefix[e] = units;
     units += dy.n_chunks * ((f + c.ch_tile - 1) / c.ch_tile);
@@ -253,12 +256,14 @@ __global__ void k_plan(ScoreCtx c) {
   if (row > c.max_rows_perm || part > c.max_part) {
     atomicExch(&c.totals->status, (int)CAMERA_ERR_WORKSPACE);
     units = 0;
+    chunks = 0;
     for (int e = 0; e <= c.n_experts; ++e) c.unit_prefix[e] = 0;
-    for (int e = 0; e < c.n_experts; ++e) { c.edyn[e].n_chunks = 0; c.edyn[e].rows = 0; }
+    for (int e = 0; e < c.n_experts; ++e) { c.edyn[e].n_chunks = 0; c.edyn[e].rows = 0; c.edyn[e].chunk_begin = 0; }
   }
   c.unit_prefix[c.n_experts] = units;
   c.totals->total_units = units;
   c.totals->total_rows = row;
+  c.totals->total_chunks = chunks;
 }
 
 // One warp per token: copies the token's hidden state to its row in every chosen expert's list.

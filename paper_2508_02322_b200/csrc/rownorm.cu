@@ -25,7 +25,7 @@ __global__ void __launch_bounds__(NORM_THREADS) k_colnorm_hf(ScoreCtx c) {
     if (c.est[mid].norm_blk_begin <= (int)blockIdx.x) lo = mid; else hi = mid;
   }
   const ExpertStatic es = c.est[lo];
-  const int f = es.d_ff, d = c.d_model;
+  const int f = es.d_ff, d = c.d_model, ld = es.down_ld;
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   const int col = ((int)blockIdx.x - es.norm_blk_begin) * 32 * VN + lane * VN;
   const T* W = static_cast<const T*>(es.w_down);
@@ -37,7 +37,7 @@ __global__ void __launch_bounds__(NORM_THREADS) k_colnorm_hf(ScoreCtx c) {
     for (; r + 3 * NORM_WARPS < d; r += 4 * NORM_WARPS) {
       float v[4][VN];
 #pragma unroll
-      for (int u = 0; u < 4; ++u) Vec16<T>::load(W + (size_t)(r + u * NORM_WARPS) * f + col, v[u]);
+      for (int u = 0; u < 4; ++u) Vec16<T>::load(W + (size_t)(r + u * NORM_WARPS) * ld + col, v[u]);
 #pragma unroll
       for (int u = 0; u < 4; ++u)
 #pragma unroll
@@ -45,7 +45,7 @@ __global__ void __launch_bounds__(NORM_THREADS) k_colnorm_hf(ScoreCtx c) {
     }
     for (; r < d; r += NORM_WARPS) {
       float v[VN];
-      Vec16<T>::load(W + (size_t)r * f + col, v);
+      Vec16<T>::load(W + (size_t)r * ld + col, v);
 #pragma unroll
       for (int i = 0; i < VN; ++i) s[i] = fmaf(v[i], v[i], s[i]);
     }

@@ -39,7 +39,10 @@ constexpr int U_SMEM_BYTES = U_STAGES * U_STAGE_BYTES + U_WBUF_BYTES + 256 + 102
 static_assert(CH_TILE == 128, "one micro-expert per TMEM lane");
 
 // lambda = a_t * SiLU(g) * u for 16 tokens of this thread's micro-expert; folds lambda^2 and |lambda|.
-__device__ __forceinline__ void fold16(const uint32_t* vg, const uint32_t* vu, const float* wb, float& s, float& m) {
+// WRITE_H (layer forward): lambda is also stored, as bf16, to h[token][micro-expert] for the first n_store tokens.
+template <bool WRITE_H>
+__device__ __forceinline__ void fold16(const uint32_t* vg, const uint32_t* vu, const float* wb, float& s, float& m,
+                                       __nv_bfloat16* hcol, int h_ld, int n_store) {
   float a[16];
 #pragma unroll
   for (int q = 0; q < 4; ++q) {
@@ -53,9 +56,11 @@ __device__ __forceinline__ void fold16(const uint32_t* vg, const uint32_t* vu, c
     const float lam = (a[j] * up) * (g * sig);
     s = fmaf(lam, lam, s);
     m = fmaxf(m, fabsf(lam));
+    if (WRITE_H && j < n_store) hcol[(size_t)j * h_ld] = __float2bfloat16_rn(lam);
   }
 }
 
+template <bool WRITE_H>
 __global__ void __launch_bounds__(U_THREADS, 1) k_score_umma(const ScoreCtx c) {
   extern __shared__ uint8_t smem_raw[];
   const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
@@ -179,9 +184,20 @@ __global__ void __launch_bounds__(U_THREADS, 1) k_score_umma(const ScoreCtx c) {
       const int n_tiles = (u.rows + UMMA_TOK - 1) / UMMA_TOK;
       const float* wsrc = u.shared_idx < 0 ? c.perm_w + u.row0 : c.shared_w + (size_t)u.shared_idx * c.n_tokens + u.row0;
       float s = 0.f, m = 0.f;
+      // layer forward: where this thread's micro-expert goes in h, and the last row h has
+      __nv_bfloat16* hbase = nullptr;
+      int h_ld = 0, row_limit = 0;
+      if (WRITE_H) {
+        const ExpertStatic es = c.est[u.e];
+        h_ld = es.h_ld;
+        hbase = static_cast<__nv_bfloat16*>(es.h) + (size_t)u.row0 * h_ld + u.ch0 + warp * 32 + lane;
+        row_limit = (u.shared_idx < 0 ? c.max_rows_perm : c.n_tokens) - u.row0;
+      }
       for (int tt = 0; ok && tt < n_tiles; ++tt) {
         const int valid = min(UMMA_TOK, u.rows - tt * UMMA_TOK);
         const int nv = (valid + 15) & ~15;
+        __nv_bfloat16* const htile = hbase + (size_t)tt * UMMA_TOK * h_ld;
+        const int rows_left = row_limit - tt * UMMA_TOK;
         // each warp stages the tile's router weights for itself (while the MMAs of the tile run), so
         // the four warps never wait on one another and a wait that runs out can be left warp by warp
         __syncwarp();
@@ -197,11 +213,11 @@ __global__ void __launch_bounds__(U_THREADS, 1) k_score_umma(const ScoreCtx c) {
         for (int c0 = 0; c0 < nv; c0 += 32) {
           tmem_ld_wait(g0, u0);
           if (c0 + 16 < nv) { tmem_ld16(t_gate + c0 + 16, g1); tmem_ld16(t_up + c0 + 16, u1); }
-          fold16(g0, u0, wb + c0, s, m);
+          fold16<WRITE_H>(g0, u0, wb + c0, s, m, htile + (size_t)c0 * h_ld, h_ld, rows_left - c0);
           if (c0 + 16 < nv) {
             tmem_ld_wait(g1, u1);
             if (c0 + 32 < nv) { tmem_ld16(t_gate + c0 + 32, g0); tmem_ld16(t_up + c0 + 32, u0); }
-            fold16(g1, u1, wb + c0 + 16, s, m);
+            fold16<WRITE_H>(g1, u1, wb + c0 + 16, s, m, htile + (size_t)(c0 + 16) * h_ld, h_ld, rows_left - c0 - 16);
           }
         }
         tc_fence_before();
@@ -209,7 +225,7 @@ __global__ void __launch_bounds__(U_THREADS, 1) k_score_umma(const ScoreCtx c) {
         tile_phase ^= 1u;
       }
       const int ch = u.ch0 + warp * 32 + lane;
-      if (ok && ch < u.f) {
+      if (!WRITE_H && ok && ch < u.f) {
         const size_t slot = (size_t)u.part_slot + warp * 32 + lane;
         c.part_sum[slot] = s;
         c.part_max[slot] = m;
@@ -244,11 +260,12 @@ EncodeTiledFn get_encode_fn() {
 }
 
 // bf16 row-major [rows, d] matrix, box = 64 columns (128 bytes) x box_rows rows, 128-byte swizzle.
-bool encode_2d(EncodeTiledFn fn, void* out, const void* ptr, uint64_t rows, uint64_t d, uint32_t box_rows) {
-  if (ptr == nullptr || rows == 0) { memset(out, 0, 128); return true; }
+bool encode_2d(EncodeTiledFn fn, void* out, const void* ptr, uint64_t rows, uint64_t d, uint32_t box_rows,
+               uint64_t pitch = 0) {
+  if (ptr == nullptr || rows == 0 || d == 0) { memset(out, 0, 128); return true; }
   CUtensorMap m;
   const cuuint64_t dims[2] = {d, rows};
-  const cuuint64_t strides[1] = {d * 2};
+  const cuuint64_t strides[1] = {(pitch ? pitch : d) * 2};
   const cuuint32_t box[2] = {(cuuint32_t)U_BK, box_rows};
   const cuuint32_t estr[2] = {1, 1};
   const CUresult r = fn(&m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(ptr), dims, strides, box, estr,
@@ -264,6 +281,11 @@ bool encode_2d(EncodeTiledFn fn, void* out, const void* ptr, uint64_t rows, uint
 bool encode_bf16_2d(void* out, const void* ptr, uint64_t rows, uint64_t d, uint32_t box_rows) {
   EncodeTiledFn fn = get_encode_fn();
   return fn != nullptr && encode_2d(fn, out, ptr, rows, d, box_rows);
+}
+
+bool encode_bf16_2d_pitch(void* out, const void* ptr, uint64_t rows, uint64_t cols, uint64_t pitch, uint32_t box_rows) {
+  EncodeTiledFn fn = get_encode_fn();
+  return fn != nullptr && encode_2d(fn, out, ptr, rows, cols, box_rows, pitch);
 }
 
 bool umma_shape_ok(const camera_layer_t* L) {
@@ -304,9 +326,20 @@ cudaError_t launch_score_umma(const ScoreCtx& c, cudaStream_t st) {
   int dev = 0, sms = 148;
   cudaGetDevice(&dev);
   cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
-  cudaError_t e = cudaFuncSetAttribute(k_score_umma, cudaFuncAttributeMaxDynamicSharedMemorySize, U_SMEM_BYTES);
+  cudaError_t e = cudaFuncSetAttribute(k_score_umma<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, U_SMEM_BYTES);
   if (e != cudaSuccess) return e;
-  k_score_umma<<<sms, U_THREADS, U_SMEM_BYTES, st>>>(c);
+  k_score_umma<false><<<sms, U_THREADS, U_SMEM_BYTES, st>>>(c);
+  return cudaGetLastError();
+}
+
+// The same kernel with the epilogue that stores h (layer forward).
+cudaError_t launch_score_umma_write_h(const ScoreCtx& c, cudaStream_t st) {
+  int dev = 0, sms = 148;
+  cudaGetDevice(&dev);
+  cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+  cudaError_t e = cudaFuncSetAttribute(k_score_umma<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, U_SMEM_BYTES);
+  if (e != cudaSuccess) return e;
+  k_score_umma<true><<<sms, U_THREADS, U_SMEM_BYTES, st>>>(c);
   return cudaGetLastError();
 }
 

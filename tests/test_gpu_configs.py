@@ -150,3 +150,20 @@ def test_deepseek_moe_shape_heavy_tails_bit_budget(P):
 
 def test_qwen2_57b_shape_one_full_layer(P):
     run_config(P, "qwen2_57b_a14b", 3, 6, 0.95, (0.2, 0.4, 0.6), ([0.2, 0.6, 0.2], [3, 2, 1]), False)
+
+
+def test_qwen15_moe_shape_layer_output_on_sampled_tokens(P):
+    """The layer output at a full-size config: the oracle computes Eq. 1-2 for a sample of tokens under the GPU's
+    routing of those tokens (every expert's full weights take part)."""
+    from test_gpu_forward import assert_output_close, oracle_forward
+    from _util import to_oracle_layer
+    cfg = W().CONFIGS["qwen15_moe_a27b"]
+    L = W().make_layer(cfg, seed=0, device=DEV)
+    X = W().make_tokens(cfg, seed=0, device=DEV)
+    y, (gi, gw) = P.camera_layer_forward(P.Layer.from_workload(L), X, want_routing=True)
+    tok = np.sort(np.random.default_rng(3).choice(cfg.n_tokens, size=48, replace=False))
+    tok[0], tok[-1] = 0, cfg.n_tokens - 1
+    ol = to_oracle_layer(L)
+    ref = oracle_forward(ol, f64(X[torch.from_numpy(tok).to(DEV)]),
+                         (gi.cpu().numpy().astype(np.int64)[tok], gw.cpu().numpy().astype(np.float64)[tok]))
+    assert_output_close("qwen15 layer output", y.cpu().numpy()[tok], ref)

@@ -1,0 +1,141 @@
+"""GPU parity of the layer output (Eq. 1-2) and of the output of a sliced layer (Y_hat = Phi[:,S] W[S,:], Eq. 7)
+against the float64 oracle, and of the error metrics against their definitions.
+
+Tolerance: h is rounded to bf16 between the two GEMMs (8 significant bits: relative error up to 2^-8 per term,
+independent signs), so an output element carries an error of about 2^-8 / sqrt(3) * 0.7 = 1.6e-3 of the root-sum-square
+of its terms, which for random signs is the size of the output itself: elements are compared within 1.2e-2 of their
+token's RMS (seven standard deviations; the worst of 65 k elements measured 8e-3), the whole output within 3e-3 in
+Frobenius norm.
+"""
+import numpy as np
+import pytest
+import torch
+
+import oracle as O
+from _util import f64, to_oracle_layer
+
+pytestmark = pytest.mark.gpu
+
+DEV = "cuda:0"
+ELEM_TOL, FRO_TOL = 1.2e-2, 3e-3
+
+
+@pytest.fixture(scope="module")
+def P():
+    import paper_2508_02322_b200 as pkg
+    return pkg
+
+
+def W():
+    from paper_2508_02322_b200 import workloads
+    return workloads
+
+
+def cfg_of(**kw):
+    base = dict(name="fwd", d_model=256, n_routed=6, top_k=2, d_ff_routed=256, d_ff_shared=(192,),
+                shared_gate_sigmoid=True, n_tokens=700, dtype="bf16", x_dist="normal_rms1", router_bias_std=0.3,
+                weight_std=0.05)
+    base.update(kw)
+    return W().LayerConfig(**base)
+
+
+def assert_output_close(name, got, ref):
+    got = np.asarray(got, dtype=np.float64)
+    rms = np.sqrt((ref ** 2).mean(axis=1, keepdims=True))
+    err = np.abs(got - ref)
+    assert (err <= ELEM_TOL * np.maximum(rms, 1e-30)).all(), f"{name}: worst {np.max(err / np.maximum(rms, 1e-30)):.3e} of token RMS"
+    fro = np.sqrt((err ** 2).sum() / max((ref ** 2).sum(), 1e-300))
+    assert fro <= FRO_TOL, f"{name}: relative Frobenius error {fro:.3e}"
+    assert (got[(ref == 0).all(axis=1)] == 0).all()
+
+
+def oracle_routing(ol, Xd):
+    idx, w = O.top_and_norm(O.router_probs(ol, Xd), ol.top_k, ol.norm_topk)
+    w32 = w.astype(np.float32)
+    return (torch.from_numpy(idx.astype(np.int32)), torch.from_numpy(w32)), (idx, w32.astype(np.float64))
+
+
+def oracle_forward(ol, Xd, routing):
+    """Eq. 1-2 with the routed coefficients prescribed (the ones handed to the GPU)."""
+    A = O.coefficients(ol, Xd, routing=routing)
+    Y = np.zeros((Xd.shape[0], ol.w_down[0].shape[0]))
+    for e in range(ol.n_experts):
+        Y += A[:, e:e + 1] * (O.expert_hidden(Xd, ol.w_gate[e], ol.w_up[e]) @ ol.w_down[e].T)
+    return Y
+
+
+@pytest.mark.parametrize("T", [1, 255, 700, 5000])
+def test_layer_output(P, T):
+    cfg = cfg_of(n_tokens=T)
+    L = W().make_layer(cfg, seed=30, device=DEV)
+    X = W().make_tokens(cfg, seed=30, device=DEV)
+    ol, Xd = to_oracle_layer(L), f64(X)
+    rin, rout = oracle_routing(ol, Xd)
+    y = P.camera_layer_forward(P.Layer.from_workload(L), X, routing_in=rin)
+    ref = oracle_forward(ol, Xd, rout)
+    assert np.allclose(ref, O.forward(ol, Xd), rtol=1e-5, atol=1e-6)       # the helper above is Eq. 1-2 (coefficients rounded to fp32)
+    assert_output_close("layer output", y.cpu().numpy(), ref)
+
+
+def test_layer_output_own_routing_and_no_shared(P):
+    cfg = cfg_of(n_tokens=900, d_ff_shared=(), shared_gate_sigmoid=False, n_routed=5, top_k=3, d_ff_routed=320)
+    L = W().make_layer(cfg, seed=31, device=DEV)
+    X = W().make_tokens(cfg, seed=31, device=DEV)
+    ol, Xd = to_oracle_layer(L), f64(X)
+    y, (gi, gw) = P.camera_layer_forward(P.Layer.from_workload(L), X, want_routing=True)
+    ref = oracle_forward(ol, Xd, (gi.cpu().numpy().astype(np.int64), gw.cpu().numpy().astype(np.float64)))
+    assert_output_close("layer output under the GPU's routing", y.cpu().numpy(), ref)
+
+
+def test_dense_layer_is_a_gated_ffn(P):
+    cfg = cfg_of(n_tokens=400, n_routed=0, top_k=1, d_ff_shared=(384,), shared_gate_sigmoid=False, router_bias_std=0.0)
+    L = W().make_layer(cfg, seed=32, device=DEV)
+    X = W().make_tokens(cfg, seed=32, device=DEV)
+    y = P.camera_layer_forward(P.Layer.from_workload(L), X)
+    Xd = f64(X)
+    ref = O.expert_hidden(Xd, f64(L["w_gate"][0]), f64(L["w_up"][0])) @ f64(L["w_down"][0]).T
+    assert_output_close("dense FFN", y.cpu().numpy(), ref)
+
+
+@pytest.mark.parametrize("ratio", [0.2, 0.6])
+def test_sliced_layer_output_and_error_metrics(P, ratio):
+    """Score, select, slice, run the sliced layer: its output is Phi[:,S] W[S,:] of the GPU's own mask, and the
+    reported error is the objective of Eq. 7 for that mask."""
+    cfg = cfg_of(n_tokens=1200)
+    L = W().make_layer(cfg, seed=33, device=DEV)
+    X = W().make_tokens(cfg, seed=33, device=DEV)
+    layer = P.Layer.from_workload(L)
+    ol, Xd = to_oracle_layer(L), f64(X)
+    rin, rout = oracle_routing(ol, Xd)
+    E = P.camera_score_layer(layer, X, 0.95, routing_in=rin)
+    keep = P.camera_select_prune(E, ratio)
+    keep[256:512] = 0                       # one routed expert loses every micro-expert
+    sub, counts = P.camera_sub_index(keep, P.expert_offsets_tensor(layer), [1])
+    out = P.camera_compact_weights(layer, sub, counts, 1)
+    m = counts[:, 0].cpu().numpy()
+    assert m[1] == 0
+    sliced = P.Layer(L["w_router"], [out["w_gate"][e][:m[e]] for e in range(layer.n_experts)],
+                     [out["w_up"][e][:m[e]] for e in range(layer.n_experts)], out["w_down"], cfg.top_k, cfg.n_shared,
+                     L["router_bias"], L["w_shared_gate"], cfg.norm_topk, "hf", down_ld=layer.d_ff)
+    y = P.camera_layer_forward(layer, X, routing_in=rin)
+    y_hat = P.camera_layer_forward(sliced, X, routing_in=rin)
+    lists, _ = O.sub_index_lists(keep.cpu().numpy(), O.me_offsets(ol), [1])
+    ref_hat = oracle_forward(O.slice_layer(ol, lists), Xd, rout)
+    assert_output_close("sliced layer output", y_hat.cpu().numpy(), ref_hat)
+    # the metrics against their definitions on the same two fp32 arrays
+    got = P.camera_output_error(y, y_hat).cpu().numpy()
+    a, b = y.cpu().numpy().astype(np.float64), y_hat.cpu().numpy().astype(np.float64)
+    cos = (a * b).sum(1) / np.sqrt((a * a).sum(1) * (b * b).sum(1))
+    assert np.allclose(got, [((a - b) ** 2).sum(), (a * a).sum(), cos.mean()], rtol=1e-12)
+    # and against the oracle's decoding error of the pruned set (Eq. 7), which the bf16 rounding of h perturbs a little
+    ref_err = ((oracle_forward(ol, Xd, rout) - ref_hat) ** 2).sum()
+    assert abs(got[0] - ref_err) <= 0.02 * ref_err
+
+
+def test_forward_argument_errors(P):
+    cfg = cfg_of(dtype="f32", n_tokens=64)
+    L = W().make_layer(cfg, seed=34, device=DEV)
+    X = W().make_tokens(cfg, seed=34, device=DEV)
+    with pytest.raises(P.CameraError) as e:
+        P.camera_layer_forward(P.Layer.from_workload(L), X)
+    assert e.value.status == -2
