@@ -270,7 +270,7 @@ def main():
     ms_per_step = ms / args.steps
 
     # ---- the selection applied to the weights (Algorithm 2 lines 9-13), timed on its own after the step loop
-    compact = forward = None
+    compact = forward = decode = None
     if not args.no_compact:
         off = P.expert_offsets_tensor(layer)
         outw = {k: [torch.empty_like(w) for w in layer.tensors[k]] for k in ("w_gate", "w_up", "w_down")}
@@ -324,6 +324,37 @@ def main():
                        "relative_output_error": err[0] / err[1] if err[1] > 0 else None, "mean_cosine": err[2]}
             del ws_f, yb, yh
         del outw
+
+        # ---- decode through the layer, batch of 64 tokens, full and sliced at each prune ratio (the paper's speed table)
+        if not args.no_forward and cfg.dtype == "bf16":
+            xd = Xs[0][:64].contiguous()
+            ws_d = P.alloc_workspace(P.camera_forward_workspace_bytes(layer, 64), dev)
+            yd = torch.empty((64, cfg.d_model), dtype=torch.float32, device=dev)
+            outd = {k: [torch.empty_like(w) for w in layer.tensors[k]] for k in ("w_gate", "w_up", "w_down")}
+            def decode_ms(lay, reps=20):
+                for _ in range(3):
+                    P.camera_layer_forward(lay, xd, y=yd, workspace=ws_d)
+                sync_all()
+                f0, f1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                f0.record(stream)
+                for _ in range(reps):
+                    P.camera_layer_forward(lay, xd, y=yd, workspace=ws_d)
+                f1.record(stream); sync_all()
+                return f0.elapsed_time(f1) / reps
+            base_ms = decode_ms(layer)
+            esz = 2
+            decode = {"batch_tokens": 64, "full_layer_us": 1e3 * base_ms,
+                      "full_layer_weight_gbs": 3 * layer.n_me * cfg.d_model * esz / 1e9 / (base_ms * 1e-3), "pruned": []}
+            for j, r in enumerate(PRUNE_RATIOS):
+                sub, cnt = P.camera_sub_index(keep[j], off, [1])
+                P.camera_compact_weights(layer, sub, cnt, 1, out=outd, workspace=ws_c)
+                mj = cnt[:, 0].cpu().tolist()
+                sl = P.Layer(L["w_router"], [outd["w_gate"][e][:mj[e]] for e in range(layer.n_experts)],
+                             [outd["w_up"][e][:mj[e]] for e in range(layer.n_experts)], outd["w_down"], cfg.top_k,
+                             cfg.n_shared, L["router_bias"], L["w_shared_gate"], cfg.norm_topk, "hf", down_ld=layer.d_ff)
+                ms_j = decode_ms(sl)
+                decode["pruned"].append({"prune_ratio": r, "us": 1e3 * ms_j, "speedup": base_ms / ms_j})
+            del outd, ws_d
 
     # ---- end to end through the host-buffer entry point: H2D of the tokens, D2H of the results, every step
     e2e = None
@@ -390,7 +421,7 @@ def main():
                    "parallelism": f"layers x{world}" if world > 1 else "single GPU"},
         "model_seconds": cfg.n_layers * ms_per_step * 1e-3 / world,
         "stage_ms": stage_ms, "clocks": clocks, "e2e": e2e, "gpu_launches": LAUNCHES_PER_STEP * args.steps,
-        "roofline": roofline, "compact": compact, "forward": forward, "cpu_baseline": cpu, "context": PAPER_CONTEXT,
+        "roofline": roofline, "compact": compact, "forward": forward, "decode": decode, "cpu_baseline": cpu, "context": PAPER_CONTEXT,
     }
     print(json.dumps(out))
     if world > 1:
