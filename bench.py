@@ -44,6 +44,22 @@ def shard_layers(n_layers: int, world: int, rank: int):
     return list(range(rank, n_layers, world))
 
 
+def shard_tokens(n_tokens: int, world: int, rank: int):
+    """[t0, t1) of the calibration tokens a rank scores when one layer's tokens are spread over `world` ranks."""
+    base, extra = divmod(n_tokens, world)
+    t0 = rank * base + min(rank, extra)
+    return t0, t0 + base + (1 if rank < extra else 0)
+
+
+def reduce_components(phi2, phi_inf_sq, dist=None):
+    """The one exchange of token-sharded scoring: column sums add over the shards, column maxima take the maximum
+    (Algorithm 1 lines 7-8).  In place; a no-op without a process group."""
+    if dist is not None and dist.is_initialized() and dist.get_world_size() > 1:
+        dist.all_reduce(phi2, op=dist.ReduceOp.SUM)
+        dist.all_reduce(phi_inf_sq, op=dist.ReduceOp.MAX)
+    return phi2, phi_inf_sq
+
+
 def max_over_ranks(ms: float, dist=None, device="cpu") -> float:
     """Largest per-rank time; a collective only when a process group exists."""
     if dist is None or not dist.is_initialized() or dist.get_world_size() == 1:
@@ -181,6 +197,9 @@ def main():
     ap.add_argument("--routed", type=int, default=0, help="override the number of routed experts (profiling slices)")
     ap.add_argument("--topk", type=int, default=0, help="override top-k (with --routed and --tokens: a slice that keeps the full layer's tokens per expert)")
     ap.add_argument("--oracle-tokens", type=int, default=0, help="tokens of the CPU-oracle sample (default 512 for --impl reference, 2048 for the cpu_baseline leg)")
+    ap.add_argument("--shard", default="layers", choices=["layers", "tokens"],
+                    help="with --gpus N: every rank its own layer (weak scaling, no exchange), or one layer's tokens "
+                         "spread over the ranks with an all-reduce of the 2 x N_e score components (strong scaling)")
     ap.add_argument("--cta-pair", action="store_true", help="score on CTA pairs (tcgen05 cta_group::2) instead of single CTAs")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
@@ -211,9 +230,14 @@ def main():
         cfg = W.scaled(cfg, n_routed=args.routed, top_k=min(args.topk or cfg.top_k, args.routed))
     elif args.topk:
         cfg = W.scaled(cfg, top_k=args.topk)
+    by_tokens = args.shard == "tokens"
+    if by_tokens:
+        # one layer for all ranks; a rank scores its share of the tokens, then the components are all-reduced
+        t0, t1 = shard_tokens(cfg.n_tokens, world, rank)
+        cfg = W.scaled(cfg, n_tokens=t1 - t0)
     T = cfg.n_tokens
-    # every rank analyses its own layer (weights and tokens seeded by the layer id): no data-path collective
-    L = W.make_layer(cfg, seed=0, layer_id=rank, device=dev)
+    # layers mode: every rank analyses its own layer (weights and tokens seeded by the layer id): no data-path collective
+    L = W.make_layer(cfg, seed=0, layer_id=0 if by_tokens else rank, device=dev)
     layer = P.Layer.from_workload(L)
     Xs = [W.make_tokens(cfg, seed=0, layer_id=rank + world * i, device=dev) for i in range(2)]
     n_me = layer.n_me
@@ -224,9 +248,21 @@ def main():
     bits = torch.empty(n_me, dtype=torch.uint8, device=dev)
     stream = torch.cuda.current_stream()
 
+    phi2 = torch.empty(n_me, dtype=torch.float32, device=dev)
+    phi_inf = torch.empty_like(phi2)
+    x_none = Xs[0][:0]
+
     def step(i, events=None):
-        P.camera_score_layer(layer, Xs[i % 2], ALPHA, energy=energy, workspace=ws_score, stage_events=events,
-                             cta_pair=args.cta_pair)
+        if by_tokens:
+            P.camera_score_layer(layer, Xs[i % 2], ALPHA, energy=energy, workspace=ws_score, stage_events=events,
+                                 cta_pair=args.cta_pair, phi2=phi2, phi_inf_sq=phi_inf)
+            reduce_components(phi2, phi_inf, dist if world > 1 else None)
+            # no tokens, accumulate: folds nothing in and turns the reduced components into the energies
+            P.camera_score_layer(layer, x_none, ALPHA, energy=energy, workspace=ws_score, phi2=phi2, phi_inf_sq=phi_inf,
+                                 accumulate=True)
+        else:
+            P.camera_score_layer(layer, Xs[i % 2], ALPHA, energy=energy, workspace=ws_score, stage_events=events,
+                                 cta_pair=args.cta_pair)
         for j, r in enumerate(PRUNE_RATIOS):
             P.camera_select_prune(energy, r, workspace=ws_sel, keep_mask=keep[j])
         P.camera_alloc_bits(energy, BIT_RATIOS, BIT_LEVELS, workspace=ws_sel, bits_out=bits)
@@ -358,7 +394,7 @@ def main():
 
     # ---- end to end through the host-buffer entry point: H2D of the tokens, D2H of the results, every step
     e2e = None
-    if not args.no_e2e:
+    if not args.no_e2e and not by_tokens:
         del ws_score
         torch.cuda.empty_cache()
         ws_an = P.alloc_workspace(P.camera_analyze_workspace_bytes(layer, T, len(BIT_LEVELS)), dev)
@@ -412,15 +448,15 @@ def main():
 
     out = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
-        "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "strong" if by_tokens else "weak", "vs_baseline": None,
         "dtype": "bf16" if cfg.dtype == "bf16" else "f32", "data": "synthetic",
         "config": {"workload": f"{cfg.name} layer: d_model {cfg.d_model}, {cfg.n_routed}x{cfg.d_ff_routed} top-{cfg.top_k}"
                                f" + shared {list(cfg.d_ff_shared)}, {T} tokens", "tokens_per_layer": T,
                    "micro_experts": n_me, "alpha": ALPHA, "prune_ratios": list(PRUNE_RATIOS),
                    "bit_levels": list(BIT_LEVELS), "bit_ratios": list(BIT_RATIOS), "l2": "inputs larger than L2",
-                   "parallelism": f"layers x{world}" if world > 1 else "single GPU"},
+                   "parallelism": (f"tokens x{world}" if by_tokens else f"layers x{world}") if world > 1 else "single GPU"},
         "model_seconds": cfg.n_layers * ms_per_step * 1e-3 / world,
-        "stage_ms": stage_ms, "clocks": clocks, "e2e": e2e, "gpu_launches": LAUNCHES_PER_STEP * args.steps,
+        "stage_ms": stage_ms, "clocks": clocks, "e2e": e2e, "gpu_launches": (LAUNCHES_PER_STEP + (3 if by_tokens else 0)) * args.steps,
         "roofline": roofline, "compact": compact, "forward": forward, "decode": decode, "cpu_baseline": cpu, "context": PAPER_CONTEXT,
     }
     print(json.dumps(out))

@@ -309,3 +309,21 @@ def test_analyze_layer_host_in_batches(P):
         for j, r in enumerate((0.2, 0.6)):
             assert np.array_equal(kh[j].numpy(), O.select_prune(eh.numpy(), r))
         assert np.array_equal(bh.numpy(), O.alloc_bits(eh.numpy(), [0.2, 0.6, 0.2], [3, 2, 1])[0])
+
+
+def test_token_shards_reduced_then_finalised(P):
+    """Token-sharded scoring as a multi-GPU run does it: every shard gives its components, sums add and maxima take
+    the maximum (the all-reduce), and a call with no tokens and CAMERA_SCORE_ACCUMULATE turns them into energies."""
+    cfg = small_cfg(n_tokens=3000)
+    L = W().make_layer(cfg, seed=16, device=DEV)
+    X = W().make_tokens(cfg, seed=16, device=DEV)
+    layer = P.Layer.from_workload(L)
+    parts = []
+    for t0, t1 in ((0, 1400), (1400, 3000)):
+        o = P.camera_score_layer(layer, X[t0:t1].contiguous(), 0.95, details=True)
+        parts.append((o["phi2"], o["phi_inf_sq"]))
+    phi2 = parts[0][0] + parts[1][0]
+    phi_inf = torch.maximum(parts[0][1], parts[1][1])
+    E = P.camera_score_layer(layer, X[:0], 0.95, phi2=phi2, phi_inf_sq=phi_inf, accumulate=True)
+    whole = P.camera_score_layer(layer, X, 0.95)
+    assert_close("sharded vs one call", E.cpu().numpy(), whole.cpu().numpy(), rel=1e-5)
