@@ -392,6 +392,33 @@ def main():
                 decode["pruned"].append({"prune_ratio": r, "us": 1e3 * ms_j, "speedup": base_ms / ms_j})
             del outd, ws_d
 
+    # ---- the selections of all layers of the model in one call (one segment per layer): where a6/a7 see real bytes
+    select_model = None
+    if not args.no_compact:
+        nl = cfg.n_layers
+        Eall = energy.repeat(nl) * (1.0 + torch.arange(nl * n_me, device=dev) // n_me).float()
+        seg = [i * n_me for i in range(nl + 1)]
+        keep_all = torch.empty(nl * n_me, dtype=torch.uint8, device=dev)
+        ws_all = P.alloc_workspace(P.camera_select_workspace_bytes(nl * n_me, nl, len(BIT_LEVELS)), dev)
+        s0, s1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        def select_all():
+            for r in PRUNE_RATIOS:
+                P.camera_select_prune(Eall, r, seg_offsets=seg, workspace=ws_all, keep_mask=keep_all)
+            P.camera_alloc_bits(Eall, BIT_RATIOS, BIT_LEVELS, seg_offsets=seg, workspace=ws_all, bits_out=keep_all)
+        for _ in range(3):
+            select_all()
+        sync_all()
+        s0.record(stream)
+        for _ in range(10):
+            select_all()
+        s1.record(stream); sync_all()
+        sel_ms = s0.elapsed_time(s1) / 10
+        sel_bytes = 4 * (9 * 4 * nl * n_me + nl * n_me)     # per call: 9 passes over the fp32 keys, one byte per label out
+        select_model = {"what": f"3 prune masks + bit allocation for {nl} layers as segments of one call", "ms": sel_ms,
+                        "algorithmic_gb": sel_bytes / 1e9, "achieved_gbs": sel_bytes / 1e9 / (sel_ms * 1e-3),
+                        "frac_of_hbm_peak": sel_bytes / 1e9 / (sel_ms * 1e-3) / load_peaks()["hbm_gbs"]}
+        del Eall, keep_all, ws_all
+
     # ---- end to end through the host-buffer entry point: H2D of the tokens, D2H of the results, every step
     e2e = None
     if not args.no_e2e and not by_tokens:
@@ -457,7 +484,7 @@ def main():
                    "parallelism": (f"tokens x{world}" if by_tokens else f"layers x{world}") if world > 1 else "single GPU"},
         "model_seconds": cfg.n_layers * ms_per_step * 1e-3 / world,
         "stage_ms": stage_ms, "clocks": clocks, "e2e": e2e, "gpu_launches": (LAUNCHES_PER_STEP + (3 if by_tokens else 0)) * args.steps,
-        "roofline": roofline, "compact": compact, "forward": forward, "decode": decode, "cpu_baseline": cpu, "context": PAPER_CONTEXT,
+        "roofline": roofline, "compact": compact, "forward": forward, "decode": decode, "select_model": select_model, "cpu_baseline": cpu, "context": PAPER_CONTEXT,
     }
     print(json.dumps(out))
     if world > 1:

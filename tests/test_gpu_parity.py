@@ -327,3 +327,37 @@ def test_token_shards_reduced_then_finalised(P):
     E = P.camera_score_layer(layer, X[:0], 0.95, phi2=phi2, phi_inf_sq=phi_inf, accumulate=True)
     whole = P.camera_score_layer(layer, X, 0.95)
     assert_close("sharded vs one call", E.cpu().numpy(), whole.cpu().numpy(), rel=1e-5)
+
+
+def test_limits_of_the_router(P):
+    """The largest expert count and top-k the library takes (256 routed experts, top-16): more logit columns than
+    the tensor-core router holds, so the fp32 router runs next to the tensor-core scoring kernel."""
+    cfg = small_cfg(n_tokens=300, d_model=128, n_routed=256, top_k=16, d_ff_routed=64, d_ff_shared=(), shared_gate_sigmoid=False,
+                    router_bias_std=1.0)
+    L = W().make_layer(cfg, seed=17, device=DEV)
+    X = W().make_tokens(cfg, seed=17, device=DEV)
+    out, _ = run_and_compare(P, L, X, alpha=0.95)
+    assert int(out["expert_token_counts"].sum()) == 300 * 16
+
+
+def test_many_logit_columns_on_the_tensor_core_router(P):
+    """112 routed experts + 3 gated shared experts = 128 logit columns, the most the tensor-core router takes."""
+    cfg = small_cfg(n_tokens=1000, d_model=192, n_routed=112, top_k=5, d_ff_routed=64, d_ff_shared=(64, 64, 64),
+                    shared_gate_sigmoid=True)
+    L = W().make_layer(cfg, seed=18, device=DEV)
+    X = W().make_tokens(cfg, seed=18, device=DEV)
+    run_and_compare(P, L, X, alpha=0.95)
+
+
+def test_selection_over_28_layers_at_once(P):
+    """All layers of a model as segments of one call: every layer gets its own threshold."""
+    n, layers = 184320, 28
+    g = torch.Generator(device="cpu").manual_seed(5)
+    E = torch.rand(n * layers, generator=g) ** 3 * (1 + torch.arange(n * layers) // n).float()
+    seg = [i * n for i in range(layers + 1)]
+    keep, thr = P.camera_select_prune(E.to(DEV), 0.4, seg_offsets=seg, want_threshold=True)
+    ref = np.concatenate([O.select_prune(E.numpy()[seg[i]:seg[i + 1]], 0.4) for i in range(layers)])
+    assert np.array_equal(keep.cpu().numpy(), ref)
+    bits = P.camera_alloc_bits(E.to(DEV), [0.2, 0.6, 0.2], [3, 2, 1], seg_offsets=seg)
+    refb = np.concatenate([O.alloc_bits(E.numpy()[seg[i]:seg[i + 1]], [0.2, 0.6, 0.2], [3, 2, 1])[0] for i in range(layers)])
+    assert np.array_equal(bits.cpu().numpy(), refb)
