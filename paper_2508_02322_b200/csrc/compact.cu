@@ -14,7 +14,7 @@ namespace {
 constexpr int SUB_THREADS = 256;
 constexpr int GR_THREADS = 256;
 constexpr int GR_ROWS = GR_THREADS / 32;     // destination rows per CTA of the row gather (one warp each)
-constexpr int GC_ROWS = 4;                   // d_model rows per CTA of the column gather
+constexpr int GC_ROWS = 8;                   // d_model rows per CTA of the column gather
 
 struct LabelOrder { unsigned char v[MAX_LEVELS]; };
 
@@ -101,23 +101,46 @@ k_gather_rows(const CompactExpert* __restrict__ tab, int n_experts, const int* _
 }
 
 // Paper layout W_down [d_model, d_ff]: destination column j <- source column sub_index[j], for GC_ROWS rows of
-// d_model per CTA; the index is read once per column and used for all of the CTA's rows.
+// d_model per CTA.  A thread takes two neighbouring destination columns: their indices are read once and used for all
+// of the CTA's rows, the 2 * GC_ROWS loads are independent, and every store writes both columns at once.
+template <typename T> struct Pair;
+template <> struct Pair<__nv_bfloat16> { typedef __nv_bfloat162 type; };
+template <> struct Pair<float> { typedef float2 type; };
+
 template <typename T>
 __global__ void __launch_bounds__(GR_THREADS)
 k_gather_cols(const CompactExpert* __restrict__ tab, int n_experts, const int* __restrict__ sub_index,
               const int* __restrict__ counts, int n_labels, int n_take, int d_model) {
+  typedef typename Pair<T>::type T2;
   const int e = expert_of_block(tab, n_experts, blockIdx.x, true);
   const CompactExpert ce = tab[e];
   const int c0 = ((int)blockIdx.x - ce.col_blk_begin) * GC_ROWS;
   const int m = rows_taken(counts, e, n_labels, n_take);
-  const T* src = static_cast<const T*>(ce.src_down);
-  T* dst = static_cast<T*>(ce.dst_down);
+  const int rows = min(GC_ROWS, d_model - c0);
+  const T* src = static_cast<const T*>(ce.src_down) + (size_t)c0 * ce.d_ff;
+  T* dst = static_cast<T*>(ce.dst_down) + (size_t)c0 * ce.down_ld;
   const int* idx = sub_index + ce.me_off;
-  for (int j = threadIdx.x; j < m; j += GR_THREADS) {
-    const int s = idx[j];
+  const bool pair_ok = (ce.down_ld & 1) == 0 && (ce.me_off & 1) == 0 &&
+                       (reinterpret_cast<uintptr_t>(ce.dst_down) & (2 * sizeof(T) - 1)) == 0;
+  for (int j = 2 * threadIdx.x; j < m; j += 2 * GR_THREADS) {
+    if (pair_ok && j + 1 < m) {
+      const int2 s = *reinterpret_cast<const int2*>(idx + j);
+      T a[GC_ROWS], b[GC_ROWS];
 #pragma unroll
-    for (int r = 0; r < GC_ROWS; ++r)
-      if (c0 + r < d_model) dst[(size_t)(c0 + r) * ce.down_ld + j] = src[(size_t)(c0 + r) * ce.d_ff + s];
+      for (int r = 0; r < GC_ROWS; ++r)
+        if (r < rows) { a[r] = src[(size_t)r * ce.d_ff + s.x]; b[r] = src[(size_t)r * ce.d_ff + s.y]; }
+#pragma unroll
+      for (int r = 0; r < GC_ROWS; ++r)
+        if (r < rows) {
+          T2 v; v.x = a[r]; v.y = b[r];
+          *reinterpret_cast<T2*>(dst + (size_t)r * ce.down_ld + j) = v;
+        }
+    } else {
+      for (int jj = j; jj < min(j + 2, m); ++jj) {
+        const int s = idx[jj];
+        for (int r = 0; r < rows; ++r) dst[(size_t)r * ce.down_ld + jj] = src[(size_t)r * ce.d_ff + s];
+      }
+    }
   }
 }
 
