@@ -186,6 +186,89 @@ def run_reference(args):
         "gpu_launches": 0}))
 
 
+def run_stack(args):
+    """--stack: Algorithm 2's layer loop on a synthetic stack of MoE layers.  Per layer: output of the layer on the
+    calibration tokens (line 6), scores (line 8), selection and slicing (lines 9-13), output of the sliced layer
+    (line 14), which -- added to the residual and rescaled to RMS 1, the stand-in for the rest of a decoder layer --
+    becomes the next layer's input (line 15).  Prints one JSON line of its own."""
+    import torch
+    import paper_2508_02322_b200 as P
+    from paper_2508_02322_b200 import workloads as W
+    dev = torch.device("cuda", int(os.environ.get("LOCAL_RANK", "0")))
+    torch.cuda.set_device(dev)
+    cfg = W.CONFIGS[args.config]
+    if args.tokens:
+        cfg = W.scaled(cfg, n_tokens=args.tokens)
+    T, d = cfg.n_tokens, cfg.d_model
+    n_layers = args.stack_layers or cfg.n_layers
+    ratio = PRUNE_RATIOS[1]
+    B = min(T, 65536)
+    spans = [(t0, min(T, t0 + B)) for t0 in range(0, T, B)]
+    X = W.make_tokens(cfg, seed=0, layer_id=0, device=dev)
+    Y = torch.empty((T, d), dtype=torch.float32, device=dev)
+    Yh = torch.empty_like(Y)
+    probe = P.Layer.from_workload(W.make_layer(W.scaled(cfg, n_tokens=B), seed=0, layer_id=0, device=dev))
+    n_me = probe.n_me
+    ws_f = P.alloc_workspace(P.camera_forward_workspace_bytes(probe, B), dev)
+    ws_s = P.alloc_workspace(P.camera_score_workspace_bytes(probe, B), dev)
+    ws_sel = P.alloc_workspace(P.camera_select_workspace_bytes(n_me, 1, 2), dev)
+    ws_c = P.alloc_workspace(4096 + 64 * probe.n_experts, dev)
+    energy = torch.empty(n_me, dtype=torch.float32, device=dev)
+    phi2, phi_inf = torch.empty_like(energy), torch.empty_like(energy)
+    keep = torch.empty(n_me, dtype=torch.uint8, device=dev)
+    outw = {k: [torch.empty_like(w) for w in probe.tensors[k]] for k in ("w_gate", "w_up", "w_down")}
+    del probe
+    stream = torch.cuda.current_stream()
+    names = ("forward", "score", "select_slice", "forward_sliced", "error_next_input")
+    tot = {k: 0.0 for k in names}
+    errors = []
+    for l in range(n_layers):
+        L = W.make_layer(cfg, seed=0, layer_id=l, device=dev)        # weights of the layer: not timed
+        layer = P.Layer.from_workload(L)
+        off = P.expert_offsets_tensor(layer)
+        torch.cuda.synchronize()
+        ev = [torch.cuda.Event(enable_timing=True) for _ in range(len(names) + 1)]
+        ev[0].record(stream)
+        for t0, t1 in spans:
+            P.camera_layer_forward(layer, X[t0:t1], y=Y[t0:t1], workspace=ws_f)
+        ev[1].record(stream)
+        for i, (t0, t1) in enumerate(spans):
+            P.camera_score_layer(layer, X[t0:t1], ALPHA, energy=energy, workspace=ws_s, phi2=phi2, phi_inf_sq=phi_inf,
+                                 accumulate=i > 0)
+        ev[2].record(stream)
+        P.camera_select_prune(energy, ratio, workspace=ws_sel, keep_mask=keep)
+        sub, counts = P.camera_sub_index(keep, off, [1])
+        P.camera_compact_weights(layer, sub, counts, 1, out=outw, workspace=ws_c)
+        m = counts[:, 0].cpu().tolist()                               # the sliced layer's shape: the one host read
+        sliced = P.Layer(L["w_router"], [outw["w_gate"][e][:m[e]] for e in range(layer.n_experts)],
+                         [outw["w_up"][e][:m[e]] for e in range(layer.n_experts)], outw["w_down"], cfg.top_k, cfg.n_shared,
+                         L["router_bias"], L["w_shared_gate"], cfg.norm_topk, "hf", down_ld=layer.d_ff)
+        ev[3].record(stream)
+        for t0, t1 in spans:
+            P.camera_layer_forward(sliced, X[t0:t1], y=Yh[t0:t1], workspace=ws_f)
+        ev[4].record(stream)
+        err = P.camera_output_error(Y, Yh)
+        P.camera_residual_norm(X, Yh, out=X)
+        ev[5].record(stream)
+        torch.cuda.synchronize()
+        if P.camera_read_status(ws_s) != 0 or P.camera_read_status(ws_f) != 0:
+            raise RuntimeError("device status set in the stack run")
+        for i, k in enumerate(names):
+            tot[k] += ev[i].elapsed_time(ev[i + 1])
+        e = err.cpu().tolist()
+        errors.append(e[0] / e[1] if e[1] > 0 else 0.0)
+        del L, layer, sliced
+    total_s = sum(tot.values()) * 1e-3
+    print(json.dumps({
+        "mode": "stack", "what": "Algorithm 2 over a synthetic stack of MoE layers (layer outputs, CAMERA scores, prune, slice, "
+                                 "sliced-layer outputs fed to the next layer)",
+        "config": {"workload": f"{cfg.name} x {n_layers} layers", "tokens": T, "prune_ratio": ratio, "alpha": ALPHA},
+        "seconds": total_s, "tokens_per_s_per_layer": T * n_layers / total_s,
+        "ms_per_layer": {k: v / n_layers for k, v in tot.items()},
+        "relative_output_error": {"first_layer": errors[0], "last_layer": errors[-1], "mean": sum(errors) / len(errors)},
+        "context": PAPER_CONTEXT}))
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -205,10 +288,14 @@ def main():
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-compact", action="store_true")
     ap.add_argument("--no-forward", action="store_true")
+    ap.add_argument("--stack", action="store_true", help="run Algorithm 2's layer loop over a synthetic stack instead of the step benchmark")
+    ap.add_argument("--stack-layers", type=int, default=0, help="layers of the stack (default: the config's)")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
     if args.impl == "reference":
         return run_reference(args)
+    if args.stack:
+        return run_stack(args)
 
     import torch
     import torch.distributed as dist

@@ -260,6 +260,15 @@ size_t camera_output_error_workspace_bytes(int64_t n_tokens);
 int camera_output_error(const float* y, const float* y_hat, int64_t n_tokens, int32_t d_model, double* out,
                         void* workspace, size_t workspace_bytes, void* cuda_stream);
 
+/*
+ * Glue for running Algorithm 2's layer loop ("I <- O", line 15) on a synthetic stack of MoE layers, where no
+ * attention block or trained norm exists (the paper has no counterpart: its layers are whole decoder layers):
+ * out_t = (x_t + y_t) / sqrt(mean((x_t + y_t)^2) + eps), rounded to the dtype of x.  x: DEVICE [n_tokens, d_model]
+ * bf16 (CAMERA_BF16) or fp32, y: DEVICE fp32 (a layer output), out: DEVICE like x (may be x itself).  d_model % 8 == 0.
+ */
+int camera_residual_norm(const void* x, int32_t dtype, const float* y, int64_t n_tokens, int32_t d_model, float eps,
+                         void* out, void* cuda_stream);
+
 /* Scratch for camera_analyze_layer_host: score + select scratch for one batch of tokens, two staging
  * buffers for batches of x, and the results. */
 size_t camera_analyze_workspace_bytes(const camera_layer_t* layer, int64_t n_tokens, int32_t n_levels);

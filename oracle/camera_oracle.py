@@ -41,7 +41,7 @@ __all__ = [
     "coefficients", "expert_hidden", "forward", "phi_matrix", "basis",
     "me_offsets", "camera_components_dense", "camera_components", "energy",
     "camera_rank", "n_pruned", "select_prune", "class_boundaries",
-    "alloc_bits", "sub_index", "sub_index_lists", "slice_layer", "decode_error", "best_subset_error",
+    "alloc_bits", "sub_index", "sub_index_lists", "slice_layer", "next_layer_input", "decode_error", "best_subset_error",
     "average_bits",
 ]
 
@@ -348,6 +348,16 @@ def slice_layer(layer: OracleLayer, lists: Sequence[np.ndarray]) -> OracleLayer:
         w_down=[w[:, np.asarray(ix, dtype=np.int64)] for w, ix in zip(layer.w_down, lists)],
         router_bias=layer.router_bias, norm_topk=layer.norm_topk, n_shared=layer.n_shared,
         w_shared_gate=layer.w_shared_gate)
+
+
+def next_layer_input(X: np.ndarray, Y: np.ndarray, eps: float = 1e-6) -> np.ndarray:
+    """Glue of the synthetic multi-layer stack (NO counterpart in the paper, whose
+    layers are whole decoder layers of a trained model): the next layer's input
+    is the residual sum x + y of a token, rescaled to root-mean-square 1.  It
+    stands in for "I <- O" of Algorithm 2 line 15 where no attention block,
+    norm weights or trained model exist."""
+    Z = X + Y
+    return Z / np.sqrt((Z * Z).mean(axis=1, keepdims=True) + eps)
 
 
 # ----------------------------------------------------------------------------

@@ -88,6 +88,9 @@ def _load() -> C.CDLL:
     lib.camera_output_error.restype = C.c_int
     lib.camera_output_error.argtypes = [C.c_void_p, C.c_void_p, C.c_int64, C.c_int32, C.c_void_p, C.c_void_p, C.c_size_t,
                                         C.c_void_p]
+    lib.camera_residual_norm.restype = C.c_int
+    lib.camera_residual_norm.argtypes = [C.c_void_p, C.c_int32, C.c_void_p, C.c_int64, C.c_int32, C.c_float, C.c_void_p,
+                                         C.c_void_p]
     lib.camera_sub_index.restype = C.c_int
     lib.camera_sub_index.argtypes = [C.c_void_p, C.c_void_p, C.c_int32, C.POINTER(C.c_int32), C.c_int32, C.c_void_p,
                                      C.c_void_p, C.c_void_p]
@@ -438,4 +441,17 @@ def camera_output_error(y: torch.Tensor, y_hat: torch.Tensor, *, stream: Optiona
     ws = alloc_workspace(int(lib.camera_output_error_workspace_bytes(T)), y.device)
     _check(lib.camera_output_error(y.contiguous().data_ptr(), y_hat.contiguous().data_ptr(), T, d, out.data_ptr(),
                                    ws.data_ptr(), ws.numel(), _stream_ptr(stream)), "camera_output_error")
+    return out
+
+
+def camera_residual_norm(x: torch.Tensor, y: torch.Tensor, *, eps: float = 1e-6, out: Optional[torch.Tensor] = None,
+                         stream: Optional[torch.cuda.Stream] = None) -> torch.Tensor:
+    """Next layer's input of a synthetic stack: (x + y) rescaled to RMS 1 per token, in the dtype of x."""
+    if x.shape != y.shape or y.dtype != torch.float32 or x.dtype not in (torch.bfloat16, torch.float32):
+        raise ValueError("x: bf16 or fp32 [T, d_model], y: fp32 of the same shape")
+    if out is None:
+        out = torch.empty_like(x)
+    _check(lib.camera_residual_norm(x.contiguous().data_ptr(), CAMERA_BF16 if x.dtype == torch.bfloat16 else CAMERA_F32,
+                                    y.contiguous().data_ptr(), int(x.shape[0]), int(x.shape[1]), float(eps), out.data_ptr(),
+                                    _stream_ptr(stream)), "camera_residual_norm")
     return out

@@ -276,6 +276,39 @@ __global__ void __launch_bounds__(256) k_error_final(const double* __restrict__ 
   }
 }
 
+// One warp per token: z = x + y, out = z / sqrt(mean(z^2) + eps) in the dtype of x.  The row stays in registers
+// between the two passes for d_model <= 8192; longer rows are read twice.
+template <typename T>
+__global__ void __launch_bounds__(256) k_residual_norm(const T* __restrict__ x, const float* __restrict__ y, long long n_tokens,
+                                                       int d, float eps, T* __restrict__ out) {
+  constexpr int VN = Vec16<T>::N;
+  const int lane = threadIdx.x & 31;
+  const long long t = (long long)blockIdx.x * 8 + (threadIdx.x >> 5);
+  if (t >= n_tokens) return;
+  const T* xr = x + (size_t)t * d;
+  const float* yr = y + (size_t)t * d;
+  float ss = 0.f;
+  for (int v = lane * VN; v < d; v += 32 * VN) {
+    float xv[VN];
+    Vec16<T>::load(xr + v, xv);
+#pragma unroll
+    for (int i = 0; i < VN; ++i) { const float z = xv[i] + yr[v + i]; ss = fmaf(z, z, ss); }
+  }
+#pragma unroll
+  for (int o = 16; o; o >>= 1) ss += __shfl_xor_sync(0xffffffffu, ss, o);
+  const float scale = rsqrtf(ss / (float)d + eps);
+  T* orow = out + (size_t)t * d;
+  for (int v = lane * VN; v < d; v += 32 * VN) {
+    float xv[VN];
+    Vec16<T>::load(xr + v, xv);
+#pragma unroll
+    for (int i = 0; i < VN; ++i) {
+      const float z = (xv[i] + yr[v + i]) * scale;
+      if constexpr (sizeof(T) == 2) orow[v + i] = __float2bfloat16_rn(z); else orow[v + i] = z;
+    }
+  }
+}
+
 size_t up256(size_t v) { return (v + 255) & ~(size_t)255; }
 
 struct FwdLayout {
@@ -405,5 +438,23 @@ extern "C" int camera_output_error(const float* y, const float* y_hat, int64_t n
   const long long n_part = (n_tokens + 7) / 8;
   if (n_part > 0) k_error_partials<<<(unsigned)n_part, 256, 0, st>>>(y, y_hat, n_tokens, d_model, part);
   k_error_final<<<1, 256, 0, st>>>(part, n_part, n_tokens, out);
+  return cudaGetLastError() == cudaSuccess ? CAMERA_OK : CAMERA_ERR_CUDA;
+}
+
+extern "C" int camera_residual_norm(const void* x, int32_t dtype, const float* y, int64_t n_tokens, int32_t d_model, float eps,
+                                    void* out, void* cuda_stream) {
+  if (n_tokens < 0 || d_model < 8 || d_model % 8 != 0 || !(eps >= 0.f) || (dtype != CAMERA_BF16 && dtype != CAMERA_F32))
+    return CAMERA_ERR_INVALID_ARG;
+  if (n_tokens == 0) return CAMERA_OK;
+  if (x == nullptr || y == nullptr || out == nullptr ||
+      ((reinterpret_cast<uintptr_t>(x) | reinterpret_cast<uintptr_t>(y) | reinterpret_cast<uintptr_t>(out)) & 15))
+    return CAMERA_ERR_INVALID_ARG;
+  cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+  const unsigned grid = (unsigned)((n_tokens + 7) / 8);
+  if (dtype == CAMERA_BF16)
+    k_residual_norm<__nv_bfloat16><<<grid, 256, 0, st>>>(static_cast<const __nv_bfloat16*>(x), y, n_tokens, d_model, eps,
+                                                          static_cast<__nv_bfloat16*>(out));
+  else
+    k_residual_norm<float><<<grid, 256, 0, st>>>(static_cast<const float*>(x), y, n_tokens, d_model, eps, static_cast<float*>(out));
   return cudaGetLastError() == cudaSuccess ? CAMERA_OK : CAMERA_ERR_CUDA;
 }

@@ -139,3 +139,15 @@ def test_forward_argument_errors(P):
     with pytest.raises(P.CameraError) as e:
         P.camera_layer_forward(P.Layer.from_workload(L), X)
     assert e.value.status == -2
+
+
+@pytest.mark.parametrize("dtype", [torch.bfloat16, torch.float32])
+def test_residual_norm(P, dtype):
+    g = torch.Generator(device="cpu").manual_seed(3)
+    x = (torch.randn(1001, 256, generator=g) * 2).to(dtype).to(DEV)
+    y = (torch.randn(1001, 256, generator=g) * 0.5).to(DEV)
+    out = P.camera_residual_norm(x, y, eps=1e-6)
+    ref = O.next_layer_input(f64(x), f64(y), eps=1e-6)
+    tol = 2.0 ** -8 if dtype == torch.bfloat16 else 1e-6       # one rounding to the output dtype
+    assert np.abs(f64(out) - ref).max() <= tol * np.abs(ref).max()
+    assert out.dtype == dtype

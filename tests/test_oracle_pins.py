@@ -423,3 +423,14 @@ def test_sub_index_leaves_out_other_labels_and_handles_empty_experts():
     lists, counts = O.sub_index_lists(labels, np.array([0, 4, 4, 7, 9]), [1])
     assert [l.tolist() for l in lists] == [[0, 2, 3], [], [], [0]]
     assert counts[:, 0].tolist() == [3, 0, 0, 1]
+
+
+def test_next_layer_input_is_the_unit_rms_residual():
+    r = rng(42)
+    X, Y = r.standard_normal((9, 16)), r.standard_normal((9, 16)) * 3
+    Z = O.next_layer_input(X, Y, eps=0.0)
+    assert np.allclose((Z * Z).mean(axis=1), 1.0, atol=1e-12)                  # RMS 1 per token
+    assert np.allclose(Z * np.sqrt(((X + Y) ** 2).mean(axis=1, keepdims=True)), X + Y, atol=1e-12)   # same direction as x + y
+    assert np.allclose(O.next_layer_input(2 * X, 2 * Y, eps=0.0), Z, atol=1e-12)   # scale invariant
+    ref = torch.nn.functional.rms_norm(torch.from_numpy(X + Y), (16,), eps=1e-6).numpy()
+    assert np.allclose(O.next_layer_input(X, Y, eps=1e-6), ref, rtol=1e-12)
