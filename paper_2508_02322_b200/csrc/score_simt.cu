@@ -115,22 +115,34 @@ __global__ void __launch_bounds__(SS_THREADS) k_score_simt(ScoreCtx c) {
   }
 }
 
-// Adds the chunk partials of every micro-expert in chunk order (fp64), squares the max and
-// blends: E_i = [(1-alpha) phi2_i + alpha phi_inf_i] * omega2_i   (Eq. 11).
-__global__ void __launch_bounds__(256) k_combine(ScoreCtx c) {
-  const int i = blockIdx.x * blockDim.x + threadIdx.x;
-  if (i >= c.n_me) return;
-  const int e = upper_segment(c.me_prefix, c.n_experts, i);
-  const int ch = i - c.me_prefix[e];
-  const ExpertDyn dy = c.edyn[e];
-  const int f = c.est[e].d_ff;
+// Adds the chunk partials of every micro-expert (fp64, fixed order: eight interleaved running sums, then those in
+// order), squares the max and blends: E_i = [(1-alpha) phi2_i + alpha phi_inf_i] * omega2_i   (Eq. 11).
+// Block = 32 micro-experts x 8 chunk lanes, so that eight loads per micro-expert are in flight.
+constexpr int CB_X = 32, CB_Y = 8;
+__global__ void __launch_bounds__(CB_X * CB_Y) k_combine(ScoreCtx c) {
+  __shared__ double ssum[CB_Y][CB_X];
+  __shared__ float smax[CB_Y][CB_X];
+  const int i = blockIdx.x * CB_X + threadIdx.x;
   double s = 0.0;
   float m = 0.f;
-  for (int j = 0; j < dy.n_chunks; ++j) {
-    const size_t slot = (size_t)dy.part_begin + (size_t)j * f + ch;
-    s += (double)c.part_sum[slot];
-    m = fmaxf(m, c.part_max[slot]);
+  if (i < c.n_me) {
+    const int e = upper_segment(c.me_prefix, c.n_experts, i);
+    const int ch = i - c.me_prefix[e];
+    const ExpertDyn dy = c.edyn[e];
+    const int f = c.est[e].d_ff;
+    for (int j = threadIdx.y; j < dy.n_chunks; j += CB_Y) {
+      const size_t slot = (size_t)dy.part_begin + (size_t)j * f + ch;
+      s += (double)c.part_sum[slot];
+      m = fmaxf(m, c.part_max[slot]);
+    }
   }
+  ssum[threadIdx.y][threadIdx.x] = s;
+  smax[threadIdx.y][threadIdx.x] = m;
+  __syncthreads();
+  if (threadIdx.y != 0 || i >= c.n_me) return;
+  s = 0.0; m = 0.f;
+#pragma unroll
+  for (int y = 0; y < CB_Y; ++y) { s += ssum[y][threadIdx.x]; m = fmaxf(m, smax[y][threadIdx.x]); }
   double m2 = (double)m * (double)m;
   if (c.accumulate) {     // earlier batches of tokens: sums add, maxima take the maximum
     s += (double)c.phi2[i];
@@ -156,7 +168,7 @@ cudaError_t launch_score_simt(const ScoreCtx& c, cudaStream_t st) {
 
 cudaError_t launch_combine(const ScoreCtx& c, cudaStream_t st) {
   if (c.n_me == 0) return cudaSuccess;
-  k_combine<<<(c.n_me + 255) / 256, 256, 0, st>>>(c);
+  k_combine<<<(c.n_me + CB_X - 1) / CB_X, dim3(CB_X, CB_Y), 0, st>>>(c);
   return cudaGetLastError();
 }
 
