@@ -34,6 +34,7 @@ constexpr int U_A_BYTES = CH_TILE * 128;         // 128 weight rows x 128 B (one
 constexpr int U_B_BYTES = UMMA_TOK * 128;        // 256 token rows x 128 B
 constexpr int U_STAGE_BYTES = 2 * U_A_BYTES + U_B_BYTES;
 constexpr int U_TMEM_COLS = 512;
+constexpr int U_SCHED = 2;                       // depth of the ring that passes unit numbers between the warps
 constexpr int U_WBUF_BYTES = 4 * UMMA_TOK * 4;   // router weights of a token tile, one copy per epilogue warp
 constexpr int U_SMEM_BYTES = U_STAGES * U_STAGE_BYTES + U_WBUF_BYTES + 256 + 1024;
 static_assert(CH_TILE == 128, "one micro-expert per TMEM lane");
@@ -72,9 +73,14 @@ __global__ void __launch_bounds__(U_THREADS, 1) k_score_umma(const ScoreCtx c) {
   auto empty_bar = [&](int s) { return bars + 8u * (U_STAGES + s); };
   const uint32_t tfull_bar = bars + 8u * (2 * U_STAGES);
   const uint32_t tempty_bar = bars + 8u * (2 * U_STAGES + 1);
-  uint8_t* const tail = base_ptr + U_STAGES * U_STAGE_BYTES + U_WBUF_BYTES + 8 * (2 * U_STAGES + 2);
+  // work units are handed out in order from a counter in global memory: the producer thread takes the next one and
+  // passes its number to the MMA thread and the epilogue warps through a small ring
+  auto sfull_bar = [&](int q) { return bars + 8u * (2 * U_STAGES + 2 + q); };
+  auto sempty_bar = [&](int q) { return bars + 8u * (2 * U_STAGES + 2 + U_SCHED + q); };
+  uint8_t* const tail = base_ptr + U_STAGES * U_STAGE_BYTES + U_WBUF_BYTES + 8 * (2 * U_STAGES + 2 + 2 * U_SCHED);
   volatile uint32_t* const tmem_slot = reinterpret_cast<volatile uint32_t*>(tail);
   volatile int* const abort_flag = reinterpret_cast<volatile int*>(tail + 8);
+  volatile int* const sched_unit = reinterpret_cast<volatile int*>(tail + 16);
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int total_units = c.totals->total_units;
@@ -84,6 +90,7 @@ __global__ void __launch_bounds__(U_THREADS, 1) k_score_umma(const ScoreCtx c) {
     for (int s = 0; s < U_STAGES; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
     mbar_init(tfull_bar, 1);
     mbar_init(tempty_bar, 128);
+    for (int q = 0; q < U_SCHED; ++q) { mbar_init(sfull_bar(q), 1); mbar_init(sempty_bar(q), 5); }
     *abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
@@ -106,7 +113,16 @@ __global__ void __launch_bounds__(U_THREADS, 1) k_score_umma(const ScoreCtx c) {
       uint32_t phase = 0;
       bool ok = true;
       const char* maps = static_cast<const char*>(c.tensor_maps);
-      for (int unit = blockIdx.x; ok && unit < total_units; unit += gridDim.x) {
+      int q = 0;
+      uint32_t qphase = 0;
+      while (ok) {
+        if (!mbar_wait(sempty_bar(q), qphase ^ 1u, abort_flag)) { ok = false; break; }
+        int unit = atomicAdd(&c.totals->unit_counter, 1);
+        if (unit >= total_units) unit = -1;
+        sched_unit[q] = unit;
+        mbar_arrive(sfull_bar(q));
+        if (++q == U_SCHED) { q = 0; qphase ^= 1u; }
+        if (unit < 0) break;
         const UnitInfo u = decode_unit(c, unit);
         const int n_tiles = (u.rows + UMMA_TOK - 1) / UMMA_TOK;
         const void* map_g = maps + (size_t)128 * (2 * u.e);
@@ -141,7 +157,14 @@ __global__ void __launch_bounds__(U_THREADS, 1) k_score_umma(const ScoreCtx c) {
       int stage = 0;
       uint32_t phase = 0, tile_phase = 0;
       bool ok = true;
-      for (int unit = blockIdx.x; ok && unit < total_units; unit += gridDim.x) {
+      int q = 0;
+      uint32_t qphase = 0;
+      while (ok) {
+        if (!mbar_wait(sfull_bar(q), qphase, abort_flag)) { ok = false; break; }
+        const int unit = sched_unit[q];
+        mbar_arrive(sempty_bar(q));
+        if (++q == U_SCHED) { q = 0; qphase ^= 1u; }
+        if (unit < 0) break;
         const UnitInfo u = decode_unit(c, unit);
         const int n_tiles = (u.rows + UMMA_TOK - 1) / UMMA_TOK;
         for (int tt = 0; ok && tt < n_tiles; ++tt) {
@@ -179,7 +202,16 @@ __global__ void __launch_bounds__(U_THREADS, 1) k_score_umma(const ScoreCtx c) {
     float* const wb = wbuf + warp * UMMA_TOK;
     const uint32_t t_gate = tmem_base + ((uint32_t)(warp * 32) << 16);
     const uint32_t t_up = t_gate + UMMA_TOK;
-    for (int unit = blockIdx.x; ok && unit < total_units; unit += gridDim.x) {
+    int q = 0;
+    uint32_t qphase = 0;
+    while (ok) {
+      ok = __all_sync(0xffffffffu, mbar_wait(sfull_bar(q), qphase, abort_flag));
+      if (!ok) break;
+      const int unit = sched_unit[q];
+      __syncwarp();
+      if (lane == 0) mbar_arrive(sempty_bar(q));
+      if (++q == U_SCHED) { q = 0; qphase ^= 1u; }
+      if (unit < 0) break;
       const UnitInfo u = decode_unit(c, unit);
       const int n_tiles = (u.rows + UMMA_TOK - 1) / UMMA_TOK;
       const float* wsrc = u.shared_idx < 0 ? c.perm_w + u.row0 : c.shared_w + (size_t)u.shared_idx * c.n_tokens + u.row0;
