@@ -28,6 +28,7 @@ constexpr int P_A_BYTES = 128 * 128;             // 128 weight rows x 128 B (one
 constexpr int P_B_BYTES = 128 * 128;             // this CTA's half of the token tile
 constexpr int P_STAGE_BYTES = 2 * P_A_BYTES + P_B_BYTES;
 constexpr int P_TMEM_COLS = 512;
+constexpr int P_SCHED = 2;                       // depth of the ring that passes unit numbers around the pair
 constexpr int P_WBUF_BYTES = 4 * UMMA_TOK * 4;
 constexpr int P_SMEM_BYTES = P_STAGES * P_STAGE_BYTES + P_WBUF_BYTES + 256 + 1024;
 
@@ -45,6 +46,35 @@ __device__ __forceinline__ uint32_t map_to_cta(uint32_t addr, uint32_t rank) {
   uint32_t r;
   asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(addr), "r"(rank));
   return r;
+}
+// try_wait that also orders what another CTA of the cluster wrote before it arrived.
+__device__ __forceinline__ bool mbar_try_wait_cluster(uint32_t bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n"
+      ".reg .pred p;\n"
+      "mbarrier.try_wait.parity.acquire.cluster.shared::cta.b64 p, [%1], %2;\n"
+      "selp.u32 %0, 1, 0, p;\n"
+      "}\n"
+      : "=r"(ok)
+      : "r"(bar), "r"(parity)
+      : "memory");
+  return ok != 0;
+}
+__device__ __forceinline__ bool mbar_wait_cluster(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
+  if (mbar_try_wait_cluster(bar, parity)) return true;
+  const unsigned long long t0 = globaltimer_ns();
+  unsigned spins = 0;
+  for (;;) {
+    if (mbar_try_wait_cluster(bar, parity)) return true;
+    if ((++spins & 63u) == 0u) {
+      if (*abort_flag) return false;
+      if (globaltimer_ns() - t0 > WAIT_LIMIT_NS) { *abort_flag = 1; return false; }
+    }
+  }
+}
+__device__ __forceinline__ void st_cluster_u32(uint32_t cluster_addr, uint32_t v) {
+  asm volatile("st.shared::cluster.u32 [%0], %1;" ::"r"(cluster_addr), "r"(v) : "memory");
 }
 __device__ __forceinline__ void mbar_arrive_cluster(uint32_t cluster_addr) {
   asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
@@ -107,13 +137,18 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(P_THREADS, 1) k_scor
   auto empty_bar = [&](int s) { return bars + 8u * (P_STAGES + s); };
   const uint32_t tfull_bar = bars + 8u * (2 * P_STAGES);
   const uint32_t tempty_bar = bars + 8u * (2 * P_STAGES + 1);
-  uint8_t* const tail = base_ptr + P_STAGES * P_STAGE_BYTES + P_WBUF_BYTES + 8 * (2 * P_STAGES + 2);
+  // work units are handed out in order: the first CTA's producer takes the next one from a counter in global memory and
+  // writes its number into the ring of both CTAs; sfull (each CTA) = a number is there, sempty (first CTA) = the
+  // ten readers of the pair (MMA thread, second CTA's producer, eight epilogue warps) have taken it
+  auto sfull_bar = [&](int q) { return bars + 8u * (2 * P_STAGES + 2 + q); };
+  auto sempty_bar = [&](int q) { return bars + 8u * (2 * P_STAGES + 2 + P_SCHED + q); };
+  uint8_t* const tail = base_ptr + P_STAGES * P_STAGE_BYTES + P_WBUF_BYTES + 8 * (2 * P_STAGES + 2 + 2 * P_SCHED);
   volatile uint32_t* const tmem_slot = reinterpret_cast<volatile uint32_t*>(tail);
   volatile int* const abort_flag = reinterpret_cast<volatile int*>(tail + 8);
+  volatile int* const sched_unit = reinterpret_cast<volatile int*>(tail + 16);
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const uint32_t rank = cluster_ctarank();
-  const int pair = blockIdx.x >> 1, n_pairs = gridDim.x >> 1;
   const int total_units = c.totals->total_units;
   const int n_kb = c.d_model / UMMA_BK;
 
@@ -121,6 +156,7 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(P_THREADS, 1) k_scor
     for (int s = 0; s < P_STAGES; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
     mbar_init(tfull_bar, 1);
     mbar_init(tempty_bar, 256);
+    for (int q = 0; q < P_SCHED; ++q) { mbar_init(sfull_bar(q), 1); mbar_init(sempty_bar(q), 10); }
     *abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
@@ -144,7 +180,25 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(P_THREADS, 1) k_scor
       uint32_t phase = 0;
       bool ok = true;
       const char* maps = static_cast<const char*>(c.tensor_maps);
-      for (int unit = pair; ok && unit < total_units; unit += n_pairs) {
+      int q = 0;
+      uint32_t qphase = 0;
+      while (ok) {
+        int unit;
+        if (rank == 0) {
+          if (!mbar_wait_cluster(sempty_bar(q), qphase ^ 1u, abort_flag)) { ok = false; break; }
+          unit = atomicAdd(&c.totals->unit_counter, 1);
+          if (unit >= total_units) unit = -1;
+          sched_unit[q] = unit;
+          st_cluster_u32(map_to_cta(smem_u32((const void*)(sched_unit + q)), 1), (uint32_t)unit);
+          mbar_arrive(sfull_bar(q));
+          mbar_arrive_cluster(map_to_cta(sfull_bar(q), 1));
+        } else {
+          if (!mbar_wait_cluster(sfull_bar(q), qphase, abort_flag)) { ok = false; break; }
+          unit = sched_unit[q];
+          mbar_arrive_cluster(map_to_cta(sempty_bar(q), 0));
+        }
+        if (++q == P_SCHED) { q = 0; qphase ^= 1u; }
+        if (unit < 0) break;
         const UnitInfo u = decode_unit(c, unit);
         const int n_tiles = (u.rows + UMMA_TOK - 1) / UMMA_TOK;
         const void* map_g = maps + (size_t)128 * (2 * u.e);
@@ -180,7 +234,14 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(P_THREADS, 1) k_scor
       int stage = 0;
       uint32_t phase = 0, tile_phase = 0;
       bool ok = true;
-      for (int unit = pair; ok && unit < total_units; unit += n_pairs) {
+      int q = 0;
+      uint32_t qphase = 0;
+      while (ok) {
+        if (!mbar_wait(sfull_bar(q), qphase, abort_flag)) { ok = false; break; }
+        const int unit = sched_unit[q];
+        mbar_arrive(sempty_bar(q));
+        if (++q == P_SCHED) { q = 0; qphase ^= 1u; }
+        if (unit < 0) break;
         const UnitInfo u = decode_unit(c, unit);
         const int n_tiles = (u.rows + UMMA_TOK - 1) / UMMA_TOK;
         for (int tt = 0; ok && tt < n_tiles; ++tt) {
@@ -218,7 +279,17 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(P_THREADS, 1) k_scor
     const uint32_t t_gate = tmem_base + ((uint32_t)(warp * 32) << 16);
     const uint32_t t_up = t_gate + UMMA_TOK;
     const uint32_t tempty0 = map_to_cta(tempty_bar, 0);
-    for (int unit = pair; ok && unit < total_units; unit += n_pairs) {
+    const uint32_t sempty0[P_SCHED] = {map_to_cta(sempty_bar(0), 0), map_to_cta(sempty_bar(1), 0)};
+    int q = 0;
+    uint32_t qphase = 0;
+    while (ok) {
+      ok = __all_sync(0xffffffffu, mbar_wait_cluster(sfull_bar(q), qphase, abort_flag));
+      if (!ok) break;
+      const int unit = sched_unit[q];
+      __syncwarp();
+      if (lane == 0) mbar_arrive_cluster(sempty0[q]);
+      if (++q == P_SCHED) { q = 0; qphase ^= 1u; }
+      if (unit < 0) break;
       const UnitInfo u = decode_unit(c, unit);
       const int n_tiles = (u.rows + UMMA_TOK - 1) / UMMA_TOK;
       const float* wsrc = u.shared_idx < 0 ? c.perm_w + u.row0 : c.shared_w + (size_t)u.shared_idx * c.n_tokens + u.row0;
