@@ -283,7 +283,8 @@ def main():
     ap.add_argument("--shard", default="layers", choices=["layers", "tokens"],
                     help="with --gpus N: every rank its own layer (weak scaling, no exchange), or one layer's tokens "
                          "spread over the ranks with an all-reduce of the 2 x N_e score components (strong scaling)")
-    ap.add_argument("--cta-pair", action="store_true", help="score on CTA pairs (tcgen05 cta_group::2) instead of single CTAs")
+    ap.add_argument("--cta-pair", action="store_true", help="force scoring on CTA pairs (tcgen05 cta_group::2)")
+    ap.add_argument("--single-cta", action="store_true", help="force scoring with one CTA per MMA")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-compact", action="store_true")
@@ -342,14 +343,14 @@ def main():
     def step(i, events=None):
         if by_tokens:
             P.camera_score_layer(layer, Xs[i % 2], ALPHA, energy=energy, workspace=ws_score, stage_events=events,
-                                 cta_pair=args.cta_pair, phi2=phi2, phi_inf_sq=phi_inf)
+                                 cta_pair=(True if args.cta_pair else (False if args.single_cta else None)), phi2=phi2, phi_inf_sq=phi_inf)
             reduce_components(phi2, phi_inf, dist if world > 1 else None)
             # no tokens, accumulate: folds nothing in and turns the reduced components into the energies
             P.camera_score_layer(layer, x_none, ALPHA, energy=energy, workspace=ws_score, phi2=phi2, phi_inf_sq=phi_inf,
                                  accumulate=True)
         else:
             P.camera_score_layer(layer, Xs[i % 2], ALPHA, energy=energy, workspace=ws_score, stage_events=events,
-                                 cta_pair=args.cta_pair)
+                                 cta_pair=(True if args.cta_pair else (False if args.single_cta else None)))
         for j, r in enumerate(PRUNE_RATIOS):
             P.camera_select_prune(energy, r, workspace=ws_sel, keep_mask=keep[j])
         P.camera_alloc_bits(energy, BIT_RATIOS, BIT_LEVELS, workspace=ws_sel, bits_out=bits)
@@ -543,12 +544,12 @@ def main():
     flop = cfg.gate_up_flop
     score_ms = stage_ms["score"]
     achieved = flop / (score_ms * 1e-3) / 1e12
-    roofline = {"kernel": "k_score_umma", "bound": "tensor", "achieved": achieved,
+    roofline = {"kernel": "k_score_umma" if args.single_cta else "k_score_umma_pair / k_score_umma (library's choice)", "bound": "tensor", "achieved": achieved,
                 "peak": peaks["bf16_tflops_sustained"], "unit": "TFLOP/s", "frac": achieved / peaks["bf16_tflops_sustained"],
                 "frac_of_burst_peak": achieved / peaks["bf16_tflops"], "peak_source": peaks["source"] + " (sustained bf16)",
                 "flop_per_launch": flop, "ms_per_launch": score_ms,
                 "traffic": SCORE_KERNEL_DRAM_BYTES_PER_FLOP * flop
-                if (args.config == "qwen2_57b_a14b" and not args.cta_pair) else None}
+                if (args.config == "qwen2_57b_a14b" and not args.single_cta) else None}
 
     cpu = None
     if not args.no_cpu_baseline:

@@ -59,8 +59,10 @@ enum {
 /* camera_score_aux_t.flags */
 enum {
   CAMERA_SCORE_FORCE_SIMT = 1u,    /* run the fp32-FMA kernels even where the tensor-core kernels apply */
-  CAMERA_SCORE_CTA_PAIR = 2u,      /* tensor-core scoring on CTA pairs (tcgen05 cta_group::2): less L2 and shared-memory
-                                      traffic per flop, but measured slower under the power cap; off by default */
+  CAMERA_SCORE_CTA_PAIR = 2u,      /* force tensor-core scoring on CTA pairs (tcgen05 cta_group::2, 256 micro-experts per
+                                      work unit: less L2 and shared-memory traffic per flop).  By default the library takes
+                                      pairs unless padding d_ff to multiples of 256 would add more than 6 % of work */
+  CAMERA_SCORE_SINGLE_CTA = 8u,    /* force one CTA per MMA (128 micro-experts per work unit) */
   CAMERA_SCORE_ACCUMULATE = 4u     /* phi2 and phi_inf_sq (both required) already hold the result of earlier batches of
                                       calibration tokens of this layer; this call folds its batch in (the column sums of
                                       Alg. 1 line 7 add up over batches, the column maxima of line 8 take the maximum)

@@ -21,6 +21,7 @@ CAMERA_ROUTER_NORM_TOPK, CAMERA_SHARED_GATE_SIGMOID = 1, 2
 CAMERA_SCORE_FORCE_SIMT = 1
 CAMERA_SCORE_CTA_PAIR = 2
 CAMERA_SCORE_ACCUMULATE = 4
+CAMERA_SCORE_SINGLE_CTA = 8
 STAGES = ("router", "permute", "rownorm", "score", "combine")
 
 
@@ -195,7 +196,7 @@ def alloc_workspace(nbytes: int, device) -> torch.Tensor:
 
 def camera_score_layer(layer: Layer, x: torch.Tensor, alpha: float, *, energy: Optional[torch.Tensor] = None,
                        workspace: Optional[torch.Tensor] = None, details: bool = False,
-                       routing_in=None, force_simt: bool = False, cta_pair: bool = False, stage_events=None,
+                       routing_in=None, force_simt: bool = False, cta_pair: Optional[bool] = None, stage_events=None,
                        phi2: Optional[torch.Tensor] = None, phi_inf_sq: Optional[torch.Tensor] = None,
                        accumulate: bool = False,
                        stream: Optional[torch.cuda.Stream] = None, check_status: bool = False):
@@ -239,7 +240,7 @@ def camera_score_layer(layer: Layer, x: torch.Tensor, alpha: float, *, energy: O
                 raise ValueError(f"{name} must be a contiguous fp32 [N_e] tensor on the device of x")
             out[name] = t
             setattr(aux, name, t.data_ptr())
-    aux.flags = ((CAMERA_SCORE_FORCE_SIMT if force_simt else 0) | (CAMERA_SCORE_CTA_PAIR if cta_pair else 0) |
+    aux.flags = ((CAMERA_SCORE_FORCE_SIMT if force_simt else 0) | (CAMERA_SCORE_CTA_PAIR if cta_pair else 0) | (CAMERA_SCORE_SINGLE_CTA if cta_pair is False else 0) |
                  (CAMERA_SCORE_ACCUMULATE if accumulate else 0))
     if stage_events:
         for name, (e0, e1) in stage_events.items():

@@ -269,7 +269,25 @@ int score_front(const camera_layer_t* L, const void* x, int64_t T, float alpha, 
 
   const bool use_umma = umma_shape_ok(L) && !(aux && (aux->flags & CAMERA_SCORE_FORCE_SIMT)) &&
                         (reinterpret_cast<uintptr_t>(x) & 15) == 0;
-  const bool use_pair = use_umma && fwd == nullptr && aux && (aux->flags & CAMERA_SCORE_CTA_PAIR);
+  bool use_pair = false;
+  if (use_umma && fwd == nullptr) {
+    if (aux && (aux->flags & CAMERA_SCORE_CTA_PAIR)) use_pair = true;
+    else if (aux && (aux->flags & CAMERA_SCORE_SINGLE_CTA)) use_pair = false;
+    else {
+      // pairs move fewer bytes per flop but work on 256 micro-experts at a time: measured 2 % ahead where d_ff fills
+      // the pairs (Qwen2, Mixtral shapes), 6 % behind where a ninth of every expert's last pair is padding (d_ff 1408)
+      double work1 = 0.0, work2 = 0.0;
+      for (int e = 0; e < E; ++e) {
+        const double rows = e < L->n_routed ? (double)T * c.top_k / L->n_routed : (double)T;
+        work1 += rows * (double)((L->d_ff[e] + CH_TILE - 1) / CH_TILE * CH_TILE);
+        work2 += rows * (double)((L->d_ff[e] + 2 * CH_TILE - 1) / (2 * CH_TILE) * (2 * CH_TILE));
+      }
+      int dev_sms = 0, cur = 0;
+      cudaGetDevice(&cur);
+      cudaDeviceGetAttribute(&dev_sms, cudaDevAttrMultiProcessorCount, cur);
+      use_pair = work2 <= 1.06 * work1 && dev_sms % 2 == 0;
+    }
+  }
   c.ch_tile = use_pair ? 2 * CH_TILE : CH_TILE;
   c.ct_group = score_group_channels() / c.ch_tile;
   const bool use_router_umma = use_umma && router_umma_ok(c);

@@ -54,7 +54,7 @@ def check_routing(olayer, Xd, topk_idx, topk_w):
     return int((~same).sum())
 
 
-def run_and_compare(P, L, X, alpha=0.95, channels=None, force_simt=False, check_dense=False, cta_pair=False):
+def run_and_compare(P, L, X, alpha=0.95, channels=None, force_simt=False, check_dense=False, cta_pair=None):
     """Scores one layer on the GPU (own routing, then the oracle's routing injected) and checks
     every component against the oracle.  `channels` restricts the oracle to sampled micro-experts."""
     layer = P.Layer.from_workload(L)

@@ -41,8 +41,9 @@ def test_random_layers(P, seed):
     L = W.make_layer(cfg, seed=seed, device=DEV, down_layout=str(r.choice(["hf", "me_major"])))
     X = W.make_tokens(cfg, seed=seed, device=DEV)
     alpha = float(r.choice([0.0, 0.5, 0.95, 1.0]))
-    kernel = ["umma", "umma_pair", "simt"][seed % 3]
-    out, _ = run_and_compare(P, L, X, alpha=alpha, force_simt=kernel == "simt", cta_pair=kernel == "umma_pair")
+    kernel = ["umma", "umma_pair", "simt", "auto"][seed % 4]
+    out, _ = run_and_compare(P, L, X, alpha=alpha, force_simt=kernel == "simt",
+                              cta_pair={"umma": False, "umma_pair": True}.get(kernel))
     # selections on these scores, and the weights they select
     E = out["energy"]
     ratio = float(r.choice([0.0, 0.3, 0.7]))
