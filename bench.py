@@ -36,7 +36,7 @@ PAPER_CONTEXT = "paper: <5 min for the full Qwen2-57B-A14B analysis on one A100-
 LAUNCHES_PER_STEP = 8 + 9 * (len(PRUNE_RATIOS) + 1)
 # DRAM bytes (read + write) per gate/up flop of the scoring kernel, from the committed ncu capture of a
 # 1/8 slice of the layer whose traffic grows in proportion to the flop (profiles/k_score_umma_qwen2_slice.md).
-SCORE_KERNEL_DRAM_BYTES_PER_FLOP = 5.245e9 / 1.924e13
+SCORE_KERNEL_DRAM_BYTES_PER_FLOP = 4.469e9 / 1.924e13
 
 
 def shard_layers(n_layers: int, world: int, rank: int):
