@@ -52,7 +52,8 @@ struct PlanTotals {
   int32_t status;        // device status word (0 = fine)
   int32_t total_chunks;  // sum over experts of n_chunks
   int32_t unit_counter;  // next scoring work unit to hand out (the scoring kernel's CTAs take units in order)
-  int32_t pad[3];
+  int32_t down_counter;  // the same for the W_down GEMM of the layer forward
+  int32_t pad[2];
 };
 
 // Everything the kernels of one camera_score_layer call need.

@@ -23,6 +23,7 @@ constexpr int D_A_BYTES = D_TILE * 128;
 constexpr int D_B_BYTES = UMMA_TOK * 128;
 constexpr int D_STAGE_BYTES = D_A_BYTES + D_B_BYTES;
 constexpr int D_TMEM_COLS = 512;
+constexpr int D_SCHED = 2;                        // ring that passes unit numbers from the producer to the other warps
 constexpr int D_SMEM_BYTES = D_STAGES * D_STAGE_BYTES + 256 + 1024;
 
 struct DownUnit {
@@ -62,9 +63,12 @@ __global__ void __launch_bounds__(D_THREADS, 1) k_down_umma(const ScoreCtx c, co
   auto empty_bar = [&](int s) { return bars + 8u * (D_STAGES + s); };
   auto tfull_bar = [&](int a) { return bars + 8u * (2 * D_STAGES + a); };
   auto tempty_bar = [&](int a) { return bars + 8u * (2 * D_STAGES + 2 + a); };
-  uint8_t* const tail = base_ptr + D_STAGES * D_STAGE_BYTES + 8 * (2 * D_STAGES + 4);
+  auto sfull_bar = [&](int q) { return bars + 8u * (2 * D_STAGES + 4 + q); };
+  auto sempty_bar = [&](int q) { return bars + 8u * (2 * D_STAGES + 4 + D_SCHED + q); };
+  uint8_t* const tail = base_ptr + D_STAGES * D_STAGE_BYTES + 8 * (2 * D_STAGES + 4 + 2 * D_SCHED);
   volatile uint32_t* const tmem_slot = reinterpret_cast<volatile uint32_t*>(tail);
   volatile int* const abort_flag = reinterpret_cast<volatile int*>(tail + 8);
+  volatile int* const sched_unit = reinterpret_cast<volatile int*>(tail + 16);
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int total_units = c.totals->total_chunks * n_dt;
@@ -72,6 +76,7 @@ __global__ void __launch_bounds__(D_THREADS, 1) k_down_umma(const ScoreCtx c, co
   if (tid == 0) {
     for (int s = 0; s < D_STAGES; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
     for (int a = 0; a < 2; ++a) { mbar_init(tfull_bar(a), 1); mbar_init(tempty_bar(a), 128); }
+    for (int q = 0; q < D_SCHED; ++q) { mbar_init(sfull_bar(q), 1); mbar_init(sempty_bar(q), 5); }
     *abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
@@ -94,7 +99,16 @@ __global__ void __launch_bounds__(D_THREADS, 1) k_down_umma(const ScoreCtx c, co
       uint32_t phase = 0;
       bool ok = true;
       const char* maps = static_cast<const char*>(maps_raw);
-      for (int unit = blockIdx.x; ok && unit < total_units; unit += gridDim.x) {
+      int q = 0;
+      uint32_t qphase = 0;
+      while (ok) {   // units are taken in order from a counter, as in the scoring kernel
+        if (!mbar_wait(sempty_bar(q), qphase ^ 1u, abort_flag)) { ok = false; break; }
+        int unit = atomicAdd(&c.totals->down_counter, 1);
+        if (unit >= total_units) unit = -1;
+        sched_unit[q] = unit;
+        mbar_arrive(sfull_bar(q));
+        if (++q == D_SCHED) { q = 0; qphase ^= 1u; }
+        if (unit < 0) break;
         const DownUnit u = decode_down_unit(c, unit, n_dt);
         if (u.n_kb == 0) continue;
         const int n_tiles = (u.rows + UMMA_TOK - 1) / UMMA_TOK;
@@ -126,7 +140,14 @@ __global__ void __launch_bounds__(D_THREADS, 1) k_down_umma(const ScoreCtx c, co
       int stage = 0, acc = 0;
       uint32_t phase = 0, acc_phase = 0;
       bool ok = true;
-      for (int unit = blockIdx.x; ok && unit < total_units; unit += gridDim.x) {
+      int q = 0;
+      uint32_t qphase = 0;
+      while (ok) {
+        if (!mbar_wait(sfull_bar(q), qphase, abort_flag)) { ok = false; break; }
+        const int unit = sched_unit[q];
+        mbar_arrive(sempty_bar(q));
+        if (++q == D_SCHED) { q = 0; qphase ^= 1u; }
+        if (unit < 0) break;
         const DownUnit u = decode_down_unit(c, unit, n_dt);
         if (u.n_kb == 0) continue;
         const int n_tiles = (u.rows + UMMA_TOK - 1) / UMMA_TOK;
@@ -159,7 +180,16 @@ __global__ void __launch_bounds__(D_THREADS, 1) k_down_umma(const ScoreCtx c, co
     int acc = 0;
     uint32_t acc_phase = 0;
     bool ok = true;
-    for (int unit = blockIdx.x; ok && unit < total_units; unit += gridDim.x) {
+    int q = 0;
+    uint32_t qphase = 0;
+    while (ok) {
+      ok = __all_sync(0xffffffffu, mbar_wait(sfull_bar(q), qphase, abort_flag));
+      if (!ok) break;
+      const int unit = sched_unit[q];
+      __syncwarp();
+      if (lane == 0) mbar_arrive(sempty_bar(q));
+      if (++q == D_SCHED) { q = 0; qphase ^= 1u; }
+      if (unit < 0) break;
       const DownUnit u = decode_down_unit(c, unit, n_dt);
       const int n_tiles = (u.rows + UMMA_TOK - 1) / UMMA_TOK;
       const int ch = u.c0 + warp * 32 + lane;

@@ -265,6 +265,7 @@ __global__ void k_plan(ScoreCtx c) {
   c.totals->total_rows = row;
   c.totals->total_chunks = chunks;
   c.totals->unit_counter = 0;
+  c.totals->down_counter = 0;
 }
 
 // One warp per token: copies the token's hidden state to its row in every chosen expert's list.
