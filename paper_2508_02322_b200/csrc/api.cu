@@ -13,8 +13,6 @@ int rownorm_blocks(int down_layout, int dtype, int f);
 
 namespace {
 
-constexpr int PLAN_SMS = 148;   // used only to size work units; the result is valid on any device
-
 size_t up256(size_t v) { return (v + 255) & ~(size_t)255; }
 
 // Micro-experts per scheduling group.  2560 of them are 37 MB of gate+up rows at d_model 3584,
@@ -79,31 +77,17 @@ ScoreLayout score_layout(const camera_layer_t* L, int64_t T) {
   s.n_experts = E;
   s.n_blocks = (int)((T + ROUTER_TOK - 1) / ROUTER_TOK);
   long long n_me = 0;
-  double tiles = 0.0;
   int f_routed_max = 0;
   for (int e = 0; e < E; ++e) {
     n_me += L->d_ff[e];
-    const double ct = (double)((L->d_ff[e] + CH_TILE - 1) / CH_TILE);
-    if (e < L->n_routed) {
-      f_routed_max = L->d_ff[e] > f_routed_max ? L->d_ff[e] : f_routed_max;
-    } else {
-      tiles += ct * (double)((T + UMMA_TOK - 1) / UMMA_TOK);
-    }
-  }
-  if (L->n_routed > 0) {
-    double avg_ct = 0.0;
-    for (int e = 0; e < L->n_routed; ++e) avg_ct += (double)((L->d_ff[e] + CH_TILE - 1) / CH_TILE);
-    avg_ct /= L->n_routed;
-    tiles += avg_ct * (double)(T * k) / UMMA_TOK;
+    if (e < L->n_routed && L->d_ff[e] > f_routed_max) f_routed_max = L->d_ff[e];
   }
   s.n_me = (int)n_me;
   // tokens per work unit: one tile.  Units of a group are numbered (token tile, channel tile), so with one-tile units
   // the CTAs running at one time work on a handful of *neighbouring* token tiles and move on together; measured on the
   // Qwen2-shaped layer, units of 1 / 2 / 4 / 8 / 16 tiles: 1320 / 1279 / 1276 / 1239 / 1199 TFLOP/s (DRAM reads of the
   // 1/8 slice 7.3 GB with 1 tile against 10.7 GB with 8).  The price is one partial per micro-expert and token tile.
-  const int chunk_tiles = 1;
-  (void)tiles;
-  s.chunk_tokens = chunk_tiles * UMMA_TOK;
+  s.chunk_tokens = UMMA_TOK;
   s.max_rows_perm = (int)(T * k + (long long)ROW_ALIGN * L->n_routed);
   long long part = 0;
   if (L->n_routed > 0) part += (long long)f_routed_max * ((T * k) / s.chunk_tokens + L->n_routed);

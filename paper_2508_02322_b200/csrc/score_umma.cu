@@ -14,6 +14,10 @@
 // the tile: gate and up of a (micro-expert, token) pair arrive in the same thread, and the reduction
 // over tokens runs down its own registers.
 //
+// Work units (one channel tile x one token tile) are handed out in order from a counter in global memory, so
+// that the CTAs running at one time share a few neighbouring token tiles and one expert's weights through L2
+// and stay in step; which CTA runs a unit does not change the result (one partial per unit and micro-expert).
+//
 // Every wait on an mbarrier is bounded: when a wait runs out the CTA records
 // CAMERA_ERR_DEVICE_TIMEOUT in the status word, lets its copies land, frees its tensor memory and
 // returns.
