@@ -76,3 +76,27 @@ def test_argument_errors_return_before_any_launch(P):
     r = (C.c_double * 3)(0.2, 0.6, 0.2)
     b = (C.c_int32 * 3)(3, 2, 300)
     assert P.lib.camera_alloc_bits(4096, seg, 1, r, b, 3, None, 0, 4096, None, 4096, 1 << 20, None) == -1   # bit-width
+
+
+def test_new_entry_points_reject_bad_arguments_on_the_host(P):
+    ok = _layer_struct(P)
+    order = (C.c_int32 * 2)(1, 1)
+    assert P.lib.camera_sub_index(4096, 4096, 4, order, 2, 4096, 4096, None) == -1               # a label named twice
+    assert P.lib.camera_sub_index(None, 4096, 4, order, 1, 4096, 4096, None) == -1
+    assert P.lib.camera_compact_workspace_bytes(0) == 0 and P.lib.camera_compact_workspace_bytes(65) >= 65 * 64
+    ptrs = (C.c_void_p * 4)(*[4096] * 4)
+    assert P.lib.camera_compact_weights(C.byref(ok), 4096, 4096, 1, 2, ptrs, ptrs, ptrs, None, 4096, 1 << 20, None) == -1   # n_take > n_labels
+    assert P.lib.camera_compact_weights(C.byref(ok), 4096, 4096, 1, 1, ptrs, ptrs, ptrs, None, None, 0, None) == -3
+    assert P.lib.camera_forward_workspace_bytes(C.byref(ok), 1000) > P.lib.camera_score_workspace_bytes(C.byref(ok), 1000)
+    # the forward path takes sliced layers: any d_ff >= 0, as long as W_down rows start on 16-byte boundaries
+    odd = _layer_struct(P, d_ff=(64, 3, 0, 64))
+    assert P.lib.camera_score_workspace_bytes(C.byref(odd), 10) == 0
+    assert P.lib.camera_forward_workspace_bytes(C.byref(odd), 10) > 0
+    assert P.lib.camera_layer_forward(C.byref(ok), 4096, 10, None, None, 4096, 1 << 30, None) == -1        # no output
+    f32 = _layer_struct(P, dtype=0)
+    assert P.lib.camera_layer_forward(C.byref(f32), 4096, 10, 4096, None, 4096, 1 << 30, None) == -2       # bf16 only
+    assert P.lib.camera_output_error(4096, 4096, 10, 0, 4096, 4096, 1 << 20, None) == -1
+    assert P.lib.camera_output_error(4096, 4096, 10, 64, 4096, None, 0, None) == -3
+    assert P.lib.camera_residual_norm(4096, 1, 4096, 10, 60, C.c_float(1e-6), 4096, None) == -1             # d_model % 8
+    assert P.lib.camera_residual_norm(4096, 5, 4096, 10, 64, C.c_float(1e-6), 4096, None) == -1             # dtype
+    assert P.lib.camera_residual_norm(None, 1, None, 0, 64, C.c_float(1e-6), None, None) == 0              # nothing to do
