@@ -167,3 +167,18 @@ def test_qwen15_moe_shape_layer_output_on_sampled_tokens(P):
     ref = oracle_forward(ol, f64(X[torch.from_numpy(tok).to(DEV)]),
                          (gi.cpu().numpy().astype(np.int64)[tok], gw.cpu().numpy().astype(np.float64)[tok]))
     assert_output_close("qwen15 layer output", y.cpu().numpy()[tok], ref)
+
+
+def test_qwen2_57b_shape_layer_output_on_sampled_tokens(P):
+    """The same at the Qwen2-57B-A14B shape, on one 65536-token batch (the size the benchmark's forward leg uses)."""
+    from test_gpu_forward import assert_output_close, oracle_forward
+    from _util import to_oracle_layer
+    cfg = W().scaled(W().CONFIGS["qwen2_57b_a14b"], n_tokens=65536)
+    L = W().make_layer(cfg, seed=0, device=DEV)
+    X = W().make_tokens(cfg, seed=0, device=DEV)
+    y, (gi, gw) = P.camera_layer_forward(P.Layer.from_workload(L), X, want_routing=True)
+    tok = np.sort(np.random.default_rng(4).choice(cfg.n_tokens, size=24, replace=False))
+    tok[0], tok[-1] = 0, cfg.n_tokens - 1
+    ref = oracle_forward(to_oracle_layer(L), f64(X[torch.from_numpy(tok).to(DEV)]),
+                         (gi.cpu().numpy().astype(np.int64)[tok], gw.cpu().numpy().astype(np.float64)[tok]))
+    assert_output_close("qwen2 layer output", y.cpu().numpy()[tok], ref)
