@@ -239,7 +239,8 @@ size_t camera_forward_workspace_bytes(const camera_layer_t* layer, int64_t n_tok
 /*
  * The layer's output, Eq. 1-2:  y_t = sum_e A_{t,e} W_down_e [ SiLU(W_gate_e x_t) * (W_up_e x_t) ],  with the
  * router coefficients A of camera_score_layer (aux: topk_idx_in / topk_w_in prescribe them, topk_idx / topk_w /
- * shared_w / expert_token_counts export them; other fields are ignored).  Applied to a layer sliced by
+ * shared_w / expert_token_counts export them; flags CAMERA_SCORE_CTA_PAIR / CAMERA_SCORE_SINGLE_CTA force the
+ * gate/up kernel; other fields and flags are ignored).  Applied to a layer sliced by
  * camera_compact_weights it gives Y_hat = Phi[:,S] W[S,:], the retained micro-experts' output of Eq. 7.
  * x: DEVICE [n_tokens, d_model] bf16;  y: DEVICE [n_tokens, d_model] fp32, 16-byte aligned.
  * bf16 layers in CAMERA_DOWN_HF layout with d_model % 64 == 0 only (else CAMERA_ERR_UNSUPPORTED_SHAPE); d_ff[e] may

@@ -254,7 +254,7 @@ int score_front(const camera_layer_t* L, const void* x, int64_t T, float alpha, 
   const bool use_umma = umma_shape_ok(L) && !(aux && (aux->flags & CAMERA_SCORE_FORCE_SIMT)) &&
                         (reinterpret_cast<uintptr_t>(x) & 15) == 0;
   bool use_pair = false;
-  if (use_umma && fwd == nullptr) {
+  if (use_umma) {
     if (aux && (aux->flags & CAMERA_SCORE_CTA_PAIR)) use_pair = true;
     else if (aux && (aux->flags & CAMERA_SCORE_SINGLE_CTA)) use_pair = false;
     else {

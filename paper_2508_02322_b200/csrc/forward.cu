@@ -415,7 +415,7 @@ extern "C" int camera_layer_forward(const camera_layer_t* L, const void* x, int6
   const ForwardBuffers fb{h.data(), fl.h_ld.data(), yp.data()};
   camera_score_aux_t a2;
   memset(&a2, 0, sizeof(a2));
-  if (aux) { a2 = *aux; a2.flags &= ~(uint32_t)(CAMERA_SCORE_FORCE_SIMT | CAMERA_SCORE_CTA_PAIR | CAMERA_SCORE_ACCUMULATE); }
+  if (aux) { a2 = *aux; a2.flags &= ~(uint32_t)(CAMERA_SCORE_FORCE_SIMT | CAMERA_SCORE_ACCUMULATE); }
   ScoreFront f;
   int rc = score_front(L, x, T, 0.f, nullptr, &a2, ws + fl.score, fl.score_bytes, st, &fb, &f);
   if (rc != CAMERA_OK) return rc;
@@ -438,7 +438,10 @@ extern "C" int camera_layer_forward(const camera_layer_t* L, const void* x, int6
     cudaGetLastError();
     return CAMERA_ERR_CUDA;
   }
-  if (launch_score_umma_write_h(c, st) != cudaSuccess) { cudaGetLastError(); return CAMERA_ERR_CUDA; }
+  if ((f.use_pair ? launch_score_umma_pair_write_h(c, st) : launch_score_umma_write_h(c, st)) != cudaSuccess) {
+    cudaGetLastError();
+    return CAMERA_ERR_CUDA;
+  }
   int dev = 0, sms = 148;
   cudaGetDevice(&dev);
   cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);

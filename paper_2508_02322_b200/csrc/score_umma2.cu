@@ -109,7 +109,10 @@ __device__ __forceinline__ void umma_commit_pair(uint32_t bar) {
                : "memory");
 }
 
-__device__ __forceinline__ void fold16_pair(const uint32_t* vg, const uint32_t* vu, const float* wb, float& s, float& m) {
+// WRITE_H (layer forward): lambda is also stored, as bf16, to h[token][micro-expert] for the first n_store tokens.
+template <bool WRITE_H>
+__device__ __forceinline__ void fold16_pair(const uint32_t* vg, const uint32_t* vu, const float* wb, float& s, float& m,
+                                            __nv_bfloat16* hcol, int h_ld, int n_store) {
   float a[16];
 #pragma unroll
   for (int q = 0; q < 4; ++q) {
@@ -123,9 +126,11 @@ __device__ __forceinline__ void fold16_pair(const uint32_t* vg, const uint32_t* 
     const float lam = (a[j] * up) * (g * sig);
     s = fmaf(lam, lam, s);
     m = fmaxf(m, fabsf(lam));
+    if (WRITE_H && j < n_store) hcol[(size_t)j * h_ld] = __float2bfloat16_rn(lam);
   }
 }
 
+template <bool WRITE_H>
 __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(P_THREADS, 1) k_score_umma_pair(const ScoreCtx c) {
   extern __shared__ uint8_t smem_raw[];
   const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
@@ -294,9 +299,21 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(P_THREADS, 1) k_scor
       const int n_tiles = (u.rows + UMMA_TOK - 1) / UMMA_TOK;
       const float* wsrc = u.shared_idx < 0 ? c.perm_w + u.row0 : c.shared_w + (size_t)u.shared_idx * c.n_tokens + u.row0;
       float s = 0.f, m = 0.f;
+      __nv_bfloat16* hbase = nullptr;
+      int h_ld = 0, row_limit = 0;
+      if (WRITE_H) {
+        const ExpertStatic es = c.est[u.e];
+        h_ld = es.h_ld;
+        hbase = static_cast<__nv_bfloat16*>(es.h) + (size_t)u.row0 * h_ld + u.ch0 + 128 * (int)rank + warp * 32 + lane;
+        row_limit = (u.shared_idx < 0 ? c.max_rows_perm : c.n_tokens) - u.row0;
+        // h is padded to 128 columns, a pair covers 256: the second CTA of an expert's last pair may have no column
+        if (u.ch0 + 128 * (int)rank + warp * 32 + lane >= h_ld) row_limit = 0;
+      }
       for (int tt = 0; ok && tt < n_tiles; ++tt) {
         const int valid = min(UMMA_TOK, u.rows - tt * UMMA_TOK);
         const int nv = (valid + 15) & ~15;
+        __nv_bfloat16* const htile = hbase + (size_t)tt * UMMA_TOK * h_ld;
+        const int rows_left = row_limit - tt * UMMA_TOK;
         __syncwarp();
         for (int i = lane; i < UMMA_TOK; i += 32) wb[i] = i < valid ? wsrc[tt * UMMA_TOK + i] : 0.f;
         __syncwarp();
@@ -309,11 +326,11 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(P_THREADS, 1) k_scor
         for (int c0 = 0; c0 < nv; c0 += 32) {
           tmem_ld_wait(g0, u0);
           if (c0 + 16 < nv) { tmem_ld16(t_gate + c0 + 16, g1); tmem_ld16(t_up + c0 + 16, u1); }
-          fold16_pair(g0, u0, wb + c0, s, m);
+          fold16_pair<WRITE_H>(g0, u0, wb + c0, s, m, htile + (size_t)c0 * h_ld, h_ld, rows_left - c0);
           if (c0 + 16 < nv) {
             tmem_ld_wait(g1, u1);
             if (c0 + 32 < nv) { tmem_ld16(t_gate + c0 + 32, g0); tmem_ld16(t_up + c0 + 32, u0); }
-            fold16_pair(g1, u1, wb + c0 + 16, s, m);
+            fold16_pair<WRITE_H>(g1, u1, wb + c0 + 16, s, m, htile + (size_t)(c0 + 16) * h_ld, h_ld, rows_left - c0 - 16);
           }
         }
         tc_fence_before();
@@ -321,7 +338,7 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(P_THREADS, 1) k_scor
         tile_phase ^= 1u;
       }
       const int ch = u.ch0 + 128 * (int)rank + warp * 32 + lane;
-      if (ok && ch < u.f) {
+      if (!WRITE_H && ok && ch < u.f) {
         const size_t slot = (size_t)u.part_slot + 128 * rank + warp * 32 + lane;
         c.part_sum[slot] = s;
         c.part_max[slot] = m;
@@ -345,9 +362,20 @@ cudaError_t launch_score_umma_pair(const ScoreCtx& c, cudaStream_t st) {
   int dev = 0, sms = 148;
   cudaGetDevice(&dev);
   cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
-  cudaError_t e = cudaFuncSetAttribute(k_score_umma_pair, cudaFuncAttributeMaxDynamicSharedMemorySize, P_SMEM_BYTES);
+  cudaError_t e = cudaFuncSetAttribute(k_score_umma_pair<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, P_SMEM_BYTES);
   if (e != cudaSuccess) return e;
-  k_score_umma_pair<<<sms & ~1, P_THREADS, P_SMEM_BYTES, st>>>(c);
+  k_score_umma_pair<false><<<sms & ~1, P_THREADS, P_SMEM_BYTES, st>>>(c);
+  return cudaGetLastError();
+}
+
+// The same kernel with the epilogue that stores h (layer forward).
+cudaError_t launch_score_umma_pair_write_h(const ScoreCtx& c, cudaStream_t st) {
+  int dev = 0, sms = 148;
+  cudaGetDevice(&dev);
+  cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+  cudaError_t e = cudaFuncSetAttribute(k_score_umma_pair<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, P_SMEM_BYTES);
+  if (e != cudaSuccess) return e;
+  k_score_umma_pair<true><<<sms & ~1, P_THREADS, P_SMEM_BYTES, st>>>(c);
   return cudaGetLastError();
 }
 

@@ -67,25 +67,28 @@ def oracle_forward(ol, Xd, routing):
     return Y
 
 
+@pytest.mark.parametrize("cta_pair", [False, True])
 @pytest.mark.parametrize("T", [1, 255, 700, 5000])
-def test_layer_output(P, T):
+def test_layer_output(P, T, cta_pair):
     cfg = cfg_of(n_tokens=T)
     L = W().make_layer(cfg, seed=30, device=DEV)
     X = W().make_tokens(cfg, seed=30, device=DEV)
     ol, Xd = to_oracle_layer(L), f64(X)
     rin, rout = oracle_routing(ol, Xd)
-    y = P.camera_layer_forward(P.Layer.from_workload(L), X, routing_in=rin)
+    y = P.camera_layer_forward(P.Layer.from_workload(L), X, routing_in=rin, cta_pair=cta_pair)
     ref = oracle_forward(ol, Xd, rout)
     assert np.allclose(ref, O.forward(ol, Xd), rtol=1e-5, atol=1e-6)       # the helper above is Eq. 1-2 (coefficients rounded to fp32)
     assert_output_close("layer output", y.cpu().numpy(), ref)
 
 
-def test_layer_output_own_routing_and_no_shared(P):
+@pytest.mark.parametrize("cta_pair", [False, True])
+def test_layer_output_own_routing_and_no_shared(P, cta_pair):
+    # d_ff 320 = 2.5 tiles of 128: a pair's second CTA has a half tile, then none, of h's 384 padded columns
     cfg = cfg_of(n_tokens=900, d_ff_shared=(), shared_gate_sigmoid=False, n_routed=5, top_k=3, d_ff_routed=320)
     L = W().make_layer(cfg, seed=31, device=DEV)
     X = W().make_tokens(cfg, seed=31, device=DEV)
     ol, Xd = to_oracle_layer(L), f64(X)
-    y, (gi, gw) = P.camera_layer_forward(P.Layer.from_workload(L), X, want_routing=True)
+    y, (gi, gw) = P.camera_layer_forward(P.Layer.from_workload(L), X, want_routing=True, cta_pair=cta_pair)
     ref = oracle_forward(ol, Xd, (gi.cpu().numpy().astype(np.int64), gw.cpu().numpy().astype(np.float64)))
     assert_output_close("layer output under the GPU's routing", y.cpu().numpy(), ref)
 
