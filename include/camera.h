@@ -63,6 +63,11 @@ enum {
                                       work unit: less L2 and shared-memory traffic per flop).  By default the library takes
                                       pairs unless padding d_ff to multiples of 256 would add more than 6 % of work */
   CAMERA_SCORE_SINGLE_CTA = 8u,    /* force one CTA per MMA (128 micro-experts per work unit) */
+  CAMERA_FORWARD_TOKEN_ROWS = 16u, /* camera_layer_forward only: force the gate/up kernel that keeps the tokens on the
+                                      accumulator rows (CTA pairs, 256-token tiles; an epilogue thread writes runs of
+                                      consecutive micro-experts of its token).  By default the library takes it when
+                                      the experts' token lists are long enough for whole 256-token tiles to cost no
+                                      more than they save; CTA_PAIR / SINGLE_CTA force the scoring orientation */
   CAMERA_SCORE_ACCUMULATE = 4u     /* phi2 and phi_inf_sq (both required) already hold the result of earlier batches of
                                       calibration tokens of this layer; this call folds its batch in (the column sums of
                                       Alg. 1 line 7 add up over batches, the column maxima of line 8 take the maximum)
@@ -239,8 +244,8 @@ size_t camera_forward_workspace_bytes(const camera_layer_t* layer, int64_t n_tok
 /*
  * The layer's output, Eq. 1-2:  y_t = sum_e A_{t,e} W_down_e [ SiLU(W_gate_e x_t) * (W_up_e x_t) ],  with the
  * router coefficients A of camera_score_layer (aux: topk_idx_in / topk_w_in prescribe them, topk_idx / topk_w /
- * shared_w / expert_token_counts export them; flags CAMERA_SCORE_CTA_PAIR / CAMERA_SCORE_SINGLE_CTA force the
- * gate/up kernel; other fields and flags are ignored).  Applied to a layer sliced by
+ * shared_w / expert_token_counts export them; flags CAMERA_SCORE_CTA_PAIR / CAMERA_SCORE_SINGLE_CTA /
+ * CAMERA_FORWARD_TOKEN_ROWS force the gate/up kernel; other fields and flags are ignored).  Applied to a layer sliced by
  * camera_compact_weights it gives Y_hat = Phi[:,S] W[S,:], the retained micro-experts' output of Eq. 7.
  * x: DEVICE [n_tokens, d_model] bf16;  y: DEVICE [n_tokens, d_model] fp32, 16-byte aligned.
  * bf16 layers in CAMERA_DOWN_HF layout with d_model % 64 == 0 only (else CAMERA_ERR_UNSUPPORTED_SHAPE); d_ff[e] may

@@ -22,6 +22,7 @@ CAMERA_SCORE_FORCE_SIMT = 1
 CAMERA_SCORE_CTA_PAIR = 2
 CAMERA_SCORE_ACCUMULATE = 4
 CAMERA_SCORE_SINGLE_CTA = 8
+CAMERA_FORWARD_TOKEN_ROWS = 16
 STAGES = ("router", "permute", "rownorm", "score", "combine")
 
 
@@ -407,10 +408,12 @@ def camera_forward_workspace_bytes(layer: Layer, n_tokens: int) -> int:
 
 def camera_layer_forward(layer: Layer, x: torch.Tensor, *, y: Optional[torch.Tensor] = None, routing_in=None,
                          workspace: Optional[torch.Tensor] = None, want_routing: bool = False,
-                         cta_pair: Optional[bool] = None, stream: Optional[torch.cuda.Stream] = None):
+                         cta_pair: Optional[bool] = None, token_rows: bool = False,
+                         stream: Optional[torch.cuda.Stream] = None):
     """The layer's output y [T, d_model] fp32 (Eq. 1-2).  routing_in = (topk_idx, topk_w) prescribes the routed
     coefficients; want_routing also returns the (topk_idx, topk_w) the call used; cta_pair forces the CTA-pair
-    (True) or single-CTA (False) gate/up kernel instead of the library's choice."""
+    (True) or single-CTA (False) gate/up kernel of the scoring orientation, token_rows the kernel with the tokens on
+    the accumulator rows, instead of the library's choice."""
     T = int(x.shape[0])
     dev = x.device
     if y is None:
@@ -418,7 +421,8 @@ def camera_layer_forward(layer: Layer, x: torch.Tensor, *, y: Optional[torch.Ten
     if workspace is None:
         workspace = alloc_workspace(camera_forward_workspace_bytes(layer, T), dev)
     aux = camera_score_aux_t()
-    aux.flags = (CAMERA_SCORE_CTA_PAIR if cta_pair else 0) | (CAMERA_SCORE_SINGLE_CTA if cta_pair is False else 0)
+    aux.flags = ((CAMERA_SCORE_CTA_PAIR if cta_pair else 0) | (CAMERA_SCORE_SINGLE_CTA if cta_pair is False else 0) |
+                 (CAMERA_FORWARD_TOKEN_ROWS if token_rows else 0))
     keep_alive = []
     if routing_in is not None:
         idx = routing_in[0].to(device=dev, dtype=torch.int32).contiguous()

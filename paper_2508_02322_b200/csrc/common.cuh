@@ -125,7 +125,7 @@ cudaError_t launch_score_umma_pair(const ScoreCtx& c, cudaStream_t st);
 cudaError_t launch_combine(const ScoreCtx& c, cudaStream_t st);
 cudaError_t launch_router_umma(const ScoreCtx& c, const int32_t* idx_in, const float* w_in, cudaStream_t st);
 cudaError_t launch_score_umma_write_h(const ScoreCtx& c, cudaStream_t st);
-cudaError_t launch_score_umma_pair_write_h(const ScoreCtx& c, cudaStream_t st);
+cudaError_t launch_score_umma_pair_write_h(const ScoreCtx& c, bool token_rows, cudaStream_t st);
 bool umma_shape_ok(const camera_layer_t* L);
 bool router_umma_ok(const ScoreCtx& c);
 int encode_tensor_maps(const camera_layer_t* L, const ScoreCtx& c, void* host_maps /* 128 B each */);

@@ -5,6 +5,7 @@
 //   k_score_umma<WRITE_H>   h = A * SiLU(W_gate x) * (W_up x) per (token row, micro-expert), bf16      (score_umma.cu)
 //   k_down_umma             y_part[row, :] = W_down h[row, :] per expert, tcgen05, fp32 out
 //   k_unpermute_sum         y[t, :] = sum over the token's k routed rows and its shared-expert rows, fixed order
+#include <math.h>
 #include <string.h>
 
 #include <vector>
@@ -376,6 +377,28 @@ FwdLayout fwd_layout(const camera_layer_t* L, int64_t T) {
   return f;
 }
 
+// Which gate/up kernel the layer forward runs.  With the tokens on the accumulator rows the epilogue is short (a
+// thread packs 16 micro-experts of its token into two 16-byte stores) but every token tile costs 256 rows, where the
+// scoring orientation trims a list's last tile to a multiple of 16 tokens; its stores of single bf16 values cost
+// about a tenth of the kernel.  Token lists are taken at their average length: the routing is not known here.
+bool forward_token_rows(const camera_layer_t* L, int64_t T, uint32_t flags) {
+  int dev = 0, sms = 0;
+  cudaGetDevice(&dev);
+  cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+  if (sms % 2 != 0) return false;
+  if (flags & CAMERA_FORWARD_TOKEN_ROWS) return true;
+  if (flags & (CAMERA_SCORE_CTA_PAIR | CAMERA_SCORE_SINGLE_CTA)) return false;
+  const int E = L->n_routed + L->n_shared;
+  double rows_tile = 0.0, cols_tile = 0.0;
+  for (int e = 0; e < E; ++e) {
+    const double rows = e < L->n_routed ? (double)T * L->top_k / L->n_routed : (double)T;
+    const double f = (double)L->d_ff[e];
+    rows_tile += ceil(rows / UMMA_TOK) * UMMA_TOK * ceil(f / UMMA_BK) * UMMA_BK;
+    cols_tile += ceil(rows / ROW_ALIGN) * ROW_ALIGN * ceil(f / CH_TILE) * CH_TILE;
+  }
+  return rows_tile <= 1.10 * cols_tile;
+}
+
 }  // namespace
 }  // namespace camera
 
@@ -416,6 +439,8 @@ extern "C" int camera_layer_forward(const camera_layer_t* L, const void* x, int6
   camera_score_aux_t a2;
   memset(&a2, 0, sizeof(a2));
   if (aux) { a2 = *aux; a2.flags &= ~(uint32_t)(CAMERA_SCORE_FORCE_SIMT | CAMERA_SCORE_ACCUMULATE); }
+  const bool token_rows = forward_token_rows(L, T, a2.flags);
+  if (token_rows) a2.flags = (a2.flags & ~(uint32_t)CAMERA_SCORE_SINGLE_CTA) | CAMERA_SCORE_CTA_PAIR;
   ScoreFront f;
   int rc = score_front(L, x, T, 0.f, nullptr, &a2, ws + fl.score, fl.score_bytes, st, &fb, &f);
   if (rc != CAMERA_OK) return rc;
@@ -438,7 +463,7 @@ extern "C" int camera_layer_forward(const camera_layer_t* L, const void* x, int6
     cudaGetLastError();
     return CAMERA_ERR_CUDA;
   }
-  if ((f.use_pair ? launch_score_umma_pair_write_h(c, st) : launch_score_umma_write_h(c, st)) != cudaSuccess) {
+  if ((f.use_pair ? launch_score_umma_pair_write_h(c, token_rows, st) : launch_score_umma_write_h(c, st)) != cudaSuccess) {
     cudaGetLastError();
     return CAMERA_ERR_CUDA;
   }

@@ -130,8 +130,33 @@ __device__ __forceinline__ void fold16_pair(const uint32_t* vg, const uint32_t* 
   }
 }
 
-template <bool WRITE_H>
+// The layer-forward epilogue with a token on every accumulator row: h = a * SiLU(g) * u for 16 consecutive
+// micro-experts of the thread's token, rounded to bf16 and packed into 32 contiguous bytes.
+__device__ __forceinline__ void silu_mul16(const uint32_t* vg, const uint32_t* vu, float a, uint4& lo, uint4& hi) {
+  uint32_t p[8];
+#pragma unroll
+  for (int j = 0; j < 16; j += 2) {
+    const float g0 = __uint_as_float(vg[j]), g1 = __uint_as_float(vg[j + 1]);
+    const float l0 = (a * __uint_as_float(vu[j])) * (g0 * __fdividef(1.f, 1.f + __expf(-g0)));
+    const float l1 = (a * __uint_as_float(vu[j + 1])) * (g1 * __fdividef(1.f, 1.f + __expf(-g1)));
+    const __nv_bfloat162 b = __floats2bfloat162_rn(l0, l1);
+    p[j >> 1] = *reinterpret_cast<const uint32_t*>(&b);
+  }
+  lo = make_uint4(p[0], p[1], p[2], p[3]);
+  hi = make_uint4(p[4], p[5], p[6], p[7]);
+}
+
+// MODE 0: scoring (partial sums and maxima per micro-expert).  MODE 1: layer forward, h stored from the scoring
+// orientation (micro-experts on the accumulator rows, tokens on the columns).  MODE 2: layer forward with the operands
+// exchanged: the token tile is the M operand (128 tokens per CTA), the gate and up weights are the N operands (each CTA
+// supplies half of the tile's micro-experts), so a thread of the epilogue owns a token and writes runs of consecutive
+// micro-experts.  The shared-memory tiles, the loads and the barriers are the same in all three.
+enum { PAIR_SCORE = 0, PAIR_H_COLS = 1, PAIR_H_ROWS = 2 };
+constexpr int H_TILE_CH = 2 * CH_TILE;          // micro-experts per work unit
+
+template <int MODE>
 __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(P_THREADS, 1) k_score_umma_pair(const ScoreCtx c) {
+  constexpr bool WRITE_H = MODE == PAIR_H_COLS;
   extern __shared__ uint8_t smem_raw[];
   const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
   uint8_t* const base_ptr = smem_raw + (base - smem_u32(smem_raw));
@@ -212,10 +237,14 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(P_THREADS, 1) k_scor
         tensormap_acquire(map_g);
         tensormap_acquire(map_u);
         tensormap_acquire(map_x);
-        const int ch = u.ch0 + 128 * (int)rank;     // past d_ff for the second CTA of an odd last tile: reads zeros
+        // MODE 2: the tile's micro-experts, in whole k-blocks of the second GEMM (h is read 64 columns at a time)
+        const int ncv = min(H_TILE_CH, (u.f - u.ch0 + UMMA_BK - 1) & ~(UMMA_BK - 1));
+        // past d_ff for the second CTA of an odd last tile: reads zeros
+        const int ch = u.ch0 + (MODE == PAIR_H_ROWS ? (int)rank * (ncv >> 1) : 128 * (int)rank);
         for (int tt = 0; ok && tt < n_tiles; ++tt) {
           const int nv = (min(UMMA_TOK, u.rows - tt * UMMA_TOK) + 15) & ~15;
-          const int row = u.row0 + tt * UMMA_TOK + (int)rank * (nv >> 1);   // this CTA holds tokens [rank * nv/2, +nv/2)
+          // this CTA holds tokens [rank * nv/2, +nv/2) of the N operand, or rows [128 rank, +128) of the M operand
+          const int row = u.row0 + tt * UMMA_TOK + (int)rank * (MODE == PAIR_H_ROWS ? 128 : (nv >> 1));
           for (int kb = 0; kb < n_kb; ++kb) {
             if (!mbar_wait(empty_bar(stage), phase ^ 1u, abort_flag)) { ok = false; break; }
             const uint32_t a_dst = base + stage * P_STAGE_BYTES;
@@ -251,7 +280,8 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(P_THREADS, 1) k_scor
         const int n_tiles = (u.rows + UMMA_TOK - 1) / UMMA_TOK;
         for (int tt = 0; ok && tt < n_tiles; ++tt) {
           const int nv = (min(UMMA_TOK, u.rows - tt * UMMA_TOK) + 15) & ~15;
-          const uint32_t idesc = make_idesc_pair(nv);
+          const int ncv = min(H_TILE_CH, (u.f - u.ch0 + UMMA_BK - 1) & ~(UMMA_BK - 1));
+          const uint32_t idesc = make_idesc_pair(MODE == PAIR_H_ROWS ? ncv : nv);
           if (!mbar_wait(tempty_bar, tile_phase ^ 1u, abort_flag)) { ok = false; break; }
           tc_fence_after();
           for (int kb = 0; kb < n_kb; ++kb) {
@@ -264,8 +294,13 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(P_THREADS, 1) k_scor
 #pragma unroll
             for (int k = 0; k < UMMA_BK / 16; ++k) {
               const uint32_t acc = (uint32_t)((kb | k) != 0);
-              umma_bf16_pair(tmem_base, g_desc + 2 * k, b_desc + 2 * k, idesc, acc);
-              umma_bf16_pair(tmem_base + UMMA_TOK, u_desc + 2 * k, b_desc + 2 * k, idesc, acc);
+              if (MODE == PAIR_H_ROWS) {   // [tokens] x [micro-experts]: gate in columns 0-255, up in 256-511
+                umma_bf16_pair(tmem_base, b_desc + 2 * k, g_desc + 2 * k, idesc, acc);
+                umma_bf16_pair(tmem_base + H_TILE_CH, b_desc + 2 * k, u_desc + 2 * k, idesc, acc);
+              } else {                     // [micro-experts] x [tokens]
+                umma_bf16_pair(tmem_base, g_desc + 2 * k, b_desc + 2 * k, idesc, acc);
+                umma_bf16_pair(tmem_base + UMMA_TOK, u_desc + 2 * k, b_desc + 2 * k, idesc, acc);
+              }
             }
             umma_commit_pair(empty_bar(stage));
             if (++stage == P_STAGES) { stage = 0; phase ^= 1u; }
@@ -309,39 +344,82 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(P_THREADS, 1) k_scor
         // h is padded to 128 columns, a pair covers 256: the second CTA of an expert's last pair may have no column
         if (u.ch0 + 128 * (int)rank + warp * 32 + lane >= h_ld) row_limit = 0;
       }
-      for (int tt = 0; ok && tt < n_tiles; ++tt) {
-        const int valid = min(UMMA_TOK, u.rows - tt * UMMA_TOK);
-        const int nv = (valid + 15) & ~15;
-        __nv_bfloat16* const htile = hbase + (size_t)tt * UMMA_TOK * h_ld;
-        const int rows_left = row_limit - tt * UMMA_TOK;
-        __syncwarp();
-        for (int i = lane; i < UMMA_TOK; i += 32) wb[i] = i < valid ? wsrc[tt * UMMA_TOK + i] : 0.f;
-        __syncwarp();
-        ok = __all_sync(0xffffffffu, mbar_wait(tfull_bar, tile_phase, abort_flag));
-        if (!ok) break;
-        tc_fence_after();
-        uint32_t g0[16], u0[16], g1[16], u1[16];
-        tmem_ld16(t_gate, g0);
-        tmem_ld16(t_up, u0);
-        for (int c0 = 0; c0 < nv; c0 += 32) {
-          tmem_ld_wait(g0, u0);
-          if (c0 + 16 < nv) { tmem_ld16(t_gate + c0 + 16, g1); tmem_ld16(t_up + c0 + 16, u1); }
-          fold16_pair<WRITE_H>(g0, u0, wb + c0, s, m, htile + (size_t)c0 * h_ld, h_ld, rows_left - c0);
-          if (c0 + 16 < nv) {
-            tmem_ld_wait(g1, u1);
-            if (c0 + 32 < nv) { tmem_ld16(t_gate + c0 + 32, g0); tmem_ld16(t_up + c0 + 32, u0); }
-            fold16_pair<WRITE_H>(g1, u1, wb + c0 + 16, s, m, htile + (size_t)(c0 + 16) * h_ld, h_ld, rows_left - c0 - 16);
+      if constexpr (MODE == PAIR_H_ROWS) {
+        const ExpertStatic es = c.est[u.e];
+        const int ncv = min(H_TILE_CH, (u.f - u.ch0 + UMMA_BK - 1) & ~(UMMA_BK - 1));
+        const int r = 128 * (int)rank + warp * 32 + lane;            // this thread's token row of the tile
+        const int buf_rows = (u.shared_idx < 0 ? c.max_rows_perm : c.n_tokens) - u.row0;
+        for (int tt = 0; ok && tt < n_tiles; ++tt) {
+          const int valid = min(UMMA_TOK, u.rows - tt * UMMA_TOK);
+          const int rt = tt * UMMA_TOK + r;
+          // rows up to the next multiple of 16 are written (zeros: the second GEMM reads them), none past the buffer
+          const bool store = r < ((valid + 15) & ~15) && rt < buf_rows;
+          const float a = r < valid ? wsrc[rt] : 0.f;
+          __nv_bfloat16* const hrow = static_cast<__nv_bfloat16*>(es.h) + (size_t)(u.row0 + rt) * es.h_ld + u.ch0;
+          ok = __all_sync(0xffffffffu, mbar_wait(tfull_bar, tile_phase, abort_flag));
+          if (!ok) break;
+          tc_fence_after();
+          uint32_t g0[16], u0[16], g1[16], u1[16];
+          uint4 lo, hi;
+          tmem_ld16(t_gate, g0);
+          tmem_ld16(t_gate + H_TILE_CH, u0);
+          for (int c0 = 0; c0 < ncv; c0 += 32) {
+            tmem_ld_wait(g0, u0);
+            if (c0 + 16 < ncv) { tmem_ld16(t_gate + c0 + 16, g1); tmem_ld16(t_gate + H_TILE_CH + c0 + 16, u1); }
+            silu_mul16(g0, u0, a, lo, hi);
+            if (store) {
+              *reinterpret_cast<uint4*>(hrow + c0) = lo;
+              *reinterpret_cast<uint4*>(hrow + c0 + 8) = hi;
+            }
+            if (c0 + 16 < ncv) {
+              tmem_ld_wait(g1, u1);
+              if (c0 + 32 < ncv) { tmem_ld16(t_gate + c0 + 32, g0); tmem_ld16(t_gate + H_TILE_CH + c0 + 32, u0); }
+              silu_mul16(g1, u1, a, lo, hi);
+              if (store) {
+                *reinterpret_cast<uint4*>(hrow + c0 + 16) = lo;
+                *reinterpret_cast<uint4*>(hrow + c0 + 24) = hi;
+              }
+            }
           }
+          tc_fence_before();
+          mbar_arrive_cluster(tempty0);
+          tile_phase ^= 1u;
         }
-        tc_fence_before();
-        mbar_arrive_cluster(tempty0);
-        tile_phase ^= 1u;
-      }
-      const int ch = u.ch0 + 128 * (int)rank + warp * 32 + lane;
-      if (!WRITE_H && ok && ch < u.f) {
-        const size_t slot = (size_t)u.part_slot + 128 * rank + warp * 32 + lane;
-        c.part_sum[slot] = s;
-        c.part_max[slot] = m;
+      } else {
+        for (int tt = 0; ok && tt < n_tiles; ++tt) {
+          const int valid = min(UMMA_TOK, u.rows - tt * UMMA_TOK);
+          const int nv = (valid + 15) & ~15;
+          __nv_bfloat16* const htile = hbase + (size_t)tt * UMMA_TOK * h_ld;
+          const int rows_left = row_limit - tt * UMMA_TOK;
+          __syncwarp();
+          for (int i = lane; i < UMMA_TOK; i += 32) wb[i] = i < valid ? wsrc[tt * UMMA_TOK + i] : 0.f;
+          __syncwarp();
+          ok = __all_sync(0xffffffffu, mbar_wait(tfull_bar, tile_phase, abort_flag));
+          if (!ok) break;
+          tc_fence_after();
+          uint32_t g0[16], u0[16], g1[16], u1[16];
+          tmem_ld16(t_gate, g0);
+          tmem_ld16(t_up, u0);
+          for (int c0 = 0; c0 < nv; c0 += 32) {
+            tmem_ld_wait(g0, u0);
+            if (c0 + 16 < nv) { tmem_ld16(t_gate + c0 + 16, g1); tmem_ld16(t_up + c0 + 16, u1); }
+            fold16_pair<WRITE_H>(g0, u0, wb + c0, s, m, htile + (size_t)c0 * h_ld, h_ld, rows_left - c0);
+            if (c0 + 16 < nv) {
+              tmem_ld_wait(g1, u1);
+              if (c0 + 32 < nv) { tmem_ld16(t_gate + c0 + 32, g0); tmem_ld16(t_up + c0 + 32, u0); }
+              fold16_pair<WRITE_H>(g1, u1, wb + c0 + 16, s, m, htile + (size_t)(c0 + 16) * h_ld, h_ld, rows_left - c0 - 16);
+            }
+          }
+          tc_fence_before();
+          mbar_arrive_cluster(tempty0);
+          tile_phase ^= 1u;
+        }
+        const int ch = u.ch0 + 128 * (int)rank + warp * 32 + lane;
+        if (MODE == PAIR_SCORE && ok && ch < u.f) {
+          const size_t slot = (size_t)u.part_slot + 128 * rank + warp * 32 + lane;
+          c.part_sum[slot] = s;
+          c.part_max[slot] = m;
+        }
       }
     }
   }
@@ -362,20 +440,22 @@ cudaError_t launch_score_umma_pair(const ScoreCtx& c, cudaStream_t st) {
   int dev = 0, sms = 148;
   cudaGetDevice(&dev);
   cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
-  cudaError_t e = cudaFuncSetAttribute(k_score_umma_pair<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, P_SMEM_BYTES);
+  cudaError_t e = cudaFuncSetAttribute(k_score_umma_pair<PAIR_SCORE>, cudaFuncAttributeMaxDynamicSharedMemorySize, P_SMEM_BYTES);
   if (e != cudaSuccess) return e;
-  k_score_umma_pair<false><<<sms & ~1, P_THREADS, P_SMEM_BYTES, st>>>(c);
+  k_score_umma_pair<PAIR_SCORE><<<sms & ~1, P_THREADS, P_SMEM_BYTES, st>>>(c);
   return cudaGetLastError();
 }
 
-// The same kernel with the epilogue that stores h (layer forward).
-cudaError_t launch_score_umma_pair_write_h(const ScoreCtx& c, cudaStream_t st) {
+// The same kernel with an epilogue that stores h (layer forward); token_rows picks the orientation with the token
+// tile as the M operand.
+cudaError_t launch_score_umma_pair_write_h(const ScoreCtx& c, bool token_rows, cudaStream_t st) {
   int dev = 0, sms = 148;
   cudaGetDevice(&dev);
   cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
-  cudaError_t e = cudaFuncSetAttribute(k_score_umma_pair<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, P_SMEM_BYTES);
+  auto kern = token_rows ? k_score_umma_pair<PAIR_H_ROWS> : k_score_umma_pair<PAIR_H_COLS>;
+  cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, P_SMEM_BYTES);
   if (e != cudaSuccess) return e;
-  k_score_umma_pair<true><<<sms & ~1, P_THREADS, P_SMEM_BYTES, st>>>(c);
+  kern<<<sms & ~1, P_THREADS, P_SMEM_BYTES, st>>>(c);
   return cudaGetLastError();
 }
 

@@ -67,30 +67,46 @@ def oracle_forward(ol, Xd, routing):
     return Y
 
 
-@pytest.mark.parametrize("cta_pair", [False, True])
+KERNELS = {"single": dict(cta_pair=False), "pair": dict(cta_pair=True), "token_rows": dict(token_rows=True)}
+
+
+@pytest.mark.parametrize("kernel", list(KERNELS))
 @pytest.mark.parametrize("T", [1, 255, 700, 5000])
-def test_layer_output(P, T, cta_pair):
+def test_layer_output(P, T, kernel):
     cfg = cfg_of(n_tokens=T)
     L = W().make_layer(cfg, seed=30, device=DEV)
     X = W().make_tokens(cfg, seed=30, device=DEV)
     ol, Xd = to_oracle_layer(L), f64(X)
     rin, rout = oracle_routing(ol, Xd)
-    y = P.camera_layer_forward(P.Layer.from_workload(L), X, routing_in=rin, cta_pair=cta_pair)
+    y = P.camera_layer_forward(P.Layer.from_workload(L), X, routing_in=rin, **KERNELS[kernel])
     ref = oracle_forward(ol, Xd, rout)
     assert np.allclose(ref, O.forward(ol, Xd), rtol=1e-5, atol=1e-6)       # the helper above is Eq. 1-2 (coefficients rounded to fp32)
     assert_output_close("layer output", y.cpu().numpy(), ref)
 
 
-@pytest.mark.parametrize("cta_pair", [False, True])
-def test_layer_output_own_routing_and_no_shared(P, cta_pair):
-    # d_ff 320 = 2.5 tiles of 128: a pair's second CTA has a half tile, then none, of h's 384 padded columns
+@pytest.mark.parametrize("kernel", list(KERNELS))
+def test_layer_output_own_routing_and_no_shared(P, kernel):
+    # d_ff 320 = 2.5 tiles of 128: a pair's second CTA has a half tile, then none, of h's 384 padded columns; with the
+    # tokens on the accumulator rows the second unit of an expert is 64 micro-experts wide
     cfg = cfg_of(n_tokens=900, d_ff_shared=(), shared_gate_sigmoid=False, n_routed=5, top_k=3, d_ff_routed=320)
     L = W().make_layer(cfg, seed=31, device=DEV)
     X = W().make_tokens(cfg, seed=31, device=DEV)
     ol, Xd = to_oracle_layer(L), f64(X)
-    y, (gi, gw) = P.camera_layer_forward(P.Layer.from_workload(L), X, want_routing=True, cta_pair=cta_pair)
+    y, (gi, gw) = P.camera_layer_forward(P.Layer.from_workload(L), X, want_routing=True, **KERNELS[kernel])
     ref = oracle_forward(ol, Xd, (gi.cpu().numpy().astype(np.int64), gw.cpu().numpy().astype(np.float64)))
     assert_output_close("layer output under the GPU's routing", y.cpu().numpy(), ref)
+
+
+@pytest.mark.parametrize("d_ff", [8, 72, 200, 264, 648])
+def test_token_rows_kernel_ragged_widths(P, d_ff):
+    """Widths that leave the last unit 64, 128 or 192 micro-experts wide, or the only unit narrower than a k-block."""
+    cfg = cfg_of(n_tokens=1500, n_routed=3, top_k=2, d_ff_routed=d_ff, d_ff_shared=(d_ff + 64,))
+    L = W().make_layer(cfg, seed=35, device=DEV)
+    X = W().make_tokens(cfg, seed=35, device=DEV)
+    ol, Xd = to_oracle_layer(L), f64(X)
+    rin, rout = oracle_routing(ol, Xd)
+    y = P.camera_layer_forward(P.Layer.from_workload(L), X, routing_in=rin, token_rows=True)
+    assert_output_close(f"token rows, d_ff {d_ff}", y.cpu().numpy(), oracle_forward(ol, Xd, rout))
 
 
 def test_dense_layer_is_a_gated_ffn(P):
@@ -124,7 +140,7 @@ def test_sliced_layer_output_and_error_metrics(P, ratio):
                      [out["w_up"][e][:m[e]] for e in range(layer.n_experts)], out["w_down"], cfg.top_k, cfg.n_shared,
                      L["router_bias"], L["w_shared_gate"], cfg.norm_topk, "hf", down_ld=layer.d_ff)
     y = P.camera_layer_forward(layer, X, routing_in=rin)
-    y_hat = P.camera_layer_forward(sliced, X, routing_in=rin)
+    y_hat = P.camera_layer_forward(sliced, X, routing_in=rin, token_rows=ratio > 0.5)
     lists, _ = O.sub_index_lists(keep.cpu().numpy(), O.me_offsets(ol), [1])
     ref_hat = oracle_forward(O.slice_layer(ol, lists), Xd, rout)
     assert_output_close("sliced layer output", y_hat.cpu().numpy(), ref_hat)

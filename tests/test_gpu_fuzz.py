@@ -64,7 +64,7 @@ def test_random_layers(P, seed):
     # the layer output, where the forward path takes the layout
     if L["down_layout"] == "hf":
         from test_gpu_forward import assert_output_close, oracle_forward
-        y, routing = P.camera_layer_forward(layer, X, want_routing=True, cta_pair=[None, False, True][seed % 3])
+        y, routing = P.camera_layer_forward(layer, X, want_routing=True, **[dict(), dict(cta_pair=False), dict(cta_pair=True), dict(token_rows=True)][(seed // 2) % 4])
         gi, gw = routing
         ref_y = oracle_forward(to_oracle_layer(L), f64(X), (gi.cpu().numpy().astype(np.int64), gw.cpu().numpy().astype(np.float64)))
         assert_output_close(f"fuzz {seed} layer output", y.cpu().numpy(), ref_y)
