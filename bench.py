@@ -188,7 +188,8 @@ def run_reference(args):
 
 def run_stack(args):
     """--stack: Algorithm 2's layer loop on a synthetic stack of MoE layers.  Per layer: output of the layer on the
-    calibration tokens (line 6), scores (line 8), selection and slicing (lines 9-13), output of the sliced layer
+    calibration tokens (line 6) and scores (line 8) from one pass over the gate/up weights
+    (camera_score_forward_layer), selection and slicing (lines 9-13), output of the sliced layer
     (line 14), which -- added to the residual and rescaled to RMS 1, the stand-in for the rest of a decoder layer --
     becomes the next layer's input (line 15).  Prints one JSON line of its own."""
     import torch
@@ -210,7 +211,6 @@ def run_stack(args):
     probe = P.Layer.from_workload(W.make_layer(W.scaled(cfg, n_tokens=B), seed=0, layer_id=0, device=dev))
     n_me = probe.n_me
     ws_f = P.alloc_workspace(P.camera_forward_workspace_bytes(probe, B), dev)
-    ws_s = P.alloc_workspace(P.camera_score_workspace_bytes(probe, B), dev)
     ws_sel = P.alloc_workspace(P.camera_select_workspace_bytes(n_me, 1, 2), dev)
     ws_c = P.alloc_workspace(4096 + 64 * probe.n_experts, dev)
     energy = torch.empty(n_me, dtype=torch.float32, device=dev)
@@ -219,7 +219,7 @@ def run_stack(args):
     outw = {k: [torch.empty_like(w) for w in probe.tensors[k]] for k in ("w_gate", "w_up", "w_down")}
     del probe
     stream = torch.cuda.current_stream()
-    names = ("forward", "score", "select_slice", "forward_sliced", "error_next_input")
+    names = ("forward_and_score", "select_slice", "forward_sliced", "error_next_input")
     tot = {k: 0.0 for k in names}
     errors = []
     for l in range(n_layers):
@@ -229,13 +229,10 @@ def run_stack(args):
         torch.cuda.synchronize()
         ev = [torch.cuda.Event(enable_timing=True) for _ in range(len(names) + 1)]
         ev[0].record(stream)
-        for t0, t1 in spans:
-            P.camera_layer_forward(layer, X[t0:t1], y=Y[t0:t1], workspace=ws_f)
-        ev[1].record(stream)
         for i, (t0, t1) in enumerate(spans):
-            P.camera_score_layer(layer, X[t0:t1], ALPHA, energy=energy, workspace=ws_s, phi2=phi2, phi_inf_sq=phi_inf,
-                                 accumulate=i > 0)
-        ev[2].record(stream)
+            P.camera_score_forward_layer(layer, X[t0:t1], ALPHA, energy=energy, y=Y[t0:t1], workspace=ws_f, phi2=phi2,
+                                         phi_inf_sq=phi_inf, accumulate=i > 0)
+        ev[1].record(stream)
         P.camera_select_prune(energy, ratio, workspace=ws_sel, keep_mask=keep)
         sub, counts = P.camera_sub_index(keep, off, [1])
         P.camera_compact_weights(layer, sub, counts, 1, out=outw, workspace=ws_c)
@@ -243,15 +240,15 @@ def run_stack(args):
         sliced = P.Layer(L["w_router"], [outw["w_gate"][e][:m[e]] for e in range(layer.n_experts)],
                          [outw["w_up"][e][:m[e]] for e in range(layer.n_experts)], outw["w_down"], cfg.top_k, cfg.n_shared,
                          L["router_bias"], L["w_shared_gate"], cfg.norm_topk, "hf", down_ld=layer.d_ff)
-        ev[3].record(stream)
+        ev[2].record(stream)
         for t0, t1 in spans:
             P.camera_layer_forward(sliced, X[t0:t1], y=Yh[t0:t1], workspace=ws_f)
-        ev[4].record(stream)
+        ev[3].record(stream)
         err = P.camera_output_error(Y, Yh)
         P.camera_residual_norm(X, Yh, out=X)
-        ev[5].record(stream)
+        ev[4].record(stream)
         torch.cuda.synchronize()
-        if P.camera_read_status(ws_s) != 0 or P.camera_read_status(ws_f) != 0:
+        if P.camera_read_status(ws_f) != 0:
             raise RuntimeError("device status set in the stack run")
         for i, k in enumerate(names):
             tot[k] += ev[i].elapsed_time(ev[i + 1])

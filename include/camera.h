@@ -257,6 +257,19 @@ size_t camera_forward_workspace_bytes(const camera_layer_t* layer, int64_t n_tok
 int camera_layer_forward(const camera_layer_t* layer, const void* x, int64_t n_tokens, float* y,
                          const camera_score_aux_t* aux, void* workspace, size_t workspace_bytes, void* cuda_stream);
 
+/*
+ * Lines 6 and 8 of Algorithm 2 on one batch of tokens, from one pass over W_gate and W_up: the energies of
+ * camera_score_layer (Algorithm 1: same alpha, energy, aux fields and flags, CAMERA_SCORE_ACCUMULATE included) and the
+ * layer output y of camera_layer_forward (Eq. 1-2).  The gate/up GEMM runs once, in the scoring orientation; its
+ * epilogue folds lambda into the per-micro-expert sums and maxima and stores it as h for the W_down GEMM.  The
+ * energies are bit-identical to camera_score_layer's and y to camera_layer_forward's under the same kernel flags.
+ * Arguments, layouts, restrictions and errors as for those two calls; energy must not be NULL (CAMERA_ERR_INVALID_ARG);
+ * workspace: camera_forward_workspace_bytes.  With n_tokens == 0 only the energies are written.
+ */
+int camera_score_forward_layer(const camera_layer_t* layer, const void* x, int64_t n_tokens, float alpha, float* energy,
+                               float* y, const camera_score_aux_t* aux, void* workspace, size_t workspace_bytes,
+                               void* cuda_stream);
+
 /* Scratch for camera_output_error. */
 size_t camera_output_error_workspace_bytes(int64_t n_tokens);
 

@@ -85,6 +85,10 @@ def _load() -> C.CDLL:
     lib.camera_layer_forward.restype = C.c_int
     lib.camera_layer_forward.argtypes = [C.POINTER(camera_layer_t), C.c_void_p, C.c_int64, C.c_void_p,
                                          C.POINTER(camera_score_aux_t), C.c_void_p, C.c_size_t, C.c_void_p]
+    lib.camera_score_forward_layer.restype = C.c_int
+    lib.camera_score_forward_layer.argtypes = [C.POINTER(camera_layer_t), C.c_void_p, C.c_int64, C.c_float, C.c_void_p,
+                                               C.c_void_p, C.POINTER(camera_score_aux_t), C.c_void_p, C.c_size_t,
+                                               C.c_void_p]
     lib.camera_output_error_workspace_bytes.restype = C.c_size_t
     lib.camera_output_error_workspace_bytes.argtypes = [C.c_int64]
     lib.camera_output_error.restype = C.c_int
@@ -437,6 +441,41 @@ def camera_layer_forward(layer: Layer, x: torch.Tensor, *, y: Optional[torch.Ten
     _check(lib.camera_layer_forward(C.byref(layer.c), x.data_ptr(), T, y.data_ptr(), C.byref(aux), workspace.data_ptr(),
                                     workspace.numel(), _stream_ptr(stream)), "camera_layer_forward")
     return (y, routing) if want_routing else y
+
+
+def camera_score_forward_layer(layer: Layer, x: torch.Tensor, alpha: float, *, energy: Optional[torch.Tensor] = None,
+                               y: Optional[torch.Tensor] = None, routing_in=None, workspace: Optional[torch.Tensor] = None,
+                               phi2: Optional[torch.Tensor] = None, phi_inf_sq: Optional[torch.Tensor] = None,
+                               accumulate: bool = False, cta_pair: Optional[bool] = None,
+                               stream: Optional[torch.cuda.Stream] = None):
+    """Energies (Algorithm 1) and layer output (Eq. 1-2) of one batch from one pass over W_gate and W_up.
+    Returns (energy [N_e] fp32, y [T, d_model] fp32); arguments as for camera_score_layer and camera_layer_forward."""
+    T = int(x.shape[0])
+    dev = x.device
+    if energy is None:
+        energy = torch.empty(layer.n_me, dtype=torch.float32, device=dev)
+    if y is None:
+        y = torch.empty((T, layer.d_model), dtype=torch.float32, device=dev)
+    if workspace is None:
+        workspace = alloc_workspace(camera_forward_workspace_bytes(layer, T), dev)
+    aux = camera_score_aux_t()
+    aux.flags = ((CAMERA_SCORE_CTA_PAIR if cta_pair else 0) | (CAMERA_SCORE_SINGLE_CTA if cta_pair is False else 0) |
+                 (CAMERA_SCORE_ACCUMULATE if accumulate else 0))
+    keep_alive = []
+    if routing_in is not None:
+        idx = routing_in[0].to(device=dev, dtype=torch.int32).contiguous()
+        w = routing_in[1].to(device=dev, dtype=torch.float32).contiguous()
+        keep_alive += [idx, w]
+        aux.topk_idx_in, aux.topk_w_in = idx.data_ptr(), w.data_ptr()
+    for name, t in (("phi2", phi2), ("phi_inf_sq", phi_inf_sq)):
+        if t is not None:
+            if not (t.is_contiguous() and t.dtype == torch.float32 and t.numel() == layer.n_me and t.device == dev):
+                raise ValueError(f"{name} must be a contiguous fp32 [N_e] tensor on the device of x")
+            setattr(aux, name, t.data_ptr())
+    _check(lib.camera_score_forward_layer(C.byref(layer.c), x.data_ptr(), T, float(alpha), energy.data_ptr(), y.data_ptr(),
+                                          C.byref(aux), workspace.data_ptr(), workspace.numel(), _stream_ptr(stream)),
+           "camera_score_forward_layer")
+    return energy, y
 
 
 def camera_output_error(y: torch.Tensor, y_hat: torch.Tensor, *, stream: Optional[torch.cuda.Stream] = None) -> torch.Tensor:

@@ -409,10 +409,13 @@ extern "C" size_t camera_forward_workspace_bytes(const camera_layer_t* layer, in
   return fwd_layout(layer, n_tokens).total;
 }
 
-extern "C" int camera_layer_forward(const camera_layer_t* L, const void* x, int64_t T, float* y,
-                                    const camera_score_aux_t* aux, void* workspace, size_t workspace_bytes,
-                                    void* cuda_stream) {
-  if (L == nullptr || y == nullptr || (reinterpret_cast<uintptr_t>(y) & 15)) return CAMERA_ERR_INVALID_ARG;
+namespace camera {
+namespace {
+
+// The layer output, and with `energy` also the scores, from one pass over W_gate and W_up.
+int forward_impl(const camera_layer_t* L, const void* x, int64_t T, float alpha, float* energy, float* y,
+                 const camera_score_aux_t* aux, void* workspace, size_t workspace_bytes, void* cuda_stream) {
+  if (L == nullptr || (y == nullptr && T > 0) || (reinterpret_cast<uintptr_t>(y) & 15)) return CAMERA_ERR_INVALID_ARG;
   if (score_workspace_bytes_any(L, T, true) == 0) return CAMERA_ERR_INVALID_ARG;
   if (L->dtype != CAMERA_BF16 || L->down_layout != CAMERA_DOWN_HF || L->d_model % UMMA_BK != 0 || !umma_shape_ok(L) ||
       (reinterpret_cast<uintptr_t>(x) & 15))
@@ -438,15 +441,24 @@ extern "C" int camera_layer_forward(const camera_layer_t* L, const void* x, int6
   const ForwardBuffers fb{h.data(), fl.h_ld.data(), yp.data()};
   camera_score_aux_t a2;
   memset(&a2, 0, sizeof(a2));
-  if (aux) { a2 = *aux; a2.flags &= ~(uint32_t)(CAMERA_SCORE_FORCE_SIMT | CAMERA_SCORE_ACCUMULATE); }
-  const bool token_rows = forward_token_rows(L, T, a2.flags);
+  if (aux) {
+    a2 = *aux;
+    a2.flags &= ~(uint32_t)CAMERA_SCORE_FORCE_SIMT;
+    if (energy == nullptr) a2.flags &= ~(uint32_t)CAMERA_SCORE_ACCUMULATE;
+  }
+  // the scores are sums and maxima over a micro-expert's tokens: they need the scoring orientation
+  const bool token_rows = energy == nullptr && forward_token_rows(L, T, a2.flags);
   if (token_rows) a2.flags = (a2.flags & ~(uint32_t)CAMERA_SCORE_SINGLE_CTA) | CAMERA_SCORE_CTA_PAIR;
   ScoreFront f;
-  int rc = score_front(L, x, T, 0.f, nullptr, &a2, ws + fl.score, fl.score_bytes, st, &fb, &f);
+  int rc = score_front(L, x, T, alpha, energy, &a2, ws + fl.score, fl.score_bytes, st, &fb, &f);
   if (rc != CAMERA_OK) return rc;
   if (!f.use_umma) return CAMERA_ERR_UNSUPPORTED_SHAPE;
-  if (T == 0) return CAMERA_OK;
   const ScoreCtx& c = f.c;
+  if (energy != nullptr && launch_rownorm(c, f.norm_blocks, st) != cudaSuccess) { cudaGetLastError(); return CAMERA_ERR_CUDA; }
+  if (T == 0) {   // no tokens: the scores of the batches so far (or zeros), no output rows
+    if (energy != nullptr && launch_combine(c, st) != cudaSuccess) { cudaGetLastError(); return CAMERA_ERR_CUDA; }
+    return CAMERA_OK;
+  }
 
   // tensor maps of the second GEMM: per expert W_down [d_model rows, d_ff] and h [rows, h_ld]
   std::vector<char> maps((size_t)128 * 2 * E);
@@ -467,6 +479,7 @@ extern "C" int camera_layer_forward(const camera_layer_t* L, const void* x, int6
     cudaGetLastError();
     return CAMERA_ERR_CUDA;
   }
+  if (energy != nullptr && launch_combine(c, st) != cudaSuccess) { cudaGetLastError(); return CAMERA_ERR_CUDA; }
   int dev = 0, sms = 148;
   cudaGetDevice(&dev);
   cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
@@ -478,6 +491,22 @@ extern "C" int camera_layer_forward(const camera_layer_t* L, const void* x, int6
   k_down_umma<<<sms, D_THREADS, D_SMEM_BYTES, st>>>(c, ws + fl.maps, n_dt);
   k_unpermute_sum<<<(unsigned)((T + 7) / 8), 256, 0, st>>>(c, y);
   return cudaGetLastError() == cudaSuccess ? CAMERA_OK : CAMERA_ERR_CUDA;
+}
+
+}  // namespace
+}  // namespace camera
+
+extern "C" int camera_layer_forward(const camera_layer_t* L, const void* x, int64_t T, float* y,
+                                    const camera_score_aux_t* aux, void* workspace, size_t workspace_bytes,
+                                    void* cuda_stream) {
+  return forward_impl(L, x, T, 0.f, nullptr, y, aux, workspace, workspace_bytes, cuda_stream);
+}
+
+extern "C" int camera_score_forward_layer(const camera_layer_t* L, const void* x, int64_t T, float alpha, float* energy,
+                                          float* y, const camera_score_aux_t* aux, void* workspace,
+                                          size_t workspace_bytes, void* cuda_stream) {
+  if (energy == nullptr) return CAMERA_ERR_INVALID_ARG;
+  return forward_impl(L, x, T, alpha, energy, y, aux, workspace, workspace_bytes, cuda_stream);
 }
 
 extern "C" size_t camera_output_error_workspace_bytes(int64_t n_tokens) {

@@ -261,7 +261,8 @@ __global__ void __launch_bounds__(U_THREADS, 1) k_score_umma(const ScoreCtx c) {
         tile_phase ^= 1u;
       }
       const int ch = u.ch0 + warp * 32 + lane;
-      if (!WRITE_H && ok && ch < u.f) {
+      // the partials are the scores' input: always when scoring, with the layer forward when scores were asked for
+      if ((!WRITE_H || c.energy != nullptr) && ok && ch < u.f) {
         const size_t slot = (size_t)u.part_slot + warp * 32 + lane;
         c.part_sum[slot] = s;
         c.part_max[slot] = m;

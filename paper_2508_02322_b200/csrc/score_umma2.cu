@@ -415,7 +415,8 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(P_THREADS, 1) k_scor
           tile_phase ^= 1u;
         }
         const int ch = u.ch0 + 128 * (int)rank + warp * 32 + lane;
-        if (MODE == PAIR_SCORE && ok && ch < u.f) {
+        // the partials are the scores' input: always when scoring, with the layer forward when scores were asked for
+        if ((MODE == PAIR_SCORE || c.energy != nullptr) && ok && ch < u.f) {
           const size_t slot = (size_t)u.part_slot + 128 * rank + warp * 32 + lane;
           c.part_sum[slot] = s;
           c.part_max[slot] = m;

@@ -109,6 +109,49 @@ def test_token_rows_kernel_ragged_widths(P, d_ff):
     assert_output_close(f"token rows, d_ff {d_ff}", y.cpu().numpy(), oracle_forward(ol, Xd, rout))
 
 
+@pytest.mark.parametrize("cta_pair", [False, True])
+def test_scores_and_output_from_one_pass(P, cta_pair):
+    """camera_score_forward_layer: the energies against the oracle's (Algorithm 1) and bit for bit against
+    camera_score_layer's, the output bit for bit against camera_layer_forward's, also when the tokens come in two
+    batches that accumulate."""
+    from _gpu import assert_close
+    cfg = cfg_of(n_tokens=1300, d_ff_routed=320)
+    L = W().make_layer(cfg, seed=36, device=DEV)
+    X = W().make_tokens(cfg, seed=36, device=DEV)
+    layer = P.Layer.from_workload(L)
+    ol, Xd = to_oracle_layer(L), f64(X)
+    rin, rout = oracle_routing(ol, Xd)
+    E, y = P.camera_score_forward_layer(layer, X, 0.95, routing_in=rin, cta_pair=cta_pair)
+    E_ref = P.camera_score_layer(layer, X, 0.95, routing_in=rin, cta_pair=cta_pair)
+    y_ref = P.camera_layer_forward(layer, X, routing_in=rin, cta_pair=cta_pair)
+    assert torch.equal(E, E_ref) and torch.equal(y, y_ref)
+    p2, pinf, w2 = O.camera_components(ol, Xd, routing=rout)
+    assert_close("energy from the one-pass call", E.cpu().numpy(), O.energy(p2, pinf, w2, float(np.float32(0.95))))
+    assert_output_close("output from the one-pass call", y.cpu().numpy(), oracle_forward(ol, Xd, rout))
+    # two batches: the components accumulate, the outputs are the batches' rows
+    phi2 = torch.empty(layer.n_me, dtype=torch.float32, device=DEV)
+    pinf_t = torch.empty_like(phi2)
+    E2 = torch.empty_like(phi2)
+    y2 = torch.empty_like(y)
+    ws = P.alloc_workspace(P.camera_forward_workspace_bytes(layer, 800), DEV)
+    for i, (t0, t1) in enumerate([(0, 800), (800, 1300)]):
+        P.camera_score_forward_layer(layer, X[t0:t1], 0.95, energy=E2, y=y2[t0:t1], workspace=ws, phi2=phi2,
+                                     phi_inf_sq=pinf_t, accumulate=i > 0, cta_pair=cta_pair,
+                                     routing_in=(rin[0][t0:t1], rin[1][t0:t1]))
+    assert P.camera_read_status(ws) == 0
+    assert_close("energy accumulated over two batches", E2.cpu().numpy(), O.energy(p2, pinf, w2, float(np.float32(0.95))))
+    assert_output_close("output in two batches", y2.cpu().numpy(), oracle_forward(ol, Xd, rout))
+
+
+def test_one_pass_call_without_tokens(P):
+    cfg = cfg_of(n_tokens=0)
+    L = W().make_layer(cfg, seed=37, device=DEV)
+    layer = P.Layer.from_workload(L)
+    X = torch.empty((0, cfg.d_model), dtype=torch.bfloat16, device=DEV)
+    E, y = P.camera_score_forward_layer(layer, X, 0.95)
+    assert y.shape == (0, cfg.d_model) and float(E.abs().max()) == 0.0
+
+
 def test_dense_layer_is_a_gated_ffn(P):
     cfg = cfg_of(n_tokens=400, n_routed=0, top_k=1, d_ff_shared=(384,), shared_gate_sigmoid=False, router_bias_std=0.0)
     L = W().make_layer(cfg, seed=32, device=DEV)
