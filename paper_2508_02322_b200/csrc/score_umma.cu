@@ -40,30 +40,9 @@ constexpr int U_STAGE_BYTES = 2 * U_A_BYTES + U_B_BYTES;
 constexpr int U_TMEM_COLS = 512;
 constexpr int U_SCHED = 2;                       // depth of the ring that passes unit numbers between the warps
 constexpr int U_WBUF_BYTES = 4 * UMMA_TOK * 4;   // router weights of a token tile, one copy per epilogue warp
-constexpr int U_SMEM_BYTES = U_STAGES * U_STAGE_BYTES + U_WBUF_BYTES + 256 + 1024;
+constexpr int U_STG_BYTES = 4 * FOLD_STG_BYTES;   // layer forward: where an epilogue warp turns its 16 x 32 values of h
+constexpr int U_SMEM_BYTES = U_STAGES * U_STAGE_BYTES + U_WBUF_BYTES + U_STG_BYTES + 256 + 1024;
 static_assert(CH_TILE == 128, "one micro-expert per TMEM lane");
-
-// lambda = a_t * SiLU(g) * u for 16 tokens of this thread's micro-expert; folds lambda^2 and |lambda|.
-// WRITE_H (layer forward): lambda is also stored, as bf16, to h[token][micro-expert] for the first n_store tokens.
-template <bool WRITE_H>
-__device__ __forceinline__ void fold16(const uint32_t* vg, const uint32_t* vu, const float* wb, float& s, float& m,
-                                       __nv_bfloat16* hcol, int h_ld, int n_store) {
-  float a[16];
-#pragma unroll
-  for (int q = 0; q < 4; ++q) {
-    const float4 w4 = *reinterpret_cast<const float4*>(wb + 4 * q);
-    a[4 * q] = w4.x; a[4 * q + 1] = w4.y; a[4 * q + 2] = w4.z; a[4 * q + 3] = w4.w;
-  }
-#pragma unroll
-  for (int j = 0; j < 16; ++j) {
-    const float g = __uint_as_float(vg[j]), up = __uint_as_float(vu[j]);
-    const float sig = __fdividef(1.f, 1.f + __expf(-g));
-    const float lam = (a[j] * up) * (g * sig);
-    s = fmaf(lam, lam, s);
-    m = fmaxf(m, fabsf(lam));
-    if (WRITE_H && j < n_store) hcol[(size_t)j * h_ld] = __float2bfloat16_rn(lam);
-  }
-}
 
 template <bool WRITE_H>
 __global__ void __launch_bounds__(U_THREADS, 1) k_score_umma(const ScoreCtx c) {
@@ -72,7 +51,8 @@ __global__ void __launch_bounds__(U_THREADS, 1) k_score_umma(const ScoreCtx c) {
   uint8_t* const base_ptr = smem_raw + (base - smem_u32(smem_raw));
   // [stages: A_gate | A_up | B] [wbuf 4 warps x 256 floats] [barriers] [tmem slot] [abort flag]
   float* const wbuf = reinterpret_cast<float*>(base_ptr + U_STAGES * U_STAGE_BYTES);
-  const uint32_t bars = base + U_STAGES * U_STAGE_BYTES + U_WBUF_BYTES;
+  uint8_t* const stg_all = base_ptr + U_STAGES * U_STAGE_BYTES + U_WBUF_BYTES;
+  const uint32_t bars = base + U_STAGES * U_STAGE_BYTES + U_WBUF_BYTES + U_STG_BYTES;
   auto full_bar = [&](int s) { return bars + 8u * s; };
   auto empty_bar = [&](int s) { return bars + 8u * (U_STAGES + s); };
   const uint32_t tfull_bar = bars + 8u * (2 * U_STAGES);
@@ -81,7 +61,7 @@ __global__ void __launch_bounds__(U_THREADS, 1) k_score_umma(const ScoreCtx c) {
   // passes its number to the MMA thread and the epilogue warps through a small ring
   auto sfull_bar = [&](int q) { return bars + 8u * (2 * U_STAGES + 2 + q); };
   auto sempty_bar = [&](int q) { return bars + 8u * (2 * U_STAGES + 2 + U_SCHED + q); };
-  uint8_t* const tail = base_ptr + U_STAGES * U_STAGE_BYTES + U_WBUF_BYTES + 8 * (2 * U_STAGES + 2 + 2 * U_SCHED);
+  uint8_t* const tail = base_ptr + U_STAGES * U_STAGE_BYTES + U_WBUF_BYTES + U_STG_BYTES + 8 * (2 * U_STAGES + 2 + 2 * U_SCHED);
   volatile uint32_t* const tmem_slot = reinterpret_cast<volatile uint32_t*>(tail);
   volatile int* const abort_flag = reinterpret_cast<volatile int*>(tail + 8);
   volatile int* const sched_unit = reinterpret_cast<volatile int*>(tail + 16);
@@ -204,6 +184,7 @@ __global__ void __launch_bounds__(U_THREADS, 1) k_score_umma(const ScoreCtx c) {
     uint32_t tile_phase = 0;
     bool ok = true;
     float* const wb = wbuf + warp * UMMA_TOK;
+    uint8_t* const stg = stg_all + warp * FOLD_STG_BYTES;
     const uint32_t t_gate = tmem_base + ((uint32_t)(warp * 32) << 16);
     const uint32_t t_up = t_gate + UMMA_TOK;
     int q = 0;
@@ -220,13 +201,13 @@ __global__ void __launch_bounds__(U_THREADS, 1) k_score_umma(const ScoreCtx c) {
       const int n_tiles = (u.rows + UMMA_TOK - 1) / UMMA_TOK;
       const float* wsrc = u.shared_idx < 0 ? c.perm_w + u.row0 : c.shared_w + (size_t)u.shared_idx * c.n_tokens + u.row0;
       float s = 0.f, m = 0.f;
-      // layer forward: where this thread's micro-expert goes in h, and the last row h has
+      // layer forward: where the warp's 32 micro-experts go in h, and the last row h has
       __nv_bfloat16* hbase = nullptr;
       int h_ld = 0, row_limit = 0;
       if (WRITE_H) {
         const ExpertStatic es = c.est[u.e];
         h_ld = es.h_ld;
-        hbase = static_cast<__nv_bfloat16*>(es.h) + (size_t)u.row0 * h_ld + u.ch0 + warp * 32 + lane;
+        hbase = static_cast<__nv_bfloat16*>(es.h) + (size_t)u.row0 * h_ld + u.ch0 + warp * 32;
         row_limit = (u.shared_idx < 0 ? c.max_rows_perm : c.n_tokens) - u.row0;
       }
       for (int tt = 0; ok && tt < n_tiles; ++tt) {
@@ -249,11 +230,11 @@ __global__ void __launch_bounds__(U_THREADS, 1) k_score_umma(const ScoreCtx c) {
         for (int c0 = 0; c0 < nv; c0 += 32) {
           tmem_ld_wait(g0, u0);
           if (c0 + 16 < nv) { tmem_ld16(t_gate + c0 + 16, g1); tmem_ld16(t_up + c0 + 16, u1); }
-          fold16<WRITE_H>(g0, u0, wb + c0, s, m, htile + (size_t)c0 * h_ld, h_ld, rows_left - c0);
+          fold16<WRITE_H>(g0, u0, wb + c0, s, m, htile + (size_t)c0 * h_ld, h_ld, rows_left - c0, stg, lane);
           if (c0 + 16 < nv) {
             tmem_ld_wait(g1, u1);
             if (c0 + 32 < nv) { tmem_ld16(t_gate + c0 + 32, g0); tmem_ld16(t_up + c0 + 32, u0); }
-            fold16<WRITE_H>(g1, u1, wb + c0 + 16, s, m, htile + (size_t)(c0 + 16) * h_ld, h_ld, rows_left - c0 - 16);
+            fold16<WRITE_H>(g1, u1, wb + c0 + 16, s, m, htile + (size_t)(c0 + 16) * h_ld, h_ld, rows_left - c0 - 16, stg, lane);
           }
         }
         tc_fence_before();

@@ -30,7 +30,8 @@ constexpr int P_STAGE_BYTES = 2 * P_A_BYTES + P_B_BYTES;
 constexpr int P_TMEM_COLS = 512;
 constexpr int P_SCHED = 2;                       // depth of the ring that passes unit numbers around the pair
 constexpr int P_WBUF_BYTES = 4 * UMMA_TOK * 4;
-constexpr int P_SMEM_BYTES = P_STAGES * P_STAGE_BYTES + P_WBUF_BYTES + 256 + 1024;
+constexpr int P_STG_BYTES = 4 * FOLD_STG_BYTES;   // layer forward: where an epilogue warp turns its 16 x 32 values of h
+constexpr int P_SMEM_BYTES = P_STAGES * P_STAGE_BYTES + P_WBUF_BYTES + P_STG_BYTES + 256 + 1024;
 
 __device__ __forceinline__ uint32_t cluster_ctarank() {
   uint32_t r;
@@ -109,27 +110,6 @@ __device__ __forceinline__ void umma_commit_pair(uint32_t bar) {
                : "memory");
 }
 
-// WRITE_H (layer forward): lambda is also stored, as bf16, to h[token][micro-expert] for the first n_store tokens.
-template <bool WRITE_H>
-__device__ __forceinline__ void fold16_pair(const uint32_t* vg, const uint32_t* vu, const float* wb, float& s, float& m,
-                                            __nv_bfloat16* hcol, int h_ld, int n_store) {
-  float a[16];
-#pragma unroll
-  for (int q = 0; q < 4; ++q) {
-    const float4 w4 = *reinterpret_cast<const float4*>(wb + 4 * q);
-    a[4 * q] = w4.x; a[4 * q + 1] = w4.y; a[4 * q + 2] = w4.z; a[4 * q + 3] = w4.w;
-  }
-#pragma unroll
-  for (int j = 0; j < 16; ++j) {
-    const float g = __uint_as_float(vg[j]), up = __uint_as_float(vu[j]);
-    const float sig = __fdividef(1.f, 1.f + __expf(-g));
-    const float lam = (a[j] * up) * (g * sig);
-    s = fmaf(lam, lam, s);
-    m = fmaxf(m, fabsf(lam));
-    if (WRITE_H && j < n_store) hcol[(size_t)j * h_ld] = __float2bfloat16_rn(lam);
-  }
-}
-
 // The layer-forward epilogue with a token on every accumulator row: h = a * SiLU(g) * u for 16 consecutive
 // micro-experts of the thread's token, rounded to bf16 and packed into 32 contiguous bytes.
 __device__ __forceinline__ void silu_mul16(const uint32_t* vg, const uint32_t* vu, float a, uint4& lo, uint4& hi) {
@@ -162,7 +142,8 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(P_THREADS, 1) k_scor
   uint8_t* const base_ptr = smem_raw + (base - smem_u32(smem_raw));
   // [stages: A_gate | A_up | B half] [wbuf 4 warps x 256 floats] [barriers] [tmem slot] [abort flag]
   float* const wbuf = reinterpret_cast<float*>(base_ptr + P_STAGES * P_STAGE_BYTES);
-  const uint32_t bars = base + P_STAGES * P_STAGE_BYTES + P_WBUF_BYTES;
+  uint8_t* const stg_all = base_ptr + P_STAGES * P_STAGE_BYTES + P_WBUF_BYTES;
+  const uint32_t bars = base + P_STAGES * P_STAGE_BYTES + P_WBUF_BYTES + P_STG_BYTES;
   auto full_bar = [&](int s) { return bars + 8u * s; };
   auto empty_bar = [&](int s) { return bars + 8u * (P_STAGES + s); };
   const uint32_t tfull_bar = bars + 8u * (2 * P_STAGES);
@@ -172,7 +153,7 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(P_THREADS, 1) k_scor
   // ten readers of the pair (MMA thread, second CTA's producer, eight epilogue warps) have taken it
   auto sfull_bar = [&](int q) { return bars + 8u * (2 * P_STAGES + 2 + q); };
   auto sempty_bar = [&](int q) { return bars + 8u * (2 * P_STAGES + 2 + P_SCHED + q); };
-  uint8_t* const tail = base_ptr + P_STAGES * P_STAGE_BYTES + P_WBUF_BYTES + 8 * (2 * P_STAGES + 2 + 2 * P_SCHED);
+  uint8_t* const tail = base_ptr + P_STAGES * P_STAGE_BYTES + P_WBUF_BYTES + P_STG_BYTES + 8 * (2 * P_STAGES + 2 + 2 * P_SCHED);
   volatile uint32_t* const tmem_slot = reinterpret_cast<volatile uint32_t*>(tail);
   volatile int* const abort_flag = reinterpret_cast<volatile int*>(tail + 8);
   volatile int* const sched_unit = reinterpret_cast<volatile int*>(tail + 16);
@@ -316,6 +297,7 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(P_THREADS, 1) k_scor
     uint32_t tile_phase = 0;
     bool ok = true;
     float* const wb = wbuf + warp * UMMA_TOK;
+    uint8_t* const stg = stg_all + warp * FOLD_STG_BYTES;
     const uint32_t t_gate = tmem_base + ((uint32_t)(warp * 32) << 16);
     const uint32_t t_up = t_gate + UMMA_TOK;
     const uint32_t tempty0 = map_to_cta(tempty_bar, 0);
@@ -339,10 +321,10 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(P_THREADS, 1) k_scor
       if (WRITE_H) {
         const ExpertStatic es = c.est[u.e];
         h_ld = es.h_ld;
-        hbase = static_cast<__nv_bfloat16*>(es.h) + (size_t)u.row0 * h_ld + u.ch0 + 128 * (int)rank + warp * 32 + lane;
+        hbase = static_cast<__nv_bfloat16*>(es.h) + (size_t)u.row0 * h_ld + u.ch0 + 128 * (int)rank + warp * 32;
         row_limit = (u.shared_idx < 0 ? c.max_rows_perm : c.n_tokens) - u.row0;
         // h is padded to 128 columns, a pair covers 256: the second CTA of an expert's last pair may have no column
-        if (u.ch0 + 128 * (int)rank + warp * 32 + lane >= h_ld) row_limit = 0;
+        if (u.ch0 + 128 * (int)rank + warp * 32 >= h_ld) row_limit = 0;
       }
       if constexpr (MODE == PAIR_H_ROWS) {
         const ExpertStatic es = c.est[u.e];
@@ -403,11 +385,11 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(P_THREADS, 1) k_scor
           for (int c0 = 0; c0 < nv; c0 += 32) {
             tmem_ld_wait(g0, u0);
             if (c0 + 16 < nv) { tmem_ld16(t_gate + c0 + 16, g1); tmem_ld16(t_up + c0 + 16, u1); }
-            fold16_pair<WRITE_H>(g0, u0, wb + c0, s, m, htile + (size_t)c0 * h_ld, h_ld, rows_left - c0);
+            fold16<WRITE_H>(g0, u0, wb + c0, s, m, htile + (size_t)c0 * h_ld, h_ld, rows_left - c0, stg, lane);
             if (c0 + 16 < nv) {
               tmem_ld_wait(g1, u1);
               if (c0 + 32 < nv) { tmem_ld16(t_gate + c0 + 32, g0); tmem_ld16(t_up + c0 + 32, u0); }
-              fold16_pair<WRITE_H>(g1, u1, wb + c0 + 16, s, m, htile + (size_t)(c0 + 16) * h_ld, h_ld, rows_left - c0 - 16);
+              fold16<WRITE_H>(g1, u1, wb + c0 + 16, s, m, htile + (size_t)(c0 + 16) * h_ld, h_ld, rows_left - c0 - 16, stg, lane);
             }
           }
           tc_fence_before();

@@ -130,4 +130,42 @@ __device__ __forceinline__ void tmem_ld_wait(uint32_t* a, uint32_t* b) {
                : "memory");
 }
 
+// Epilogue of the scoring orientation (a thread = a micro-expert, 16 tokens per call):
+// lambda = a_t * SiLU(g) * u; folds lambda^2 and |lambda| into s and m.
+// WRITE_H (layer forward): lambda also goes, as bf16, to h[token][micro-expert].  The 16 x 32 values of the warp are
+// turned in shared memory (stg: 1 KB of the warp's own, 16-byte aligned) so that a lane stores 16 bytes = 8 consecutive
+// micro-experts of one token: two vector stores per lane instead of sixteen 2-byte ones.  hwarp points at
+// h[first of the 16 tokens][first of the warp's 32 micro-experts]; tokens from n_store on are not stored.
+constexpr int FOLD_STG_BYTES = 16 * 32 * 2;
+template <bool WRITE_H>
+__device__ __forceinline__ void fold16(const uint32_t* vg, const uint32_t* vu, const float* wb, float& s, float& m,
+                                       __nv_bfloat16* hwarp, int h_ld, int n_store, uint8_t* stg, int lane) {
+  float a[16];
+#pragma unroll
+  for (int q = 0; q < 4; ++q) {
+    const float4 w4 = *reinterpret_cast<const float4*>(wb + 4 * q);
+    a[4 * q] = w4.x; a[4 * q + 1] = w4.y; a[4 * q + 2] = w4.z; a[4 * q + 3] = w4.w;
+  }
+  __nv_bfloat16* const col = reinterpret_cast<__nv_bfloat16*>(stg) + lane;
+#pragma unroll
+  for (int j = 0; j < 16; ++j) {
+    const float g = __uint_as_float(vg[j]), up = __uint_as_float(vu[j]);
+    const float sig = __fdividef(1.f, 1.f + __expf(-g));
+    const float lam = (a[j] * up) * (g * sig);
+    s = fmaf(lam, lam, s);
+    m = fmaxf(m, fabsf(lam));
+    if (WRITE_H) col[j * 32] = __float2bfloat16_rn(lam);
+  }
+  if (WRITE_H) {
+    __syncwarp();
+#pragma unroll
+    for (int i = 0; i < 2; ++i) {
+      const int q = lane + 32 * i, row = q >> 2, part = q & 3;      // 64 pieces of 16 bytes: 4 per token row
+      const uint4 v = *reinterpret_cast<const uint4*>(stg + 16 * q);
+      if (row < n_store) *reinterpret_cast<uint4*>(hwarp + (size_t)row * h_ld + 8 * part) = v;
+    }
+    __syncwarp();
+  }
+}
+
 }  // namespace camera
