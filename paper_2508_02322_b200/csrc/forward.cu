@@ -3,7 +3,7 @@
 // Y_hat = Phi[:,S] W[S,:] of Eq. 7, and camera_output_error gives ||Y - Y_hat||_F^2 and the cosine similarity.
 //
 //   k_score_umma<WRITE_H>   h = A * SiLU(W_gate x) * (W_up x) per (token row, micro-expert), bf16      (score_umma.cu)
-//   k_down_umma             y_part[row, :] = W_down h[row, :] per expert, tcgen05, fp32 out
+//   k_down_umma(_pair)      y_part[row, :] = W_down h[row, :] per expert, tcgen05, fp32 out (pairs: long token lists)
 //   k_unpermute_sum         y[t, :] = sum over the token's k routed rows and its shared-expert rows, fixed order
 #include <math.h>
 #include <string.h>
@@ -12,6 +12,7 @@
 
 #include "common.cuh"
 #include "umma.cuh"
+#include "umma_pair.cuh"
 
 namespace camera {
 
@@ -34,7 +35,7 @@ struct DownUnit {
 
 // Work units are numbered (token chunk, output-channel tile) with the tile fastest: the CTAs running at one time
 // share a chunk of h through L2 while an expert's W_down stays resident.
-__device__ __forceinline__ DownUnit decode_down_unit(const ScoreCtx& c, int unit, int n_dt) {
+__device__ __forceinline__ DownUnit decode_down_unit(const ScoreCtx& c, int unit, int n_dt, int tile = D_TILE) {
   DownUnit u;
   const int chunk = unit / n_dt;
   int lo = 0, hi = c.n_experts;
@@ -48,7 +49,7 @@ __device__ __forceinline__ DownUnit decode_down_unit(const ScoreCtx& c, int unit
   const int ck = chunk - dy.chunk_begin;
   u.rows = min(c.chunk_tokens, dy.rows - ck * c.chunk_tokens);
   u.row0 = dy.row_base + ck * c.chunk_tokens;
-  u.c0 = (unit % n_dt) * D_TILE;
+  u.c0 = (unit % n_dt) * tile;
   u.n_kb = (es.d_ff + UMMA_BK - 1) / UMMA_BK;
   u.row_limit = (es.shared_idx < 0 ? c.max_rows_perm : c.n_tokens) - u.row0;
   u.y = es.y_part;
@@ -232,6 +233,234 @@ __global__ void __launch_bounds__(D_THREADS, 1) k_down_umma(const ScoreCtx c, co
     __syncwarp();
     tc_fence_after();
     asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(D_TMEM_COLS) : "memory");
+  }
+}
+
+// The same GEMM on CTA pairs with the token tile as the M operand: the pair computes 256 tokens x 512 output channels
+// as two MMAs of N = 256 that share the token tile, so a CTA pulls 48 KB per k-block from L2 for 16.8 Mflop (k_down_umma:
+// 48 KB for 4.2 Mflop, which keeps the tensor pipe waiting for L2).  Each CTA holds its 128 token rows of h and its
+// halves of the two W_down tiles; the two accumulators fill the 512 TMEM columns, so the short epilogue (a thread owns
+// a token and writes 64 contiguous bytes of its output row per 16 columns) runs between tiles.  Barriers and the
+// hand-out of work units are those of k_score_umma_pair; every token tile costs 256 rows, so short token lists stay
+// with k_down_umma.
+constexpr int DP_STAGES = 4;
+constexpr int DP_HALF = 256;                      // output channels per MMA
+constexpr int DP_TILE = 2 * DP_HALF;              // output channels per work unit
+constexpr int DP_A_BYTES = 128 * 128;             // this CTA's 128 token rows of h x 128 B
+constexpr int DP_B_BYTES = 128 * 128;             // this CTA's half of one W_down tile
+constexpr int DP_STAGE_BYTES = DP_A_BYTES + 2 * DP_B_BYTES;
+constexpr int DP_SMEM_BYTES = DP_STAGES * DP_STAGE_BYTES + 256 + 1024;
+
+// 32 bytes in one store (the address is 32-byte aligned).
+__device__ __forceinline__ void st_global_v8(void* p, const uint32_t* v) {
+  asm volatile("st.global.v8.b32 [%0], {%1,%2,%3,%4,%5,%6,%7,%8};" ::"l"(p), "r"(v[0]), "r"(v[1]), "r"(v[2]), "r"(v[3]),
+               "r"(v[4]), "r"(v[5]), "r"(v[6]), "r"(v[7])
+               : "memory");
+}
+
+__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(D_THREADS, 1)
+    k_down_umma_pair(const ScoreCtx c, const void* maps_raw, int n_dt) {
+  extern __shared__ uint8_t smem_raw[];
+  const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+  uint8_t* const base_ptr = smem_raw + (base - smem_u32(smem_raw));
+  const uint32_t bars = base + DP_STAGES * DP_STAGE_BYTES;
+  auto full_bar = [&](int s) { return bars + 8u * s; };                                   // first CTA
+  auto empty_bar = [&](int s) { return bars + 8u * (DP_STAGES + s); };                    // each CTA
+  const uint32_t tfull_bar = bars + 8u * (2 * DP_STAGES);                                 // each CTA
+  const uint32_t tempty_bar = bars + 8u * (2 * DP_STAGES + 1);                            // first CTA, 256 readers
+  auto sfull_bar = [&](int q) { return bars + 8u * (2 * DP_STAGES + 2 + q); };            // each CTA
+  auto sempty_bar = [&](int q) { return bars + 8u * (2 * DP_STAGES + 2 + D_SCHED + q); }; // first CTA, 10 readers
+  uint8_t* const tail = base_ptr + DP_STAGES * DP_STAGE_BYTES + 8 * (2 * DP_STAGES + 2 + 2 * D_SCHED);
+  volatile uint32_t* const tmem_slot = reinterpret_cast<volatile uint32_t*>(tail);
+  volatile int* const abort_flag = reinterpret_cast<volatile int*>(tail + 8);
+  volatile int* const sched_unit = reinterpret_cast<volatile int*>(tail + 16);
+
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const uint32_t rank = cluster_ctarank();
+  const int total_units = c.totals->total_chunks * n_dt;
+
+  if (tid == 0) {
+    for (int s = 0; s < DP_STAGES; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
+    mbar_init(tfull_bar, 1);
+    mbar_init(tempty_bar, 256);
+    for (int q = 0; q < D_SCHED; ++q) { mbar_init(sfull_bar(q), 1); mbar_init(sempty_bar(q), 10); }
+    *abort_flag = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+  }
+  if (warp == 5) {
+    asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32((const void*)tmem_slot)),
+                 "r"(D_TMEM_COLS)
+                 : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
+  }
+  tc_fence_before();
+  __syncthreads();
+  cluster_sync_all();     // the other CTA's barriers are initialised before anything arrives on them
+  tc_fence_after();
+  const uint32_t tmem_base = *tmem_slot;
+
+  if (warp == 4) {
+    // ------------------------------------------------------------------ TMA producer (each CTA loads its own share)
+    if (lane == 0) {
+      int stage = 0;
+      uint32_t phase = 0;
+      bool ok = true;
+      const char* maps = static_cast<const char*>(maps_raw);
+      int q = 0;
+      uint32_t qphase = 0;
+      while (ok) {
+        int unit;
+        if (rank == 0) {
+          if (!mbar_wait_cluster(sempty_bar(q), qphase ^ 1u, abort_flag)) { ok = false; break; }
+          unit = atomicAdd(&c.totals->down_counter, 1);
+          if (unit >= total_units) unit = -1;
+          sched_unit[q] = unit;
+          st_cluster_u32(map_to_cta(smem_u32((const void*)(sched_unit + q)), 1), (uint32_t)unit);
+          mbar_arrive(sfull_bar(q));
+          mbar_arrive_cluster(map_to_cta(sfull_bar(q), 1));
+        } else {
+          if (!mbar_wait_cluster(sfull_bar(q), qphase, abort_flag)) { ok = false; break; }
+          unit = sched_unit[q];
+          mbar_arrive_cluster(map_to_cta(sempty_bar(q), 0));
+        }
+        if (++q == D_SCHED) { q = 0; qphase ^= 1u; }
+        if (unit < 0) break;
+        const DownUnit u = decode_down_unit(c, unit, n_dt, DP_TILE);
+        if (u.n_kb == 0) continue;
+        const int n_tiles = (u.rows + UMMA_TOK - 1) / UMMA_TOK;
+        const void* map_w = maps + (size_t)128 * (2 * u.e);
+        const void* map_h = maps + (size_t)128 * (2 * u.e + 1);
+        tensormap_acquire(map_w);
+        tensormap_acquire(map_h);
+        // the two N operands (d_model is a multiple of 64); this CTA holds the upper or lower half of each
+        const int ncv0 = min(DP_HALF, c.d_model - u.c0), ncv1 = max(0, min(DP_HALF, c.d_model - u.c0 - DP_HALF));
+        const int wrow0 = u.c0 + (int)rank * (ncv0 >> 1), wrow1 = u.c0 + DP_HALF + (int)rank * (ncv1 >> 1);
+        for (int tt = 0; ok && tt < n_tiles; ++tt) {
+          const int row = u.row0 + tt * UMMA_TOK + 128 * (int)rank;  // this CTA's rows of the M operand
+          for (int kb = 0; kb < u.n_kb; ++kb) {
+            if (!mbar_wait(empty_bar(stage), phase ^ 1u, abort_flag)) { ok = false; break; }
+            const uint32_t a_dst = base + stage * DP_STAGE_BYTES;
+            const uint32_t full0 = map_to_cta(full_bar(stage), 0);
+            if (rank == 0) mbar_expect_tx(full_bar(stage), 2 * DP_STAGE_BYTES);
+            // h rows past the buffer, W_down columns past d_ff and rows past d_model: filled with zeros
+            tma_load_2d_pair(a_dst, map_h, full0, kb * UMMA_BK, row);
+            tma_load_2d_pair(a_dst + DP_A_BYTES, map_w, full0, kb * UMMA_BK, wrow0);
+            tma_load_2d_pair(a_dst + DP_A_BYTES + DP_B_BYTES, map_w, full0, kb * UMMA_BK, wrow1);
+            if (++stage == DP_STAGES) { stage = 0; phase ^= 1u; }
+          }
+        }
+      }
+      if (!ok) {
+        const unsigned long long t0 = globaltimer_ns();
+        while (globaltimer_ns() - t0 < 2000000ull) __nanosleep(1000);
+      }
+    }
+  } else if (warp == 5) {
+    // ------------------------------------------------------------------ MMA issuer (first CTA of the pair only)
+    if (lane == 0 && rank == 0) {
+      int stage = 0;
+      uint32_t phase = 0, tile_phase = 0;
+      bool ok = true;
+      int q = 0;
+      uint32_t qphase = 0;
+      while (ok) {
+        if (!mbar_wait(sfull_bar(q), qphase, abort_flag)) { ok = false; break; }
+        const int unit = sched_unit[q];
+        mbar_arrive(sempty_bar(q));
+        if (++q == D_SCHED) { q = 0; qphase ^= 1u; }
+        if (unit < 0) break;
+        const DownUnit u = decode_down_unit(c, unit, n_dt, DP_TILE);
+        if (u.n_kb == 0) continue;
+        const int n_tiles = (u.rows + UMMA_TOK - 1) / UMMA_TOK;
+        const int ncv0 = min(DP_HALF, c.d_model - u.c0), ncv1 = max(0, min(DP_HALF, c.d_model - u.c0 - DP_HALF));
+        const uint32_t idesc0 = make_idesc_pair(ncv0), idesc1 = make_idesc_pair(ncv1);
+        for (int tt = 0; ok && tt < n_tiles; ++tt) {
+          if (!mbar_wait_cluster(tempty_bar, tile_phase ^ 1u, abort_flag)) { ok = false; break; }
+          tc_fence_after();
+          for (int kb = 0; kb < u.n_kb; ++kb) {
+            if (!mbar_wait(full_bar(stage), phase, abort_flag)) { ok = false; break; }
+            tc_fence_after();
+            const uint32_t a_addr = base + stage * DP_STAGE_BYTES;
+            const unsigned long long a_desc = make_smem_desc(a_addr);
+            const unsigned long long b0_desc = make_smem_desc(a_addr + DP_A_BYTES);
+            const unsigned long long b1_desc = make_smem_desc(a_addr + DP_A_BYTES + DP_B_BYTES);
+#pragma unroll
+            for (int k = 0; k < UMMA_BK / 16; ++k) {
+              const uint32_t accum = (uint32_t)((kb | k) != 0);
+              umma_bf16_pair(tmem_base, a_desc + 2 * k, b0_desc + 2 * k, idesc0, accum);
+              if (ncv1 > 0) umma_bf16_pair(tmem_base + DP_HALF, a_desc + 2 * k, b1_desc + 2 * k, idesc1, accum);
+            }
+            umma_commit_pair(empty_bar(stage));
+            if (++stage == DP_STAGES) { stage = 0; phase ^= 1u; }
+          }
+          if (!ok) break;
+          umma_commit_pair(tfull_bar);
+          tile_phase ^= 1u;
+        }
+      }
+    }
+  } else {
+    // ------------------------------------------------------------------ epilogue (warps 0-3 of both CTAs): lane = token
+    uint32_t tile_phase = 0;
+    bool ok = true;
+    const uint32_t tempty0 = map_to_cta(tempty_bar, 0);
+    const uint32_t sempty0[D_SCHED] = {map_to_cta(sempty_bar(0), 0), map_to_cta(sempty_bar(1), 0)};
+    const int r = 128 * (int)rank + warp * 32 + lane;               // this thread's token row of the tile
+    int q = 0;
+    uint32_t qphase = 0;
+    while (ok) {
+      ok = __all_sync(0xffffffffu, mbar_wait_cluster(sfull_bar(q), qphase, abort_flag));
+      if (!ok) break;
+      const int unit = sched_unit[q];
+      __syncwarp();
+      if (lane == 0) mbar_arrive_cluster(sempty0[q]);
+      if (++q == D_SCHED) { q = 0; qphase ^= 1u; }
+      if (unit < 0) break;
+      const DownUnit u = decode_down_unit(c, unit, n_dt, DP_TILE);
+      const int n_tiles = (u.rows + UMMA_TOK - 1) / UMMA_TOK;
+      const int ncv = min(DP_TILE, c.d_model - u.c0);
+      for (int tt = 0; ok && tt < n_tiles; ++tt) {
+        const int nv = (min(UMMA_TOK, u.rows - tt * UMMA_TOK) + 15) & ~15;
+        const int rt = tt * UMMA_TOK + r;
+        const bool store = r < nv && rt < u.row_limit;
+        float* const yrow = u.y + (size_t)(u.row0 + rt) * c.d_model + u.c0;
+        if (u.n_kb == 0) {   // an expert without micro-experts contributes zeros
+          if (store)
+            for (int j = 0; j < ncv; j += 4) *reinterpret_cast<float4*>(yrow + j) = make_float4(0.f, 0.f, 0.f, 0.f);
+          continue;
+        }
+        ok = __all_sync(0xffffffffu, mbar_wait(tfull_bar, tile_phase, abort_flag));
+        if (!ok) break;
+        tc_fence_after();
+        // the unit's output channels are consecutive accumulator columns (the first MMA fills 256 unless it is the last)
+        const uint32_t taddr = tmem_base + ((uint32_t)(warp * 32) << 16);
+        uint32_t v0[16], v1[16];
+        tmem_ld16(taddr, v0);
+        for (int c0 = 0; c0 < ncv; c0 += 32) {
+          tmem_ld_wait(v0);
+          if (c0 + 16 < ncv) tmem_ld16(taddr + c0 + 16, v1);
+          if (store) { st_global_v8(yrow + c0, v0); st_global_v8(yrow + c0 + 8, v0 + 8); }
+          if (c0 + 16 < ncv) {
+            tmem_ld_wait(v1);
+            if (c0 + 32 < ncv) tmem_ld16(taddr + c0 + 32, v0);
+            if (store) { st_global_v8(yrow + c0 + 16, v1); st_global_v8(yrow + c0 + 24, v1 + 8); }
+          }
+        }
+        tc_fence_before();
+        mbar_arrive_cluster(tempty0);
+        tile_phase ^= 1u;
+      }
+    }
+  }
+
+  tc_fence_before();
+  __syncthreads();
+  if (*abort_flag && tid == 0) atomicExch(&c.totals->status, (int)CAMERA_ERR_DEVICE_TIMEOUT);
+  cluster_sync_all();     // neither CTA leaves while the other may still read its shared or tensor memory
+  if (warp == 5) {
+    tc_fence_after();
+    asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(D_TMEM_COLS) : "memory");
   }
 }
 
@@ -447,7 +676,8 @@ int forward_impl(const camera_layer_t* L, const void* x, int64_t T, float alpha,
     if (energy == nullptr) a2.flags &= ~(uint32_t)CAMERA_SCORE_ACCUMULATE;
   }
   // the scores are sums and maxima over a micro-expert's tokens: they need the scoring orientation
-  const bool token_rows = energy == nullptr && forward_token_rows(L, T, a2.flags);
+  const bool long_lists = forward_token_rows(L, T, a2.flags);
+  const bool token_rows = energy == nullptr && long_lists;
   if (token_rows) a2.flags = (a2.flags & ~(uint32_t)CAMERA_SCORE_SINGLE_CTA) | CAMERA_SCORE_CTA_PAIR;
   ScoreFront f;
   int rc = score_front(L, x, T, alpha, energy, &a2, ws + fl.score, fl.score_bytes, st, &fb, &f);
@@ -468,7 +698,7 @@ int forward_impl(const camera_layer_t* L, const void* x, int64_t T, float alpha,
     if (!encode_bf16_2d_pitch(maps.data() + (size_t)128 * (2 * e), L->d_ff[e] > 0 ? L->w_down[e] : nullptr,
                               (uint64_t)L->d_model, (uint64_t)L->d_ff[e], (uint64_t)ld, D_TILE) ||
         !encode_bf16_2d_pitch(maps.data() + (size_t)128 * (2 * e + 1), h[e], rows_h, (uint64_t)fl.h_ld[e],
-                              (uint64_t)fl.h_ld[e], UMMA_TOK))
+                              (uint64_t)fl.h_ld[e], long_lists ? 128 : UMMA_TOK))
       return CAMERA_ERR_CUDA;
   }
   if (cudaMemcpyAsync(ws + fl.maps, maps.data(), maps.size(), cudaMemcpyHostToDevice, st) != cudaSuccess) {
@@ -483,12 +713,19 @@ int forward_impl(const camera_layer_t* L, const void* x, int64_t T, float alpha,
   int dev = 0, sms = 148;
   cudaGetDevice(&dev);
   cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
-  if (cudaFuncSetAttribute(k_down_umma, cudaFuncAttributeMaxDynamicSharedMemorySize, D_SMEM_BYTES) != cudaSuccess) {
-    cudaGetLastError();
-    return CAMERA_ERR_CUDA;
+  if (long_lists) {   // whole 256-token tiles cost little: CTA pairs, tokens on the accumulator rows
+    if (cudaFuncSetAttribute(k_down_umma_pair, cudaFuncAttributeMaxDynamicSharedMemorySize, DP_SMEM_BYTES) != cudaSuccess) {
+      cudaGetLastError();
+      return CAMERA_ERR_CUDA;
+    }
+    k_down_umma_pair<<<sms & ~1, D_THREADS, DP_SMEM_BYTES, st>>>(c, ws + fl.maps, (L->d_model + DP_TILE - 1) / DP_TILE);
+  } else {
+    if (cudaFuncSetAttribute(k_down_umma, cudaFuncAttributeMaxDynamicSharedMemorySize, D_SMEM_BYTES) != cudaSuccess) {
+      cudaGetLastError();
+      return CAMERA_ERR_CUDA;
+    }
+    k_down_umma<<<sms, D_THREADS, D_SMEM_BYTES, st>>>(c, ws + fl.maps, (L->d_model + D_TILE - 1) / D_TILE);
   }
-  const int n_dt = (L->d_model + D_TILE - 1) / D_TILE;
-  k_down_umma<<<sms, D_THREADS, D_SMEM_BYTES, st>>>(c, ws + fl.maps, n_dt);
   k_unpermute_sum<<<(unsigned)((T + 7) / 8), 256, 0, st>>>(c, y);
   return cudaGetLastError() == cudaSuccess ? CAMERA_OK : CAMERA_ERR_CUDA;
 }
