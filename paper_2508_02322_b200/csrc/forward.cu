@@ -251,13 +251,6 @@ constexpr int DP_B_BYTES = 128 * 128;             // this CTA's half of one W_do
 constexpr int DP_STAGE_BYTES = DP_A_BYTES + 2 * DP_B_BYTES;
 constexpr int DP_SMEM_BYTES = DP_STAGES * DP_STAGE_BYTES + 256 + 1024;
 
-// 32 bytes in one store (the address is 32-byte aligned).
-__device__ __forceinline__ void st_global_v8(void* p, const uint32_t* v) {
-  asm volatile("st.global.v8.b32 [%0], {%1,%2,%3,%4,%5,%6,%7,%8};" ::"l"(p), "r"(v[0]), "r"(v[1]), "r"(v[2]), "r"(v[3]),
-               "r"(v[4]), "r"(v[5]), "r"(v[6]), "r"(v[7])
-               : "memory");
-}
-
 __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(D_THREADS, 1)
     k_down_umma_pair(const ScoreCtx c, const void* maps_raw, int n_dt) {
   extern __shared__ uint8_t smem_raw[];
@@ -607,7 +600,7 @@ FwdLayout fwd_layout(const camera_layer_t* L, int64_t T) {
 }
 
 // Which gate/up kernel the layer forward runs.  With the tokens on the accumulator rows the epilogue is short (a
-// thread packs 16 micro-experts of its token into two 16-byte stores) but every token tile costs 256 rows, where the
+// thread packs 16 micro-experts of its token into one 32-byte store) but every token tile costs 256 rows, where the
 // scoring orientation trims a list's last tile to a multiple of 16 tokens; its stores of single bf16 values cost
 // about a tenth of the kernel.  Token lists are taken at their average length: the routing is not known here.
 bool forward_token_rows(const camera_layer_t* L, int64_t T, uint32_t flags) {

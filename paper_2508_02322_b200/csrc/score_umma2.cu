@@ -35,9 +35,8 @@ constexpr int P_STG_BYTES = 4 * FOLD_STG_BYTES;   // layer forward: where an epi
 constexpr int P_SMEM_BYTES = P_STAGES * P_STAGE_BYTES + P_WBUF_BYTES + P_STG_BYTES + 256 + 1024;
 
 // The layer-forward epilogue with a token on every accumulator row: h = a * SiLU(g) * u for 16 consecutive
-// micro-experts of the thread's token, rounded to bf16 and packed into 32 contiguous bytes.
-__device__ __forceinline__ void silu_mul16(const uint32_t* vg, const uint32_t* vu, float a, uint4& lo, uint4& hi) {
-  uint32_t p[8];
+// micro-experts of the thread's token, rounded to bf16 and packed into 32 contiguous bytes (one store).
+__device__ __forceinline__ void silu_mul16(const uint32_t* vg, const uint32_t* vu, float a, uint32_t* p) {
 #pragma unroll
   for (int j = 0; j < 16; j += 2) {
     const float g0 = __uint_as_float(vg[j]), g1 = __uint_as_float(vg[j + 1]);
@@ -46,8 +45,6 @@ __device__ __forceinline__ void silu_mul16(const uint32_t* vg, const uint32_t* v
     const __nv_bfloat162 b = __floats2bfloat162_rn(l0, l1);
     p[j >> 1] = *reinterpret_cast<const uint32_t*>(&b);
   }
-  lo = make_uint4(p[0], p[1], p[2], p[3]);
-  hi = make_uint4(p[4], p[5], p[6], p[7]);
 }
 
 // MODE 0: scoring (partial sums and maxima per micro-expert).  MODE 1: layer forward, h stored from the scoring
@@ -266,25 +263,19 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(P_THREADS, 1) k_scor
           if (!ok) break;
           tc_fence_after();
           uint32_t g0[16], u0[16], g1[16], u1[16];
-          uint4 lo, hi;
+          uint32_t pk[8];
           tmem_ld16(t_gate, g0);
           tmem_ld16(t_gate + H_TILE_CH, u0);
           for (int c0 = 0; c0 < ncv; c0 += 32) {
             tmem_ld_wait(g0, u0);
             if (c0 + 16 < ncv) { tmem_ld16(t_gate + c0 + 16, g1); tmem_ld16(t_gate + H_TILE_CH + c0 + 16, u1); }
-            silu_mul16(g0, u0, a, lo, hi);
-            if (store) {
-              *reinterpret_cast<uint4*>(hrow + c0) = lo;
-              *reinterpret_cast<uint4*>(hrow + c0 + 8) = hi;
-            }
+            silu_mul16(g0, u0, a, pk);
+            if (store) st_global_v8(hrow + c0, pk);
             if (c0 + 16 < ncv) {
               tmem_ld_wait(g1, u1);
               if (c0 + 32 < ncv) { tmem_ld16(t_gate + c0 + 32, g0); tmem_ld16(t_gate + H_TILE_CH + c0 + 32, u0); }
-              silu_mul16(g1, u1, a, lo, hi);
-              if (store) {
-                *reinterpret_cast<uint4*>(hrow + c0 + 16) = lo;
-                *reinterpret_cast<uint4*>(hrow + c0 + 24) = hi;
-              }
+              silu_mul16(g1, u1, a, pk);
+              if (store) st_global_v8(hrow + c0 + 16, pk);
             }
           }
           tc_fence_before();

@@ -130,6 +130,13 @@ __device__ __forceinline__ void tmem_ld_wait(uint32_t* a, uint32_t* b) {
                : "memory");
 }
 
+// 32 bytes in one store (the address is 32-byte aligned).
+__device__ __forceinline__ void st_global_v8(void* p, const uint32_t* v) {
+  asm volatile("st.global.v8.b32 [%0], {%1,%2,%3,%4,%5,%6,%7,%8};" ::"l"(p), "r"(v[0]), "r"(v[1]), "r"(v[2]), "r"(v[3]),
+               "r"(v[4]), "r"(v[5]), "r"(v[6]), "r"(v[7])
+               : "memory");
+}
+
 // Epilogue of the scoring orientation (a thread = a micro-expert, 16 tokens per call):
 // lambda = a_t * SiLU(g) * u; folds lambda^2 and |lambda| into s and m.
 // WRITE_H (layer forward): lambda also goes, as bf16, to h[token][micro-expert].  The 16 x 32 values of the warp are
