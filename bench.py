@@ -36,7 +36,7 @@ PAPER_CONTEXT = "paper: <5 min for the full Qwen2-57B-A14B analysis on one A100-
 LAUNCHES_PER_STEP = 8 + 9 * (len(PRUNE_RATIOS) + 1)
 # DRAM bytes (read + write) per gate/up flop of the scoring kernel, from the committed ncu capture of a
 # 1/8 slice of the layer whose traffic grows in proportion to the flop (profiles/k_score_umma_qwen2_slice.md).
-SCORE_KERNEL_DRAM_BYTES_PER_FLOP = 4.469e9 / 1.924e13
+SCORE_KERNEL_DRAM_BYTES_PER_FLOP = 4.483e9 / 1.924e13
 
 
 def shard_layers(n_layers: int, world: int, rank: int):
@@ -453,10 +453,12 @@ def main():
                 return f0.elapsed_time(f1) / reps
             full_ms = timed(lambda: P.camera_layer_forward(layer, xb, y=yb, workspace=ws_f))
             sl_ms = timed(lambda: P.camera_layer_forward(sliced, xb, y=yh, workspace=ws_f))
+            e_tmp = torch.empty(n_me, dtype=torch.float32, device=dev)
+            both_ms = timed(lambda: P.camera_score_forward_layer(layer, xb, ALPHA, energy=e_tmp, y=yb, workspace=ws_f))
             err = P.camera_output_error(yb, yh).cpu().tolist()
             flop_full = 1.5 * cfg.gate_up_flop * Tb / T
             forward = {"tokens": Tb, "full_layer_ms": full_ms, "full_layer_tflops": flop_full / (full_ms * 1e-3) / 1e12,
-                       "sliced_layer_ms": sl_ms, "prune_ratio": PRUNE_RATIOS[1],
+                       "sliced_layer_ms": sl_ms, "full_layer_and_scores_ms": both_ms, "prune_ratio": PRUNE_RATIOS[1],
                        "relative_output_error": err[0] / err[1] if err[1] > 0 else None, "mean_cosine": err[2]}
             del ws_f, yb, yh
         del outw
