@@ -53,7 +53,7 @@ def shard_tokens(n_tokens: int, world: int, rank: int):
 
 def reduce_components(phi2, phi_inf_sq, dist=None):
     """The one exchange of token-sharded scoring: column sums add over the shards, column maxima take the maximum
-    (Algorithm 1 lines 7-8).  In place; a no-op without a process group."""
+    (Algorithm 1's ColumnSum and ColumnMax).  In place; a no-op without a process group."""
     if dist is not None and dist.is_initialized() and dist.get_world_size() > 1:
         dist.all_reduce(phi2, op=dist.ReduceOp.SUM)
         dist.all_reduce(phi_inf_sq, op=dist.ReduceOp.MAX)
@@ -188,10 +188,10 @@ def run_reference(args):
 
 def run_stack(args):
     """--stack: Algorithm 2's layer loop on a synthetic stack of MoE layers.  Per layer: output of the layer on the
-    calibration tokens (line 6) and scores (line 8) from one pass over the gate/up weights
-    (camera_score_forward_layer), selection and slicing (lines 9-13), output of the sliced layer
-    (line 14), which -- added to the residual and rescaled to RMS 1, the stand-in for the rest of a decoder layer --
-    becomes the next layer's input (line 15).  Prints one JSON line of its own."""
+    calibration tokens and scores from one pass over the gate/up weights
+    (camera_score_forward_layer), selection and slicing, output of the sliced layer,
+    which -- added to the residual and rescaled to RMS 1, the stand-in for the rest of a decoder layer --
+    becomes the next layer's input ("I <- O").  Prints one JSON line of its own."""
     import torch
     import paper_2508_02322_b200 as P
     from paper_2508_02322_b200 import workloads as W
@@ -405,7 +405,7 @@ def main():
     value = world * T * args.steps / (ms * 1e-3)
     ms_per_step = ms / args.steps
 
-    # ---- the selection applied to the weights (Algorithm 2 lines 9-13), timed on its own after the step loop
+    # ---- the selection applied to the weights (Algorithm 2, TopSelect to the slicing), timed on its own after the step loop
     compact = forward = decode = None
     if not args.no_compact:
         off = P.expert_offsets_tensor(layer)

@@ -7,7 +7,7 @@
  * channel i of an expert: row i of W_gate and W_up plus column i of W_down
  * (paper Eq. 3).  Experts are ordered routed[0..n_routed) then
  * shared[0..n_shared); the global micro-expert index is off[e] + i with off the
- * prefix sum of d_ff (Algorithm 1 line 4, generalised to unequal d_ff).
+ * prefix sum of d_ff (Algorithm 1's global index, generalised to unequal d_ff).
  *
  * General rules
  *  - "DEVICE" pointers are CUDA device memory of the current device, "HOST"
@@ -70,7 +70,7 @@ enum {
                                       more than they save; CTA_PAIR / SINGLE_CTA force the scoring orientation */
   CAMERA_SCORE_ACCUMULATE = 4u     /* phi2 and phi_inf_sq (both required) already hold the result of earlier batches of
                                       calibration tokens of this layer; this call folds its batch in (the column sums of
-                                      Alg. 1 line 7 add up over batches, the column maxima of line 8 take the maximum)
+                                      Algorithm 1 add up over batches, the column maxima take the maximum)
                                       and writes the energy of all batches so far; the workspace's status word is
                                       not cleared by such a call, so one camera_read_status after the last batch
                                       reports trouble in any of them (use the same workspace for all batches) */
@@ -105,9 +105,9 @@ typedef struct {
 
 /* Optional inputs/outputs of camera_score_layer; any pointer may be NULL. All DEVICE. */
 typedef struct {
-  float* phi2;                  /* [N_e]  ||Phi_i||_2^2       (Alg. 1 line 7) */
-  float* phi_inf_sq;            /* [N_e]  ||Phi_i||_inf^2     (Alg. 1 line 8) */
-  float* omega2;                /* [N_e]  ||w_i||_2^2         (Alg. 1 line 5) */
+  float* phi2;                  /* [N_e]  ||Phi_i||_2^2       (Alg. 1, ColumnSum) */
+  float* phi_inf_sq;            /* [N_e]  ||Phi_i||_inf^2     (Alg. 1, ColumnMax) */
+  float* omega2;                /* [N_e]  ||w_i||_2^2         (Alg. 1, omega) */
   int32_t* topk_idx;            /* [T, top_k] chosen experts, by decreasing probability */
   float* topk_w;                /* [T, top_k] their coefficients A */
   const int32_t* topk_idx_in;   /* if both *_in are set the router is skipped and this routing is used */
@@ -125,12 +125,12 @@ int camera_version(void);
 size_t camera_score_workspace_bytes(const camera_layer_t* layer, int64_t n_tokens);
 
 /*
- * Algorithm 1 of the paper (micro-expert ranking) up to and including line 10:
- *   A      <- Top&Norm(softmax(R x))                               line 2
- *   omega2 <- ColumnSum(W_down * W_down)                           line 5
- *   Lambda <- A[:,e] * SiLU(W_gate X) * (W_up X)                   line 6  (never stored)
- *   phi2   <- ColumnSum(Lambda*Lambda), phi_inf <- ColumnMax|Lambda|^2   lines 7-8
- *   energy <- [(1-alpha) phi2 + alpha phi_inf] * omega2            line 10, Eq. 11
+ * Algorithm 1 of the paper (micro-expert ranking) up to and including the energies:
+ *   A      <- Top&Norm(softmax(R x))
+ *   omega2 <- ColumnSum(W_down * W_down)
+ *   Lambda <- A[:,e] * SiLU(W_gate X) * (W_up X)                   (never stored)
+ *   phi2   <- ColumnSum(Lambda*Lambda), phi_inf <- ColumnMax|Lambda|^2
+ *   energy <- [(1-alpha) phi2 + alpha phi_inf] * omega2            Eq. 11
  * x: DEVICE [n_tokens, d_model] row-major, dtype layer->dtype.  energy: DEVICE [N_e] fp32.
  * The calibration set may be fed in several calls (batches of tokens) with CAMERA_SCORE_ACCUMULATE.
  * Arithmetic: inputs as stored, products and sums in fp32 (bf16: tensor cores with fp32
@@ -151,7 +151,7 @@ int camera_read_status(const void* workspace, void* cuda_stream, int32_t* status
 size_t camera_select_workspace_bytes(int64_t n_total, int32_t n_segments, int32_t n_levels);
 
 /*
- * CAMERA-P selection (Algorithm 2 line 9, S <- TopSelect(R, 1 - lambda)), for one or many
+ * CAMERA-P selection (Algorithm 2, S <- TopSelect(R, 1 - lambda)), for one or many
  * layers at once.  energy: DEVICE [n_total] fp32, non-negative.  seg_offsets: HOST
  * [n_segments+1] increasing, seg_offsets[0] = 0, last = n_total; one segment = one layer.  In
  * every segment of n elements the floor(prune_ratio * n + 1e-9) lowest-energy micro-experts get
@@ -166,7 +166,7 @@ int camera_select_prune(const float* energy, const int64_t* seg_offsets, int32_t
                         void* workspace, size_t workspace_bytes, void* cuda_stream);
 
 /*
- * CAMERA-Q class split (Algorithm 3 lines 5-8: ListSplitByRatio + GetSubIndex).  ratios: HOST
+ * CAMERA-Q class split (Algorithm 3: ListSplitByRatio + GetSubIndex).  ratios: HOST
  * [n_levels] (2..8 levels), most important class first, summing to 1; bits: HOST [n_levels]
  * bit-widths 0..255.  Within a segment of n elements ranked from highest to lowest energy
  * (equal energies: higher index first), class j takes ranks [c_{j-1}, c_j) with
@@ -204,7 +204,7 @@ int camera_select_prune_static(const float* energy, const int64_t* seg_offsets, 
                                void* cuda_stream);
 
 /*
- * GetSubIndex (Algorithm 3 line 8; the per-expert retained sets S of Algorithm 2 lines 9-10).
+ * GetSubIndex (Algorithm 3; the per-expert retained sets S of Algorithm 2).
  * labels: DEVICE [N_e] uint8, one per micro-expert -- a keep mask of camera_select_prune, or the
  * bits_out of camera_alloc_bits.  expert_offsets: DEVICE int64 [n_experts+1], global micro-expert
  * offsets.  label_order: HOST [n_labels] (1..8 distinct values 0..255).  For every expert e the
@@ -224,7 +224,7 @@ int camera_sub_index(const uint8_t* labels, const int64_t* expert_offsets, int32
 size_t camera_compact_workspace_bytes(int32_t n_experts);
 
 /*
- * Algorithm 2 lines 11-13: W_up <- W_up[S,:], W_gate <- W_gate[S,:], W_down <- W_down[:,S], with S
+ * The slicing step of Algorithm 2: W_up <- W_up[S,:], W_gate <- W_gate[S,:], W_down <- W_down[:,S], with S
  * the first m_e = counts[e,0] + .. + counts[e,n_take-1] entries of expert e's list in sub_index
  * (both as written by camera_sub_index; DEVICE).  w_gate_out / w_up_out / w_down_out: HOST arrays
  * of DEVICE pointers, one per expert, 16-byte aligned, with room for the worst case the caller
@@ -258,7 +258,7 @@ int camera_layer_forward(const camera_layer_t* layer, const void* x, int64_t n_t
                          const camera_score_aux_t* aux, void* workspace, size_t workspace_bytes, void* cuda_stream);
 
 /*
- * Lines 6 and 8 of Algorithm 2 on one batch of tokens, from one pass over W_gate and W_up: the energies of
+ * The layer-output step and the scoring step of Algorithm 2's loop on one batch of tokens, from one pass over W_gate and W_up: the energies of
  * camera_score_layer (Algorithm 1: same alpha, energy, aux fields and flags, CAMERA_SCORE_ACCUMULATE included) and the
  * layer output y of camera_layer_forward (Eq. 1-2).  The gate/up GEMM runs once, in the scoring orientation; its
  * epilogue folds lambda into the per-micro-expert sums and maxima and stores it as h for the W_down GEMM.  The
@@ -282,7 +282,7 @@ int camera_output_error(const float* y, const float* y_hat, int64_t n_tokens, in
                         void* workspace, size_t workspace_bytes, void* cuda_stream);
 
 /*
- * Glue for running Algorithm 2's layer loop ("I <- O", line 15) on a synthetic stack of MoE layers, where no
+ * Glue for running Algorithm 2's layer loop ("I <- O") on a synthetic stack of MoE layers, where no
  * attention block or trained norm exists (the paper has no counterpart: its layers are whole decoder layers):
  * out_t = (x_t + y_t) / sqrt(mean((x_t + y_t)^2) + eps), rounded to the dtype of x.  x: DEVICE [n_tokens, d_model]
  * bf16 (CAMERA_BF16) or fp32, y: DEVICE fp32 (a layer output), out: DEVICE like x (may be x itself).  d_model % 8 == 0.

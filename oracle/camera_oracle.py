@@ -14,7 +14,7 @@ Conventions (paper, Section "From Expert to Micro-Expert"):
     column i of W_down                                                   (Eq. 3);
   * experts are ordered routed[0..n_routed) then shared[0..n_shared); the
     global micro-expert index is offset[e] + i with offset the prefix sum of
-    the experts' d_ff (Algorithm 1 line 4, generalised to unequal d_ff).
+    the experts' d_ff (Algorithm 1's global index, generalised to unequal d_ff).
 
 Every input array is float64 and holds the *storage-rounded* values (a bf16
 tensor widened exactly), so the only difference to the CUDA path is the
@@ -89,12 +89,12 @@ def silu(g: np.ndarray) -> np.ndarray:
 
 
 def me_offsets(layer: OracleLayer) -> np.ndarray:
-    """Start of each expert's micro-experts in the global index (Alg. 1 line 4)."""
+    """Start of each expert's micro-experts in the global index (the global index of Alg. 1)."""
     return np.concatenate([[0], np.cumsum(layer.d_ff)]).astype(np.int64)
 
 
 # ----------------------------------------------------------------------------
-# Router: A <- Top&Norm(R X)                                   (Alg. 1 line 2)
+# Router: A <- Top&Norm(R X)                                   (Alg. 1, Top&Norm)
 # ----------------------------------------------------------------------------
 def router_probs(layer: OracleLayer, X: np.ndarray) -> np.ndarray:
     """softmax over the routed experts of z = X R^T (+ bias); shape [T, n_routed]."""
@@ -184,16 +184,16 @@ def basis(layer: OracleLayer) -> np.ndarray:
 # Algorithm 1: phi^2, phi^inf, omega^2 and the energy (Eq. 11)
 # ----------------------------------------------------------------------------
 def camera_components_dense(layer: OracleLayer, X: np.ndarray):
-    """Algorithm 1 lines 1-9 taken literally: Lambda is formed over *all* n
+    """Algorithm 1 up to the components, taken literally: Lambda is formed over *all* n
     tokens with the dense column A[:, e].  Returns (phi2, phi_inf_sq, omega2),
     each of length N_e."""
     A = coefficients(layer, X)
     phi2, phi_inf, omega2 = [], [], []
     for e in range(layer.n_experts):
-        omega2.append((layer.w_down[e] * layer.w_down[e]).sum(axis=0))        # line 5
-        Lam = A[:, e:e + 1] * expert_hidden(X, layer.w_gate[e], layer.w_up[e])  # line 6
-        phi2.append((Lam * Lam).sum(axis=0))                                   # line 7
-        phi_inf.append(np.abs(Lam).max(axis=0) ** 2 if Lam.shape[0] else np.zeros(Lam.shape[1]))  # line 8
+        omega2.append((layer.w_down[e] * layer.w_down[e]).sum(axis=0))        # omega
+        Lam = A[:, e:e + 1] * expert_hidden(X, layer.w_gate[e], layer.w_up[e])  # Lambda
+        phi2.append((Lam * Lam).sum(axis=0))                                   # ColumnSum
+        phi_inf.append(np.abs(Lam).max(axis=0) ** 2 if Lam.shape[0] else np.zeros(Lam.shape[1]))  # ColumnMax
     return np.concatenate(phi2), np.concatenate(phi_inf), np.concatenate(omega2)
 
 
@@ -247,18 +247,18 @@ def camera_components(layer: OracleLayer, X: np.ndarray,
 
 
 def energy(phi2: np.ndarray, phi_inf_sq: np.ndarray, omega2: np.ndarray, alpha: float) -> np.ndarray:
-    """E_i = [(1 - alpha) ||Phi_i||_2^2 + alpha ||Phi_i||_inf^2] ||w_i||_2^2   (Eq. 11, Alg. 1 line 10)."""
+    """E_i = [(1 - alpha) ||Phi_i||_2^2 + alpha ||Phi_i||_inf^2] ||w_i||_2^2   (Eq. 11, the energy step of Alg. 1)."""
     return ((1.0 - alpha) * phi2 + alpha * phi_inf_sq) * omega2
 
 
 def camera_rank(E: np.ndarray) -> np.ndarray:
-    """Alg. 1 line 11: all micro-experts from least to most important
+    """The Argsort step of Alg. 1: all micro-experts from least to most important
     (energy ascending, lower index first among equal energies)."""
     return np.argsort(E, kind="stable")
 
 
 # ----------------------------------------------------------------------------
-# Selection: CAMERA-P keep mask (Alg. 2 line 9), CAMERA-Q classes (Alg. 3 l. 5-8)
+# Selection: CAMERA-P keep mask (Alg. 2, TopSelect), CAMERA-Q classes (Alg. 3, ListSplitByRatio / GetSubIndex)
 # ----------------------------------------------------------------------------
 def _floor_count(ratio: float, n: int) -> int:
     return int(math.floor(ratio * float(n) + 1e-9))
@@ -315,7 +315,7 @@ def sub_index(cls_or_mask: np.ndarray, offsets: np.ndarray, n_classes: int) -> n
 
 
 def sub_index_lists(labels: np.ndarray, offsets: np.ndarray, order: Sequence[int]):
-    """GetSubIndex (Algorithm 3 line 8; the per-expert retained sets of Algorithm 2 lines 9-10).
+    """GetSubIndex (Algorithm 3; the per-expert retained sets of Algorithm 2).
 
     For every expert, its micro-experts (channel numbers inside the expert)
     listed label by label in the given `order` of label values, ascending
@@ -338,7 +338,7 @@ def sub_index_lists(labels: np.ndarray, offsets: np.ndarray, order: Sequence[int
 
 
 def slice_layer(layer: OracleLayer, lists: Sequence[np.ndarray]) -> OracleLayer:
-    """Algorithm 2 lines 11-13: W_up <- W_up[S,:], W_gate <- W_gate[S,:],
+    """The slicing step of Algorithm 2: W_up <- W_up[S,:], W_gate <- W_gate[S,:],
     W_down <- W_down[:,S] for every expert, S given as channel lists (any
     order; a permutation of all channels merely reorders the micro-experts)."""
     return OracleLayer(
@@ -354,7 +354,7 @@ def next_layer_input(X: np.ndarray, Y: np.ndarray, eps: float = 1e-6) -> np.ndar
     """Glue of the synthetic multi-layer stack (NO counterpart in the paper, whose
     layers are whole decoder layers of a trained model): the next layer's input
     is the residual sum x + y of a token, rescaled to root-mean-square 1.  It
-    stands in for "I <- O" of Algorithm 2 line 15 where no attention block,
+    stands in for "I <- O" of Algorithm 2 where no attention block,
     norm weights or trained model exist."""
     Z = X + Y
     return Z / np.sqrt((Z * Z).mean(axis=1, keepdims=True) + eps)

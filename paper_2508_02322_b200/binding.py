@@ -386,7 +386,7 @@ def camera_sub_index(labels: torch.Tensor, expert_offsets: torch.Tensor, label_o
 def camera_compact_weights(layer: Layer, sub_index: torch.Tensor, counts: torch.Tensor, n_take: int, *,
                            out: Optional[Dict[str, List[torch.Tensor]]] = None, down_ld: Optional[Sequence[int]] = None,
                            workspace: Optional[torch.Tensor] = None, stream: Optional[torch.cuda.Stream] = None):
-    """Gathers W_gate[S,:], W_up[S,:], W_down[:,S] (Algorithm 2 lines 11-13) with S the entries of the first n_take
+    """Gathers W_gate[S,:], W_up[S,:], W_down[:,S] (Algorithm 2, the slicing step) with S the entries of the first n_take
     labels of every expert's list.  `out` = {"w_gate": [...], "w_up": [...], "w_down": [...]} (per expert, sized
     like the sources unless down_ld says otherwise); allocated when missing.  Returns `out`; the rows / columns
     actually written per expert are counts[:, :n_take].sum(1)."""

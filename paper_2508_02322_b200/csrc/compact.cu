@@ -1,6 +1,6 @@
-// Applying a selection to the weights: the per-expert index lists (GetSubIndex, Algorithm 3 line 8;
-// the retained sets of Algorithm 2 lines 9-10) and the gathers W_up[S,:], W_gate[S,:], W_down[:,S]
-// (Algorithm 2 lines 11-13).  Pure data movement: every kernel is bound by HBM bandwidth.
+// Applying a selection to the weights: the per-expert index lists (GetSubIndex, Algorithm 3;
+// the retained sets of Algorithm 2) and the gathers W_up[S,:], W_gate[S,:], W_down[:,S]
+// (Algorithm 2, the slicing step).  Pure data movement: every kernel is bound by HBM bandwidth.
 #include <string.h>
 
 #include <vector>

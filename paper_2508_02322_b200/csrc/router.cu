@@ -1,4 +1,4 @@
-// Router (Algorithm 1 line 2: A <- Top&Norm(R X)), the stable counting sort of (token, expert)
+// Router (Algorithm 1: A <- Top&Norm(R X)), the stable counting sort of (token, expert)
 // pairs by expert, and the token permutation that lays every expert's tokens out contiguously.
 #include "common.cuh"
 

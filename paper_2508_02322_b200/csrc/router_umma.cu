@@ -1,4 +1,4 @@
-// Tensor-core router for bf16 layers (Algorithm 1 line 2: A <- Top&Norm(R X)).
+// Tensor-core router for bf16 layers (Algorithm 1: A <- Top&Norm(R X)).
 //
 // The logit GEMM z = X W_r^T (plus the gate logits of sigmoid-gated shared experts) runs on
 // tcgen05 with tokens on the 128 TMEM lanes and experts on the columns, so X is streamed from HBM

@@ -1,4 +1,4 @@
-// omega^2_i = ||w_i||_2^2 over the W_down of every expert (Algorithm 1 line 5).  Pure HBM stream:
+// omega^2_i = ||w_i||_2^2 over the W_down of every expert (Algorithm 1, the ColumnSum of W_down * W_down).  Pure HBM stream:
 // every element of W_down is read exactly once with 16-byte loads, sums in fp32.
 #include "common.cuh"
 

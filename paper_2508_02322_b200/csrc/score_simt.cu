@@ -1,5 +1,5 @@
-// fp32-FMA scoring kernel (Algorithm 1 lines 6-8 with Lambda kept in registers) and the final
-// combine (line 10, Eq. 11).  This kernel serves fp32 layers and shapes the tensor-core kernel
+// fp32-FMA scoring kernel (Algorithm 1's Lambda, ColumnSum and ColumnMax steps with Lambda kept in registers) and the final
+// combine (the energy step, Eq. 11).  This kernel serves fp32 layers and shapes the tensor-core kernel
 // does not take; it uses the same work units and partial layout as the tensor-core kernel.
 #include "common.cuh"
 

@@ -1,4 +1,4 @@
-// Tensor-core scoring kernel for bf16 layers (Algorithm 1 lines 6-8):
+// Tensor-core scoring kernel for bf16 layers (Algorithm 1: Lambda, ColumnSum, ColumnMax):
 //   Lambda = A[:,e] * SiLU(W_gate X) * (W_up X) is formed tile by tile in tensor memory and reduced
 //   to per-micro-expert sum(Lambda^2) and max|Lambda| in the epilogue; it never reaches HBM.
 //

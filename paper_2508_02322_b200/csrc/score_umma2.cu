@@ -1,4 +1,4 @@
-// Tensor-core scoring kernel for bf16 layers on CTA pairs (Algorithm 1 lines 6-8).
+// Tensor-core scoring kernel for bf16 layers on CTA pairs (Algorithm 1: Lambda, ColumnSum, ColumnMax).
 //
 // Same computation and the same epilogue as k_score_umma, but two CTAs on neighbouring SMs share one
 // MMA (tcgen05 cta_group::2): the pair handles 256 micro-experts x 256 tokens, each CTA keeps the

@@ -1,5 +1,5 @@
-// Device-wide segmented rank selection for CAMERA-P (Algorithm 2 line 9, TopSelect) and CAMERA-Q
-// (Algorithm 3 lines 5-8, ListSplitByRatio / GetSubIndex).
+// Device-wide segmented rank selection for CAMERA-P (Algorithm 2, TopSelect) and CAMERA-Q
+// (Algorithm 3, ListSplitByRatio / GetSubIndex).
 //
 // Every micro-expert gets the 64-bit key (order-preserving image of its fp32 energy) << 32 | index
 // within its segment.  Keys are unique, so "the r-th smallest key" is unambiguous and equal

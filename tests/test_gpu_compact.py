@@ -1,5 +1,4 @@
-"""GPU parity of the selection's application to the weights: GetSubIndex (Algorithm 3 line 8, Algorithm 2
-lines 9-10) and the gathers W_up[S,:], W_gate[S,:], W_down[:,S] (Algorithm 2 lines 11-13), bit for bit against
+"""GPU parity of the selection's application to the weights: GetSubIndex (Algorithm 3, Algorithm 2) and the gathers W_up[S,:], W_gate[S,:], W_down[:,S] (Algorithm 2, the slicing step), bit for bit against
 the oracle's index lists and slices."""
 import numpy as np
 import pytest

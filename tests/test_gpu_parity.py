@@ -262,7 +262,7 @@ def test_analyze_layer_host(P):
 # ------------------------------------------------------------------ the calibration set fed in batches
 @pytest.mark.parametrize("kernel", ["umma", "simt"])
 def test_accumulate_over_token_batches(P, kernel):
-    """Column sums add up and column maxima take the maximum over batches of tokens (Algorithm 1 lines 7-8):
+    """Column sums add up and column maxima take the maximum over batches of tokens (Algorithm 1's ColumnSum and ColumnMax):
     three uneven batches must give the scores of the whole set."""
     cfg = small_cfg(n_tokens=2500)
     L = W().make_layer(cfg, seed=14, device=DEV)

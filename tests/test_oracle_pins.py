@@ -37,7 +37,7 @@ def test_silu_closed_forms_and_library():
     assert np.allclose(s, ref, rtol=1e-14, atol=1e-300)
 
 
-# ---------------------------------------------------------------- router (Alg. 1 line 2)
+# ---------------------------------------------------------------- router (Alg. 1, Top&Norm)
 @pytest.mark.parametrize("norm", [True, False])
 def test_router_against_library_softmax_topk(norm):
     r = rng(1)
@@ -374,9 +374,9 @@ def test_float32_rerun_within_tolerance():
     assert np.abs(s32 / s64 - 1).max() < 1e-4 and np.abs(m32 / m64 - 1).max() < 1e-4
 
 
-# ---------------------------------------------------------------- GetSubIndex and weight slicing (Alg. 2 lines 9-13, Alg. 3 line 8)
+# ---------------------------------------------------------------- GetSubIndex and weight slicing (Alg. 2, Alg. 3)
 def test_sliced_layer_decodes_like_the_retained_micro_experts():
-    """Slicing W_up[S,:], W_gate[S,:], W_down[:,S] (Alg. 2 lines 11-13) must give the layer whose output is
+    """Slicing W_up[S,:], W_gate[S,:], W_down[:,S] (Alg. 2, the slicing step) must give the layer whose output is
     Phi[:,S] W[S,:], the Y-hat of Eq. 7 -- computed here from the full Phi and W, never from the slices."""
     r = rng(40)
     layer = random_layer(r, d=7, d_ff=(5, 4, 6, 3), n_shared=1, top_k=2, shared_gate=True, bias=True)
