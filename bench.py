@@ -189,7 +189,9 @@ def run_reference(args):
 def run_stack(args):
     """--stack: Algorithm 2's layer loop on a synthetic stack of MoE layers.  Per layer: output of the layer on the
     calibration tokens and scores from one pass over the gate/up weights
-    (camera_score_forward_layer), selection and slicing, output of the sliced layer,
+    (camera_score_forward_layer; every batch keeps its workspace, so Phi stays in HBM as h), selection and slicing,
+    output of the retained micro-experts from the stored h and W_down with the pruned columns zeroed
+    (camera_pruned_output: Phi[:,S] W[S,:] of Eq. 7 without a second pass over the gate/up weights),
     which -- added to the residual and rescaled to RMS 1, the stand-in for the rest of a decoder layer --
     becomes the next layer's input ("I <- O").  Prints one JSON line of its own."""
     import torch
@@ -210,7 +212,8 @@ def run_stack(args):
     Yh = torch.empty_like(Y)
     probe = P.Layer.from_workload(W.make_layer(W.scaled(cfg, n_tokens=B), seed=0, layer_id=0, device=dev))
     n_me = probe.n_me
-    ws_f = P.alloc_workspace(P.camera_forward_workspace_bytes(probe, B), dev)
+    ws_f = [P.alloc_workspace(P.camera_forward_workspace_bytes(probe, B), dev) for _ in spans]
+    w_masked = [torch.empty_like(w) for w in probe.tensors["w_down"]]
     ws_sel = P.alloc_workspace(P.camera_select_workspace_bytes(n_me, 1, 2), dev)
     ws_c = P.alloc_workspace(4096 + 64 * probe.n_experts, dev)
     energy = torch.empty(n_me, dtype=torch.float32, device=dev)
@@ -219,7 +222,7 @@ def run_stack(args):
     outw = {k: [torch.empty_like(w) for w in probe.tensors[k]] for k in ("w_gate", "w_up", "w_down")}
     del probe
     stream = torch.cuda.current_stream()
-    names = ("forward_and_score", "select_slice", "forward_sliced", "error_next_input")
+    names = ("forward_and_score", "select_slice", "pruned_output", "error_next_input")
     tot = {k: 0.0 for k in names}
     errors = []
     for l in range(n_layers):
@@ -230,35 +233,32 @@ def run_stack(args):
         ev = [torch.cuda.Event(enable_timing=True) for _ in range(len(names) + 1)]
         ev[0].record(stream)
         for i, (t0, t1) in enumerate(spans):
-            P.camera_score_forward_layer(layer, X[t0:t1], ALPHA, energy=energy, y=Y[t0:t1], workspace=ws_f, phi2=phi2,
+            P.camera_score_forward_layer(layer, X[t0:t1], ALPHA, energy=energy, y=Y[t0:t1], workspace=ws_f[i], phi2=phi2,
                                          phi_inf_sq=phi_inf, accumulate=i > 0)
         ev[1].record(stream)
         P.camera_select_prune(energy, ratio, workspace=ws_sel, keep_mask=keep)
         sub, counts = P.camera_sub_index(keep, off, [1])
         P.camera_compact_weights(layer, sub, counts, 1, out=outw, workspace=ws_c)
-        m = counts[:, 0].cpu().tolist()                               # the sliced layer's shape: the one host read
-        sliced = P.Layer(L["w_router"], [outw["w_gate"][e][:m[e]] for e in range(layer.n_experts)],
-                         [outw["w_up"][e][:m[e]] for e in range(layer.n_experts)], outw["w_down"], cfg.top_k, cfg.n_shared,
-                         L["router_bias"], L["w_shared_gate"], cfg.norm_topk, "hf", down_ld=layer.d_ff)
         ev[2].record(stream)
-        for t0, t1 in spans:
-            P.camera_layer_forward(sliced, X[t0:t1], y=Yh[t0:t1], workspace=ws_f)
+        P.camera_mask_down_columns(layer, keep, out=w_masked)
+        for i, (t0, t1) in enumerate(spans):
+            P.camera_pruned_output(layer, w_masked, t1 - t0, ws_f[i], y=Yh[t0:t1])
         ev[3].record(stream)
         err = P.camera_output_error(Y, Yh)
         P.camera_residual_norm(X, Yh, out=X)
         ev[4].record(stream)
         torch.cuda.synchronize()
-        if P.camera_read_status(ws_f) != 0:
+        if any(P.camera_read_status(w) != 0 for w in ws_f):
             raise RuntimeError("device status set in the stack run")
         for i, k in enumerate(names):
             tot[k] += ev[i].elapsed_time(ev[i + 1])
         e = err.cpu().tolist()
         errors.append(e[0] / e[1] if e[1] > 0 else 0.0)
-        del L, layer, sliced
+        del L, layer
     total_s = sum(tot.values()) * 1e-3
     print(json.dumps({
         "mode": "stack", "what": "Algorithm 2 over a synthetic stack of MoE layers (layer outputs, CAMERA scores, prune, slice, "
-                                 "sliced-layer outputs fed to the next layer)",
+                                 "retained micro-experts' outputs fed to the next layer)",
         "config": {"workload": f"{cfg.name} x {n_layers} layers", "tokens": T, "prune_ratio": ratio, "alpha": ALPHA},
         "seconds": total_s, "tokens_per_s_per_layer": T * n_layers / total_s,
         "ms_per_layer": {k: v / n_layers for k, v in tot.items()},

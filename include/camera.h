@@ -270,6 +270,28 @@ int camera_score_forward_layer(const camera_layer_t* layer, const void* x, int64
                                float* y, const camera_score_aux_t* aux, void* workspace, size_t workspace_bytes,
                                void* cuda_stream);
 
+/*
+ * The retained micro-experts' output Y_hat = Phi[:,S] W[S,:] (Eq. 7) without running the pruned layer again.  After
+ * camera_score_forward_layer or camera_layer_forward the workspace still holds Phi as h (bf16) and the token lists;
+ * once the selection S is known, Y_hat is h times W_down with the columns outside S set to zero: the W_down GEMM alone,
+ * a third of the pruned layer's flops.  (The paper's loop, Algorithm 2, runs the pruned layer on the same input.)
+ *
+ * camera_mask_down_columns: w_down_out[e][r, i] = keep_mask[offset_e + i] ? w_down[e][r, i] : 0.  keep_mask: DEVICE
+ * uint8 [N_e], 8-byte aligned (the mask of camera_select_prune); w_down_out: HOST array [n_experts] of DEVICE pointers
+ * to buffers of the shape and pitch of the layer's W_down (not the layer's own).  bf16 layers in CAMERA_DOWN_HF
+ * layout with d_ff[e] % 8 == 0, else CAMERA_ERR_UNSUPPORTED_SHAPE.
+ *
+ * camera_pruned_output: y_hat [n_tokens, d_model] fp32 from the h of the last forward call on this workspace.  layer,
+ * n_tokens and aux->topk_idx (if that call exported the routing through it) must be those of that call, and nothing
+ * else may have used the workspace since; w_down_masked as written by camera_mask_down_columns (any matrices of that
+ * shape work: the call multiplies h by what it is given).  Other arguments and errors as for camera_layer_forward.
+ * The result equals camera_layer_forward on the sliced layer up to the order of the fp32 sums over d_ff.
+ */
+int camera_mask_down_columns(const camera_layer_t* layer, const uint8_t* keep_mask, void* const* w_down_out,
+                             void* cuda_stream);
+int camera_pruned_output(const camera_layer_t* layer, const void* const* w_down_masked, int64_t n_tokens, float* y_hat,
+                         const camera_score_aux_t* aux, void* workspace, size_t workspace_bytes, void* cuda_stream);
+
 /* Scratch for camera_output_error. */
 size_t camera_output_error_workspace_bytes(int64_t n_tokens);
 

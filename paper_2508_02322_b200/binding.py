@@ -89,6 +89,11 @@ def _load() -> C.CDLL:
     lib.camera_score_forward_layer.argtypes = [C.POINTER(camera_layer_t), C.c_void_p, C.c_int64, C.c_float, C.c_void_p,
                                                C.c_void_p, C.POINTER(camera_score_aux_t), C.c_void_p, C.c_size_t,
                                                C.c_void_p]
+    lib.camera_mask_down_columns.restype = C.c_int
+    lib.camera_mask_down_columns.argtypes = [C.POINTER(camera_layer_t), C.c_void_p, C.POINTER(C.c_void_p), C.c_void_p]
+    lib.camera_pruned_output.restype = C.c_int
+    lib.camera_pruned_output.argtypes = [C.POINTER(camera_layer_t), C.POINTER(C.c_void_p), C.c_int64, C.c_void_p,
+                                         C.POINTER(camera_score_aux_t), C.c_void_p, C.c_size_t, C.c_void_p]
     lib.camera_output_error_workspace_bytes.restype = C.c_size_t
     lib.camera_output_error_workspace_bytes.argtypes = [C.c_int64]
     lib.camera_output_error.restype = C.c_int
@@ -476,6 +481,29 @@ def camera_score_forward_layer(layer: Layer, x: torch.Tensor, alpha: float, *, e
                                           C.byref(aux), workspace.data_ptr(), workspace.numel(), _stream_ptr(stream)),
            "camera_score_forward_layer")
     return energy, y
+
+
+def camera_mask_down_columns(layer: Layer, keep: torch.Tensor, *, out=None, stream: Optional[torch.cuda.Stream] = None):
+    """W_down of every expert with the columns of the micro-experts outside the selection set to zero.
+    keep: uint8 [N_e] on the device; out: list of tensors shaped like the layer's W_down (allocated if None)."""
+    if out is None:
+        out = [torch.empty_like(w) for w in layer.tensors["w_down"]]
+    ptrs = (C.c_void_p * layer.n_experts)(*[t.data_ptr() for t in out])
+    _check(lib.camera_mask_down_columns(C.byref(layer.c), keep.data_ptr(), ptrs, _stream_ptr(stream)),
+           "camera_mask_down_columns")
+    return out
+
+
+def camera_pruned_output(layer: Layer, w_down_masked, n_tokens: int, workspace: torch.Tensor, *,
+                         y: Optional[torch.Tensor] = None, stream: Optional[torch.cuda.Stream] = None) -> torch.Tensor:
+    """Y_hat = Phi[:,S] W[S,:] (Eq. 7) from the h that the last camera_score_forward_layer / camera_layer_forward
+    call left in `workspace` (same layer, same number of tokens) and W_down with the pruned columns zeroed."""
+    if y is None:
+        y = torch.empty((n_tokens, layer.d_model), dtype=torch.float32, device=workspace.device)
+    ptrs = (C.c_void_p * layer.n_experts)(*[t.data_ptr() for t in w_down_masked])
+    _check(lib.camera_pruned_output(C.byref(layer.c), ptrs, int(n_tokens), y.data_ptr(), None, workspace.data_ptr(),
+                                    workspace.numel(), _stream_ptr(stream)), "camera_pruned_output")
+    return y
 
 
 def camera_output_error(y: torch.Tensor, y_hat: torch.Tensor, *, stream: Optional[torch.cuda.Stream] = None) -> torch.Tensor:

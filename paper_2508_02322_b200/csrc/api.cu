@@ -179,7 +179,8 @@ int score_front(const camera_layer_t* L, const void* x, int64_t T, float alpha, 
                 const ForwardBuffers* fwd, ScoreFront* out) {
   int rc = validate_layer(L, T, fwd != nullptr);
   if (rc != CAMERA_OK) return rc;
-  if (!(alpha >= 0.f && alpha <= 1.f) || (energy == nullptr && fwd == nullptr) || (T > 0 && x == nullptr))
+  const bool reuse = fwd != nullptr && fwd->reuse;
+  if (!(alpha >= 0.f && alpha <= 1.f) || (energy == nullptr && fwd == nullptr) || (T > 0 && x == nullptr && !reuse))
     return CAMERA_ERR_INVALID_ARG;
   if (aux && ((aux->topk_idx_in == nullptr) != (aux->topk_w_in == nullptr))) return CAMERA_ERR_INVALID_ARG;
   const bool accumulate = aux && (aux->flags & CAMERA_SCORE_ACCUMULATE);
@@ -231,6 +232,13 @@ int score_front(const camera_layer_t* L, const void* x, int64_t T, float alpha, 
   c.omega2 = (aux && aux->omega2) ? aux->omega2 : reinterpret_cast<float*>(ws + lay.omega2);
   c.energy = energy;
   c.tensor_maps = ws + lay.tensor_maps;
+
+  if (reuse) {   // the tables, token lists and h are those of the earlier call on this workspace
+    out->norm_blocks = 0;
+    out->use_umma = umma_shape_ok(L);
+    out->use_pair = false;
+    return CAMERA_OK;
+  }
 
   // host-known tables
   std::vector<ExpertStatic> est(E);

@@ -102,6 +102,7 @@ struct ForwardBuffers {
   void* const* h;
   const int32_t* h_ld;
   float* const* y_part;
+  bool reuse;   // only rebuild the context: the workspace still holds the lists, tables and h of an earlier call
 };
 struct ScoreFront {
   ScoreCtx c;

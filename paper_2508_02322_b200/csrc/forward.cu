@@ -634,61 +634,17 @@ extern "C" size_t camera_forward_workspace_bytes(const camera_layer_t* layer, in
 namespace camera {
 namespace {
 
-// The layer output, and with `energy` also the scores, from one pass over W_gate and W_up.
-int forward_impl(const camera_layer_t* L, const void* x, int64_t T, float alpha, float* energy, float* y,
-                 const camera_score_aux_t* aux, void* workspace, size_t workspace_bytes, void* cuda_stream) {
-  if (L == nullptr || (y == nullptr && T > 0) || (reinterpret_cast<uintptr_t>(y) & 15)) return CAMERA_ERR_INVALID_ARG;
-  if (score_workspace_bytes_any(L, T, true) == 0) return CAMERA_ERR_INVALID_ARG;
-  if (L->dtype != CAMERA_BF16 || L->down_layout != CAMERA_DOWN_HF || L->d_model % UMMA_BK != 0 || !umma_shape_ok(L) ||
-      (reinterpret_cast<uintptr_t>(x) & 15))
-    return CAMERA_ERR_UNSUPPORTED_SHAPE;
-  const FwdLayout fl = fwd_layout(L, T);
-  if (workspace == nullptr || workspace_bytes < fl.total || (reinterpret_cast<uintptr_t>(workspace) & 255))
-    return CAMERA_ERR_WORKSPACE;
-  cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
-  char* ws = static_cast<char*>(workspace);
+// The second GEMM and the sum over a token's experts, on the token lists, tables and h that the workspace holds.
+// w_down: per expert (HOST array of DEVICE pointers) the matrix that multiplies h.
+int down_and_sum(const camera_layer_t* L, const void* const* w_down, int64_t T, float* y, const ScoreCtx& c,
+                 const FwdLayout& fl, void* const* h, char* ws, bool long_lists, cudaStream_t st) {
   const int E = L->n_routed + L->n_shared;
-  std::vector<void*> h(E);
-  std::vector<float*> yp(E);
-  for (int e = 0; e < E; ++e) {
-    if (e < L->n_routed) {
-      h[e] = ws + fl.h_routed;
-      yp[e] = reinterpret_cast<float*>(ws + fl.y_perm);
-    } else {
-      h[e] = ws + fl.h_shared[e - L->n_routed];
-      yp[e] = reinterpret_cast<float*>(ws + fl.y_shared[e - L->n_routed]);
-    }
-    if (L->w_down_ld == nullptr && L->d_ff[e] % 8 != 0) return CAMERA_ERR_UNSUPPORTED_SHAPE;   // TMA row pitch: 16 bytes
-  }
-  const ForwardBuffers fb{h.data(), fl.h_ld.data(), yp.data()};
-  camera_score_aux_t a2;
-  memset(&a2, 0, sizeof(a2));
-  if (aux) {
-    a2 = *aux;
-    a2.flags &= ~(uint32_t)CAMERA_SCORE_FORCE_SIMT;
-    if (energy == nullptr) a2.flags &= ~(uint32_t)CAMERA_SCORE_ACCUMULATE;
-  }
-  // the scores are sums and maxima over a micro-expert's tokens: they need the scoring orientation
-  const bool long_lists = forward_token_rows(L, T, a2.flags);
-  const bool token_rows = energy == nullptr && long_lists;
-  if (token_rows) a2.flags = (a2.flags & ~(uint32_t)CAMERA_SCORE_SINGLE_CTA) | CAMERA_SCORE_CTA_PAIR;
-  ScoreFront f;
-  int rc = score_front(L, x, T, alpha, energy, &a2, ws + fl.score, fl.score_bytes, st, &fb, &f);
-  if (rc != CAMERA_OK) return rc;
-  if (!f.use_umma) return CAMERA_ERR_UNSUPPORTED_SHAPE;
-  const ScoreCtx& c = f.c;
-  if (energy != nullptr && launch_rownorm(c, f.norm_blocks, st) != cudaSuccess) { cudaGetLastError(); return CAMERA_ERR_CUDA; }
-  if (T == 0) {   // no tokens: the scores of the batches so far (or zeros), no output rows
-    if (energy != nullptr && launch_combine(c, st) != cudaSuccess) { cudaGetLastError(); return CAMERA_ERR_CUDA; }
-    return CAMERA_OK;
-  }
-
-  // tensor maps of the second GEMM: per expert W_down [d_model rows, d_ff] and h [rows, h_ld]
+  // tensor maps: per expert W_down [d_model rows, d_ff] and h [rows, h_ld]
   std::vector<char> maps((size_t)128 * 2 * E);
   for (int e = 0; e < E; ++e) {
     const int ld = L->w_down_ld ? L->w_down_ld[e] : L->d_ff[e];
     const uint64_t rows_h = e < L->n_routed ? (uint64_t)(fl.max_rows_perm > 0 ? fl.max_rows_perm : 1) : (uint64_t)T;
-    if (!encode_bf16_2d_pitch(maps.data() + (size_t)128 * (2 * e), L->d_ff[e] > 0 ? L->w_down[e] : nullptr,
+    if (!encode_bf16_2d_pitch(maps.data() + (size_t)128 * (2 * e), L->d_ff[e] > 0 ? w_down[e] : nullptr,
                               (uint64_t)L->d_model, (uint64_t)L->d_ff[e], (uint64_t)ld, D_TILE) ||
         !encode_bf16_2d_pitch(maps.data() + (size_t)128 * (2 * e + 1), h[e], rows_h, (uint64_t)fl.h_ld[e],
                               (uint64_t)fl.h_ld[e], long_lists ? 128 : UMMA_TOK))
@@ -698,11 +654,6 @@ int forward_impl(const camera_layer_t* L, const void* x, int64_t T, float alpha,
     cudaGetLastError();
     return CAMERA_ERR_CUDA;
   }
-  if ((f.use_pair ? launch_score_umma_pair_write_h(c, token_rows, st) : launch_score_umma_write_h(c, st)) != cudaSuccess) {
-    cudaGetLastError();
-    return CAMERA_ERR_CUDA;
-  }
-  if (energy != nullptr && launch_combine(c, st) != cudaSuccess) { cudaGetLastError(); return CAMERA_ERR_CUDA; }
   int dev = 0, sms = 148;
   cudaGetDevice(&dev);
   cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
@@ -723,6 +674,80 @@ int forward_impl(const camera_layer_t* L, const void* x, int64_t T, float alpha,
   return cudaGetLastError() == cudaSuccess ? CAMERA_OK : CAMERA_ERR_CUDA;
 }
 
+// Per-expert buffers of the forward workspace and the argument checks the forward entry points share.
+struct FwdSetup {
+  FwdLayout fl;
+  std::vector<void*> h;
+  std::vector<float*> yp;
+};
+int forward_setup(const camera_layer_t* L, const void* x, int64_t T, const float* y, void* workspace,
+                  size_t workspace_bytes, FwdSetup* s) {
+  if (L == nullptr || (y == nullptr && T > 0) || (reinterpret_cast<uintptr_t>(y) & 15)) return CAMERA_ERR_INVALID_ARG;
+  if (score_workspace_bytes_any(L, T, true) == 0) return CAMERA_ERR_INVALID_ARG;
+  if (L->dtype != CAMERA_BF16 || L->down_layout != CAMERA_DOWN_HF || L->d_model % UMMA_BK != 0 || !umma_shape_ok(L) ||
+      (reinterpret_cast<uintptr_t>(x) & 15))
+    return CAMERA_ERR_UNSUPPORTED_SHAPE;
+  s->fl = fwd_layout(L, T);
+  const FwdLayout& fl = s->fl;
+  if (workspace == nullptr || workspace_bytes < fl.total || (reinterpret_cast<uintptr_t>(workspace) & 255))
+    return CAMERA_ERR_WORKSPACE;
+  char* ws = static_cast<char*>(workspace);
+  const int E = L->n_routed + L->n_shared;
+  s->h.resize(E);
+  s->yp.resize(E);
+  for (int e = 0; e < E; ++e) {
+    if (e < L->n_routed) {
+      s->h[e] = ws + fl.h_routed;
+      s->yp[e] = reinterpret_cast<float*>(ws + fl.y_perm);
+    } else {
+      s->h[e] = ws + fl.h_shared[e - L->n_routed];
+      s->yp[e] = reinterpret_cast<float*>(ws + fl.y_shared[e - L->n_routed]);
+    }
+    if (L->w_down_ld == nullptr && L->d_ff[e] % 8 != 0) return CAMERA_ERR_UNSUPPORTED_SHAPE;   // TMA row pitch: 16 bytes
+  }
+  return CAMERA_OK;
+}
+
+// The layer output, and with `energy` also the scores, from one pass over W_gate and W_up.
+int forward_impl(const camera_layer_t* L, const void* x, int64_t T, float alpha, float* energy, float* y,
+                 const camera_score_aux_t* aux, void* workspace, size_t workspace_bytes, void* cuda_stream) {
+  FwdSetup fs;
+  int rc = forward_setup(L, x, T, y, workspace, workspace_bytes, &fs);
+  if (rc != CAMERA_OK) return rc;
+  const FwdLayout& fl = fs.fl;
+  cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+  char* ws = static_cast<char*>(workspace);
+  const ForwardBuffers fb{fs.h.data(), fl.h_ld.data(), fs.yp.data(), false};
+  camera_score_aux_t a2;
+  memset(&a2, 0, sizeof(a2));
+  if (aux) {
+    a2 = *aux;
+    a2.flags &= ~(uint32_t)CAMERA_SCORE_FORCE_SIMT;
+    if (energy == nullptr) a2.flags &= ~(uint32_t)CAMERA_SCORE_ACCUMULATE;
+  }
+  // the scores are sums and maxima over a micro-expert's tokens: they need the scoring orientation
+  const bool long_lists = forward_token_rows(L, T, a2.flags);
+  const bool token_rows = energy == nullptr && long_lists;
+  if (token_rows) a2.flags = (a2.flags & ~(uint32_t)CAMERA_SCORE_SINGLE_CTA) | CAMERA_SCORE_CTA_PAIR;
+  ScoreFront f;
+  rc = score_front(L, x, T, alpha, energy, &a2, ws + fl.score, fl.score_bytes, st, &fb, &f);
+  if (rc != CAMERA_OK) return rc;
+  if (!f.use_umma) return CAMERA_ERR_UNSUPPORTED_SHAPE;
+  const ScoreCtx& c = f.c;
+  if (energy != nullptr && launch_rownorm(c, f.norm_blocks, st) != cudaSuccess) { cudaGetLastError(); return CAMERA_ERR_CUDA; }
+  if (T == 0) {   // no tokens: the scores of the batches so far (or zeros), no output rows
+    if (energy != nullptr && launch_combine(c, st) != cudaSuccess) { cudaGetLastError(); return CAMERA_ERR_CUDA; }
+    return CAMERA_OK;
+  }
+
+  if ((f.use_pair ? launch_score_umma_pair_write_h(c, token_rows, st) : launch_score_umma_write_h(c, st)) != cudaSuccess) {
+    cudaGetLastError();
+    return CAMERA_ERR_CUDA;
+  }
+  if (energy != nullptr && launch_combine(c, st) != cudaSuccess) { cudaGetLastError(); return CAMERA_ERR_CUDA; }
+  return down_and_sum(L, L->w_down, T, y, c, fl, fs.h.data(), ws, long_lists, st);
+}
+
 }  // namespace
 }  // namespace camera
 
@@ -737,6 +762,102 @@ extern "C" int camera_score_forward_layer(const camera_layer_t* L, const void* x
                                           size_t workspace_bytes, void* cuda_stream) {
   if (energy == nullptr) return CAMERA_ERR_INVALID_ARG;
   return forward_impl(L, x, T, alpha, energy, y, aux, workspace, workspace_bytes, cuda_stream);
+}
+
+namespace camera {
+namespace {
+
+constexpr int MASK_EXPERTS = 64;    // experts per launch of k_mask_down (their pointers travel as kernel arguments)
+struct MaskArgs {
+  const void* src[MASK_EXPERTS];
+  void* dst[MASK_EXPERTS];
+  int d_ff[MASK_EXPERTS], ld[MASK_EXPERTS], me_off[MASK_EXPERTS];
+};
+
+// dst[r, i] = keep[me_off + i] ? src[r, i] : 0 for the W_down [d_model, d_ff] of the expert blockIdx.y names:
+// 8 micro-experts (16 bytes of a row, 8 bytes of the mask) per thread and step.
+__global__ void __launch_bounds__(256) k_mask_down(const MaskArgs a, const uint8_t* __restrict__ keep, int d_model) {
+  const int e = blockIdx.y;
+  const int vecs = a.d_ff[e] >> 3;
+  const long long total = (long long)d_model * vecs;
+  const __nv_bfloat16* src = static_cast<const __nv_bfloat16*>(a.src[e]);
+  __nv_bfloat16* dst = static_cast<__nv_bfloat16*>(a.dst[e]);
+  const uint8_t* k = keep + a.me_off[e];
+  for (long long v = (long long)blockIdx.x * blockDim.x + threadIdx.x; v < total; v += (long long)gridDim.x * blockDim.x) {
+    const int r = (int)(v / vecs), cv = (int)(v - (long long)r * vecs);
+    uint4 w = *reinterpret_cast<const uint4*>(src + (size_t)r * a.ld[e] + 8 * cv);
+    const uint2 m = *reinterpret_cast<const uint2*>(k + 8 * cv);
+    auto sel = [](uint32_t word, uint32_t lo_keep, uint32_t hi_keep) {
+      return (lo_keep ? word & 0x0000ffffu : 0u) | (hi_keep ? word & 0xffff0000u : 0u);
+    };
+    w.x = sel(w.x, m.x & 0xffu, m.x & 0xff00u);
+    w.y = sel(w.y, m.x & 0xff0000u, m.x & 0xff000000u);
+    w.z = sel(w.z, m.y & 0xffu, m.y & 0xff00u);
+    w.w = sel(w.w, m.y & 0xff0000u, m.y & 0xff000000u);
+    *reinterpret_cast<uint4*>(dst + (size_t)r * a.ld[e] + 8 * cv) = w;
+  }
+}
+
+}  // namespace
+}  // namespace camera
+
+extern "C" int camera_mask_down_columns(const camera_layer_t* L, const uint8_t* keep_mask, void* const* w_down_out,
+                                        void* cuda_stream) {
+  if (L == nullptr || keep_mask == nullptr || w_down_out == nullptr || (reinterpret_cast<uintptr_t>(keep_mask) & 7))
+    return CAMERA_ERR_INVALID_ARG;
+  if (score_workspace_bytes_any(L, 0, true) == 0) return CAMERA_ERR_INVALID_ARG;
+  if (L->dtype != CAMERA_BF16 || L->down_layout != CAMERA_DOWN_HF) return CAMERA_ERR_UNSUPPORTED_SHAPE;
+  const int E = L->n_routed + L->n_shared;
+  cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+  int me = 0;
+  for (int e0 = 0; e0 < E; e0 += MASK_EXPERTS) {
+    MaskArgs a;
+    memset(&a, 0, sizeof(a));
+    const int n = E - e0 < MASK_EXPERTS ? E - e0 : MASK_EXPERTS;
+    long long most = 0;
+    for (int i = 0; i < n; ++i) {
+      const int e = e0 + i;
+      const int ld = L->w_down_ld ? L->w_down_ld[e] : L->d_ff[e];
+      if (L->d_ff[e] % 8 != 0 || ld % 8 != 0) return CAMERA_ERR_UNSUPPORTED_SHAPE;        // 16-byte pieces of a row
+      if (L->d_ff[e] > 0 && (w_down_out[e] == nullptr || (reinterpret_cast<uintptr_t>(w_down_out[e]) & 15)))
+        return CAMERA_ERR_INVALID_ARG;
+      a.src[i] = L->w_down[e]; a.dst[i] = w_down_out[e]; a.d_ff[i] = L->d_ff[e]; a.ld[i] = ld; a.me_off[i] = me;
+      me += L->d_ff[e];
+      const long long v = (long long)L->d_model * (L->d_ff[e] >> 3);
+      most = v > most ? v : most;
+    }
+    if (most == 0) continue;
+    const long long blocks = (most + 255) / 256;
+    k_mask_down<<<dim3((unsigned)(blocks < 1024 ? blocks : 1024), (unsigned)n), 256, 0, st>>>(a, keep_mask, L->d_model);
+  }
+  return cudaGetLastError() == cudaSuccess ? CAMERA_OK : CAMERA_ERR_CUDA;
+}
+
+extern "C" int camera_pruned_output(const camera_layer_t* L, const void* const* w_down_masked, int64_t T, float* y_hat,
+                                    const camera_score_aux_t* aux, void* workspace, size_t workspace_bytes,
+                                    void* cuda_stream) {
+  if (w_down_masked == nullptr) return CAMERA_ERR_INVALID_ARG;
+  FwdSetup fs;
+  int rc = forward_setup(L, nullptr, T, y_hat, workspace, workspace_bytes, &fs);
+  if (rc != CAMERA_OK) return rc;
+  for (int e = 0; e < L->n_routed + L->n_shared; ++e)
+    if (L->d_ff[e] > 0 && (w_down_masked[e] == nullptr || (reinterpret_cast<uintptr_t>(w_down_masked[e]) & 15)))
+      return CAMERA_ERR_INVALID_ARG;
+  const FwdLayout& fl = fs.fl;
+  cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+  char* ws = static_cast<char*>(workspace);
+  const ForwardBuffers fb{fs.h.data(), fl.h_ld.data(), fs.yp.data(), true};
+  camera_score_aux_t a2;
+  memset(&a2, 0, sizeof(a2));
+  if (aux) { a2 = *aux; a2.flags &= ~(uint32_t)(CAMERA_SCORE_FORCE_SIMT | CAMERA_SCORE_ACCUMULATE); }
+  ScoreFront f;
+  rc = score_front(L, nullptr, T, 0.f, nullptr, &a2, ws + fl.score, fl.score_bytes, st, &fb, &f);
+  if (rc != CAMERA_OK) return rc;
+  if (!f.use_umma) return CAMERA_ERR_UNSUPPORTED_SHAPE;
+  if (T == 0) return CAMERA_OK;
+  // the work-unit counter of the second GEMM is the one thing the earlier call left used up
+  if (cudaMemsetAsync(&f.c.totals->down_counter, 0, sizeof(int), st) != cudaSuccess) { cudaGetLastError(); return CAMERA_ERR_CUDA; }
+  return down_and_sum(L, w_down_masked, T, y_hat, f.c, fl, fs.h.data(), ws, forward_token_rows(L, T, a2.flags), st);
 }
 
 extern "C" size_t camera_output_error_workspace_bytes(int64_t n_tokens) {

@@ -98,6 +98,12 @@ def test_new_entry_points_reject_bad_arguments_on_the_host(P):
     assert P.lib.camera_score_forward_layer(C.byref(ok), 4096, 10, C.c_float(0.5), None, 4096, None, 4096, 1 << 30, None) == -1   # no energy
     assert P.lib.camera_score_forward_layer(C.byref(ok), 4096, 10, C.c_float(0.5), 4096, None, None, 4096, 1 << 30, None) == -1   # no output
     assert P.lib.camera_score_forward_layer(C.byref(f32), 4096, 10, C.c_float(0.5), 4096, 4096, None, 4096, 1 << 30, None) == -2
+    ptrs4 = (C.c_void_p * 4)(*[4096] * 4)
+    assert P.lib.camera_mask_down_columns(C.byref(ok), None, ptrs4, None) == -1                             # no mask
+    assert P.lib.camera_mask_down_columns(C.byref(ok), 4100, ptrs4, None) == -1                             # mask not 8-byte aligned
+    assert P.lib.camera_mask_down_columns(C.byref(f32), 4096, ptrs4, None) == -2
+    assert P.lib.camera_pruned_output(C.byref(ok), None, 10, 4096, None, 4096, 1 << 30, None) == -1
+    assert P.lib.camera_pruned_output(C.byref(ok), ptrs4, 10, 4096, None, None, 0, None) == -3
     assert P.lib.camera_output_error(4096, 4096, 10, 0, 4096, 4096, 1 << 20, None) == -1
     assert P.lib.camera_output_error(4096, 4096, 10, 64, 4096, None, 0, None) == -3
     assert P.lib.camera_residual_norm(4096, 1, 4096, 10, 60, C.c_float(1e-6), 4096, None) == -1             # d_model % 8

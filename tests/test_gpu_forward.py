@@ -143,6 +143,49 @@ def test_scores_and_output_from_one_pass(P, cta_pair):
     assert_output_close("output in two batches", y2.cpu().numpy(), oracle_forward(ol, Xd, rout))
 
 
+@pytest.mark.parametrize("T,ratio", [(1300, 0.4), (5000, 0.7), (70, 0.2)])
+def test_pruned_output_from_stored_h(P, T, ratio):
+    """Phi[:,S] W[S,:] of Eq. 7 from the h the one-pass call left in its workspace and W_down with the pruned columns
+    zeroed: against the oracle's sliced layer, and against the sliced layer run through camera_layer_forward (the same
+    products, another order of the fp32 sums over d_ff)."""
+    cfg = cfg_of(n_tokens=T, d_ff_routed=320, d_ff_shared=(192,))
+    L = W().make_layer(cfg, seed=38, device=DEV)
+    X = W().make_tokens(cfg, seed=38, device=DEV)
+    layer = P.Layer.from_workload(L)
+    ol, Xd = to_oracle_layer(L), f64(X)
+    rin, rout = oracle_routing(ol, Xd)
+    ws = P.alloc_workspace(P.camera_forward_workspace_bytes(layer, T), DEV)
+    E, y = P.camera_score_forward_layer(layer, X, 0.95, routing_in=rin, workspace=ws)
+    keep = P.camera_select_prune(E, ratio)
+    keep[320:640] = 0                       # one routed expert loses every micro-expert
+    masked = P.camera_mask_down_columns(layer, keep)
+    off = O.me_offsets(ol)
+    for e in range(layer.n_experts):        # the masking itself, bit for bit
+        k = keep[off[e]:off[e + 1]].bool()
+        assert torch.equal(masked[e], torch.where(k[None, :], L["w_down"][e], torch.zeros_like(L["w_down"][e])))
+    y_hat = P.camera_pruned_output(layer, masked, T, ws)
+    y_hat2 = P.camera_pruned_output(layer, masked, T, ws)          # the call leaves the workspace reusable
+    assert torch.equal(y_hat, y_hat2)
+    assert P.camera_read_status(ws) == 0
+    lists, _ = O.sub_index_lists(keep.cpu().numpy(), off, [1])
+    ref_hat = oracle_forward(O.slice_layer(ol, lists), Xd, rout)
+    assert_output_close("pruned output from stored h", y_hat.cpu().numpy(), ref_hat)
+    # the sliced layer through the forward call
+    sub, counts = P.camera_sub_index(keep, P.expert_offsets_tensor(layer), [1])
+    out = P.camera_compact_weights(layer, sub, counts, 1)
+    m = counts[:, 0].cpu().numpy()
+    sliced = P.Layer(L["w_router"], [out["w_gate"][e][:m[e]] for e in range(layer.n_experts)],
+                     [out["w_up"][e][:m[e]] for e in range(layer.n_experts)], out["w_down"], cfg.top_k, cfg.n_shared,
+                     L["router_bias"], L["w_shared_gate"], cfg.norm_topk, "hf", down_ld=layer.d_ff)
+    y_sl = P.camera_layer_forward(sliced, X, routing_in=rin).cpu().numpy().astype(np.float64)
+    got = y_hat.cpu().numpy().astype(np.float64)
+    rms = np.sqrt((y_sl ** 2).mean(axis=1, keepdims=True))
+    assert (np.abs(got - y_sl) <= 1e-5 * np.maximum(rms, 1e-30)).all()
+    # and the full mask gives back the layer's own output
+    full = P.camera_mask_down_columns(layer, torch.ones_like(keep))
+    assert torch.equal(P.camera_pruned_output(layer, full, T, ws), y)
+
+
 def test_one_pass_call_without_tokens(P):
     cfg = cfg_of(n_tokens=0)
     L = W().make_layer(cfg, seed=37, device=DEV)
