@@ -365,6 +365,7 @@ extern "C" int camera_read_status(const void* workspace, void* cuda_stream, int3
 
 namespace {
 constexpr int64_t ANALYZE_BATCH_TOKENS = 65536;   // tokens per host-to-device batch of camera_analyze_layer_host
+constexpr int64_t ANALYZE_FIRST_BATCH_TOKENS = 8192;
 
 struct AnalyzeLayout {
   size_t score, select, x[2], energy, phi2, phi_inf, keep, bits, total;
@@ -396,12 +397,13 @@ AnalyzeLayout analyze_layout(const camera_layer_t* L, int64_t T, int n_levels) {
 // The copy stream and the events that order it against the caller's stream; destroyed when the call returns.
 struct CopyPipe {
   cudaStream_t copy = nullptr;
-  cudaEvent_t copied[2] = {nullptr, nullptr}, consumed[2] = {nullptr, nullptr};
+  cudaEvent_t copied[2] = {nullptr, nullptr}, consumed[2] = {nullptr, nullptr}, timed[2] = {nullptr, nullptr};
   bool create() {
     if (cudaStreamCreateWithFlags(&copy, cudaStreamNonBlocking) != cudaSuccess) return false;
     for (int i = 0; i < 2; ++i)
       if (cudaEventCreateWithFlags(&copied[i], cudaEventDisableTiming) != cudaSuccess ||
-          cudaEventCreateWithFlags(&consumed[i], cudaEventDisableTiming) != cudaSuccess)
+          cudaEventCreateWithFlags(&consumed[i], cudaEventDisableTiming) != cudaSuccess ||
+          cudaEventCreate(&timed[i]) != cudaSuccess)
         return false;
     return true;
   }
@@ -409,6 +411,7 @@ struct CopyPipe {
     for (int i = 0; i < 2; ++i) {
       if (copied[i]) cudaEventDestroy(copied[i]);
       if (consumed[i]) cudaEventDestroy(consumed[i]);
+      if (timed[i]) cudaEventDestroy(timed[i]);
     }
     if (copy) cudaStreamDestroy(copy);
   }
@@ -447,29 +450,51 @@ extern "C" int camera_analyze_layer_host(const camera_layer_t* L, const void* x_
   aux.phi2 = reinterpret_cast<float*>(ws + a.phi2);
   aux.phi_inf_sq = reinterpret_cast<float*>(ws + a.phi_inf);
 
-  // the first batch is a quarter of the others: its copy is the only one nothing overlaps
-  const int64_t first = T > a.batch ? a.batch / 4 : T;
-  const int64_t n_batches = T > a.batch ? 1 + (T - first + a.batch - 1) / a.batch : 1;
+  // Batch sizes.  Nothing overlaps the copy of the first batch, so it is small.  The copy of batch b+1 hides behind the
+  // scoring of batch b as long as their sizes differ by less than the ratio of the two rates, tokens copied per ms to
+  // tokens scored per ms.  The call times its first copy (the GPU has nothing to do until it lands) and lets the
+  // batches grow by 0.85 of that ratio, between 1.5 and 4, up to the workspace's batch: three batches to get there on
+  // a fast link, six on a link half as fast (measured on this kind of host: 1.5 to 3 for the Qwen2 shape).
+  const bool batched = T > a.batch;
   CopyPipe pipe;
-  if (n_batches > 1 && !pipe.create()) { cudaGetLastError(); return CAMERA_ERR_CUDA; }
-  for (int64_t b = 0; b < n_batches; ++b) {
+  if (batched && !pipe.create()) { cudaGetLastError(); return CAMERA_ERR_CUDA; }
+  double growth = 1.5;
+  int64_t t0 = 0, n = batched ? ANALYZE_FIRST_BATCH_TOKENS : T;
+  for (int64_t b = 0; b == 0 || t0 < T; ++b) {
     const int buf = (int)(b & 1);
-    const int64_t t0 = b == 0 ? 0 : first + (b - 1) * a.batch;
-    const int64_t n = b == 0 ? first : (T - t0 < a.batch ? T - t0 : a.batch);
+    if (n > T - t0) n = T - t0;
     const char* src = static_cast<const char*>(x_host) + (size_t)t0 * row_bytes;
-    if (n_batches == 1) {
+    if (!batched) {
       if (n > 0) CK(cudaMemcpyAsync(ws + a.x[0], src, (size_t)n * row_bytes, cudaMemcpyHostToDevice, st));
     } else {
       // batch b travels on the copy stream while batch b-1 is being scored on the caller's stream
       if (b >= 2) CK(cudaStreamWaitEvent(pipe.copy, pipe.consumed[buf], 0));
+      if (b == 0) CK(cudaEventRecord(pipe.timed[0], pipe.copy));
       CK(cudaMemcpyAsync(ws + a.x[buf], src, (size_t)n * row_bytes, cudaMemcpyHostToDevice, pipe.copy));
+      if (b == 0) CK(cudaEventRecord(pipe.timed[1], pipe.copy));
       CK(cudaEventRecord(pipe.copied[buf], pipe.copy));
       CK(cudaStreamWaitEvent(st, pipe.copied[buf], 0));
     }
     aux.flags = b > 0 ? CAMERA_SCORE_ACCUMULATE : 0u;
     rc = camera_score_layer(L, ws + a.x[buf], n, alpha, d_energy, &aux, ws + a.score, a.score_bytes, cuda_stream);
     if (rc != CAMERA_OK) return rc;
-    if (n_batches > 1) CK(cudaEventRecord(pipe.consumed[buf], st));
+    if (batched) CK(cudaEventRecord(pipe.consumed[buf], st));
+    if (batched && b == 0) {
+      float copy_ms = 0.f;
+      CK(cudaEventSynchronize(pipe.timed[1]));
+      CK(cudaEventElapsedTime(&copy_ms, pipe.timed[0], pipe.timed[1]));
+      // tokens scored per ms at 1.4 Pflop/s of gate/up work (4 d f flop per token and active micro-expert)
+      double f_active = 0.0;
+      for (int e = 0; e < L->n_routed + L->n_shared; ++e)
+        f_active += e < L->n_routed ? (double)L->d_ff[e] * L->top_k / L->n_routed : (double)L->d_ff[e];
+      const double scored_per_ms = 1.4e12 / (4.0 * L->d_model * (f_active > 1.0 ? f_active : 1.0));
+      const double copied_per_ms = copy_ms > 0.f ? (double)n / copy_ms : 4.0 * scored_per_ms;
+      growth = 0.85 * copied_per_ms / scored_per_ms;
+      growth = growth < 1.5 ? 1.5 : (growth > 4.0 ? 4.0 : growth);
+    }
+    t0 += n;
+    const int64_t next = ((int64_t)((double)n * growth) + 255) / 256 * 256;
+    n = next < a.batch ? next : a.batch;
   }
   if (energy_host) CK(cudaMemcpyAsync(energy_host, d_energy, sizeof(float) * (size_t)n_me, cudaMemcpyDeviceToHost, st));
   const int64_t seg[2] = {0, n_me};

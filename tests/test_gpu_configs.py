@@ -182,3 +182,32 @@ def test_qwen2_57b_shape_layer_output_on_sampled_tokens(P):
     ref = oracle_forward(to_oracle_layer(L), f64(X[torch.from_numpy(tok).to(DEV)]),
                          (gi.cpu().numpy().astype(np.int64)[tok], gw.cpu().numpy().astype(np.float64)[tok]))
     assert_output_close("qwen2 layer output", y.cpu().numpy()[tok], ref)
+
+
+def test_qwen2_57b_shape_one_pass_scores_output_and_pruned_output(P):
+    """The calls of the Algorithm 2 loop on one 65536-token batch of the Qwen2-57B-A14B shape: the one-pass call gives
+    camera_score_layer's energies bit for bit and the layer output within the forward tolerance on sampled tokens; the
+    retained micro-experts' output from the stored h agrees with the oracle's sliced layer on those tokens."""
+    from test_gpu_forward import assert_output_close, oracle_forward
+    from _util import to_oracle_layer
+    cfg = W().scaled(W().CONFIGS["qwen2_57b_a14b"], n_tokens=65536)
+    L = W().make_layer(cfg, seed=0, device=DEV)
+    X = W().make_tokens(cfg, seed=0, device=DEV)
+    layer = P.Layer.from_workload(L)
+    ws = P.alloc_workspace(P.camera_forward_workspace_bytes(layer, cfg.n_tokens), DEV)
+    ref = P.camera_score_layer(layer, X, 0.95, details=True)
+    E, y = P.camera_score_forward_layer(layer, X, 0.95, workspace=ws,
+                                        routing_in=(ref["topk_idx"], ref["topk_w"]))
+    assert P.camera_read_status(ws) == 0
+    assert torch.equal(E, ref["energy"])
+    tok = np.sort(np.random.default_rng(5).choice(cfg.n_tokens, size=16, replace=False))
+    tok[0], tok[-1] = 0, cfg.n_tokens - 1
+    ol = to_oracle_layer(L)
+    Xs = f64(X[torch.from_numpy(tok).to(DEV)])
+    routing = (ref["topk_idx"].cpu().numpy().astype(np.int64)[tok], ref["topk_w"].cpu().numpy().astype(np.float64)[tok])
+    assert_output_close("qwen2 one-pass output", y.cpu().numpy()[tok], oracle_forward(ol, Xs, routing))
+    keep = P.camera_select_prune(E, 0.4)
+    y_hat = P.camera_pruned_output(layer, P.camera_mask_down_columns(layer, keep), cfg.n_tokens, ws)
+    assert P.camera_read_status(ws) == 0
+    lists, _ = O.sub_index_lists(keep.cpu().numpy(), O.me_offsets(ol), [1])
+    assert_output_close("qwen2 pruned output", y_hat.cpu().numpy()[tok], oracle_forward(O.slice_layer(ol, lists), Xs, routing))
