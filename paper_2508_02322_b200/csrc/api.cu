@@ -475,7 +475,7 @@ extern "C" int camera_analyze_layer_host(const camera_layer_t* L, const void* x_
       CK(cudaEventRecord(pipe.copied[buf], pipe.copy));
       CK(cudaStreamWaitEvent(st, pipe.copied[buf], 0));
     }
-    aux.flags = b > 0 ? CAMERA_SCORE_ACCUMULATE : 0u;
+    aux.flags = b > 0 ? (uint32_t)CAMERA_SCORE_ACCUMULATE : 0u;
     rc = camera_score_layer(L, ws + a.x[buf], n, alpha, d_energy, &aux, ws + a.score, a.score_bytes, cuda_stream);
     if (rc != CAMERA_OK) return rc;
     if (batched) CK(cudaEventRecord(pipe.consumed[buf], st));
