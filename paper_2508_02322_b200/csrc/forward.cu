@@ -56,7 +56,9 @@ __device__ __forceinline__ DownUnit decode_down_unit(const ScoreCtx& c, int unit
   return u;
 }
 
-__global__ void __launch_bounds__(D_THREADS, 1) k_down_umma(const ScoreCtx c, const void* maps_raw, int n_dt) {
+// b_bytes: size of the box of h rows one load brings (128 bytes per row; the map's box is as many rows as a token list
+// can have, at most a tile: with a few tokens per expert a full tile's box would triple the bytes L2 has to deliver).
+__global__ void __launch_bounds__(D_THREADS, 1) k_down_umma(const ScoreCtx c, const void* maps_raw, int n_dt, int b_bytes) {
   extern __shared__ uint8_t smem_raw[];
   const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
   uint8_t* const base_ptr = smem_raw + (base - smem_u32(smem_raw));
@@ -105,8 +107,10 @@ __global__ void __launch_bounds__(D_THREADS, 1) k_down_umma(const ScoreCtx c, co
       uint32_t qphase = 0;
       while (ok) {   // units are taken in order from a counter, as in the scoring kernel
         if (!mbar_wait(sempty_bar(q), qphase ^ 1u, abort_flag)) { ok = false; break; }
+        // last expert first: the shared experts come last in the numbering and have the longest K, so their
+        // units start early instead of forming the tail (with 64 tokens they are 8 times a routed expert's unit)
         int unit = atomicAdd(&c.totals->down_counter, 1);
-        if (unit >= total_units) unit = -1;
+        unit = unit >= total_units ? -1 : total_units - 1 - unit;
         sched_unit[q] = unit;
         mbar_arrive(sfull_bar(q));
         if (++q == D_SCHED) { q = 0; qphase ^= 1u; }
@@ -123,7 +127,7 @@ __global__ void __launch_bounds__(D_THREADS, 1) k_down_umma(const ScoreCtx c, co
           for (int kb = 0; kb < u.n_kb; ++kb) {
             if (!mbar_wait(empty_bar(stage), phase ^ 1u, abort_flag)) { ok = false; break; }
             const uint32_t a_dst = base + stage * D_STAGE_BYTES;
-            mbar_expect_tx(full_bar(stage), D_STAGE_BYTES);
+            mbar_expect_tx(full_bar(stage), D_A_BYTES + b_bytes);
             // W_down columns past d_ff and rows past d_model, h rows past the buffer: filled with zeros
             tma_load_2d(a_dst, map_w, full_bar(stage), kb * UMMA_BK, u.c0);
             tma_load_2d(a_dst + D_A_BYTES, map_h, full_bar(stage), kb * UMMA_BK, row);
@@ -307,7 +311,7 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(D_THREADS, 1)
         if (rank == 0) {
           if (!mbar_wait_cluster(sempty_bar(q), qphase ^ 1u, abort_flag)) { ok = false; break; }
           unit = atomicAdd(&c.totals->down_counter, 1);
-          if (unit >= total_units) unit = -1;
+          unit = unit >= total_units ? -1 : total_units - 1 - unit;     // last expert first, as in k_down_umma
           sched_unit[q] = unit;
           st_cluster_u32(map_to_cta(smem_u32((const void*)(sched_unit + q)), 1), (uint32_t)unit);
           mbar_arrive(sfull_bar(q));
@@ -457,31 +461,33 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(D_THREADS, 1)
   }
 }
 
-// One warp per token: y[t, :] = its k routed rows of y_perm (in slot order) plus its row of every shared expert.
+// y[t, :] = the token's k routed rows of y_perm (in slot order) plus its row of every shared expert.  A block owns up
+// to 1024 consecutive output channels of one token (four per thread), so a 64-token decode batch still fills the GPU
+// with independent loads; the rows' positions are worked out once per block.
 __global__ void __launch_bounds__(256) k_unpermute_sum(const ScoreCtx c, float* __restrict__ y) {
-  const int lane = threadIdx.x & 31;
-  const int t = blockIdx.x * 8 + (threadIdx.x >> 5);
-  if (t >= c.n_tokens) return;
+  __shared__ long long pos_s[MAX_TOPK];
   const int k = c.top_k, d = c.d_model;
-  long long pos_l = 0;
-  if (lane < k) {
-    const int e = c.topk_idx[(size_t)t * k + lane];
-    pos_l = c.edyn[e].row_base + c.block_hist[(size_t)(t / ROUTER_TOK) * c.n_routed + e] + c.local_rank[(size_t)t * k + lane];
+  const int t = blockIdx.x;
+  if ((int)threadIdx.x < k) {
+    const int e = c.topk_idx[(size_t)t * k + threadIdx.x];
+    pos_s[threadIdx.x] = (long long)c.edyn[e].row_base + c.block_hist[(size_t)(t / ROUTER_TOK) * c.n_routed + e] +
+                         c.local_rank[(size_t)t * k + threadIdx.x];
   }
+  __syncthreads();
+  const int v = (blockIdx.y * 256 + threadIdx.x) << 2;
+  if (v >= d) return;
   const float* routed = c.n_routed > 0 ? c.est[0].y_part : nullptr;
-  for (int v = lane * 4; v < d; v += 128) {
-    float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
-    for (int s = 0; s < k; ++s) {
-      const long long pos = __shfl_sync(0xffffffffu, pos_l, s);
-      const float4 p = *reinterpret_cast<const float4*>(routed + (size_t)pos * d + v);
-      acc.x += p.x; acc.y += p.y; acc.z += p.z; acc.w += p.w;
-    }
-    for (int s = 0; s < c.n_shared; ++s) {
-      const float4 p = *reinterpret_cast<const float4*>(c.est[c.n_routed + s].y_part + (size_t)t * d + v);
-      acc.x += p.x; acc.y += p.y; acc.z += p.z; acc.w += p.w;
-    }
-    *reinterpret_cast<float4*>(y + (size_t)t * d + v) = acc;
+  float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll 4
+  for (int s = 0; s < k; ++s) {
+    const float4 p = *reinterpret_cast<const float4*>(routed + (size_t)pos_s[s] * d + v);
+    acc.x += p.x; acc.y += p.y; acc.z += p.z; acc.w += p.w;
   }
+  for (int s = 0; s < c.n_shared; ++s) {
+    const float4 p = *reinterpret_cast<const float4*>(c.est[c.n_routed + s].y_part + (size_t)t * d + v);
+    acc.x += p.x; acc.y += p.y; acc.z += p.z; acc.w += p.w;
+  }
+  *reinterpret_cast<float4*>(y + (size_t)t * d + v) = acc;
 }
 
 // Per CTA of 8 tokens: sum (y - y_hat)^2, sum y^2, sum of the tokens' cosine similarities, in double.
@@ -639,6 +645,9 @@ namespace {
 int down_and_sum(const camera_layer_t* L, const void* const* w_down, int64_t T, float* y, const ScoreCtx& c,
                  const FwdLayout& fl, void* const* h, char* ws, bool long_lists, cudaStream_t st) {
   const int E = L->n_routed + L->n_shared;
+  // rows of h per load: the pair kernel's 128 per CTA; else a tile, or less where no list can be longer (an expert
+  // sees a token at most once)
+  const int h_box = long_lists ? 128 : (T <= 32 ? 32 : T <= 64 ? 64 : T <= 128 ? 128 : UMMA_TOK);
   // tensor maps: per expert W_down [d_model rows, d_ff] and h [rows, h_ld]
   std::vector<char> maps((size_t)128 * 2 * E);
   for (int e = 0; e < E; ++e) {
@@ -647,7 +656,7 @@ int down_and_sum(const camera_layer_t* L, const void* const* w_down, int64_t T, 
     if (!encode_bf16_2d_pitch(maps.data() + (size_t)128 * (2 * e), L->d_ff[e] > 0 ? w_down[e] : nullptr,
                               (uint64_t)L->d_model, (uint64_t)L->d_ff[e], (uint64_t)ld, D_TILE) ||
         !encode_bf16_2d_pitch(maps.data() + (size_t)128 * (2 * e + 1), h[e], rows_h, (uint64_t)fl.h_ld[e],
-                              (uint64_t)fl.h_ld[e], long_lists ? 128 : UMMA_TOK))
+                              (uint64_t)fl.h_ld[e], h_box))
       return CAMERA_ERR_CUDA;
   }
   if (cudaMemcpyAsync(ws + fl.maps, maps.data(), maps.size(), cudaMemcpyHostToDevice, st) != cudaSuccess) {
@@ -668,9 +677,9 @@ int down_and_sum(const camera_layer_t* L, const void* const* w_down, int64_t T, 
       cudaGetLastError();
       return CAMERA_ERR_CUDA;
     }
-    k_down_umma<<<sms, D_THREADS, D_SMEM_BYTES, st>>>(c, ws + fl.maps, (L->d_model + D_TILE - 1) / D_TILE);
+    k_down_umma<<<sms, D_THREADS, D_SMEM_BYTES, st>>>(c, ws + fl.maps, (L->d_model + D_TILE - 1) / D_TILE, h_box * 128);
   }
-  k_unpermute_sum<<<(unsigned)((T + 7) / 8), 256, 0, st>>>(c, y);
+  k_unpermute_sum<<<dim3((unsigned)T, (unsigned)((L->d_model + 1023) / 1024)), 256, 0, st>>>(c, y);
   return cudaGetLastError() == cudaSuccess ? CAMERA_OK : CAMERA_ERR_CUDA;
 }
 
