@@ -184,6 +184,10 @@ def test_pruned_output_from_stored_h(P, T, ratio):
     # and the full mask gives back the layer's own output
     full = P.camera_mask_down_columns(layer, torch.ones_like(keep))
     assert torch.equal(P.camera_pruned_output(layer, full, T, ws), y)
+    # the h that camera_layer_forward leaves behind serves as well
+    y_fw = P.camera_layer_forward(layer, X, routing_in=rin, workspace=ws)
+    assert torch.equal(P.camera_pruned_output(layer, full, T, ws), y_fw)
+    assert torch.equal(P.camera_pruned_output(layer, masked, T, ws), y_hat)
 
 
 def test_one_pass_call_without_tokens(P):
