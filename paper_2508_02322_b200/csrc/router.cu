@@ -224,48 +224,67 @@ __global__ void __launch_bounds__(256) k_block_scan(ScoreCtx c) {
   if (tid == 0) c.counts[e] = run;
 }
 
-// Single thread: lays the experts' token lists out back to back (each padded to ROW_ALIGN rows)
-// and numbers the scoring work units and partial slots.
-__global__ void k_plan(ScoreCtx c) {
-  if (threadIdx.x != 0 || blockIdx.x != 0) return;
+// One warp: lays the experts' token lists out back to back (each padded to ROW_ALIGN rows) and numbers the scoring
+// work units and partial slots.  A lane takes an expert; the running offsets are warp scans.
+__global__ void __launch_bounds__(32) k_plan(ScoreCtx c) {
+  const int lane = threadIdx.x;
   int row = 0, units = 0, chunks = 0;
   long long part = 0;
-  for (int e = 0; e < c.n_experts; ++e) {
-    ExpertDyn dy;
-    if (e < c.n_routed) {
-      dy.rows = c.counts[e];
-      dy.row_base = row;
-      row += (dy.rows + ROW_ALIGN - 1) / ROW_ALIGN * ROW_ALIGN;
-    } else {
-      dy.rows = c.n_tokens;
-      dy.row_base = 0;
-      c.counts[e] = c.n_tokens;
+  for (int base = 0; base < c.n_experts; base += 32) {
+    const int e = base + lane;
+    const bool valid = e < c.n_experts, routed = e < c.n_routed;
+    const int rows = valid ? (routed ? c.counts[e] : c.n_tokens) : 0;
+    const int f = valid ? c.est[e].d_ff : 0;
+    const int n_chunks = (rows + c.chunk_tokens - 1) / c.chunk_tokens;
+    // what this expert adds to the four running offsets, then inclusive scans over the 32 lanes
+    int a_row = valid && routed ? (rows + ROW_ALIGN - 1) / ROW_ALIGN * ROW_ALIGN : 0;
+    int a_units = n_chunks * ((f + c.ch_tile - 1) / c.ch_tile), a_chunks = n_chunks;
+    long long a_part = (long long)n_chunks * f;
+    int s_row = a_row, s_units = a_units, s_chunks = a_chunks;
+    long long s_part = a_part;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+      const int t_row = __shfl_up_sync(0xffffffffu, s_row, o), t_units = __shfl_up_sync(0xffffffffu, s_units, o);
+      const int t_chunks = __shfl_up_sync(0xffffffffu, s_chunks, o);
+      const long long t_part = __shfl_up_sync(0xffffffffu, s_part, o);
+      if (lane >= o) { s_row += t_row; s_units += t_units; s_chunks += t_chunks; s_part += t_part; }
     }
-    const int f = c.est[e].d_ff;
-    dy.n_chunks = (dy.rows + c.chunk_tokens - 1) / c.chunk_tokens;
-    dy.unit_begin = units;
-    dy.part_begin = part;
-    dy.chunk_begin = chunks;
-    dy.pad = 0;
-    chunks += dy.n_chunks;
-    c.edyn[e] = dy;
-    c.unit_prefix[e] = units;
-    units += dy.n_chunks * ((f + c.ch_tile - 1) / c.ch_tile);
-    part += (long long)dy.n_chunks * f;
+    if (valid) {
+      ExpertDyn dy;
+      dy.rows = rows;
+      dy.row_base = routed ? row + s_row - a_row : 0;
+      dy.n_chunks = n_chunks;
+      dy.unit_begin = units + s_units - a_units;
+      dy.part_begin = part + s_part - a_part;
+      dy.chunk_begin = chunks + s_chunks - a_chunks;
+      dy.pad = 0;
+      c.edyn[e] = dy;
+      c.unit_prefix[e] = dy.unit_begin;
+      if (!routed) c.counts[e] = c.n_tokens;
+    }
+    row += __shfl_sync(0xffffffffu, s_row, 31);
+    units += __shfl_sync(0xffffffffu, s_units, 31);
+    chunks += __shfl_sync(0xffffffffu, s_chunks, 31);
+    part += __shfl_sync(0xffffffffu, s_part, 31);
   }
-  if (row > c.max_rows_perm || part > c.max_part) {
-    atomicExch(&c.totals->status, (int)CAMERA_ERR_WORKSPACE);
+  if (row > c.max_rows_perm || part > c.max_part) {   // cannot happen with a workspace of the size the query gives
+    if (lane == 0) atomicExch(&c.totals->status, (int)CAMERA_ERR_WORKSPACE);
     units = 0;
     chunks = 0;
-    for (int e = 0; e <= c.n_experts; ++e) c.unit_prefix[e] = 0;
-    for (int e = 0; e < c.n_experts; ++e) { c.edyn[e].n_chunks = 0; c.edyn[e].rows = 0; c.edyn[e].chunk_begin = 0; }
+    __syncwarp();
+    for (int e = lane; e < c.n_experts; e += 32) {
+      c.unit_prefix[e] = 0;
+      c.edyn[e].n_chunks = 0; c.edyn[e].rows = 0; c.edyn[e].chunk_begin = 0;
+    }
   }
-  c.unit_prefix[c.n_experts] = units;
-  c.totals->total_units = units;
-  c.totals->total_rows = row;
-  c.totals->total_chunks = chunks;
-  c.totals->unit_counter = 0;
-  c.totals->down_counter = 0;
+  if (lane == 0) {
+    c.unit_prefix[c.n_experts] = units;
+    c.totals->total_units = units;
+    c.totals->total_rows = row;
+    c.totals->total_chunks = chunks;
+    c.totals->unit_counter = 0;
+    c.totals->down_counter = 0;
+  }
 }
 
 // One warp per token: copies the token's hidden state to its row in every chosen expert's list.
