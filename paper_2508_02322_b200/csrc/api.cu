@@ -397,13 +397,12 @@ AnalyzeLayout analyze_layout(const camera_layer_t* L, int64_t T, int n_levels) {
 // The copy stream and the events that order it against the caller's stream; destroyed when the call returns.
 struct CopyPipe {
   cudaStream_t copy = nullptr;
-  cudaEvent_t copied[2] = {nullptr, nullptr}, consumed[2] = {nullptr, nullptr}, timed[2] = {nullptr, nullptr};
+  cudaEvent_t copied[2] = {nullptr, nullptr}, consumed[2] = {nullptr, nullptr};
   bool create() {
     if (cudaStreamCreateWithFlags(&copy, cudaStreamNonBlocking) != cudaSuccess) return false;
     for (int i = 0; i < 2; ++i)
       if (cudaEventCreateWithFlags(&copied[i], cudaEventDisableTiming) != cudaSuccess ||
-          cudaEventCreateWithFlags(&consumed[i], cudaEventDisableTiming) != cudaSuccess ||
-          cudaEventCreate(&timed[i]) != cudaSuccess)
+          cudaEventCreateWithFlags(&consumed[i], cudaEventDisableTiming) != cudaSuccess)
         return false;
     return true;
   }
@@ -411,7 +410,6 @@ struct CopyPipe {
     for (int i = 0; i < 2; ++i) {
       if (copied[i]) cudaEventDestroy(copied[i]);
       if (consumed[i]) cudaEventDestroy(consumed[i]);
-      if (timed[i]) cudaEventDestroy(timed[i]);
     }
     if (copy) cudaStreamDestroy(copy);
   }
@@ -452,13 +450,12 @@ extern "C" int camera_analyze_layer_host(const camera_layer_t* L, const void* x_
 
   // Batch sizes.  Nothing overlaps the copy of the first batch, so it is small.  The copy of batch b+1 hides behind the
   // scoring of batch b as long as their sizes differ by less than the ratio of the two rates, tokens copied per ms to
-  // tokens scored per ms.  The call times its first copy (the GPU has nothing to do until it lands) and lets the
-  // batches grow by 0.85 of that ratio, between 1.5 and 4, up to the workspace's batch: three batches to get there on
-  // a fast link, six on a link half as fast (measured on this kind of host: 1.5 to 3 for the Qwen2 shape).
+  // tokens scored per ms: 1.5 to 3 for the Qwen2 shape on the hosts this was measured on.  The batches grow by half
+  // from one to the next, up to the workspace's batch.  The schedule depends on nothing but the sizes: the same input
+  // gives the same bits on every run and host (a batch's tokens decide which tokens share a tile's fp32 partial sum).
   const bool batched = T > a.batch;
   CopyPipe pipe;
   if (batched && !pipe.create()) { cudaGetLastError(); return CAMERA_ERR_CUDA; }
-  double growth = 1.5;
   int64_t t0 = 0, n = batched ? ANALYZE_FIRST_BATCH_TOKENS : T;
   for (int64_t b = 0; b == 0 || t0 < T; ++b) {
     const int buf = (int)(b & 1);
@@ -469,9 +466,7 @@ extern "C" int camera_analyze_layer_host(const camera_layer_t* L, const void* x_
     } else {
       // batch b travels on the copy stream while batch b-1 is being scored on the caller's stream
       if (b >= 2) CK(cudaStreamWaitEvent(pipe.copy, pipe.consumed[buf], 0));
-      if (b == 0) CK(cudaEventRecord(pipe.timed[0], pipe.copy));
       CK(cudaMemcpyAsync(ws + a.x[buf], src, (size_t)n * row_bytes, cudaMemcpyHostToDevice, pipe.copy));
-      if (b == 0) CK(cudaEventRecord(pipe.timed[1], pipe.copy));
       CK(cudaEventRecord(pipe.copied[buf], pipe.copy));
       CK(cudaStreamWaitEvent(st, pipe.copied[buf], 0));
     }
@@ -479,21 +474,8 @@ extern "C" int camera_analyze_layer_host(const camera_layer_t* L, const void* x_
     rc = camera_score_layer(L, ws + a.x[buf], n, alpha, d_energy, &aux, ws + a.score, a.score_bytes, cuda_stream);
     if (rc != CAMERA_OK) return rc;
     if (batched) CK(cudaEventRecord(pipe.consumed[buf], st));
-    if (batched && b == 0) {
-      float copy_ms = 0.f;
-      CK(cudaEventSynchronize(pipe.timed[1]));
-      CK(cudaEventElapsedTime(&copy_ms, pipe.timed[0], pipe.timed[1]));
-      // tokens scored per ms at 1.4 Pflop/s of gate/up work (4 d f flop per token and active micro-expert)
-      double f_active = 0.0;
-      for (int e = 0; e < L->n_routed + L->n_shared; ++e)
-        f_active += e < L->n_routed ? (double)L->d_ff[e] * L->top_k / L->n_routed : (double)L->d_ff[e];
-      const double scored_per_ms = 1.4e12 / (4.0 * L->d_model * (f_active > 1.0 ? f_active : 1.0));
-      const double copied_per_ms = copy_ms > 0.f ? (double)n / copy_ms : 4.0 * scored_per_ms;
-      growth = 0.85 * copied_per_ms / scored_per_ms;
-      growth = growth < 1.5 ? 1.5 : (growth > 4.0 ? 4.0 : growth);
-    }
     t0 += n;
-    const int64_t next = ((int64_t)((double)n * growth) + 255) / 256 * 256;
+    const int64_t next = (n + n / 2 + 255) / 256 * 256;
     n = next < a.batch ? next : a.batch;
   }
   if (energy_host) CK(cudaMemcpyAsync(energy_host, d_energy, sizeof(float) * (size_t)n_me, cudaMemcpyDeviceToHost, st));
