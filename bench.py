@@ -217,7 +217,7 @@ def run_stack(args):
     ws_sel = P.alloc_workspace(P.camera_select_workspace_bytes(n_me, 1, 2), dev)
     ws_c = P.alloc_workspace(4096 + 64 * probe.n_experts, dev)
     energy = torch.empty(n_me, dtype=torch.float32, device=dev)
-    phi2, phi_inf = torch.empty_like(energy), torch.empty_like(energy)
+    phi2, phi_inf, omega2 = torch.empty_like(energy), torch.empty_like(energy), torch.empty_like(energy)
     keep = torch.empty(n_me, dtype=torch.uint8, device=dev)
     outw = {k: [torch.empty_like(w) for w in probe.tensors[k]] for k in ("w_gate", "w_up", "w_down")}
     del probe
@@ -234,7 +234,7 @@ def run_stack(args):
         ev[0].record(stream)
         for i, (t0, t1) in enumerate(spans):
             P.camera_score_forward_layer(layer, X[t0:t1], ALPHA, energy=energy, y=Y[t0:t1], workspace=ws_f[i], phi2=phi2,
-                                         phi_inf_sq=phi_inf, accumulate=i > 0)
+                                         phi_inf_sq=phi_inf, accumulate=i > 0, omega2=omega2, omega_given=i > 0)
         ev[1].record(stream)
         P.camera_select_prune(energy, ratio, workspace=ws_sel, keep_mask=keep)
         sub, counts = P.camera_sub_index(keep, off, [1])

@@ -63,6 +63,8 @@ enum {
                                       work unit: less L2 and shared-memory traffic per flop).  By default the library takes
                                       pairs unless padding d_ff to multiples of 256 would add more than 6 % of work */
   CAMERA_SCORE_SINGLE_CTA = 8u,    /* force one CTA per MMA (128 micro-experts per work unit) */
+  CAMERA_SCORE_OMEGA_GIVEN = 32u,  /* omega2 (required) already holds ||w_i||^2 of this layer's W_down, e.g. from the call on
+                                      the first batch of tokens: the pass over W_down is skipped */
   CAMERA_FORWARD_TOKEN_ROWS = 16u, /* camera_layer_forward only: force the gate/up kernel that keeps the tokens on the
                                       accumulator rows (CTA pairs, 256-token tiles; an epilogue thread writes runs of
                                       consecutive micro-experts of its token).  By default the library takes it when

@@ -23,6 +23,7 @@ CAMERA_SCORE_CTA_PAIR = 2
 CAMERA_SCORE_ACCUMULATE = 4
 CAMERA_SCORE_SINGLE_CTA = 8
 CAMERA_FORWARD_TOKEN_ROWS = 16
+CAMERA_SCORE_OMEGA_GIVEN = 32
 STAGES = ("router", "permute", "rownorm", "score", "combine")
 
 
@@ -208,14 +209,15 @@ def camera_score_layer(layer: Layer, x: torch.Tensor, alpha: float, *, energy: O
                        workspace: Optional[torch.Tensor] = None, details: bool = False,
                        routing_in=None, force_simt: bool = False, cta_pair: Optional[bool] = None, stage_events=None,
                        phi2: Optional[torch.Tensor] = None, phi_inf_sq: Optional[torch.Tensor] = None,
-                       accumulate: bool = False,
+                       accumulate: bool = False, omega2: Optional[torch.Tensor] = None, omega_given: bool = False,
                        stream: Optional[torch.cuda.Stream] = None, check_status: bool = False):
     """Algorithm 1 up to the energies.  Returns energy [N_e] fp32, or with details=True a dict that
     also holds phi2, phi_inf_sq, omega2, topk_idx, topk_w, shared_w and expert_token_counts.
     routing_in = (topk_idx int32 [T,k], topk_w fp32 [T,k]) prescribes the routing.
     stage_events = {stage: (torch.cuda.Event, torch.cuda.Event)} records per-stage timing events.
     phi2 / phi_inf_sq name the tensors that receive those components; with accumulate=True they must
-    hold the result of earlier batches of tokens, and this batch is folded into them."""
+    hold the result of earlier batches of tokens, and this batch is folded into them.  omega2 names the tensor
+    for the W_down norms; with omega_given=True it already holds them and the pass over W_down is skipped."""
     if not (x.is_contiguous() and x.dtype == layer.dtype and x.dim() == 2 and x.shape[1] == layer.d_model):
         raise ValueError("x must be a contiguous [T, d_model] tensor of the layer's dtype")
     T = int(x.shape[0])
@@ -244,14 +246,14 @@ def camera_score_layer(layer: Layer, x: torch.Tensor, alpha: float, *, energy: O
         w = w.to(device=dev, dtype=torch.float32).contiguous()
         keep_alive += [idx, w]
         aux.topk_idx_in, aux.topk_w_in = idx.data_ptr(), w.data_ptr()
-    for name, t in (("phi2", phi2), ("phi_inf_sq", phi_inf_sq)):
+    for name, t in (("phi2", phi2), ("phi_inf_sq", phi_inf_sq), ("omega2", omega2)):
         if t is not None:
             if not (t.is_contiguous() and t.dtype == torch.float32 and t.numel() == layer.n_me and t.device == dev):
                 raise ValueError(f"{name} must be a contiguous fp32 [N_e] tensor on the device of x")
             out[name] = t
             setattr(aux, name, t.data_ptr())
     aux.flags = ((CAMERA_SCORE_FORCE_SIMT if force_simt else 0) | (CAMERA_SCORE_CTA_PAIR if cta_pair else 0) | (CAMERA_SCORE_SINGLE_CTA if cta_pair is False else 0) |
-                 (CAMERA_SCORE_ACCUMULATE if accumulate else 0))
+                 (CAMERA_SCORE_ACCUMULATE if accumulate else 0) | (CAMERA_SCORE_OMEGA_GIVEN if omega_given else 0))
     if stage_events:
         for name, (e0, e1) in stage_events.items():
             i = STAGES.index(name)
@@ -451,7 +453,8 @@ def camera_layer_forward(layer: Layer, x: torch.Tensor, *, y: Optional[torch.Ten
 def camera_score_forward_layer(layer: Layer, x: torch.Tensor, alpha: float, *, energy: Optional[torch.Tensor] = None,
                                y: Optional[torch.Tensor] = None, routing_in=None, workspace: Optional[torch.Tensor] = None,
                                phi2: Optional[torch.Tensor] = None, phi_inf_sq: Optional[torch.Tensor] = None,
-                               accumulate: bool = False, cta_pair: Optional[bool] = None,
+                               accumulate: bool = False, omega2: Optional[torch.Tensor] = None,
+                               omega_given: bool = False, cta_pair: Optional[bool] = None,
                                stream: Optional[torch.cuda.Stream] = None):
     """Energies (Algorithm 1) and layer output (Eq. 1-2) of one batch from one pass over W_gate and W_up.
     Returns (energy [N_e] fp32, y [T, d_model] fp32); arguments as for camera_score_layer and camera_layer_forward."""
@@ -465,14 +468,14 @@ def camera_score_forward_layer(layer: Layer, x: torch.Tensor, alpha: float, *, e
         workspace = alloc_workspace(camera_forward_workspace_bytes(layer, T), dev)
     aux = camera_score_aux_t()
     aux.flags = ((CAMERA_SCORE_CTA_PAIR if cta_pair else 0) | (CAMERA_SCORE_SINGLE_CTA if cta_pair is False else 0) |
-                 (CAMERA_SCORE_ACCUMULATE if accumulate else 0))
+                 (CAMERA_SCORE_ACCUMULATE if accumulate else 0) | (CAMERA_SCORE_OMEGA_GIVEN if omega_given else 0))
     keep_alive = []
     if routing_in is not None:
         idx = routing_in[0].to(device=dev, dtype=torch.int32).contiguous()
         w = routing_in[1].to(device=dev, dtype=torch.float32).contiguous()
         keep_alive += [idx, w]
         aux.topk_idx_in, aux.topk_w_in = idx.data_ptr(), w.data_ptr()
-    for name, t in (("phi2", phi2), ("phi_inf_sq", phi_inf_sq)):
+    for name, t in (("phi2", phi2), ("phi_inf_sq", phi_inf_sq), ("omega2", omega2)):
         if t is not None:
             if not (t.is_contiguous() and t.dtype == torch.float32 and t.numel() == layer.n_me and t.device == dev):
                 raise ValueError(f"{name} must be a contiguous fp32 [N_e] tensor on the device of x")

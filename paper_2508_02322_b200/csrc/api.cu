@@ -185,6 +185,7 @@ int score_front(const camera_layer_t* L, const void* x, int64_t T, float alpha, 
   if (aux && ((aux->topk_idx_in == nullptr) != (aux->topk_w_in == nullptr))) return CAMERA_ERR_INVALID_ARG;
   const bool accumulate = aux && (aux->flags & CAMERA_SCORE_ACCUMULATE);
   if (accumulate && (aux->phi2 == nullptr || aux->phi_inf_sq == nullptr)) return CAMERA_ERR_INVALID_ARG;
+  if (aux && (aux->flags & CAMERA_SCORE_OMEGA_GIVEN) && aux->omega2 == nullptr) return CAMERA_ERR_INVALID_ARG;
   {  // every matrix is read with 16-byte vector loads
     uintptr_t bits = reinterpret_cast<uintptr_t>(x) | reinterpret_cast<uintptr_t>(L->w_router) |
                      reinterpret_cast<uintptr_t>(L->w_shared_gate);
@@ -336,7 +337,7 @@ extern "C" int camera_score_layer(const camera_layer_t* L, const void* x, int64_
   const StageTimer tm{aux, st};
 
   tm.begin(CAMERA_STAGE_ROWNORM);
-  CK(launch_rownorm(c, norm_blocks, st));
+  if (!(aux && (aux->flags & CAMERA_SCORE_OMEGA_GIVEN))) CK(launch_rownorm(c, norm_blocks, st));
   tm.end(CAMERA_STAGE_ROWNORM);
 
   tm.begin(CAMERA_STAGE_SCORE);
@@ -368,7 +369,7 @@ constexpr int64_t ANALYZE_BATCH_TOKENS = 65536;   // tokens per host-to-device b
 constexpr int64_t ANALYZE_FIRST_BATCH_TOKENS = 8192;
 
 struct AnalyzeLayout {
-  size_t score, select, x[2], energy, phi2, phi_inf, keep, bits, total;
+  size_t score, select, x[2], energy, phi2, phi_inf, omega2, keep, bits, total;
   size_t score_bytes, select_bytes;
   int64_t batch;
 };
@@ -388,6 +389,7 @@ AnalyzeLayout analyze_layout(const camera_layer_t* L, int64_t T, int n_levels) {
   a.energy = take(sizeof(float) * (size_t)s.n_me);
   a.phi2 = take(sizeof(float) * (size_t)s.n_me);
   a.phi_inf = take(sizeof(float) * (size_t)s.n_me);
+  a.omega2 = take(sizeof(float) * (size_t)s.n_me);
   a.keep = take((size_t)s.n_me);
   a.bits = take((size_t)s.n_me);
   a.total = o;
@@ -447,6 +449,7 @@ extern "C" int camera_analyze_layer_host(const camera_layer_t* L, const void* x_
   memset(&aux, 0, sizeof(aux));
   aux.phi2 = reinterpret_cast<float*>(ws + a.phi2);
   aux.phi_inf_sq = reinterpret_cast<float*>(ws + a.phi_inf);
+  aux.omega2 = reinterpret_cast<float*>(ws + a.omega2);      // the norms of W_down: computed with the first batch only
 
   // Batch sizes.  Nothing overlaps the copy of the first batch, so it is small.  The copy of batch b+1 hides behind the
   // scoring of batch b as long as their sizes differ by less than the ratio of the two rates, tokens copied per ms to
@@ -470,7 +473,7 @@ extern "C" int camera_analyze_layer_host(const camera_layer_t* L, const void* x_
       CK(cudaEventRecord(pipe.copied[buf], pipe.copy));
       CK(cudaStreamWaitEvent(st, pipe.copied[buf], 0));
     }
-    aux.flags = b > 0 ? (uint32_t)CAMERA_SCORE_ACCUMULATE : 0u;
+    aux.flags = b > 0 ? (uint32_t)(CAMERA_SCORE_ACCUMULATE | CAMERA_SCORE_OMEGA_GIVEN) : 0u;
     rc = camera_score_layer(L, ws + a.x[buf], n, alpha, d_energy, &aux, ws + a.score, a.score_bytes, cuda_stream);
     if (rc != CAMERA_OK) return rc;
     if (batched) CK(cudaEventRecord(pipe.consumed[buf], st));

@@ -743,7 +743,10 @@ int forward_impl(const camera_layer_t* L, const void* x, int64_t T, float alpha,
   if (rc != CAMERA_OK) return rc;
   if (!f.use_umma) return CAMERA_ERR_UNSUPPORTED_SHAPE;
   const ScoreCtx& c = f.c;
-  if (energy != nullptr && launch_rownorm(c, f.norm_blocks, st) != cudaSuccess) { cudaGetLastError(); return CAMERA_ERR_CUDA; }
+  if (energy != nullptr && !(a2.flags & CAMERA_SCORE_OMEGA_GIVEN) && launch_rownorm(c, f.norm_blocks, st) != cudaSuccess) {
+    cudaGetLastError();
+    return CAMERA_ERR_CUDA;
+  }
   if (T == 0) {   // no tokens: the scores of the batches so far (or zeros), no output rows
     if (energy != nullptr && launch_combine(c, st) != cudaSuccess) { cudaGetLastError(); return CAMERA_ERR_CUDA; }
     return CAMERA_OK;

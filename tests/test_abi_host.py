@@ -65,6 +65,10 @@ def test_argument_errors_return_before_any_launch(P):
     assert P.lib.camera_score_layer(C.byref(ok), 4096, 10, C.c_float(1.5), 4096, None, 4096, 1 << 30, None) == -1
     assert P.lib.camera_score_layer(C.byref(ok), 4096, 10, C.c_float(0.5), None, None, 4096, 1 << 30, None) == -1
     assert P.lib.camera_score_layer(C.byref(ok), 4096, 10, C.c_float(0.5), 4096, None, None, 0, None) == -3
+    from paper_2508_02322_b200.binding import camera_score_aux_t, CAMERA_SCORE_OMEGA_GIVEN
+    aux = camera_score_aux_t()
+    aux.flags = CAMERA_SCORE_OMEGA_GIVEN                      # says the norms are given, gives none
+    assert P.lib.camera_score_layer(C.byref(ok), 4096, 10, C.c_float(0.5), 4096, C.byref(aux), 4096, 1 << 30, None) == -1
     seg = (C.c_int64 * 2)(0, 10)
     bad = (C.c_int64 * 2)(1, 10)
     assert P.lib.camera_select_prune(4096, seg, 1, C.c_double(1.0), None, 0, 4096, None, None, 4096, 1 << 20, None) == -1

@@ -132,11 +132,12 @@ def test_scores_and_output_from_one_pass(P, cta_pair):
     phi2 = torch.empty(layer.n_me, dtype=torch.float32, device=DEV)
     pinf_t = torch.empty_like(phi2)
     E2 = torch.empty_like(phi2)
+    om = torch.empty_like(phi2)             # the W_down norms: computed with the first batch, given to the second
     y2 = torch.empty_like(y)
     ws = P.alloc_workspace(P.camera_forward_workspace_bytes(layer, 800), DEV)
     for i, (t0, t1) in enumerate([(0, 800), (800, 1300)]):
         P.camera_score_forward_layer(layer, X[t0:t1], 0.95, energy=E2, y=y2[t0:t1], workspace=ws, phi2=phi2,
-                                     phi_inf_sq=pinf_t, accumulate=i > 0, cta_pair=cta_pair,
+                                     phi_inf_sq=pinf_t, accumulate=i > 0, cta_pair=cta_pair, omega2=om, omega_given=i > 0,
                                      routing_in=(rin[0][t0:t1], rin[1][t0:t1]))
     assert P.camera_read_status(ws) == 0
     assert_close("energy accumulated over two batches", E2.cpu().numpy(), O.energy(p2, pinf, w2, float(np.float32(0.95))))

@@ -271,11 +271,13 @@ def test_accumulate_over_token_batches(P, kernel):
     ws = P.alloc_workspace(P.camera_score_workspace_bytes(layer, 1499), DEV)
     phi2 = torch.empty(layer.n_me, dtype=torch.float32, device=DEV)
     phi_inf = torch.empty_like(phi2)
+    om = torch.empty_like(phi2)             # the W_down norms: computed with the first batch, given to the later ones
     idx, w = [], []
     out = None
     for b, (t0, t1) in enumerate(((0, 1000), (1000, 1001), (1001, 2500))):
         out = P.camera_score_layer(layer, X[t0:t1].contiguous(), 0.95, details=True, workspace=ws, phi2=phi2,
-                                   phi_inf_sq=phi_inf, accumulate=b > 0, force_simt=kernel == "simt")
+                                   phi_inf_sq=phi_inf, accumulate=b > 0, omega2=om, omega_given=b > 0,
+                                   force_simt=kernel == "simt")
         idx.append(out["topk_idx"].cpu().numpy().astype(np.int64))
         w.append(out["topk_w"].cpu().numpy().astype(np.float64))
     assert P.camera_read_status(ws) == 0
