@@ -33,7 +33,7 @@ def random_cfg(r):
         router_bias_std=float(r.choice([0.0, 0.5, 2.0])), weight_std=0.05, norm_topk=bool(r.integers(0, 2)))
 
 
-@pytest.mark.parametrize("seed", range(10))
+@pytest.mark.parametrize("seed", range(14))
 def test_random_layers(P, seed):
     from paper_2508_02322_b200 import workloads as W
     r = np.random.default_rng(1000 + seed)
@@ -68,3 +68,16 @@ def test_random_layers(P, seed):
         gi, gw = routing
         ref_y = oracle_forward(to_oracle_layer(L), f64(X), (gi.cpu().numpy().astype(np.int64), gw.cpu().numpy().astype(np.float64)))
         assert_output_close(f"fuzz {seed} layer output", y.cpu().numpy(), ref_y)
+        # scores and output from one pass, then the retained micro-experts' output from the h it leaves behind
+        from _gpu import assert_close
+        T = int(X.shape[0])
+        ws = P.alloc_workspace(P.camera_forward_workspace_bytes(layer, T), DEV)
+        E1, y1 = P.camera_score_forward_layer(layer, X, alpha, routing_in=routing, workspace=ws)
+        assert P.camera_read_status(ws) == 0
+        rt = (gi.cpu().numpy().astype(np.int64), gw.cpu().numpy().astype(np.float64))
+        p2, pinf, w2 = O.camera_components(to_oracle_layer(L), f64(X), routing=rt)
+        assert_close(f"fuzz {seed} one-pass energy", E1.cpu().numpy(), O.energy(p2, pinf, w2, float(np.float32(alpha))))
+        assert_output_close(f"fuzz {seed} one-pass output", y1.cpu().numpy(), ref_y)
+        y_hat = P.camera_pruned_output(layer, P.camera_mask_down_columns(layer, keep), T, ws)
+        ref_hat = oracle_forward(ref, f64(X), (gi.cpu().numpy().astype(np.int64), gw.cpu().numpy().astype(np.float64)))
+        assert_output_close(f"fuzz {seed} pruned output", y_hat.cpu().numpy(), ref_hat)
