@@ -395,6 +395,24 @@ def test_sliced_layer_decodes_like_the_retained_micro_experts():
     assert abs(err - O.decode_error(O.phi_matrix(layer, X), O.basis(layer), np.nonzero(keep == 0)[0])) <= 1e-10 * max(err, 1)
 
 
+def test_zeroing_pruned_columns_of_w_down_equals_slicing():
+    """Phi[:,S] W[S,:] is also Phi times W with the rows outside S set to zero: the full layer with the pruned columns
+    of W_down zeroed (gate and up untouched) gives the sliced layer's output.  The GPU's pruned-output call rests on it."""
+    import copy
+    r = rng(42)
+    layer = random_layer(r, d=6, d_ff=(5, 7, 4), n_shared=1, top_k=2, shared_gate=True)
+    X = r.standard_normal((19, 6))
+    off = O.me_offsets(layer)
+    keep = O.select_prune(O.energy(*O.camera_components(layer, X), 0.95), 0.5)
+    keep[off[1]:off[2]] = 0                                   # an expert that loses everything
+    lists, _ = O.sub_index_lists(keep, off, [1])
+    masked = copy.deepcopy(layer)
+    masked.w_down = [layer.w_down[e] * keep[off[e]:off[e + 1]][None, :] for e in range(len(layer.w_down))]
+    assert np.allclose(O.forward(masked, X), O.forward(O.slice_layer(layer, lists), X), rtol=1e-12, atol=1e-12)
+    S = np.nonzero(keep)[0]
+    assert np.allclose(O.forward(masked, X), O.phi_matrix(layer, X)[:, S] @ O.basis(layer)[S, :], rtol=1e-12, atol=1e-12)
+
+
 def test_reordering_by_class_keeps_the_layer_and_colocates_classes():
     r = rng(41)
     layer = random_layer(r, d=6, d_ff=(8, 5, 7), n_shared=0, top_k=2)
