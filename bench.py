@@ -2,8 +2,9 @@
 """Benchmark of the CAMERA analysis hot path on B200.
 
 One step = one MoE layer analysed end to end: camera_score_layer (router, permutation, W_down
-norms, fused gate/up scoring, energy), camera_select_prune at 20/40/60 % and camera_alloc_bits for a
-2.25-bit budget, on synthetic calibration tokens of the Qwen2-57B-A14B layer shape.
+norms, fused gate/up scoring, energy), then the prune masks at 20/40/60 % and the bit-widths of a 2.25-bit budget
+(camera_select_all: the results of camera_select_prune x 3 and camera_alloc_bits from one set of radix passes), on
+synthetic calibration tokens of the Qwen2-57B-A14B layer shape.
 
     python bench.py --gpus N --steps K --warmup W            (N > 1: launched by torch.distributed.run)
     python bench.py --impl reference ...                      (the float64 CPU oracle on a bounded sample)
@@ -32,8 +33,8 @@ BIT_RATIOS, BIT_LEVELS = (0.2, 0.6, 0.2), (3, 2, 1)     # average 2 bits + 0.25 
 ALPHA = 0.95
 PAPER_CONTEXT = "paper: <5 min for the full Qwen2-57B-A14B analysis on one A100-40GB (incl. model forwards)"
 # kernels launched by one step: score = router, block scan, plan, permute, pad, norms, scoring, combine;
-# every selection = 8 histogram passes + mark
-LAUNCHES_PER_STEP = 8 + 9 * (len(PRUNE_RATIOS) + 1)
+# the selections = 8 histogram passes + mark
+LAUNCHES_PER_STEP = 8 + 9
 # DRAM bytes (read + write) per gate/up flop of the scoring kernel, from the committed ncu capture of a
 # 1/8 slice of the layer whose traffic grows in proportion to the flop (profiles/k_score_umma_qwen2_slice.md).
 SCORE_KERNEL_DRAM_BYTES_PER_FLOP = 4.483e9 / 1.924e13
@@ -327,7 +328,7 @@ def main():
     Xs = [W.make_tokens(cfg, seed=0, layer_id=rank + world * i, device=dev) for i in range(2)]
     n_me = layer.n_me
     ws_score = P.alloc_workspace(P.camera_score_workspace_bytes(layer, T), dev)
-    ws_sel = P.alloc_workspace(P.camera_select_workspace_bytes(n_me, 1, len(BIT_LEVELS)), dev)
+    ws_sel = P.alloc_workspace(P.camera_select_workspace_bytes(n_me, 1, len(PRUNE_RATIOS) + len(BIT_LEVELS)), dev)
     energy = torch.empty(n_me, dtype=torch.float32, device=dev)
     keep = torch.empty((len(PRUNE_RATIOS), n_me), dtype=torch.uint8, device=dev)
     bits = torch.empty(n_me, dtype=torch.uint8, device=dev)
@@ -348,9 +349,7 @@ def main():
         else:
             P.camera_score_layer(layer, Xs[i % 2], ALPHA, energy=energy, workspace=ws_score, stage_events=events,
                                  cta_pair=(True if args.cta_pair else (False if args.single_cta else None)))
-        for j, r in enumerate(PRUNE_RATIOS):
-            P.camera_select_prune(energy, r, workspace=ws_sel, keep_mask=keep[j])
-        P.camera_alloc_bits(energy, BIT_RATIOS, BIT_LEVELS, workspace=ws_sel, bits_out=bits)
+        P.camera_select_all(energy, PRUNE_RATIOS, BIT_RATIOS, BIT_LEVELS, workspace=ws_sel, keep_masks=keep, bits_out=bits)
 
     def sync_all():
         torch.cuda.synchronize()
@@ -500,13 +499,13 @@ def main():
         nl = cfg.n_layers
         Eall = energy.repeat(nl) * (1.0 + torch.arange(nl * n_me, device=dev) // n_me).float()
         seg = [i * n_me for i in range(nl + 1)]
-        keep_all = torch.empty(nl * n_me, dtype=torch.uint8, device=dev)
-        ws_all = P.alloc_workspace(P.camera_select_workspace_bytes(nl * n_me, nl, len(BIT_LEVELS)), dev)
+        keep_all = torch.empty((len(PRUNE_RATIOS), nl * n_me), dtype=torch.uint8, device=dev)
+        bits_all = torch.empty(nl * n_me, dtype=torch.uint8, device=dev)
+        ws_all = P.alloc_workspace(P.camera_select_workspace_bytes(nl * n_me, nl, len(PRUNE_RATIOS) + len(BIT_LEVELS)), dev)
         s0, s1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         def select_all():
-            for r in PRUNE_RATIOS:
-                P.camera_select_prune(Eall, r, seg_offsets=seg, workspace=ws_all, keep_mask=keep_all)
-            P.camera_alloc_bits(Eall, BIT_RATIOS, BIT_LEVELS, seg_offsets=seg, workspace=ws_all, bits_out=keep_all)
+            P.camera_select_all(Eall, PRUNE_RATIOS, BIT_RATIOS, BIT_LEVELS, seg_offsets=seg, workspace=ws_all,
+                                keep_masks=keep_all, bits_out=bits_all)
         for _ in range(3):
             select_all()
         sync_all()
@@ -515,11 +514,11 @@ def main():
             select_all()
         s1.record(stream); sync_all()
         sel_ms = s0.elapsed_time(s1) / 10
-        sel_bytes = 4 * (9 * 4 * nl * n_me + nl * n_me)     # per call: 9 passes over the fp32 keys, one byte per label out
-        select_model = {"what": f"3 prune masks + bit allocation for {nl} layers as segments of one call", "ms": sel_ms,
+        sel_bytes = 9 * 4 * nl * n_me + 4 * nl * n_me       # 9 passes over the fp32 keys, four bytes of labels per key out
+        select_model = {"what": f"3 prune masks + bit allocation for {nl} layers as segments of one camera_select_all call", "ms": sel_ms,
                         "algorithmic_gb": sel_bytes / 1e9, "achieved_gbs": sel_bytes / 1e9 / (sel_ms * 1e-3),
                         "frac_of_hbm_peak": sel_bytes / 1e9 / (sel_ms * 1e-3) / load_peaks()["hbm_gbs"]}
-        del Eall, keep_all, ws_all
+        del Eall, keep_all, bits_all, ws_all
 
     # ---- end to end through the host-buffer entry point: H2D of the tokens, D2H of the results, every step
     e2e = None

@@ -182,6 +182,20 @@ int camera_alloc_bits(const float* energy, const int64_t* seg_offsets, int32_t n
                       void* workspace, size_t workspace_bytes, void* cuda_stream);
 
 /*
+ * Several CAMERA-P masks (Algorithm 2, TopSelect at several prune ratios) and the CAMERA-Q bit-widths (Algorithm 3,
+ * ListSplitByRatio) of the same energies from one set of radix passes: every threshold is a rank of the same keys, so
+ * the eight histogram passes find them together and one pass writes all outputs (10 launches instead of 9 per mask
+ * and 9 for the bit-widths).  The results are those of camera_select_prune / camera_alloc_bits, bit for bit.
+ * prune_ratios: HOST [n_prune];  keep_masks: DEVICE uint8 [n_prune][N] (mask p at keep_masks + p * N, N =
+ * seg_offsets[n_segments]);  ratios, bits, n_levels, bits_out as for camera_alloc_bits, bits_out may be NULL (no
+ * bit-widths; ratios, bits, n_levels are then ignored).  n_prune + n_levels - 1 <= 7, else CAMERA_ERR_INVALID_ARG.
+ * workspace: camera_select_workspace_bytes(N, n_segments, n_prune + n_levels) bytes.
+ */
+int camera_select_all(const float* energy, const int64_t* seg_offsets, int32_t n_segments, const double* prune_ratios,
+                      int32_t n_prune, uint8_t* keep_masks, const double* ratios, const int32_t* bits, int32_t n_levels,
+                      uint8_t* bits_out, void* workspace, size_t workspace_bytes, void* cuda_stream);
+
+/*
  * camera_select_prune without a workspace argument (the paper has no counterpart; this exists for
  * the sake of integration).  Some hosts of this library may not create device allocations at all:
  * a plug-in inside a serving process whose memory pool already owns the whole GPU, a callback that

@@ -90,6 +90,10 @@ def _load() -> C.CDLL:
     lib.camera_score_forward_layer.argtypes = [C.POINTER(camera_layer_t), C.c_void_p, C.c_int64, C.c_float, C.c_void_p,
                                                C.c_void_p, C.POINTER(camera_score_aux_t), C.c_void_p, C.c_size_t,
                                                C.c_void_p]
+    lib.camera_select_all.restype = C.c_int
+    lib.camera_select_all.argtypes = [C.c_void_p, C.POINTER(C.c_int64), C.c_int32, C.POINTER(C.c_double), C.c_int32,
+                                      C.c_void_p, C.POINTER(C.c_double), C.POINTER(C.c_int32), C.c_int32, C.c_void_p,
+                                      C.c_void_p, C.c_size_t, C.c_void_p]
     lib.camera_mask_down_columns.restype = C.c_int
     lib.camera_mask_down_columns.argtypes = [C.POINTER(camera_layer_t), C.c_void_p, C.POINTER(C.c_void_p), C.c_void_p]
     lib.camera_pruned_output.restype = C.c_int
@@ -276,6 +280,32 @@ def camera_read_status(workspace: torch.Tensor, stream: Optional[torch.cuda.Stre
 def _segments(n_total: int, seg_offsets):
     seg = [0, n_total] if seg_offsets is None else [int(v) for v in seg_offsets]
     return (C.c_int64 * len(seg))(*seg), len(seg) - 1
+
+
+def camera_select_all(energy: torch.Tensor, prune_ratios: Sequence[float], ratios: Optional[Sequence[float]] = None,
+                      bits: Optional[Sequence[int]] = None, *, seg_offsets=None, workspace: Optional[torch.Tensor] = None,
+                      keep_masks: Optional[torch.Tensor] = None, bits_out: Optional[torch.Tensor] = None,
+                      stream: Optional[torch.cuda.Stream] = None):
+    """The keep masks at several prune ratios (uint8 [len(prune_ratios), N]) and, with ratios / bits, the bit-widths
+    (uint8 [N]) from one set of radix passes.  Returns (keep_masks, bits_out); bits_out is None without ratios."""
+    n = energy.numel()
+    dev = energy.device
+    seg, n_seg = _segments(n, seg_offsets)
+    n_prune = len(prune_ratios)
+    L = len(ratios) if ratios is not None else 0
+    if keep_masks is None:
+        keep_masks = torch.empty((n_prune, n), dtype=torch.uint8, device=dev)
+    if ratios is not None and bits_out is None:
+        bits_out = torch.empty(n, dtype=torch.uint8, device=dev)
+    if workspace is None:
+        workspace = alloc_workspace(camera_select_workspace_bytes(n, n_seg, max(2, n_prune + max(L, 1))), dev)
+    pr = (C.c_double * max(n_prune, 1))(*[float(v) for v in prune_ratios])
+    r = (C.c_double * max(L, 1))(*[float(v) for v in (ratios or [])])
+    b = (C.c_int32 * max(L, 1))(*[int(v) for v in (bits or [])])
+    _check(lib.camera_select_all(energy.data_ptr(), seg, n_seg, pr, n_prune, keep_masks.data_ptr(), r, b, L,
+                                 _ptr(bits_out) if ratios is not None else None, workspace.data_ptr(), workspace.numel(),
+                                 _stream_ptr(stream)), "camera_select_all")
+    return keep_masks, (bits_out if ratios is not None else None)
 
 
 def camera_select_prune(energy: torch.Tensor, prune_ratio: float, *, seg_offsets=None,

@@ -379,7 +379,7 @@ AnalyzeLayout analyze_layout(const camera_layer_t* L, int64_t T, int n_levels) {
   const ScoreLayout s = score_layout(L, a.batch);
   const size_t esz = L->dtype == CAMERA_BF16 ? 2 : 4;
   a.score_bytes = s.total;
-  a.select_bytes = camera_select_workspace_bytes(s.n_me, 1, n_levels < 2 ? 2 : n_levels);
+  a.select_bytes = camera_select_workspace_bytes(s.n_me, 1, MAX_LEVELS);     // room for every mask and class boundary at once
   size_t o = 0;
   auto take = [&](size_t bytes) { size_t at = o; o = up256(o + bytes); return at; };
   a.score = take(a.score_bytes);
@@ -390,7 +390,7 @@ AnalyzeLayout analyze_layout(const camera_layer_t* L, int64_t T, int n_levels) {
   a.phi2 = take(sizeof(float) * (size_t)s.n_me);
   a.phi_inf = take(sizeof(float) * (size_t)s.n_me);
   a.omega2 = take(sizeof(float) * (size_t)s.n_me);
-  a.keep = take((size_t)s.n_me);
+  a.keep = take((size_t)s.n_me * (MAX_LEVELS - 1));                          // up to 7 masks side by side
   a.bits = take((size_t)s.n_me);
   a.total = o;
   return a;
@@ -483,6 +483,17 @@ extern "C" int camera_analyze_layer_host(const camera_layer_t* L, const void* x_
   }
   if (energy_host) CK(cudaMemcpyAsync(energy_host, d_energy, sizeof(float) * (size_t)n_me, cudaMemcpyDeviceToHost, st));
   const int64_t seg[2] = {0, n_me};
+  if (n_prune >= 1 && n_prune + n_levels - 1 <= MAX_LEVELS - 1) {
+    // every threshold from one set of radix passes
+    rc = camera_select_all(d_energy, seg, 1, prune_ratios, n_prune, d_keep, ratios, bits, n_levels, d_bits, ws + a.select,
+                           a.select_bytes, cuda_stream);
+    if (rc != CAMERA_OK) return rc;
+    if (keep_host) CK(cudaMemcpyAsync(keep_host, d_keep, (size_t)n_prune * n_me, cudaMemcpyDeviceToHost, st));
+    if (bits_host) CK(cudaMemcpyAsync(bits_host, d_bits, (size_t)n_me, cudaMemcpyDeviceToHost, st));
+    int32_t status_all = 0;
+    rc = camera_read_status(ws + a.score, cuda_stream, &status_all);
+    return rc != CAMERA_OK ? rc : status_all;
+  }
   for (int p = 0; p < n_prune; ++p) {
     rc = camera_select_prune(d_energy, seg, 1, prune_ratios[p], nullptr, 0, d_keep, nullptr, nullptr, ws + a.select,
                              a.select_bytes, cuda_stream);

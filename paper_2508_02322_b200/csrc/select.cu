@@ -10,6 +10,8 @@
 #include <math.h>
 #include <string.h>
 
+#include <vector>
+
 #include "common.cuh"
 
 namespace camera {
@@ -143,6 +145,32 @@ k_select_mark(const float* __restrict__ energy, const long long* seg_off, const 
   }
 }
 
+// The mark pass of camera_select_all: thresholds 0 .. n_prune-1 each give a keep mask of their own, the remaining
+// n_thr - n_prune thresholds are the class boundaries of the bit-width allocation.
+__global__ void __launch_bounds__(SEL_THREADS)
+k_select_mark_all(const float* __restrict__ energy, const long long* seg_off, const long long* ranks, SelState* S,
+                  const unsigned* hist, int n_seg, int n_thr, int n_prune, LevelValues lv, long long n_total,
+                  unsigned char* keep_out, unsigned char* bits_out) {
+  __shared__ SelState st[MAX_THR];
+  const int seg = blockIdx.y;
+  const long long begin = seg_off[seg], len = seg_off[seg + 1] - begin;
+  advance_state(SEL_PASSES, seg, n_thr, len, ranks, S, hist, n_seg, st);
+  __syncthreads();
+  if (blockIdx.x == 0 && threadIdx.x < n_thr)
+    S[((size_t)(SEL_PASSES - 1) * n_seg + seg) * n_thr + threadIdx.x] = st[threadIdx.x];
+  const int n_bounds = n_thr - n_prune;
+  for (long long i = (long long)blockIdx.x * SEL_THREADS + threadIdx.x; i < len; i += (long long)gridDim.x * SEL_THREADS) {
+    const unsigned long long key = make_key(energy[begin + i], (unsigned)i);
+    for (int j = 0; j < n_prune; ++j)
+      keep_out[(size_t)j * n_total + begin + i] = (st[j].rank >= 0 && key >= st[j].prefix) ? 1 : 0;
+    if (bits_out != nullptr) {
+      int above = 0;
+      for (int j = n_prune; j < n_thr; ++j) above += (st[j].rank >= 0 && key >= st[j].prefix) ? 1 : 0;
+      bits_out[begin + i] = lv.v[n_bounds - above];
+    }
+  }
+}
+
 // One CTA per expert: how many of its micro-experts fall in each class (or are retained).
 __global__ void __launch_bounds__(SEL_THREADS)
 k_class_counts(const float* __restrict__ energy, const long long* seg_off, const SelState* S, int n_seg, int n_thr,
@@ -193,9 +221,12 @@ SelLayout sel_layout(int n_seg, int n_thr) {
 long long floor_count(double ratio, long long n) { return (long long)floor(ratio * (double)n + 1e-9); }
 
 // ranks_host: [n_seg * n_thr] target ascending ranks (a rank >= the segment length selects nothing).
+// n_prune >= 0 selects the mark pass of camera_select_all: `out` then holds n_prune masks of seg_offsets[n_seg] bytes
+// and bits_out (may be null) gets the class values.
 int select_core(const float* energy, const int64_t* seg_offsets, int n_seg, int n_thr, const long long* ranks_host,
                 LevelValues lv, const int64_t* expert_offsets, int n_experts, int n_classes_out, unsigned char* out,
-                int* counts, float* thresholds, void* ws, size_t ws_bytes, cudaStream_t st) {
+                int* counts, float* thresholds, void* ws, size_t ws_bytes, cudaStream_t st, int n_prune = -1,
+                unsigned char* bits_out = nullptr) {
   const SelLayout L = sel_layout(n_seg, n_thr);
   if (ws == nullptr || ws_bytes < L.total) return CAMERA_ERR_WORKSPACE;
   char* base = static_cast<char*>(ws);
@@ -216,7 +247,11 @@ int select_core(const float* energy, const int64_t* seg_offsets, int n_seg, int 
     const dim3 grid((unsigned)gx, (unsigned)n_seg);
     for (int p = 0; p < SEL_PASSES; ++p)
       k_select_hist<<<grid, SEL_THREADS, 0, st>>>(p, energy, d_seg, d_ranks, d_state, d_hist, n_seg, n_thr);
-    k_select_mark<<<grid, SEL_THREADS, 0, st>>>(energy, d_seg, d_ranks, d_state, d_hist, n_seg, n_thr, lv, out, thresholds);
+    if (n_prune >= 0)
+      k_select_mark_all<<<grid, SEL_THREADS, 0, st>>>(energy, d_seg, d_ranks, d_state, d_hist, n_seg, n_thr, n_prune, lv,
+                                                      (long long)seg_offsets[n_seg], out, bits_out);
+    else
+      k_select_mark<<<grid, SEL_THREADS, 0, st>>>(energy, d_seg, d_ranks, d_state, d_hist, n_seg, n_thr, lv, out, thresholds);
   }
   if (counts != nullptr && expert_offsets != nullptr && n_experts > 0) {
     if (max_len > 0)
@@ -300,6 +335,47 @@ extern "C" int camera_alloc_bits(const float* energy, const int64_t* seg_offsets
                              bits_out, class_counts, nullptr, workspace, workspace_bytes, static_cast<cudaStream_t>(cuda_stream));
   delete[] ranks;
   return rc;
+}
+
+extern "C" int camera_select_all(const float* energy, const int64_t* seg_offsets, int32_t n_segments,
+                                 const double* prune_ratios, int32_t n_prune, uint8_t* keep_masks, const double* ratios,
+                                 const int32_t* bits, int32_t n_levels, uint8_t* bits_out, void* workspace,
+                                 size_t workspace_bytes, void* cuda_stream) {
+  if (!segments_ok(seg_offsets, n_segments) || n_prune < 0 || (n_prune > 0 && (prune_ratios == nullptr || keep_masks == nullptr)))
+    return CAMERA_ERR_INVALID_ARG;
+  if (bits_out != nullptr && (ratios == nullptr || bits == nullptr || n_levels < 2 || n_levels > MAX_LEVELS))
+    return CAMERA_ERR_INVALID_ARG;
+  const int n_bounds = bits_out != nullptr ? n_levels - 1 : 0;
+  const int n_thr = n_prune + n_bounds;
+  if (n_thr < 1 || n_thr > MAX_THR) return CAMERA_ERR_INVALID_ARG;
+  if (seg_offsets[n_segments] > 0 && energy == nullptr) return CAMERA_ERR_INVALID_ARG;
+  for (int p = 0; p < n_prune; ++p)
+    if (!(prune_ratios[p] >= 0.0 && prune_ratios[p] < 1.0)) return CAMERA_ERR_INVALID_ARG;
+  LevelValues lv;
+  memset(&lv, 0, sizeof(lv));
+  if (bits_out != nullptr) {
+    double sum = 0.0;
+    for (int j = 0; j < n_levels; ++j) {
+      if (!(ratios[j] >= 0.0) || bits[j] < 0 || bits[j] > 255) return CAMERA_ERR_INVALID_ARG;
+      sum += ratios[j];
+      lv.v[j] = (unsigned char)bits[j];
+    }
+    if (fabs(sum - 1.0) > 1e-9) return CAMERA_ERR_INVALID_ARG;
+  }
+  std::vector<long long> ranks((size_t)n_segments * n_thr);
+  for (int s = 0; s < n_segments; ++s) {
+    const long long n = seg_offsets[s + 1] - seg_offsets[s];
+    for (int p = 0; p < n_prune; ++p) ranks[(size_t)s * n_thr + p] = floor_count(prune_ratios[p], n);   // as camera_select_prune
+    double acc = 0.0;
+    for (int m = 1; m <= n_bounds; ++m) {                                                              // as camera_alloc_bits
+      acc += ratios[m - 1];
+      long long cm = floor_count(acc, n);
+      if (cm > n) cm = n;
+      ranks[(size_t)s * n_thr + n_prune + (m - 1)] = n - cm;
+    }
+  }
+  return select_core(energy, seg_offsets, n_segments, n_thr, ranks.data(), lv, nullptr, 0, 0, keep_masks, nullptr, nullptr,
+                     workspace, workspace_bytes, static_cast<cudaStream_t>(cuda_stream), n_prune, bits_out);
 }
 
 // ---------------------------------------------------------------------------------------------

@@ -74,6 +74,13 @@ def test_argument_errors_return_before_any_launch(P):
     assert P.lib.camera_select_prune(4096, seg, 1, C.c_double(1.0), None, 0, 4096, None, None, 4096, 1 << 20, None) == -1
     assert P.lib.camera_select_prune(4096, bad, 1, C.c_double(0.5), None, 0, 4096, None, None, 4096, 1 << 20, None) == -1
     assert P.lib.camera_select_prune(4096, seg, 1, C.c_double(0.5), None, 0, 4096, None, None, 4096, 16, None) == -3
+    pr = (C.c_double * 3)(0.2, 0.4, 0.6)
+    rt = (C.c_double * 3)(0.2, 0.6, 0.2)
+    bt = (C.c_int32 * 3)(3, 2, 1)
+    assert P.lib.camera_select_all(4096, seg, 1, pr, 3, None, rt, bt, 3, 4096, 4096, 1 << 20, None) == -1     # no masks
+    assert P.lib.camera_select_all(4096, seg, 1, pr, 0, None, rt, bt, 3, None, 4096, 1 << 20, None) == -1     # nothing asked for
+    assert P.lib.camera_select_all(4096, seg, 1, (C.c_double * 1)(1.0), 1, 4096, rt, bt, 3, 4096, 4096, 1 << 20, None) == -1
+    assert P.lib.camera_select_all(4096, seg, 1, pr, 3, 4096, rt, bt, 3, 4096, 4096, 16, None) == -3
     r = (C.c_double * 3)(0.2, 0.5, 0.2)
     b = (C.c_int32 * 3)(3, 2, 1)
     assert P.lib.camera_alloc_bits(4096, seg, 1, r, b, 3, None, 0, 4096, None, 4096, 1 << 20, None) == -1   # ratios sum

@@ -232,6 +232,39 @@ def test_alloc_bits_bit_exact(P, n, scheme):
     assert np.array_equal(counts.cpu().numpy(), O.sub_index(ref_cls, off, len(ratios)))
 
 
+@pytest.mark.parametrize("n", [1, 37, 5000, 184320])
+def test_select_all_equals_the_separate_selections(P, n):
+    """Several masks and the bit-widths from one set of radix passes: the oracle's results bit for bit (with ties),
+    also over segments of unequal length, and with the bit-widths left out."""
+    E = _energies(n, 3 * n + 1)
+    prune = [0.2, 0.4, 0.6]
+    keep, bits = P.camera_select_all(E.to(DEV), prune, [0.2, 0.6, 0.2], [3, 2, 1])
+    for j, r in enumerate(prune):
+        assert np.array_equal(keep[j].cpu().numpy(), O.select_prune(E.numpy(), r)), f"mask at {r}"
+    assert np.array_equal(bits.cpu().numpy(), O.alloc_bits(E.numpy(), [0.2, 0.6, 0.2], [3, 2, 1])[0])
+    # four classes and four masks: seven thresholds, the most one call takes; an eighth is refused
+    keep4, bits4 = P.camera_select_all(E.to(DEV), [0.0, 0.3, 0.5, 0.97], [0.25, 0.25, 0.25, 0.25], [8, 4, 3, 2])
+    for j, r in enumerate([0.0, 0.3, 0.5, 0.97]):
+        assert np.array_equal(keep4[j].cpu().numpy(), O.select_prune(E.numpy(), r))
+    assert np.array_equal(bits4.cpu().numpy(), O.alloc_bits(E.numpy(), [0.25, 0.25, 0.25, 0.25], [8, 4, 3, 2])[0])
+    with pytest.raises(P.CameraError):
+        P.camera_select_all(E.to(DEV), [0.1, 0.2, 0.3, 0.4, 0.5], [0.25, 0.25, 0.25, 0.25], [8, 4, 3, 2])
+    only, none = P.camera_select_all(E.to(DEV), [0.4])
+    assert none is None and np.array_equal(only[0].cpu().numpy(), O.select_prune(E.numpy(), 0.4))
+
+
+def test_select_all_over_segments(P):
+    sizes = [4096, 1000, 0, 7777, 3]
+    seg = np.concatenate([[0], np.cumsum(sizes)])
+    E = _energies(int(seg[-1]), 98)
+    keep, bits = P.camera_select_all(E.to(DEV), [0.2, 0.6], [0.1, 0.8, 0.1], [4, 3, 2], seg_offsets=seg.tolist())
+    for j, r in enumerate([0.2, 0.6]):
+        ref = np.concatenate([O.select_prune(E.numpy()[seg[s]:seg[s + 1]], r) for s in range(len(sizes))])
+        assert np.array_equal(keep[j].cpu().numpy(), ref)
+    ref_bits = np.concatenate([O.alloc_bits(E.numpy()[seg[s]:seg[s + 1]], [0.1, 0.8, 0.1], [4, 3, 2])[0] for s in range(len(sizes))])
+    assert np.array_equal(bits.cpu().numpy(), ref_bits)
+
+
 def test_bit_budget_on_gpu(P):
     """The appendix' worked example realised by the allocation: [3,2,1] x [0.1,0.8,0.1] averages 2 bits."""
     E = _energies(12800, 5, ties=False)
