@@ -144,8 +144,7 @@ def blas_threads() -> int:
 
 def oracle_prepare(L, X):
     """Widens the stored weights and tokens to float64 for the oracle (not timed)."""
-    sys.path.insert(0, os.path.join(ROOT, "tests"))
-    from _util import f64, to_oracle_layer
+    from oracle import f64, to_oracle_layer
     return to_oracle_layer(L), f64(X)
 
 

@@ -146,8 +146,32 @@ int camera_score_layer(const camera_layer_t* layer, const void* x, int64_t n_tok
                        void* workspace, size_t workspace_bytes, void* cuda_stream);
 
 /* Synchronises the stream, reads the workspace's status word (0 = fine, else a
- * camera_status_t recorded by a kernel) into *status_out and clears nothing. */
+ * camera_status_t recorded by a kernel) into *status_out and clears nothing.
+ * Kernels record CAMERA_ERR_DEVICE_TIMEOUT (a bounded wait ran out), CAMERA_ERR_INVALID_ARG (a
+ * token's routing cannot be used: a prescribed expert index out of range or named twice by one
+ * token, or no finite softmax because x or the router holds a NaN or an infinity; such a token
+ * is given coefficient 0 everywhere, so the call still finishes and every index stays in range)
+ * and CAMERA_ERR_WORKSPACE (the token lists outgrew a workspace smaller than the query's size). */
 int camera_read_status(const void* workspace, void* cuda_stream, int32_t* status_out);
+
+/*
+ * Limit of the waits inside the tensor-core kernels (a thread that waits for a copy or for
+ * another warp gives up after this long, the kernel records CAMERA_ERR_DEVICE_TIMEOUT and
+ * returns normally).  Process wide, read by every later call; 4 s unless set.  1 us .. 600 s,
+ * else CAMERA_ERR_INVALID_ARG.  The paper has no counterpart: this is the library's error
+ * convention (device-side trouble surfaces through the status word, never as a trap or a hang).
+ */
+int camera_set_wait_limit_ns(uint64_t limit_ns);
+uint64_t camera_get_wait_limit_ns(void);
+
+/*
+ * Self-test of that convention: launches one small CTA whose threads wait, with the library's
+ * bounded wait, on a barrier that nothing arrives on.  After limit_ns (1 us .. 1 s) the wait runs
+ * out, the kernel writes CAMERA_ERR_DEVICE_TIMEOUT into the status word of `workspace` (cleared
+ * first; at least 256 bytes, 256-byte aligned) and returns; camera_read_status then reports it.
+ * Nothing else on the device is touched and the context stays usable.
+ */
+int camera_wait_probe(void* workspace, size_t workspace_bytes, uint64_t limit_ns, void* cuda_stream);
 
 /* Scratch for camera_select_prune / camera_alloc_bits (n_levels = 2 for pruning). */
 size_t camera_select_workspace_bytes(int64_t n_total, int32_t n_segments, int32_t n_levels);
@@ -334,13 +358,16 @@ size_t camera_analyze_workspace_bytes(const camera_layer_t* layer, int64_t n_tok
 
 /*
  * One whole analysis step with HOST token and result buffers: copies x_host (pinned or
- * pageable, [n_tokens, d_model]) to the device in batches of 65536 tokens (the first one 16384) on a copy stream of its
- * own, scoring batch b (camera_score_layer, accumulating) while batch b+1 is on its way; then runs
- * camera_select_prune
- * once per entry of prune_ratios (HOST [n_prune], may be empty) and camera_alloc_bits, and copies
- * energy [N_e] fp32, keep masks [n_prune, N_e] and bits_out [N_e] back to the given HOST buffers
- * (any may be NULL).  The layer's weights stay DEVICE resident.  Synchronises the stream before
- * returning, and returns the workspace's status word if a kernel recorded one.
+ * pageable, [n_tokens, d_model]) to the device in batches on a copy stream of its own (the first
+ * batch 8192 tokens, every later one half as large again, up to 65536), scoring batch b
+ * (camera_score_layer, accumulating) while batch b+1 is on its way; then runs camera_select_all
+ * (every prune mask of prune_ratios, HOST [n_prune], may be empty, and the bit-widths from one
+ * set of radix passes; separate camera_select_prune / camera_alloc_bits calls where n_prune +
+ * n_levels - 1 > 7) and copies energy [N_e] fp32, keep masks [n_prune, N_e] and bits_out [N_e]
+ * back to the given HOST buffers (any may be NULL).  The layer's weights stay DEVICE resident.
+ * Synchronises the stream before returning, and returns the workspace's status word if a kernel
+ * recorded one.  The batch sizes depend on n_tokens alone, so a given input gives the same bits
+ * on every run.
  */
 int camera_analyze_layer_host(const camera_layer_t* layer, const void* x_host, int64_t n_tokens,
                               float alpha, const double* prune_ratios, int32_t n_prune,

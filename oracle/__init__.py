@@ -6,3 +6,4 @@ Python binding and must never be imported by them; only the test-suite, the
 smoke check and the benchmark's CPU-baseline leg call it.
 """
 from .camera_oracle import *  # noqa: F401,F403
+from .adapters import f64, to_oracle_layer  # noqa: F401

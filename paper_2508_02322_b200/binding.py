@@ -60,6 +60,12 @@ def _load() -> C.CDLL:
                                        C.POINTER(camera_score_aux_t), C.c_void_p, C.c_size_t, C.c_void_p]
     lib.camera_read_status.restype = C.c_int
     lib.camera_read_status.argtypes = [C.c_void_p, C.c_void_p, C.POINTER(C.c_int32)]
+    lib.camera_set_wait_limit_ns.restype = C.c_int
+    lib.camera_set_wait_limit_ns.argtypes = [C.c_uint64]
+    lib.camera_get_wait_limit_ns.restype = C.c_uint64
+    lib.camera_get_wait_limit_ns.argtypes = []
+    lib.camera_wait_probe.restype = C.c_int
+    lib.camera_wait_probe.argtypes = [C.c_void_p, C.c_size_t, C.c_uint64, C.c_void_p]
     lib.camera_select_workspace_bytes.restype = C.c_size_t
     lib.camera_select_workspace_bytes.argtypes = [C.c_int64, C.c_int32, C.c_int32]
     lib.camera_select_prune.restype = C.c_int
@@ -275,6 +281,21 @@ def camera_read_status(workspace: torch.Tensor, stream: Optional[torch.cuda.Stre
     st = C.c_int32(0)
     _check(lib.camera_read_status(workspace.data_ptr(), _stream_ptr(stream), C.byref(st)), "camera_read_status")
     return int(st.value)
+
+
+def camera_set_wait_limit_ns(limit_ns: int) -> None:
+    """Limit of the waits inside the tensor-core kernels, for every later call of the process."""
+    _check(lib.camera_set_wait_limit_ns(int(limit_ns)), "camera_set_wait_limit_ns")
+
+
+def camera_get_wait_limit_ns() -> int:
+    return int(lib.camera_get_wait_limit_ns())
+
+
+def camera_wait_probe(workspace: torch.Tensor, limit_ns: int, stream: Optional[torch.cuda.Stream] = None) -> None:
+    """Launches the self-test kernel whose wait runs out after limit_ns; read the result with camera_read_status."""
+    _check(lib.camera_wait_probe(workspace.data_ptr(), workspace.numel(), int(limit_ns), _stream_ptr(stream)),
+           "camera_wait_probe")
 
 
 def _segments(n_total: int, seg_offsets):

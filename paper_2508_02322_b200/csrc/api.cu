@@ -1,11 +1,12 @@
 // C ABI entry points of camera_score_layer and camera_analyze_layer_host: argument checks,
 // workspace carving, and the launch sequence.  No device memory is allocated here.
-#include <stdlib.h>
 #include <string.h>
 
+#include <atomic>
 #include <vector>
 
 #include "common.cuh"
+#include "umma.cuh"
 
 namespace camera {
 
@@ -18,15 +19,10 @@ size_t up256(size_t v) { return (v + 255) & ~(size_t)255; }
 // Micro-experts per scheduling group.  2560 of them are 37 MB of gate+up rows at d_model 3584,
 // which stay in L2 while the concurrent CTAs walk down the expert's token list (measured on the
 // Qwen2-shaped layer: 640 / 1280 / 2560 / 5120 -> 862 / 991 / 1111 / 1083 TFLOP/s).
-// CAMERA_GROUP_CHANNELS overrides it (tuning aid).
-int score_group_channels() {
-  const char* env = getenv("CAMERA_GROUP_CHANNELS");
-  if (env != nullptr) {
-    const int v = atoi(env);
-    if (v >= 256 && v <= (1 << 20)) return v;
-  }
-  return 2560;
-}
+constexpr int SCORE_GROUP_CHANNELS = 2560;
+
+// Limit of every wait inside the tensor-core kernels, process wide (camera_set_wait_limit_ns).
+std::atomic<unsigned long long> g_wait_limit_ns{DEFAULT_WAIT_LIMIT_NS};
 
 struct ScoreLayout {
   size_t totals, est, edyn, me_prefix, unit_prefix, counts, block_hist, local_rank, topk_idx, topk_w, shared_w,
@@ -166,6 +162,8 @@ extern "C" size_t camera_score_workspace_bytes(const camera_layer_t* layer, int6
 
 namespace camera {
 
+unsigned long long current_wait_limit_ns() { return g_wait_limit_ns.load(std::memory_order_relaxed); }
+
 size_t score_workspace_bytes_any(const camera_layer_t* L, int64_t T, bool forward) {
   if (validate_layer(L, T, forward) != CAMERA_OK) return 0;
   return score_layout(L, T).total;
@@ -212,6 +210,7 @@ int score_front(const camera_layer_t* L, const void* x, int64_t T, float alpha, 
   c.n_tokens = (int)T; c.n_blocks = lay.n_blocks; c.chunk_tokens = lay.chunk_tokens;
   c.max_rows_perm = lay.max_rows_perm; c.max_part = lay.max_part; c.alpha = alpha;
   c.accumulate = accumulate ? 1 : 0;
+  c.wait_limit_ns = current_wait_limit_ns();
   c.x = x; c.w_router = L->w_router; c.router_bias = L->router_bias; c.w_shared_gate = L->w_shared_gate;
   c.totals = reinterpret_cast<PlanTotals*>(ws + lay.totals);
   c.est = reinterpret_cast<ExpertStatic*>(ws + lay.est);
@@ -282,7 +281,7 @@ int score_front(const camera_layer_t* L, const void* x, int64_t T, float alpha, 
     }
   }
   c.ch_tile = use_pair ? 2 * CH_TILE : CH_TILE;
-  c.ct_group = score_group_channels() / c.ch_tile;
+  c.ct_group = SCORE_GROUP_CHANNELS / c.ch_tile;
   const bool use_router_umma = use_umma && router_umma_ok(c);
   std::vector<char> maps;
   if (use_umma) {
@@ -362,6 +361,45 @@ extern "C" int camera_read_status(const void* workspace, void* cuda_stream, int3
   CK(cudaStreamSynchronize(st));
   *status_out = t.status;
   return CAMERA_OK;
+}
+
+extern "C" int camera_set_wait_limit_ns(uint64_t limit_ns) {
+  if (limit_ns < 1000ull || limit_ns > 600000000000ull) return CAMERA_ERR_INVALID_ARG;
+  g_wait_limit_ns.store(limit_ns, std::memory_order_relaxed);
+  return CAMERA_OK;
+}
+
+extern "C" uint64_t camera_get_wait_limit_ns(void) { return current_wait_limit_ns(); }
+
+namespace camera {
+namespace {
+// One CTA whose threads wait, with the library's bounded wait, on a barrier that nothing ever arrives on: the wait
+// runs out after limit_ns, the CTA records CAMERA_ERR_DEVICE_TIMEOUT in the status word and returns.
+__global__ void __launch_bounds__(64) k_wait_probe(PlanTotals* totals, unsigned long long limit_ns) {
+  __shared__ __align__(8) unsigned long long bar;
+  __shared__ __align__(8) int wait_state[WAIT_LIMIT_SLOT + 2];
+  volatile int* const abort_flag = wait_state;
+  if (threadIdx.x == 0) {
+    mbar_init(smem_u32(&bar), 1);
+    wait_state_init(abort_flag, limit_ns);
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  __syncthreads();
+  const bool ok = mbar_wait(smem_u32(&bar), 0u, abort_flag);
+  __syncthreads();
+  if (threadIdx.x == 0 && (!ok || *abort_flag)) atomicExch(&totals->status, (int)CAMERA_ERR_DEVICE_TIMEOUT);
+}
+}  // namespace
+}  // namespace camera
+
+extern "C" int camera_wait_probe(void* workspace, size_t workspace_bytes, uint64_t limit_ns, void* cuda_stream) {
+  if (limit_ns < 1000ull || limit_ns > 1000000000ull) return CAMERA_ERR_INVALID_ARG;     // at most a second
+  if (workspace == nullptr || workspace_bytes < sizeof(PlanTotals) || (reinterpret_cast<uintptr_t>(workspace) & 255))
+    return CAMERA_ERR_WORKSPACE;
+  cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+  CK(cudaMemsetAsync(workspace, 0, sizeof(PlanTotals), st));
+  k_wait_probe<<<1, 64, 0, st>>>(static_cast<PlanTotals*>(workspace), limit_ns);
+  return cudaGetLastError() == cudaSuccess ? CAMERA_OK : CAMERA_ERR_CUDA;
 }
 
 namespace {

@@ -69,6 +69,7 @@ struct ScoreCtx {
   int64_t max_part;                 // capacity of the partial arrays in floats
   float alpha;
   int32_t accumulate;               // fold this call's tokens into the phi2 / phi_inf_sq already there
+  unsigned long long wait_limit_ns; // after this long a wait inside a tensor-core kernel gives up (camera_set_wait_limit_ns)
   const void* x;
   const void* w_router;
   const float* router_bias;
@@ -113,6 +114,7 @@ int score_front(const camera_layer_t* L, const void* x, int64_t T, float alpha, 
                 const camera_score_aux_t* aux, void* workspace, size_t workspace_bytes, cudaStream_t st,
                 const ForwardBuffers* fwd, ScoreFront* out);
 size_t score_workspace_bytes_any(const camera_layer_t* L, int64_t T, bool forward);
+unsigned long long current_wait_limit_ns();
 
 // ---- launches (each enqueues on `st`, returns the launch's cudaError_t) ------------------------
 cudaError_t launch_router(const ScoreCtx& c, cudaStream_t st);

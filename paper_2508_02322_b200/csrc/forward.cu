@@ -81,7 +81,7 @@ __global__ void __launch_bounds__(D_THREADS, 1) k_down_umma(const ScoreCtx c, co
     for (int s = 0; s < D_STAGES; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
     for (int a = 0; a < 2; ++a) { mbar_init(tfull_bar(a), 1); mbar_init(tempty_bar(a), 128); }
     for (int q = 0; q < D_SCHED; ++q) { mbar_init(sfull_bar(q), 1); mbar_init(sempty_bar(q), 5); }
-    *abort_flag = 0;
+    wait_state_init(abort_flag, c.wait_limit_ns);
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
   }
@@ -281,7 +281,7 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(D_THREADS, 1)
     mbar_init(tfull_bar, 1);
     mbar_init(tempty_bar, 256);
     for (int q = 0; q < D_SCHED; ++q) { mbar_init(sfull_bar(q), 1); mbar_init(sempty_bar(q), 10); }
-    *abort_flag = 0;
+    wait_state_init(abort_flag, c.wait_limit_ns);
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
   }
@@ -470,8 +470,13 @@ __global__ void __launch_bounds__(256) k_unpermute_sum(const ScoreCtx c, float* 
   const int t = blockIdx.x;
   if ((int)threadIdx.x < k) {
     const int e = c.topk_idx[(size_t)t * k + threadIdx.x];
-    pos_s[threadIdx.x] = (long long)c.edyn[e].row_base + c.block_hist[(size_t)(t / ROUTER_TOK) * c.n_routed + e] +
-                         c.local_rank[(size_t)t * k + threadIdx.x];
+    long long pos = -1;     // the routers only leave experts in range; anything else adds nothing
+    if (e >= 0 && e < c.n_routed) {
+      pos = (long long)c.edyn[e].row_base + c.block_hist[(size_t)(t / ROUTER_TOK) * c.n_routed + e] +
+            c.local_rank[(size_t)t * k + threadIdx.x];
+      if (pos < 0 || pos >= c.max_rows_perm) pos = -1;
+    }
+    pos_s[threadIdx.x] = pos;
   }
   __syncthreads();
   const int v = (blockIdx.y * 256 + threadIdx.x) << 2;
@@ -480,6 +485,7 @@ __global__ void __launch_bounds__(256) k_unpermute_sum(const ScoreCtx c, float* 
   float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
 #pragma unroll 4
   for (int s = 0; s < k; ++s) {
+    if (pos_s[s] < 0) continue;
     const float4 p = *reinterpret_cast<const float4*>(routed + (size_t)pos_s[s] * d + v);
     acc.x += p.x; acc.y += p.y; acc.z += p.z; acc.w += p.w;
   }

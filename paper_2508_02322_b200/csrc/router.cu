@@ -121,14 +121,17 @@ __global__ void __launch_bounds__(RT_THREADS) k_router(ScoreCtx c, const int32_t
       }
       int my_e = 0;
       float my_p = 0.f;
+      bool bad = false;     // a routing that cannot be used: see the safe pair below
       if (idx_in != nullptr) {
         if (lane < k) {
           my_e = idx_in[(size_t)t * k + lane];
           my_p = w_in[(size_t)t * k + lane];
-          if (my_e < 0 || my_e >= c.n_routed) {
-            atomicExch(&c.totals->status, (int)CAMERA_ERR_INVALID_ARG);
-            my_e = 0; my_p = 0.f;
-          }
+          bad = my_e < 0 || my_e >= c.n_routed;
+        }
+        // a prescribed routing names k distinct experts per token
+        for (int s = 0; s < k; ++s) {
+          const int other = __shfl_sync(0xffffffffu, my_e, s);
+          if (lane < k && lane != s && other == my_e) bad = true;
         }
       } else {
         float v[MAX_ROUTED / 32];
@@ -146,6 +149,8 @@ __global__ void __launch_bounds__(RT_THREADS) k_router(ScoreCtx c, const int32_t
 #pragma unroll
         for (int i = 0; i < MAX_ROUTED / 32; ++i) den += (lane + 32 * i < c.n_routed) ? expf(v[i] - zmax) : 0.f;
         den = warp_sum(den);
+        // a NaN or +inf logit (a NaN or inf in x or in the router) leaves no softmax to take
+        bad = !(den > 0.f) || !isfinite(den);
         float chosen = 0.f;
         for (int s = 0; s < k; ++s) {
           float best = -INFINITY;
@@ -159,6 +164,7 @@ __global__ void __launch_bounds__(RT_THREADS) k_router(ScoreCtx c, const int32_t
             const int oi = __shfl_xor_sync(0xffffffffu, bi, o);
             if (ov > best || (ov == best && oi < bi)) { best = ov; bi = oi; }
           }
+          if (bi >= c.n_routed) bad = true;     // fewer than k logits above -inf
           const float p = expf(best - zmax) / den;
 #pragma unroll
           for (int i = 0; i < MAX_ROUTED / 32; ++i)
@@ -167,6 +173,13 @@ __global__ void __launch_bounds__(RT_THREADS) k_router(ScoreCtx c, const int32_t
           chosen += p;
         }
         if (c.flags & CAMERA_ROUTER_NORM_TOPK) my_p /= chosen;
+      }
+      if (__any_sync(0xffffffffu, bad)) {
+        // unusable routing: record it and give the token k distinct experts with coefficient 0, so that every
+        // later index stays in range
+        if (lane == 0) atomicExch(&c.totals->status, (int)CAMERA_ERR_INVALID_ARG);
+        my_e = lane < c.n_routed ? lane : 0;
+        my_p = 0.f;
       }
       if (lane < k) {
         c.topk_idx[(size_t)t * k + lane] = my_e;
@@ -296,9 +309,15 @@ __global__ void __launch_bounds__(256) k_permute(ScoreCtx c, int row_bytes) {
   int pos_l = 0;
   if (lane < k) {
     const int e = c.topk_idx[(size_t)t * k + lane];
-    pos_l = c.edyn[e].row_base + c.block_hist[(size_t)(t / ROUTER_TOK) * c.n_routed + e] +
-            c.local_rank[(size_t)t * k + lane];
-    c.perm_w[pos_l] = c.topk_w[(size_t)t * k + lane];
+    pos_l = -1;
+    if (e >= 0 && e < c.n_routed) {
+      pos_l = c.edyn[e].row_base + c.block_hist[(size_t)(t / ROUTER_TOK) * c.n_routed + e] +
+              c.local_rank[(size_t)t * k + lane];
+      if (pos_l < 0 || pos_l >= c.max_rows_perm) pos_l = -1;
+    }
+    // the routers only write pairs that pass this; a pair that does not is skipped and reported, never written
+    if (pos_l >= 0) c.perm_w[pos_l] = c.topk_w[(size_t)t * k + lane];
+    else atomicExch(&c.totals->status, (int)CAMERA_ERR_INVALID_ARG);
   }
   int pos[MAX_TOPK];
 #pragma unroll
@@ -309,7 +328,7 @@ __global__ void __launch_bounds__(256) k_permute(ScoreCtx c, int row_bytes) {
     const uint4 val = __ldg(src + v);
 #pragma unroll
     for (int s = 0; s < MAX_TOPK; ++s)
-      if (s < k)
+      if (s < k && pos[s] >= 0)
         reinterpret_cast<uint4*>(static_cast<char*>(c.x_perm) + (size_t)pos[s] * row_bytes)[v] = val;
   }
 }

@@ -72,7 +72,7 @@ k_router_umma(const ScoreCtx c, const int32_t* idx_in, const float* w_in, int n_
   if (tid == 0) {
     for (int s = 0; s < rs.stages; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
     for (int a = 0; a < 2; ++a) { mbar_init(tfull_bar(a), 1); mbar_init(tempty_bar(a), 128); }
-    *abort_flag = 0;
+    wait_state_init(abort_flag, c.wait_limit_ns);
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
   }
@@ -188,21 +188,24 @@ k_router_umma(const ScoreCtx c, const int32_t* idx_in, const float* w_in, int n_
 #pragma unroll
       for (int s = 0; s < MAX_TOPK; ++s) my_e[s] = -1;
       if (live) {
+        float my_p[MAX_TOPK];
+        bool bad = false;     // a routing that cannot be used: see the safe pairs below
         if (idx_in != nullptr) {
 #pragma unroll
           for (int s = 0; s < MAX_TOPK; ++s) {
+            my_p[s] = 0.f;
             if (s < k) {
-              int e = idx_in[(size_t)t * k + s];
-              float p = w_in[(size_t)t * k + s];
-              if (e < 0 || e >= c.n_routed) {
-                atomicExch(&c.totals->status, (int)CAMERA_ERR_INVALID_ARG);
-                e = 0; p = 0.f;
-              }
-              my_e[s] = e;
-              c.topk_idx[(size_t)t * k + s] = e;
-              c.topk_w[(size_t)t * k + s] = p;
+              my_e[s] = idx_in[(size_t)t * k + s];
+              my_p[s] = w_in[(size_t)t * k + s];
+              bad = bad || my_e[s] < 0 || my_e[s] >= c.n_routed;
             }
           }
+          // a prescribed routing names k distinct experts per token (the ranks below count a token once per expert)
+#pragma unroll
+          for (int s = 1; s < MAX_TOPK; ++s)
+#pragma unroll
+            for (int r = 0; r < s; ++r)
+              if (s < k && my_e[s] == my_e[r]) bad = true;
         } else {
           float zmax = -INFINITY;
           for (int j = 0; j < c.n_routed; ++j) {
@@ -212,30 +215,43 @@ k_router_umma(const ScoreCtx c, const int32_t* idx_in, const float* w_in, int n_
           }
           float den = 0.f;
           for (int j = 0; j < c.n_routed; ++j) den += expf(row[j] - zmax);
-          float my_p[MAX_TOPK];
+          // a NaN or +inf logit (a NaN or inf in x or in the router) leaves no softmax to take
+          bad = !(den > 0.f) || !isfinite(den);
           float chosen = 0.f;
 #pragma unroll
           for (int s = 0; s < MAX_TOPK; ++s) {
             my_p[s] = 0.f;
             if (s < k) {
               float best = -INFINITY;
-              int bi = 0;
+              int bi = -1;
               for (int j = 0; j < c.n_routed; ++j) {     // strict >: equal logits go to the lower expert
                 const float z = row[j];
                 if (z > best) { best = z; bi = j; }
               }
+              if (bi < 0) { bad = true; bi = 0; }        // fewer than k logits above -inf
               row[bi] = -INFINITY;
               my_e[s] = bi;
               my_p[s] = expf(best - zmax) / den;
               chosen += my_p[s];
             }
           }
+          if (c.flags & CAMERA_ROUTER_NORM_TOPK) {
 #pragma unroll
-          for (int s = 0; s < MAX_TOPK; ++s) {
-            if (s < k) {
-              c.topk_idx[(size_t)t * k + s] = my_e[s];
-              c.topk_w[(size_t)t * k + s] = (c.flags & CAMERA_ROUTER_NORM_TOPK) ? my_p[s] / chosen : my_p[s];
-            }
+            for (int s = 0; s < MAX_TOPK; ++s) my_p[s] /= chosen;
+          }
+        }
+        if (bad) {
+          // unusable routing: record it and give the token k distinct experts with coefficient 0, so that every
+          // later index stays in range and every pair gets its rank
+          atomicExch(&c.totals->status, (int)CAMERA_ERR_INVALID_ARG);
+#pragma unroll
+          for (int s = 0; s < MAX_TOPK; ++s) { my_e[s] = s < k ? s : -1; my_p[s] = 0.f; }
+        }
+#pragma unroll
+        for (int s = 0; s < MAX_TOPK; ++s) {
+          if (s < k) {
+            c.topk_idx[(size_t)t * k + s] = my_e[s];
+            c.topk_w[(size_t)t * k + s] = my_p[s];
           }
         }
       }

@@ -75,7 +75,7 @@ __global__ void __launch_bounds__(U_THREADS, 1) k_score_umma(const ScoreCtx c) {
     mbar_init(tfull_bar, 1);
     mbar_init(tempty_bar, 128);
     for (int q = 0; q < U_SCHED; ++q) { mbar_init(sfull_bar(q), 1); mbar_init(sempty_bar(q), 5); }
-    *abort_flag = 0;
+    wait_state_init(abort_flag, c.wait_limit_ns);
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
   }

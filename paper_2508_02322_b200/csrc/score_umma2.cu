@@ -89,7 +89,7 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(P_THREADS, 1) k_scor
     mbar_init(tfull_bar, 1);
     mbar_init(tempty_bar, 256);
     for (int q = 0; q < P_SCHED; ++q) { mbar_init(sfull_bar(q), 1); mbar_init(sempty_bar(q), 10); }
-    *abort_flag = 0;
+    wait_state_init(abort_flag, c.wait_limit_ns);
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
   }

@@ -386,7 +386,7 @@ namespace camera {
 namespace {
 
 constexpr int STATIC_MAX_SEGMENTS = 32;
-constexpr size_t STATIC_SCRATCH_BYTES = 288 * 1024;   // sel_layout(32, 1).total = 271,360 bytes fits
+constexpr size_t STATIC_SCRATCH_BYTES = 288 * 1024;   // room for 32 segments (checked on every call)
 
 // Lives in every GPU's memory from the moment the library is loaded there until the process ends.
 static __device__ __align__(256) unsigned char g_select_scratch[STATIC_SCRATCH_BYTES];

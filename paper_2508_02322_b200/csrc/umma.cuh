@@ -7,7 +7,8 @@
 
 namespace camera {
 
-constexpr unsigned long long WAIT_LIMIT_NS = 4000000000ull;   // every mbarrier wait gives up after this long
+constexpr unsigned long long DEFAULT_WAIT_LIMIT_NS = 4000000000ull;   // every mbarrier wait gives up after this long
+                                                                      // unless the host set another limit
 constexpr int UMMA_BK = 64;                                   // bf16 elements per k-block = one 128-byte swizzle row
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
@@ -41,6 +42,17 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
   return ok != 0;
 }
 
+// The CTA's wait state in shared memory: the abort flag (an int, 8-byte aligned) and, WAIT_LIMIT_SLOT ints behind
+// it, the limit of every wait in nanoseconds.  One thread sets both up before the first wait.
+constexpr int WAIT_LIMIT_SLOT = 4;
+__device__ __forceinline__ void wait_state_init(volatile int* abort_flag, unsigned long long limit_ns) {
+  *abort_flag = 0;
+  *reinterpret_cast<volatile unsigned long long*>(abort_flag + WAIT_LIMIT_SLOT) = limit_ns;
+}
+__device__ __forceinline__ unsigned long long wait_limit_ns(volatile int* abort_flag) {
+  return *reinterpret_cast<volatile unsigned long long*>(abort_flag + WAIT_LIMIT_SLOT);
+}
+
 // Bounded wait.  Returns false when the limit ran out or another thread of the CTA gave up.
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
   if (mbar_try_wait(bar, parity)) return true;
@@ -50,7 +62,7 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
     if (mbar_try_wait(bar, parity)) return true;
     if ((++spins & 63u) == 0u) {
       if (*abort_flag) return false;
-      if (globaltimer_ns() - t0 > WAIT_LIMIT_NS) {
+      if (globaltimer_ns() - t0 > wait_limit_ns(abort_flag)) {
         *abort_flag = 1;
         return false;
       }

@@ -43,7 +43,7 @@ __device__ __forceinline__ bool mbar_wait_cluster(uint32_t bar, uint32_t parity,
     if (mbar_try_wait_cluster(bar, parity)) return true;
     if ((++spins & 63u) == 0u) {
       if (*abort_flag) return false;
-      if (globaltimer_ns() - t0 > WAIT_LIMIT_NS) { *abort_flag = 1; return false; }
+      if (globaltimer_ns() - t0 > wait_limit_ns(abort_flag)) { *abort_flag = 1; return false; }
     }
   }
 }

@@ -15,16 +15,32 @@ W_TOL = 1e-4            # router / shared-gate coefficients: a logit is an fp32 
                         # sigmoid pass an absolute logit error on as a relative error of at most the same size
 
 
-def assert_close(name, got, ref, rel=REL_TOL):
+FLOOR_LOG = []          # (name, elements compared, elements whose scale came from the floor, of those beyond `rel` on their own)
+
+
+def assert_close(name, got, ref, rel=REL_TOL, max_under_floor=0):
+    """Element by element within `rel` of max(|ref_i|, FLOOR * max|ref|).  Counts the elements whose scale came from
+    the floor (non-zero scores a million times below the largest) and fails when there are more than
+    `max_under_floor`: the floor exists for the rare micro-expert seen by one or two tokens whose fp32 dot product
+    nearly cancels, not to hide a population of small scores."""
     got = np.asarray(got, dtype=np.float64)
     ref = np.asarray(ref, dtype=np.float64)
-    scale = np.maximum(np.abs(ref), max(FLOOR * float(np.abs(ref).max(initial=0.0)), 1e-30))
+    floor = max(FLOOR * float(np.abs(ref).max(initial=0.0)), 1e-30)
+    scale = np.maximum(np.abs(ref), floor)
     err = np.abs(got - ref) / scale
     # values that are exactly zero in the oracle must be exactly zero on the GPU
     zero = ref == 0
     assert (got[zero] == 0).all(), f"{name}: non-zero where the oracle is exactly zero"
     bad = err[~zero] > rel
     assert not bad.any(), f"{name}: {bad.sum()} of {bad.size} beyond {rel}, worst {err[~zero].max():.3e}"
+    under = ~zero & (np.abs(ref) < floor)
+    needed = under & (np.abs(got - ref) > rel * np.abs(ref))
+    FLOOR_LOG.append((name, int(ref.size), int(under.sum()), int(needed.sum())))
+    if under.any():
+        print(f"[floor] {name}: {int(under.sum())} of {ref.size} elements scaled by the floor, {int(needed.sum())} needed it")
+    assert under.sum() <= max_under_floor, \
+        f"{name}: {int(under.sum())} elements below {FLOOR} of the maximum (allowed {max_under_floor}), {int(needed.sum())} of them beyond {rel} on their own"
+    return int(under.sum())
 
 
 def check_routing(olayer, Xd, topk_idx, topk_w):
@@ -54,7 +70,8 @@ def check_routing(olayer, Xd, topk_idx, topk_w):
     return int((~same).sum())
 
 
-def run_and_compare(P, L, X, alpha=0.95, channels=None, force_simt=False, check_dense=False, cta_pair=None):
+def run_and_compare(P, L, X, alpha=0.95, channels=None, force_simt=False, check_dense=False, cta_pair=None,
+                    max_under_floor=0):
     """Scores one layer on the GPU (own routing, then the oracle's routing injected) and checks
     every component against the oracle.  `channels` restricts the oracle to sampled micro-experts."""
     layer = P.Layer.from_workload(L)
@@ -74,11 +91,11 @@ def run_and_compare(P, L, X, alpha=0.95, channels=None, force_simt=False, check_
         assert_close("shared_w", shared_w, O.shared_coeff(olayer, Xd), rel=W_TOL)
     phi2, phi_inf, omega2 = O.camera_components(olayer, Xd, channels=channels, routing=routing)
     sel = ~np.isnan(phi2)
-    assert_close("omega2", out["omega2"].cpu().numpy(), omega2)
-    assert_close("phi2", out["phi2"].cpu().numpy()[sel], phi2[sel])
-    assert_close("phi_inf_sq", out["phi_inf_sq"].cpu().numpy()[sel], phi_inf[sel])
+    assert_close("omega2", out["omega2"].cpu().numpy(), omega2, max_under_floor=max_under_floor)
+    assert_close("phi2", out["phi2"].cpu().numpy()[sel], phi2[sel], max_under_floor=max_under_floor)
+    assert_close("phi_inf_sq", out["phi_inf_sq"].cpu().numpy()[sel], phi_inf[sel], max_under_floor=max_under_floor)
     E = O.energy(phi2, phi_inf, omega2, float(np.float32(alpha)))
-    assert_close("energy", out["energy"].cpu().numpy()[sel], E[sel])
+    assert_close("energy", out["energy"].cpu().numpy()[sel], E[sel], max_under_floor=max_under_floor)
     counts = out["expert_token_counts"].cpu().numpy()
     if olayer.n_routed:
         assert np.array_equal(counts[:olayer.n_routed], np.bincount(routing[0].reshape(-1), minlength=olayer.n_routed))
@@ -92,15 +109,15 @@ def run_and_compare(P, L, X, alpha=0.95, channels=None, force_simt=False, check_
                                     routing_in=(torch.from_numpy(idx_o.astype(np.int32)), torch.from_numpy(w32)))
         assert P.camera_read_status(ws) == 0
         p2, pi, w2 = O.camera_components(olayer, Xd, channels=channels, routing=(idx_o, w32.astype(np.float64)))
-        assert_close("phi2 (oracle routing)", out2["phi2"].cpu().numpy()[sel], p2[sel])
-        assert_close("phi_inf_sq (oracle routing)", out2["phi_inf_sq"].cpu().numpy()[sel], pi[sel])
+        assert_close("phi2 (oracle routing)", out2["phi2"].cpu().numpy()[sel], p2[sel], max_under_floor=max_under_floor)
+        assert_close("phi_inf_sq (oracle routing)", out2["phi_inf_sq"].cpu().numpy()[sel], pi[sel], max_under_floor=max_under_floor)
         assert_close("energy (oracle routing)", out2["energy"].cpu().numpy()[sel],
-                     O.energy(p2, pi, w2, float(np.float32(alpha)))[sel])
+                     O.energy(p2, pi, w2, float(np.float32(alpha)))[sel], max_under_floor=max_under_floor)
     if check_dense:
         d2, dinf, dw = O.camera_components_dense(olayer, Xd)
         if flips == 0:
-            assert_close("phi2 vs literal Algorithm 1", out["phi2"].cpu().numpy(), d2)
-            assert_close("phi_inf_sq vs literal Algorithm 1", out["phi_inf_sq"].cpu().numpy(), dinf)
+            assert_close("phi2 vs literal Algorithm 1", out["phi2"].cpu().numpy(), d2, max_under_floor=max_under_floor)
+            assert_close("phi_inf_sq vs literal Algorithm 1", out["phi_inf_sq"].cpu().numpy(), dinf, max_under_floor=max_under_floor)
     return out, flips
 
 

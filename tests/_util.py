@@ -1,27 +1,7 @@
-"""Test helpers: turn a generated layer (torch tensors in storage dtype) into
-the oracle's float64 layer, and small random layers for the pins."""
+"""Test helpers: the oracle's adapters for generated layers (re-exported) and small random layers for the pins."""
 import numpy as np
-import torch
 
-from oracle import OracleLayer
-
-
-def f64(t):
-    return None if t is None else t.detach().to("cpu").to(torch.float64).numpy()
-
-
-def to_oracle_layer(L) -> OracleLayer:
-    """`L` is the dict returned by workloads.make_layer."""
-    cfg = L["cfg"]
-    if L["down_layout"] == "hf":
-        w_down = [f64(w) for w in L["w_down"]]
-    else:
-        w_down = [np.ascontiguousarray(f64(w).T) for w in L["w_down"]]
-    return OracleLayer(
-        w_router=f64(L["w_router"]), top_k=cfg.top_k,
-        w_gate=[f64(w) for w in L["w_gate"]], w_up=[f64(w) for w in L["w_up"]], w_down=w_down,
-        router_bias=f64(L["router_bias"]), norm_topk=cfg.norm_topk, n_shared=cfg.n_shared,
-        w_shared_gate=f64(L["w_shared_gate"]))
+from oracle import OracleLayer, f64, to_oracle_layer  # noqa: F401
 
 
 def random_layer(rng, d=6, d_ff=(3, 3, 3), n_shared=0, top_k=2, shared_gate=False, bias=False,

@@ -3,12 +3,15 @@
 Some users of the library run where they may not allocate device memory (a plug-in inside a server
 whose pool owns the GPU, code that must not trigger cudaMalloc's device-wide synchronisation), so
 this entry point keeps its scratch in a fixed array inside the library.  It has to give exactly the
-mask of camera_select_prune, also when it is called again and the array still holds the previous
-call's histograms and thresholds.  This file sorts last on purpose: every other test has run by then.
+mask of camera_select_prune and of the oracle's selection, also when it is called again and the array
+still holds the previous call's histograms and thresholds, and it must leave the amount of free device
+memory as it found it.  This file sorts last on purpose: every other test has run by then.
 """
 import numpy as np
 import pytest
 import torch
+
+import oracle as O
 
 pytestmark = pytest.mark.gpu
 
@@ -41,6 +44,11 @@ def test_static_scratch_matches_workspace_version_twice_in_a_row():
         torch.cuda.synchronize()
         assert torch.equal(keep, ref_keep)              # masks are integer work: bit-exact
         assert np.array_equal(thr.cpu().numpy(), ref_thr.cpu().numpy())
+        # ... and against the oracle's TopSelect, segment by segment (a segment is a layer of its own)
+        E_np, got = E.cpu().numpy(), keep.cpu().numpy()
+        bounds = [0, E.numel()] if seg is None else seg
+        for s0, s1 in zip(bounds[:-1], bounds[1:]):
+            assert np.array_equal(got[s0:s1], O.select_prune(E_np[s0:s1], ratio))
     # same input twice, back to back on one stream, no synchronisation in between
     E = cases[0][0]
     a = torch.empty(E.numel(), dtype=torch.uint8, device=DEV)
@@ -49,6 +57,30 @@ def test_static_scratch_matches_workspace_version_twice_in_a_row():
     camera_select_prune_static(E, 0.4, b)
     torch.cuda.synchronize()
     assert torch.equal(a, b) and torch.equal(a, P.camera_select_prune(E, 0.4))
+
+
+def test_static_scratch_leaves_free_device_memory_unchanged():
+    """What the entry point is for: no device allocation.  The driver's count of free device memory (which sees every
+    cudaMalloc of the process, the library's included, but not torch's reuse of blocks it already holds) is the same
+    before and after a series of calls; the first call on the device, which looks the array up, comes before."""
+    from paper_2508_02322_b200.binding import camera_select_prune_static
+
+    E = _energies(184320, 5)
+    keep = torch.empty(E.numel(), dtype=torch.uint8, device=DEV)
+    thr = torch.empty(28, dtype=torch.float32, device=DEV)
+    seg = [i * (E.numel() // 28) for i in range(28)] + [E.numel()]
+    camera_select_prune_static(E, 0.4, keep)            # first call: set-up
+    torch.cuda.synchronize()
+    free_before, _ = torch.cuda.mem_get_info()
+    for ratio in (0.2, 0.4, 0.6):
+        camera_select_prune_static(E, ratio, keep)
+        camera_select_prune_static(E, ratio, keep, seg_offsets=seg, thresholds=thr)
+    torch.cuda.synchronize()
+    free_after, _ = torch.cuda.mem_get_info()
+    assert free_after == free_before
+    E_np, got = E.cpu().numpy(), keep.cpu().numpy()
+    for s0, s1 in zip(seg[:-1], seg[1:]):
+        assert np.array_equal(got[s0:s1], O.select_prune(E_np[s0:s1], 0.6))
 
 
 def test_static_scratch_rejects_too_many_segments():
