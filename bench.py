@@ -33,8 +33,8 @@ BIT_RATIOS, BIT_LEVELS = (0.2, 0.6, 0.2), (3, 2, 1)     # average 2 bits + 0.25 
 ALPHA = 0.95
 PAPER_CONTEXT = "paper: <5 min for the full Qwen2-57B-A14B analysis on one A100-40GB (incl. model forwards)"
 # kernels launched by one step: score = router, block scan, plan, permute, pad, norms, scoring, combine;
-# the selections = 8 histogram passes + mark
-LAUNCHES_PER_STEP = 8 + 9
+# the selections = one kernel (radix passes, tie break and labels behind one cooperative launch)
+LAUNCHES_PER_STEP = 8 + 1
 # DRAM bytes (read + write) per gate/up flop of the scoring kernel, from the committed ncu capture of a
 # 1/8 slice of the layer whose traffic grows in proportion to the flop (profiles/k_score_umma_qwen2_slice.md).
 SCORE_KERNEL_DRAM_BYTES_PER_FLOP = 4.483e9 / 1.924e13
@@ -266,6 +266,163 @@ def run_stack(args):
         "context": PAPER_CONTEXT}))
 
 
+def time_steps(P, torch, cfg, layer, Xs, steps, warmup, dev, stream, ws_score, ws_sel, energy, keep, bits, sampler_index,
+               cta_pair=None):
+    """`steps` whole steps (score + every selection) of one layer after `warmup`, timed with CUDA events on the
+    launching stream; the SM clock is sampled meanwhile.  Returns (ms in total, per-stage mean ms, clocks, flushed)."""
+    def step(i, events=None):
+        P.camera_score_layer(layer, Xs[i % 2], ALPHA, energy=energy, workspace=ws_score, stage_events=events, cta_pair=cta_pair)
+        P.camera_select_all(energy, PRUNE_RATIOS, BIT_RATIOS, BIT_LEVELS, workspace=ws_sel, keep_masks=keep, bits_out=bits)
+    for i in range(warmup):
+        step(i)
+    torch.cuda.synchronize()
+    status = P.camera_read_status(ws_score)
+    if status != 0:
+        raise RuntimeError(f"device status {status} after warm-up ({cfg.name})")
+    stage_ev = [{s: (torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for s in P.binding.STAGES}
+                for _ in range(steps)]
+    for evs in stage_ev:            # events must exist before their handles are passed down
+        for e0, e1 in evs.values():
+            e0.record(stream); e1.record(stream)
+    # inputs of the large configs exceed the 126 MB L2 several times over; a small config gets its L2 flushed between
+    # steps (a 256 MiB write outside the per-step event pairs)
+    esz = 2 if cfg.dtype == "bf16" else 4
+    footprint = esz * (3 * layer.n_me * cfg.d_model + 2 * cfg.n_tokens * cfg.d_model)
+    flush = torch.empty(256 << 20, dtype=torch.uint8, device=dev) if footprint < (512 << 20) else None
+    sampler = ClockSampler(sampler_index)
+    torch.cuda.synchronize()
+    sampler.start()
+    if flush is None:
+        ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        ev0.record(stream)
+        for i in range(steps):
+            step(i, stage_ev[i])
+        ev1.record(stream)
+        torch.cuda.synchronize()
+        ms = ev0.elapsed_time(ev1)
+    else:
+        per_step = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(steps)]
+        for i in range(steps):
+            flush.zero_()
+            per_step[i][0].record(stream)
+            step(i, stage_ev[i])
+            per_step[i][1].record(stream)
+        torch.cuda.synchronize()
+        ms = sum(e0.elapsed_time(e1) for e0, e1 in per_step)
+    clocks = sampler.stop()
+    stage_ms = {s: statistics.mean(e[s][0].elapsed_time(e[s][1]) for e in stage_ev) for s in P.binding.STAGES}
+    status = P.camera_read_status(ws_score)
+    if status != 0:
+        raise RuntimeError(f"device status {status} in the timed region ({cfg.name})")
+    return ms, stage_ms, clocks, flush is not None
+
+
+def time_e2e(P, torch, cfg, layer, Xs, n_steps, dev, stream):
+    """The same step through camera_analyze_layer_host: pinned host tokens in, host energies / masks / bit-widths out,
+    every step.  Returns (ms per step, bytes in per step, bytes out per step)."""
+    n_me = layer.n_me
+    ws_an = P.alloc_workspace(P.camera_analyze_workspace_bytes(layer, cfg.n_tokens, len(BIT_LEVELS)), dev)
+    xh = [x.cpu().pin_memory() for x in Xs]
+    eh = torch.empty(n_me, dtype=torch.float32).pin_memory()
+    kh = torch.empty((len(PRUNE_RATIOS), n_me), dtype=torch.uint8).pin_memory()
+    bh = torch.empty(n_me, dtype=torch.uint8).pin_memory()
+    def run(i):
+        P.camera_analyze_layer_host(layer, xh[i % 2], ALPHA, PRUNE_RATIOS, BIT_RATIOS, BIT_LEVELS, energy_host=eh,
+                                    keep_host=kh, bits_host=bh, workspace=ws_an)
+    for i in range(2):
+        run(i)
+    torch.cuda.synchronize()
+    a0, a1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    a0.record(stream)
+    for i in range(n_steps):
+        run(i)
+    a1.record(stream)
+    torch.cuda.synchronize()
+    return a0.elapsed_time(a1) / n_steps, xh[0].numel() * xh[0].element_size(), eh.numel() * 4 + kh.numel() + bh.numel()
+
+
+def bench_other_config(P, torch, W, name, dev, stream, local, peaks):
+    """One of the smaller workload configs, measured like the headline one: whole steps with the inputs resident,
+    the scoring stage's rate, and the end-to-end step through the host-buffer entry point."""
+    cfg = W.CONFIGS[name]
+    L = W.make_layer(cfg, seed=0, layer_id=0, device=dev)
+    layer = P.Layer.from_workload(L)
+    Xs = [W.make_tokens(cfg, seed=0, layer_id=i, device=dev) for i in range(2)]
+    n_me, T = layer.n_me, cfg.n_tokens
+    ws_score = P.alloc_workspace(P.camera_score_workspace_bytes(layer, T), dev)
+    ws_sel = P.alloc_workspace(P.camera_select_workspace_bytes(n_me, 1, len(PRUNE_RATIOS) + len(BIT_LEVELS)), dev)
+    energy = torch.empty(n_me, dtype=torch.float32, device=dev)
+    keep = torch.empty((len(PRUNE_RATIOS), n_me), dtype=torch.uint8, device=dev)
+    bits = torch.empty(n_me, dtype=torch.uint8, device=dev)
+    bufs = (ws_score, ws_sel, energy, keep, bits, local)
+    ms, _, _, _ = time_steps(P, torch, cfg, layer, Xs, 10, 3, dev, stream, *bufs)
+    steps = int(min(2000, max(50, 1500.0 / max(ms / 10, 1e-3))))          # about a second and a half of steps
+    ms, stage_ms, clocks, flushed = time_steps(P, torch, cfg, layer, Xs, steps, 3, dev, stream, *bufs)
+    del ws_score, bufs
+    e2e_ms, h2d, d2h = time_e2e(P, torch, cfg, layer, Xs, min(steps, 200), dev, stream)
+    out = {"workload": f"{cfg.name} layer: d_model {cfg.d_model}, {cfg.n_routed}x{cfg.d_ff_routed} top-{cfg.top_k} + shared "
+                       f"{list(cfg.d_ff_shared)}, {T} tokens, {cfg.dtype}", "steps": steps, "ms_per_step": ms / steps,
+           "tokens_per_s": T * steps / (ms * 1e-3), "stage_ms": stage_ms, "clocks": clocks,
+           "l2": "L2 flushed between steps (256 MiB write, not timed)" if flushed else "inputs larger than L2",
+           "e2e_tokens_per_s": T / (e2e_ms * 1e-3), "e2e_ms_per_step": e2e_ms, "h2d_bytes_per_step": h2d,
+           "d2h_bytes_per_step": d2h}
+    if cfg.dtype == "bf16":
+        tf = cfg.gate_up_flop / (stage_ms["score"] * 1e-3) / 1e12
+        # these runs last a second or two: the burst peak is the denominator
+        out.update({"score_tflops": tf, "score_frac_of_burst_peak": tf / peaks["bf16_tflops"], "peak": "measured burst bf16"
+                    if peaks["source"] == "measured" else "fallback burst bf16"})
+    else:
+        out.update({"score_kernel": "fp32 FMA kernel; the step is launch bound at this size: no roofline claim"})
+    return out
+
+
+def bench_whole_model(P, torch, W, cfg, dev, stream):
+    """Every MoE layer of the model with weights and calibration tokens of its own (seeded by the layer's number):
+    camera_score_layer per layer, then the prune masks and bit-widths of all layers from one camera_select_all call
+    with one segment per layer.  Generating a layer's weights and tokens is outside the event pairs and reported
+    beside the analysis time."""
+    nl, T = cfg.n_layers, cfg.n_tokens
+    probe = P.Layer.from_workload(W.make_layer(W.scaled(cfg, n_tokens=1), seed=0, layer_id=0, device=dev))
+    n_me = probe.n_me
+    ws_score = P.alloc_workspace(P.camera_score_workspace_bytes(probe, T), dev)
+    del probe
+    ws_all = P.alloc_workspace(P.camera_select_workspace_bytes(nl * n_me, nl, len(PRUNE_RATIOS) + len(BIT_LEVELS)), dev)
+    E_all = torch.empty((nl, n_me), dtype=torch.float32, device=dev)
+    keep_all = torch.empty((len(PRUNE_RATIOS), nl * n_me), dtype=torch.uint8, device=dev)
+    bits_all = torch.empty(nl * n_me, dtype=torch.uint8, device=dev)
+    score_ms, gen_s = 0.0, 0.0
+    for l in range(nl):
+        t0 = time.perf_counter()
+        L = W.make_layer(cfg, seed=0, layer_id=l, device=dev)
+        X = W.make_tokens(cfg, seed=0, layer_id=l, device=dev)
+        layer = P.Layer.from_workload(L)
+        torch.cuda.synchronize()
+        gen_s += time.perf_counter() - t0
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record(stream)
+        P.camera_score_layer(layer, X, ALPHA, energy=E_all[l], workspace=ws_score)
+        e1.record(stream)
+        torch.cuda.synchronize()
+        if P.camera_read_status(ws_score) != 0:
+            raise RuntimeError("device status set in the whole-model run")
+        score_ms += e0.elapsed_time(e1)
+        del L, X, layer
+    seg = [i * n_me for i in range(nl + 1)]
+    s0, s1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    s0.record(stream)
+    P.camera_select_all(E_all.view(-1), PRUNE_RATIOS, BIT_RATIOS, BIT_LEVELS, seg_offsets=seg, workspace=ws_all,
+                        keep_masks=keep_all, bits_out=bits_all)
+    s1.record(stream)
+    torch.cuda.synchronize()
+    sel_ms = s0.elapsed_time(s1)
+    kept = keep_all.view(len(PRUNE_RATIOS), nl, n_me).sum(dim=2)
+    ok = all(int(kept[j, l]) == n_me - int(PRUNE_RATIOS[j] * n_me + 1e-9) for j in range(len(PRUNE_RATIOS)) for l in range(nl))
+    return {"what": f"{nl} layers, each with its own seeded weights and {T} tokens: camera_score_layer per layer, one "
+                    f"camera_select_all over {nl} segments", "seconds": (score_ms + sel_ms) * 1e-3,
+            "score_seconds": score_ms * 1e-3, "select_ms": sel_ms, "input_generation_seconds_not_timed": gen_s,
+            "kept_counts_as_expected": bool(ok)}
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -286,6 +443,8 @@ def main():
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-compact", action="store_true")
     ap.add_argument("--no-forward", action="store_true")
+    ap.add_argument("--no-configs", action="store_true", help="skip the other workload configs")
+    ap.add_argument("--no-model", action="store_true", help="skip the measured loop over all layers of the model")
     ap.add_argument("--stack", action="store_true", help="run Algorithm 2's layer loop over a synthetic stack instead of the step benchmark")
     ap.add_argument("--stack-layers", type=int, default=0, help="layers of the stack (default: the config's)")
     args = ap.parse_args()
@@ -513,8 +672,20 @@ def main():
             select_all()
         s1.record(stream); sync_all()
         sel_ms = s0.elapsed_time(s1) / 10
-        sel_bytes = 9 * 4 * nl * n_me + 4 * nl * n_me       # 9 passes over the fp32 keys, four bytes of labels per key out
+        sel_bytes = 4 * nl * n_me + 4 * nl * n_me           # algorithmic: every energy read once, four label bytes per key out
+        ws_one = P.alloc_workspace(P.camera_select_workspace_bytes(n_me, 1, len(PRUNE_RATIOS) + len(BIT_LEVELS)), dev)
+        def select_one():
+            P.camera_select_all(energy, PRUNE_RATIOS, BIT_RATIOS, BIT_LEVELS, workspace=ws_one, keep_masks=keep, bits_out=bits)
+        for _ in range(3):
+            select_one()
+        sync_all()
+        s0.record(stream)
+        for _ in range(20):
+            select_one()
+        s1.record(stream); sync_all()
+        one_us = 1e3 * s0.elapsed_time(s1) / 20
         select_model = {"what": f"3 prune masks + bit allocation for {nl} layers as segments of one camera_select_all call", "ms": sel_ms,
+                        "one_layer_call_us": one_us, "launches_per_call": 1,
                         "algorithmic_gb": sel_bytes / 1e9, "achieved_gbs": sel_bytes / 1e9 / (sel_ms * 1e-3),
                         "frac_of_hbm_peak": sel_bytes / 1e9 / (sel_ms * 1e-3) / load_peaks()["hbm_gbs"]}
         del Eall, keep_all, bits_all, ws_all
@@ -553,12 +724,24 @@ def main():
         return
 
     peaks = load_peaks()
+    # ---- the other workload configs and the measured loop over the model's layers (one GPU; not part of the step loop)
+    configs = model_measured = None
+    default_run = world == 1 and args.config == "qwen2_57b_a14b" and not (args.tokens or args.routed or args.topk)
+    if default_run and not args.no_configs:
+        torch.cuda.empty_cache()
+        configs = {name: bench_other_config(P, torch, W, name, dev, stream, local, peaks)
+                   for name in ("tiny_fp32", "mixtral_8x7b", "qwen15_moe_a27b", "deepseek_moe_16b")}
+    if default_run and not args.no_model:
+        torch.cuda.empty_cache()
+        model_measured = bench_whole_model(P, torch, W, cfg, dev, stream)
     flop = cfg.gate_up_flop
     score_ms = stage_ms["score"]
     achieved = flop / (score_ms * 1e-3) / 1e12
     roofline = {"kernel": "k_score_umma" if args.single_cta else "k_score_umma_pair / k_score_umma (library's choice)", "bound": "tensor", "achieved": achieved,
                 "peak": peaks["bf16_tflops_sustained"], "unit": "TFLOP/s", "frac": achieved / peaks["bf16_tflops_sustained"],
-                "frac_of_burst_peak": achieved / peaks["bf16_tflops"], "peak_source": peaks["source"] + " (sustained bf16)",
+                "frac_of_burst_peak": achieved / peaks["bf16_tflops"], "burst_peak": peaks["bf16_tflops"],
+                "peak_source": peaks["source"] + " (cuBLAS bf16 sustained in a seconds-long loop: the kernel is timed inside "
+                                                 "a multi-second step loop; the burst figure is beside it)",
                 "flop_per_launch": flop, "ms_per_launch": score_ms,
                 "traffic": SCORE_KERNEL_DRAM_BYTES_PER_FLOP * flop
                 if (args.config == "qwen2_57b_a14b" and not args.single_cta) else None}
@@ -583,7 +766,8 @@ def main():
                    "bit_levels": list(BIT_LEVELS), "bit_ratios": list(BIT_RATIOS),
                    "l2": "inputs larger than L2" if flush is None else "L2 flushed between steps (256 MiB write, not timed)",
                    "parallelism": (f"tokens x{world}" if by_tokens else f"layers x{world}") if world > 1 else "single GPU"},
-        "model_seconds": cfg.n_layers * ms_per_step * 1e-3 / world,
+        "model_seconds": cfg.n_layers * ms_per_step * 1e-3 / world,     # extrapolated: layers x the step on one layer
+        "model_seconds_measured": model_measured, "configs": configs,
         "stage_ms": stage_ms, "clocks": clocks, "e2e": e2e, "gpu_launches": (LAUNCHES_PER_STEP + (3 if by_tokens else 0)) * args.steps,
         "roofline": roofline, "compact": compact, "forward": forward, "decode": decode, "select_model": select_model, "cpu_baseline": cpu, "context": PAPER_CONTEXT,
     }

@@ -173,7 +173,10 @@ uint64_t camera_get_wait_limit_ns(void);
  */
 int camera_wait_probe(void* workspace, size_t workspace_bytes, uint64_t limit_ns, void* cuda_stream);
 
-/* Scratch for camera_select_prune / camera_alloc_bits (n_levels = 2 for pruning). */
+/* Scratch for camera_select_prune / camera_alloc_bits (n_levels = 2 for pruning), 256-byte aligned.  The selection
+ * is one kernel whose CTAs meet at counters in this scratch (launched cooperatively, so that they are resident
+ * together); its waits are bounded like those of the scoring kernels and report through the scratch's status word,
+ * which camera_read_status reads like a scoring workspace's. */
 size_t camera_select_workspace_bytes(int64_t n_total, int32_t n_segments, int32_t n_levels);
 
 /*
@@ -208,8 +211,8 @@ int camera_alloc_bits(const float* energy, const int64_t* seg_offsets, int32_t n
 /*
  * Several CAMERA-P masks (Algorithm 2, TopSelect at several prune ratios) and the CAMERA-Q bit-widths (Algorithm 3,
  * ListSplitByRatio) of the same energies from one set of radix passes: every threshold is a rank of the same keys, so
- * the eight histogram passes find them together and one pass writes all outputs (10 launches instead of 9 per mask
- * and 9 for the bit-widths).  The results are those of camera_select_prune / camera_alloc_bits, bit for bit.
+ * the four histogram passes find them together and all outputs are written at the end of the same kernel (one launch
+ * where the separate calls take one each).  The results are those of camera_select_prune / camera_alloc_bits, bit for bit.
  * prune_ratios: HOST [n_prune];  keep_masks: DEVICE uint8 [n_prune][N] (mask p at keep_masks + p * N, N =
  * seg_offsets[n_segments]);  ratios, bits, n_levels, bits_out as for camera_alloc_bits, bits_out may be NULL (no
  * bit-widths; ratios, bits, n_levels are then ignored).  n_prune + n_levels - 1 <= 7, else CAMERA_ERR_INVALID_ARG.

@@ -1,179 +1,361 @@
 // Device-wide segmented rank selection for CAMERA-P (Algorithm 2, TopSelect) and CAMERA-Q
 // (Algorithm 3, ListSplitByRatio / GetSubIndex).
 //
-// Every micro-expert gets the 64-bit key (order-preserving image of its fp32 energy) << 32 | index
-// within its segment.  Keys are unique, so "the r-th smallest key" is unambiguous and equal
-// energies are ordered by index.  The key of rank r is found by a most-significant-digit radix
-// select: 8 passes of 8 bits, each pass a histogram (shared-memory bins, flushed with integer
-// atomics, hence deterministic) of the digit among the keys that match the prefix found so far.
-// Several ranks per segment (the class boundaries) are selected in the same passes.
+// Every micro-expert has the key (order-preserving image of its fp32 energy, index within its
+// segment), compared lexicographically: keys are unique, "the r-th smallest key" is unambiguous and
+// equal energies are ordered by index.  The key of rank r is found by a most-significant-digit radix
+// select over the 32 energy bits, 4 digits of 8 bits: each pass builds a histogram (shared-memory
+// bins, flushed with integer atomics, hence deterministic) of the next digit among the keys that
+// match the digits found so far.  The index part only matters among the keys whose energy equals
+// the threshold's, and only when some of them fall below it: then every CTA counts its share of them
+// and the one CTA that holds the boundary finds it with an ordered scan.  Several ranks per segment
+// (prune thresholds of several ratios, class boundaries) are selected in the same passes.
+//
+// All of it is ONE launch.  A segment is split over gridDim.x CTAs that keep their keys in shared
+// memory and meet after every pass at a counter in global memory (five meetings at most).  CTAs that
+// wait on one another must be resident together, so the kernel is launched cooperatively whenever a
+// segment has more than one CTA, with a grid no larger than what fits the device at once; rows of
+// CTAs walk over the segments.  The waits are bounded: one that runs out records
+// CAMERA_ERR_DEVICE_TIMEOUT in the scratch's status word and the kernel returns.
 #include <math.h>
 #include <string.h>
 
 #include <vector>
 
 #include "common.cuh"
+#include "umma.cuh"
 
 namespace camera {
 
 namespace {
 
 constexpr int SEL_THREADS = 256;
-constexpr int SEL_PASSES = 8;
+constexpr int SEL_PASSES = 4;
 constexpr int MAX_THR = MAX_LEVELS - 1;
+constexpr int SEL_CTA_KEYS = 2048;        // keys a CTA takes when the device has CTAs to spare
+constexpr int SEL_CACHE_KEYS = 6144;      // most keys a CTA keeps in shared memory (longer shares are re-read from L2);
+                                          // six CTAs of 24 KB + 7 KB fit an SM
+constexpr int SEL_MAX_GX = 2048;          // bound on CTAs per segment that the scratch is sized for
+constexpr int SEL_PARAM_SEGS = 32;        // up to this many segments the offsets and ranks travel as kernel arguments
+constexpr int SEL_BARS = 8;               // meeting counters per segment (5 used)
 
-struct SelState {
-  unsigned long long prefix;   // digits fixed so far, in place
-  long long rank;              // rank still to find among the keys that match; < 0 = no such element
+// First bytes of the scratch, laid out like the scoring workspace's so that camera_read_status reads either.
+struct SelHeader {
+  int32_t r0, r1;
+  int32_t status;
+  int32_t abort;      // set with the status: the other CTAs stop waiting
+  int32_t pad[4];
 };
 
-__device__ __forceinline__ unsigned long long make_key(float e, unsigned idx) {
-  unsigned b = __float_as_uint(e);
-  b ^= (b >> 31) ? 0xffffffffu : 0x80000000u;
-  return ((unsigned long long)b << 32) | idx;
-}
-
-__device__ __forceinline__ float key_energy(unsigned long long key) {
-  unsigned b = (unsigned)(key >> 32);
-  b = (b & 0x80000000u) ? (b ^ 0x80000000u) : ~b;
-  return __uint_as_float(b);
-}
-
-// State after `pass` passes for (segment seg, threshold j), computed by warp j of every CTA from
-// the state after pass-1 passes and the (complete) histogram of pass-1.  Result in shared st[j].
-__device__ void advance_state(int pass, int seg, int n_thr, long long seg_len, const long long* ranks,
-                              const SelState* S, const unsigned* hist, int n_seg, SelState* st) {
-  const int lane = threadIdx.x & 31, j = threadIdx.x >> 5;
-  if (j >= n_thr) return;
-  SelState cur;
-  if (pass <= 1) {
-    cur.prefix = 0ull;
-    cur.rank = ranks[seg * n_thr + j];
-    if (cur.rank >= seg_len) cur.rank = -1;
-  } else {
-    cur = S[((size_t)(pass - 2) * n_seg + seg) * n_thr + j];
-  }
-  if (pass >= 1 && cur.rank >= 0) {
-    const unsigned* h = hist + (((size_t)(pass - 1) * n_seg + seg) * n_thr + j) * 256;
-    // lane owns bins [8*lane, 8*lane+8)
-    unsigned v[8];
-    long long mine = 0;
-#pragma unroll
-    for (int i = 0; i < 8; ++i) { v[i] = h[lane * 8 + i]; mine += v[i]; }
-    long long incl = mine;
-#pragma unroll
-    for (int o = 1; o < 32; o <<= 1) {
-      const long long n = __shfl_up_sync(0xffffffffu, incl, o);
-      if (lane >= o) incl += n;
-    }
-    long long before = incl - mine;
-    const bool here = cur.rank >= before && cur.rank < incl;
-    int bin = -1;
-    long long newrank = 0;
-    if (here) {
-#pragma unroll
-      for (int i = 0; i < 8; ++i) {
-        if (bin < 0 && cur.rank < before + (long long)v[i]) { bin = lane * 8 + i; newrank = cur.rank - before; }
-        before += v[i];
-      }
-    }
-    const unsigned who = __ballot_sync(0xffffffffu, here);
-    if (who == 0u) {
-      cur.rank = -1;    // cannot happen for a rank inside the segment
-    } else {
-      const int src = __ffs(who) - 1;
-      bin = __shfl_sync(0xffffffffu, bin, src);
-      newrank = __shfl_sync(0xffffffffu, newrank, src);
-      cur.prefix |= (unsigned long long)bin << (56 - 8 * (pass - 1));
-      cur.rank = newrank;
-    }
-  }
-  if (lane == 0) st[j] = cur;
-}
-
-__global__ void __launch_bounds__(SEL_THREADS)
-k_select_hist(int pass, const float* __restrict__ energy, const long long* seg_off, const long long* ranks,
-              SelState* S, unsigned* hist, int n_seg, int n_thr) {
-  __shared__ SelState st[MAX_THR];
-  __shared__ unsigned bins[MAX_THR][256];
-  const int seg = blockIdx.y;
-  const long long begin = seg_off[seg], len = seg_off[seg + 1] - begin;
-  for (int i = threadIdx.x; i < n_thr * 256; i += SEL_THREADS) (&bins[0][0])[i] = 0u;
-  advance_state(pass, seg, n_thr, len, ranks, S, hist, n_seg, st);
-  __syncthreads();
-  if (pass >= 1 && blockIdx.x == 0 && threadIdx.x < n_thr)
-    S[((size_t)(pass - 1) * n_seg + seg) * n_thr + threadIdx.x] = st[threadIdx.x];
-  const int shift = 56 - 8 * pass;
-  for (long long i = (long long)blockIdx.x * SEL_THREADS + threadIdx.x; i < len; i += (long long)gridDim.x * SEL_THREADS) {
-    const unsigned long long key = make_key(energy[begin + i], (unsigned)i);
-    const unsigned digit = (unsigned)(key >> shift) & 0xffu;
-    for (int j = 0; j < n_thr; ++j) {
-      if (st[j].rank < 0) continue;
-      if (pass == 0 || (key >> (shift + 8)) == (st[j].prefix >> (shift + 8))) atomicAdd(&bins[j][digit], 1u);
-    }
-  }
-  __syncthreads();
-  unsigned* h = hist + (((size_t)pass * n_seg + seg) * n_thr) * 256;
-  for (int i = threadIdx.x; i < n_thr * 256; i += SEL_THREADS) {
-    const unsigned v = (&bins[0][0])[i];
-    if (v) atomicAdd(h + i, v);
-  }
-}
+// The selected key of one (segment, threshold): an element is at or above it when
+// (bits, index) >= (bits, index) lexicographically; valid == 0: nothing is.
+struct SelFinal {
+  unsigned bits;
+  unsigned index;
+  int valid;
+  int pad;
+};
 
 struct LevelValues { unsigned char v[MAX_LEVELS]; };
 
-// Labels every element with the value of its class: class = (n_thr - number of thresholds the
-// key is at or above), thresholds being the selected keys.
-__global__ void __launch_bounds__(SEL_THREADS)
-k_select_mark(const float* __restrict__ energy, const long long* seg_off, const long long* ranks, SelState* S,
-              const unsigned* hist, int n_seg, int n_thr, LevelValues lv, unsigned char* out, float* thresholds) {
-  __shared__ SelState st[MAX_THR];
-  const int seg = blockIdx.y;
-  const long long begin = seg_off[seg], len = seg_off[seg + 1] - begin;
-  advance_state(SEL_PASSES, seg, n_thr, len, ranks, S, hist, n_seg, st);
-  __syncthreads();
-  if (blockIdx.x == 0 && threadIdx.x < n_thr) {
-    S[((size_t)(SEL_PASSES - 1) * n_seg + seg) * n_thr + threadIdx.x] = st[threadIdx.x];
-    if (thresholds != nullptr && threadIdx.x == 0)
-      thresholds[seg] = st[0].rank >= 0 ? key_energy(st[0].prefix) : INFINITY;
-  }
-  for (long long i = (long long)blockIdx.x * SEL_THREADS + threadIdx.x; i < len; i += (long long)gridDim.x * SEL_THREADS) {
-    const unsigned long long key = make_key(energy[begin + i], (unsigned)i);
-    int above = 0;
-    for (int j = 0; j < n_thr; ++j) above += (st[j].rank >= 0 && key >= st[j].prefix) ? 1 : 0;
-    out[begin + i] = lv.v[n_thr - above];
-  }
+struct SelParams {
+  long long seg_off[SEL_PARAM_SEGS + 1];
+  long long ranks[SEL_PARAM_SEGS * MAX_THR];
+};
+
+struct SelArgs {
+  const float* energy;
+  const long long* seg_off;     // DEVICE copies when there are more than SEL_PARAM_SEGS segments, else null
+  const long long* ranks;
+  SelHeader* hdr;
+  unsigned* bars;               // [n_seg][SEL_BARS], zero at launch
+  unsigned* hist;               // [n_seg][SEL_PASSES][n_thr][256], zero at launch
+  unsigned* eqcnt;              // [n_seg][n_thr][gridDim.x]
+  SelFinal* fin;                // [n_seg][n_thr]
+  int n_seg, n_thr;
+  int n_prune;                  // >= 0: thresholds 0 .. n_prune-1 give keep masks, the rest class boundaries
+  LevelValues lv;
+  long long n_total;
+  unsigned char* out;           // n_prune < 0: the label of every element; else n_prune masks of n_total bytes
+  unsigned char* bits_out;      // n_prune >= 0: class values, or null
+  float* thresholds;            // [n_seg] energy of threshold 0, or null
+  unsigned long long wait_limit_ns;
+};
+
+__device__ __forceinline__ unsigned key_bits(float e) {
+  const unsigned b = __float_as_uint(e);
+  return b ^ ((b >> 31) ? 0xffffffffu : 0x80000000u);
+}
+__device__ __forceinline__ float bits_energy(unsigned b) {
+  return __uint_as_float((b & 0x80000000u) ? (b ^ 0x80000000u) : ~b);
+}
+__device__ __forceinline__ unsigned ld_acquire_u32(const unsigned* p) {
+  unsigned v;
+  asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
+  return v;
 }
 
-// The mark pass of camera_select_all: thresholds 0 .. n_prune-1 each give a keep mask of their own, the remaining
-// n_thr - n_prune thresholds are the class boundaries of the bit-width allocation.
-__global__ void __launch_bounds__(SEL_THREADS)
-k_select_mark_all(const float* __restrict__ energy, const long long* seg_off, const long long* ranks, SelState* S,
-                  const unsigned* hist, int n_seg, int n_thr, int n_prune, LevelValues lv, long long n_total,
-                  unsigned char* keep_out, unsigned char* bits_out) {
-  __shared__ SelState st[MAX_THR];
-  const int seg = blockIdx.y;
-  const long long begin = seg_off[seg], len = seg_off[seg + 1] - begin;
-  advance_state(SEL_PASSES, seg, n_thr, len, ranks, S, hist, n_seg, st);
+// The CTAs of a segment meet: everything they wrote before is visible to all of them after.  Bounded: returns false
+// (for the whole CTA) when the limit ran out here or in another CTA.
+__device__ bool seg_meet(unsigned* counter, unsigned expected, const SelArgs& a, int* s_abort) {
   __syncthreads();
-  if (blockIdx.x == 0 && threadIdx.x < n_thr)
-    S[((size_t)(SEL_PASSES - 1) * n_seg + seg) * n_thr + threadIdx.x] = st[threadIdx.x];
-  const int n_bounds = n_thr - n_prune;
-  for (long long i = (long long)blockIdx.x * SEL_THREADS + threadIdx.x; i < len; i += (long long)gridDim.x * SEL_THREADS) {
-    const unsigned long long key = make_key(energy[begin + i], (unsigned)i);
-    for (int j = 0; j < n_prune; ++j)
-      keep_out[(size_t)j * n_total + begin + i] = (st[j].rank >= 0 && key >= st[j].prefix) ? 1 : 0;
-    if (bits_out != nullptr) {
-      int above = 0;
-      for (int j = n_prune; j < n_thr; ++j) above += (st[j].rank >= 0 && key >= st[j].prefix) ? 1 : 0;
-      bits_out[begin + i] = lv.v[n_bounds - above];
+  if (threadIdx.x == 0) {
+    if (expected > 1u) {
+      __threadfence();
+      atomicAdd(counter, 1u);
+      const unsigned long long t0 = globaltimer_ns();
+      unsigned spins = 0;
+      while (ld_acquire_u32(counter) < expected) {
+        if ((++spins & 15u) == 0u) {
+          if (*reinterpret_cast<volatile int*>(&a.hdr->abort)) { *s_abort = 1; break; }
+          if (globaltimer_ns() - t0 > a.wait_limit_ns) {
+            atomicExch(&a.hdr->status, (int)CAMERA_ERR_DEVICE_TIMEOUT);
+            atomicExch(&a.hdr->abort, 1);
+            *s_abort = 1;
+            break;
+          }
+        }
+      }
+      __threadfence();
     }
+  }
+  __syncthreads();
+  return *s_abort == 0;
+}
+
+struct ThrState {
+  unsigned prefix;      // digits found so far, in place
+  int valid;            // 0: the rank is past the segment, nothing is at or above
+  long long rank;       // rank still to find among the keys that match the prefix
+};
+
+__global__ void __launch_bounds__(SEL_THREADS, 6)
+k_select_fused(const __grid_constant__ SelArgs a, const __grid_constant__ SelParams prm) {
+  extern __shared__ unsigned skeys[];                 // [SEL_CACHE_KEYS] when the grid's shares fit, else unused
+  __shared__ unsigned bins[MAX_THR][256];
+  __shared__ ThrState st[MAX_THR];
+  __shared__ unsigned eq_mine[MAX_THR];               // this CTA's keys whose energy equals the threshold's
+  __shared__ unsigned first_above[MAX_THR];           // local index from which such keys are at or above the threshold
+  __shared__ int boundary[MAX_THR];
+  __shared__ int rep[MAX_THR];
+  __shared__ unsigned boundary_skip[MAX_THR];
+  __shared__ unsigned wtot[SEL_THREADS / 32];
+  __shared__ int s_abort;
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int n_thr = a.n_thr;
+  const unsigned gx = gridDim.x, bx = blockIdx.x;
+  if (tid == 0) s_abort = 0;
+
+  for (int seg = blockIdx.y; seg < a.n_seg; seg += gridDim.y) {
+    const long long begin = a.seg_off ? a.seg_off[seg] : prm.seg_off[seg];
+    const long long len = (a.seg_off ? a.seg_off[seg + 1] : prm.seg_off[seg + 1]) - begin;
+    if (len == 0) {                                    // the same for every CTA of the row: nothing to select from
+      if (bx == 0 && tid < n_thr) {
+        SelFinal f;
+        f.bits = 0u; f.index = 0u; f.valid = 0; f.pad = 0;
+        a.fin[(size_t)seg * n_thr + tid] = f;
+        if (tid == 0 && a.thresholds != nullptr) a.thresholds[seg] = INFINITY;
+      }
+      continue;
+    }
+    const long long per = (len + gx - 1) / gx;
+    const long long c0 = per * bx < len ? per * bx : len;
+    const int n = (int)((c0 + per < len ? c0 + per : len) - c0);       // this CTA's share: [c0, c0 + n) of the segment
+    const bool cached = per <= SEL_CACHE_KEYS;
+    const float* src = a.energy + begin + c0;
+    if (cached)
+      for (int i = tid; i < n; i += SEL_THREADS) skeys[i] = key_bits(src[i]);
+    if (tid < n_thr) {
+      const long long r = a.ranks ? a.ranks[(size_t)seg * n_thr + tid] : prm.ranks[seg * n_thr + tid];
+      st[tid].prefix = 0u;
+      st[tid].valid = r >= 0 && r < len;
+      st[tid].rank = r;
+      eq_mine[tid] = 0u;
+      first_above[tid] = 0u;
+      boundary[tid] = 0;
+      rep[tid] = tid;
+    }
+    unsigned* const hseg = a.hist + (size_t)seg * SEL_PASSES * n_thr * 256;
+    unsigned* const bseg = a.bars + (size_t)seg * SEL_BARS;
+
+    for (int pass = 0; pass < SEL_PASSES; ++pass) {
+      const int nh = pass == 0 ? 1 : n_thr;            // the first digit's histogram serves every threshold
+      for (int i = tid; i < nh * 256; i += SEL_THREADS) (&bins[0][0])[i] = 0u;
+      __syncthreads();
+      const int shift = 24 - 8 * pass;
+      if (pass == 0) {
+        // energies of one layer share their leading bits: a thread counts runs of equal digits in a register and
+        // touches the bin once per run, not once per key
+        unsigned run_digit = 0u, run_len = 0u;
+        for (int i = tid; i < n; i += SEL_THREADS) {
+          const unsigned digit = (cached ? skeys[i] : key_bits(src[i])) >> 24;
+          if (digit != run_digit) {
+            if (run_len) atomicAdd(&bins[0][run_digit], run_len);
+            run_digit = digit;
+            run_len = 0u;
+          }
+          ++run_len;
+        }
+        if (run_len) atomicAdd(&bins[0][run_digit], run_len);
+      } else {
+        // thresholds whose digits so far agree share one histogram (that of the lowest-numbered among them)
+        unsigned pre[MAX_THR];
+#pragma unroll
+        for (int j = 0; j < MAX_THR; ++j)
+          pre[j] = (j < n_thr && st[j].valid && rep[j] == j) ? (st[j].prefix >> (shift + 8)) : 0xffffffffu;
+        for (int i = tid; i < n; i += SEL_THREADS) {
+          const unsigned b = cached ? skeys[i] : key_bits(src[i]);
+          const unsigned hi = b >> (shift + 8), digit = (b >> shift) & 0xffu;
+#pragma unroll
+          for (int j = 0; j < MAX_THR; ++j)
+            if (hi == pre[j]) atomicAdd(&bins[j][digit], 1u);          // pre of an unused slot matches nothing: hi < 2^24
+        }
+      }
+      __syncthreads();
+      for (int i = tid; i < nh * 256; i += SEL_THREADS) {
+        const unsigned v = (&bins[0][0])[i];
+        if (v) atomicAdd(hseg + (size_t)pass * n_thr * 256 + i, v);
+      }
+      if (!seg_meet(bseg + pass, gx, a, &s_abort)) return;
+      // warp j: the bin of threshold j's rank in the segment's histogram of this digit
+      if (warp < n_thr && st[warp].valid) {
+        const unsigned* h = hseg + ((size_t)pass * n_thr + (pass == 0 ? 0 : rep[warp])) * 256;
+        unsigned v[8];
+        long long mine = 0;
+#pragma unroll
+        for (int i = 0; i < 8; ++i) { v[i] = __ldcg(h + lane * 8 + i); mine += v[i]; }     // lane owns bins [8 lane, 8 lane + 8)
+        long long incl = mine;
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+          const long long t = __shfl_up_sync(0xffffffffu, incl, o);
+          if (lane >= o) incl += t;
+        }
+        long long before = incl - mine;
+        const long long rank = st[warp].rank;
+        if (rank >= before && rank < incl) {           // exactly one lane, for a rank inside the segment
+          int bin = lane * 8;
+#pragma unroll
+          for (int i = 0; i < 8; ++i) {
+            if (rank >= before + (long long)v[i]) { before += v[i]; bin = lane * 8 + i + 1; }
+            else break;
+          }
+          st[warp].prefix |= (unsigned)bin << shift;
+          st[warp].rank = rank - before;
+        }
+      }
+      __syncthreads();
+      if (tid < n_thr) {       // whose histogram threshold tid reads in the next pass
+        int r = tid;
+        for (int j = tid - 1; j >= 0; --j)
+          if (st[j].valid && st[tid].valid && st[j].prefix == st[tid].prefix) r = j;
+        rep[tid] = r;
+      }
+      // (the barrier after the bins are cleared orders this before the next pass reads it)
+    }
+
+    // Keys whose energy equals a threshold's: the st.rank lowest-indexed of them are below it.  With rank 0 (always,
+    // when the threshold's energy occurs once) all are at or above and nothing more is needed.  Otherwise the CTAs
+    // count theirs, and the one CTA whose share holds the first such key at or above the threshold looks it up.
+    bool ties = false;
+    for (int j = 0; j < n_thr; ++j) ties = ties || (st[j].valid && st[j].rank > 0);
+    if (ties) {
+      unsigned cnt[MAX_THR];
+#pragma unroll
+      for (int j = 0; j < MAX_THR; ++j) cnt[j] = 0u;
+      for (int i = tid; i < n; i += SEL_THREADS) {
+        const unsigned b = cached ? skeys[i] : key_bits(src[i]);
+#pragma unroll
+        for (int j = 0; j < MAX_THR; ++j)
+          if (j < n_thr && st[j].valid && b == st[j].prefix) ++cnt[j];
+      }
+#pragma unroll
+      for (int j = 0; j < MAX_THR; ++j)
+        if (j < n_thr && cnt[j]) atomicAdd(&eq_mine[j], cnt[j]);
+      __syncthreads();
+      if (tid < n_thr) a.eqcnt[((size_t)seg * n_thr + tid) * gx + bx] = eq_mine[tid];
+      if (!seg_meet(bseg + SEL_PASSES, gx, a, &s_abort)) return;
+      if (warp < n_thr && st[warp].valid && st[warp].rank > 0) {
+        const unsigned* ec = a.eqcnt + ((size_t)seg * n_thr + warp) * gx;
+        long long base = 0;                            // such keys in the CTAs before this one
+        for (unsigned c = lane; c < bx; c += 32) base += __ldcg(ec + c);
+#pragma unroll
+        for (int o = 16; o; o >>= 1) base += __shfl_xor_sync(0xffffffffu, base, o);
+        if (lane == 0) {
+          const long long r = st[warp].rank, mine = eq_mine[warp];
+          if (base + mine <= r) first_above[warp] = 0xffffffffu;       // all of this CTA's are below
+          else if (base > r) first_above[warp] = 0u;                   // all are at or above
+          else { boundary[warp] = 1; boundary_skip[warp] = (unsigned)(r - base); }   // it holds the first one at or above
+        }
+      }
+      __syncthreads();
+      // the one CTA that holds the boundary: the local index of its boundary_skip-th such key, by an ordered scan
+      for (int j = 0; j < n_thr; ++j) {
+        if (!boundary[j]) continue;                    // the same for every thread
+        const unsigned want = boundary_skip[j], tau = st[j].prefix;
+        unsigned run = 0;
+        for (int i0 = 0; i0 < n; i0 += SEL_THREADS) {
+          const int i = i0 + tid;
+          const bool m = i < n && (cached ? skeys[i] : key_bits(src[i])) == tau;
+          const unsigned bal = __ballot_sync(0xffffffffu, m);
+          if (lane == 0) wtot[warp] = __popc(bal);
+          __syncthreads();
+          unsigned woff = 0, total = 0;
+#pragma unroll
+          for (int w = 0; w < SEL_THREADS / 32; ++w) { woff += w < warp ? wtot[w] : 0u; total += wtot[w]; }
+          if (m && run + woff + __popc(bal & ((1u << lane) - 1u)) == want) first_above[j] = (unsigned)i;
+          __syncthreads();
+          run += total;
+          if (run > want) break;                       // the same for every thread
+        }
+      }
+      __syncthreads();
+    }
+
+    // the selected keys, for the per-expert counts and the thresholds' energies
+    if (tid < n_thr) {
+      const bool writer = st[tid].valid && st[tid].rank > 0 ? boundary[tid] != 0 : bx == 0;
+      if (writer) {
+        SelFinal f;
+        f.bits = st[tid].prefix;
+        f.index = st[tid].valid ? (unsigned)(c0 + (boundary[tid] ? first_above[tid] : 0u)) : 0u;
+        f.valid = st[tid].valid;
+        f.pad = 0;
+        a.fin[(size_t)seg * n_thr + tid] = f;
+      }
+      if (tid == 0 && bx == 0 && a.thresholds != nullptr)
+        a.thresholds[seg] = st[0].valid ? bits_energy(st[0].prefix) : INFINITY;
+    }
+
+    // labels
+    unsigned tau[MAX_THR], first[MAX_THR];
+#pragma unroll
+    for (int j = 0; j < MAX_THR; ++j) {
+      const bool v = j < n_thr && st[j].valid;
+      tau[j] = v ? st[j].prefix : 0xffffffffu;
+      first[j] = v ? first_above[j] : 0xffffffffu;     // (0xffffffff, 0xffffffff): no key is at or above
+    }
+    const int n_prune = a.n_prune, n_bounds = n_thr - (n_prune < 0 ? 0 : n_prune);
+    for (int i = tid; i < n; i += SEL_THREADS) {
+      const unsigned b = cached ? skeys[i] : key_bits(src[i]);
+      unsigned at = 0u;                                // bit j: at or above threshold j
+#pragma unroll
+      for (int j = 0; j < MAX_THR; ++j)
+        at |= (unsigned)(b > tau[j] || (b == tau[j] && (unsigned)i >= first[j])) << j;
+      const size_t g = (size_t)(begin + c0) + i;
+      if (n_prune < 0) {
+        a.out[g] = a.lv.v[n_thr - __popc(at)];
+      } else {
+        for (int j = 0; j < n_prune; ++j) a.out[(size_t)j * a.n_total + g] = (at >> j) & 1u;
+        if (a.bits_out != nullptr) a.bits_out[g] = a.lv.v[n_bounds - __popc(at >> n_prune)];
+      }
+    }
+    __syncthreads();       // the next segment reuses the shared arrays
   }
 }
 
 // One CTA per expert: how many of its micro-experts fall in each class (or are retained).
 __global__ void __launch_bounds__(SEL_THREADS)
-k_class_counts(const float* __restrict__ energy, const long long* seg_off, const SelState* S, int n_seg, int n_thr,
+k_class_counts(const float* __restrict__ energy, const long long* seg_off, const SelFinal* fin, int n_seg, int n_thr,
                const long long* expert_off, int n_classes_out, int* counts) {
   __shared__ int cnt[MAX_LEVELS];
   const int e = blockIdx.x;
@@ -182,14 +364,15 @@ k_class_counts(const float* __restrict__ energy, const long long* seg_off, const
   __syncthreads();
   if (en > b) {
     const int seg = upper_segment(seg_off, n_seg, b);
-    const SelState* fin = S + ((size_t)(SEL_PASSES - 1) * n_seg + seg) * n_thr;
+    const SelFinal* f = fin + (size_t)seg * n_thr;
     int local[MAX_LEVELS];
 #pragma unroll
     for (int j = 0; j < MAX_LEVELS; ++j) local[j] = 0;
     for (long long i = b + threadIdx.x; i < en; i += SEL_THREADS) {
-      const unsigned long long key = make_key(energy[i], (unsigned)(i - seg_off[seg]));
+      const unsigned kb = key_bits(energy[i]), idx = (unsigned)(i - seg_off[seg]);
       int above = 0;
-      for (int j = 0; j < n_thr; ++j) above += (fin[j].rank >= 0 && key >= fin[j].prefix) ? 1 : 0;
+      for (int j = 0; j < n_thr; ++j)
+        above += (f[j].valid && (kb > f[j].bits || (kb == f[j].bits && idx >= f[j].index))) ? 1 : 0;
       const int cls = n_thr - above;
 #pragma unroll
       for (int j = 0; j < MAX_LEVELS; ++j) local[j] += (cls == j);
@@ -202,63 +385,135 @@ k_class_counts(const float* __restrict__ energy, const long long* seg_off, const
   if (threadIdx.x < n_classes_out) counts[(size_t)e * n_classes_out + threadIdx.x] = cnt[threadIdx.x];
 }
 
+// CTAs per segment the scratch has room for: never more than the kernel is given.
+int sel_gx_bound(long long n_total, int n_seg) {
+  long long by_keys = (n_total + SEL_CTA_KEYS - 1) / SEL_CTA_KEYS;
+  long long by_segs = SEL_MAX_GX / (n_seg < SEL_MAX_GX ? n_seg : SEL_MAX_GX);
+  long long g = by_keys < by_segs ? by_keys : by_segs;
+  return (int)(g < 1 ? 1 : g);
+}
+
 struct SelLayout {
-  size_t seg_off, ranks, state, hist, total;
+  size_t hdr, bars, hist, zero_bytes, fin, eqcnt, seg_off, ranks, total;
 };
 
-SelLayout sel_layout(int n_seg, int n_thr) {
+SelLayout sel_layout(long long n_total, int n_seg, int n_thr) {
   auto up = [](size_t v) { return (v + 255) & ~(size_t)255; };
   SelLayout L;
   size_t o = 0;
+  L.hdr = o;     o = up(o + sizeof(SelHeader));
+  L.bars = o;    o = up(o + sizeof(unsigned) * (size_t)n_seg * SEL_BARS);
+  L.hist = o;    o = up(o + sizeof(unsigned) * (size_t)SEL_PASSES * n_seg * n_thr * 256);
+  L.zero_bytes = o;                                   // everything up to here starts at zero, in one memset
+  L.fin = o;     o = up(o + sizeof(SelFinal) * (size_t)n_seg * n_thr);
+  L.eqcnt = o;   o = up(o + sizeof(unsigned) * (size_t)n_seg * n_thr * sel_gx_bound(n_total, n_seg));
   L.seg_off = o; o = up(o + sizeof(long long) * (n_seg + 1));
   L.ranks = o;   o = up(o + sizeof(long long) * (size_t)n_seg * n_thr);
-  L.state = o;   o = up(o + sizeof(SelState) * (size_t)SEL_PASSES * n_seg * n_thr);
-  L.hist = o;    o = up(o + sizeof(unsigned) * (size_t)SEL_PASSES * n_seg * n_thr * 256);
   L.total = o;
   return L;
 }
 
 long long floor_count(double ratio, long long n) { return (long long)floor(ratio * (double)n + 1e-9); }
 
+// CTAs of k_select_fused that are resident at once on the current device (0 on error); asked once per device.
+int resident_ctas(size_t smem) {
+  constexpr int MAX_DEV = 64;
+  static int cache[MAX_DEV];      // 0 = not asked yet
+  int dev = 0, sms = 0, per_sm = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess) { cudaGetLastError(); return 0; }
+  if (dev >= 0 && dev < MAX_DEV && cache[dev] > 0) return cache[dev];
+  if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess ||
+      cudaFuncSetAttribute(k_select_fused, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess ||
+      cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, k_select_fused, SEL_THREADS, smem) != cudaSuccess) {
+    cudaGetLastError();
+    return 0;
+  }
+  if (dev >= 0 && dev < MAX_DEV) cache[dev] = sms * per_sm;
+  return sms * per_sm;
+}
+
 // ranks_host: [n_seg * n_thr] target ascending ranks (a rank >= the segment length selects nothing).
-// n_prune >= 0 selects the mark pass of camera_select_all: `out` then holds n_prune masks of seg_offsets[n_seg] bytes
+// n_prune >= 0 selects the labelling of camera_select_all: `out` then holds n_prune masks of seg_offsets[n_seg] bytes
 // and bits_out (may be null) gets the class values.
 int select_core(const float* energy, const int64_t* seg_offsets, int n_seg, int n_thr, const long long* ranks_host,
                 LevelValues lv, const int64_t* expert_offsets, int n_experts, int n_classes_out, unsigned char* out,
                 int* counts, float* thresholds, void* ws, size_t ws_bytes, cudaStream_t st, int n_prune = -1,
                 unsigned char* bits_out = nullptr) {
-  const SelLayout L = sel_layout(n_seg, n_thr);
-  if (ws == nullptr || ws_bytes < L.total) return CAMERA_ERR_WORKSPACE;
+  const long long n_total = seg_offsets[n_seg];
+  const SelLayout L = sel_layout(n_total, n_seg, n_thr);
+  if (ws == nullptr || ws_bytes < L.total || (reinterpret_cast<uintptr_t>(ws) & 255)) return CAMERA_ERR_WORKSPACE;
   char* base = static_cast<char*>(ws);
-  long long* d_seg = reinterpret_cast<long long*>(base + L.seg_off);
-  long long* d_ranks = reinterpret_cast<long long*>(base + L.ranks);
-  SelState* d_state = reinterpret_cast<SelState*>(base + L.state);
-  unsigned* d_hist = reinterpret_cast<unsigned*>(base + L.hist);
   long long max_len = 0;
   for (int s = 0; s < n_seg; ++s) max_len = seg_offsets[s + 1] - seg_offsets[s] > max_len ? seg_offsets[s + 1] - seg_offsets[s] : max_len;
-  if (cudaMemcpyAsync(d_seg, seg_offsets, sizeof(long long) * (n_seg + 1), cudaMemcpyHostToDevice, st) != cudaSuccess ||
-      cudaMemcpyAsync(d_ranks, ranks_host, sizeof(long long) * (size_t)n_seg * n_thr, cudaMemcpyHostToDevice, st) != cudaSuccess ||
-      cudaMemsetAsync(d_hist, 0, sizeof(unsigned) * (size_t)SEL_PASSES * n_seg * n_thr * 256, st) != cudaSuccess)
-    return CAMERA_ERR_CUDA;
-  if (max_len > 0) {
-    long long gx = (max_len + SEL_THREADS * 8 - 1) / (SEL_THREADS * 8);
-    if (gx > 1184) gx = 1184;
+
+  SelArgs a;
+  memset(&a, 0, sizeof(a));
+  SelParams prm;
+  memset(&prm, 0, sizeof(prm));
+  a.energy = energy;
+  a.hdr = reinterpret_cast<SelHeader*>(base + L.hdr);
+  a.bars = reinterpret_cast<unsigned*>(base + L.bars);
+  a.hist = reinterpret_cast<unsigned*>(base + L.hist);
+  a.eqcnt = reinterpret_cast<unsigned*>(base + L.eqcnt);
+  a.fin = reinterpret_cast<SelFinal*>(base + L.fin);
+  a.n_seg = n_seg; a.n_thr = n_thr; a.n_prune = n_prune; a.lv = lv; a.n_total = n_total;
+  a.out = out; a.bits_out = bits_out; a.thresholds = thresholds;
+  a.wait_limit_ns = current_wait_limit_ns();
+  long long* d_seg = reinterpret_cast<long long*>(base + L.seg_off);
+  if (n_seg <= SEL_PARAM_SEGS) {
+    for (int s = 0; s <= n_seg; ++s) prm.seg_off[s] = seg_offsets[s];
+    for (int i = 0; i < n_seg * n_thr; ++i) prm.ranks[i] = ranks_host[i];
+  } else {
+    a.seg_off = d_seg;
+    a.ranks = reinterpret_cast<long long*>(base + L.ranks);
+    if (cudaMemcpyAsync(d_seg, seg_offsets, sizeof(long long) * (n_seg + 1), cudaMemcpyHostToDevice, st) != cudaSuccess ||
+        cudaMemcpyAsync(const_cast<long long*>(a.ranks), ranks_host, sizeof(long long) * (size_t)n_seg * n_thr,
+                        cudaMemcpyHostToDevice, st) != cudaSuccess) {
+      cudaGetLastError();
+      return CAMERA_ERR_CUDA;
+    }
+  }
+  if (cudaMemsetAsync(base, 0, L.zero_bytes, st) != cudaSuccess) { cudaGetLastError(); return CAMERA_ERR_CUDA; }
+
+  {   // empty segments get their thresholds (infinity) from the kernel too
+    const size_t smem = sizeof(unsigned) * SEL_CACHE_KEYS;
+    const int resident = resident_ctas(smem);
+    if (resident < 1) return CAMERA_ERR_CUDA;
+    // CTAs per segment: shares of SEL_CTA_KEYS keys while the device has room, never more than the scratch holds
+    long long gx = (max_len + SEL_CTA_KEYS - 1) / SEL_CTA_KEYS;
+    const int rows_wanted = n_seg < resident ? n_seg : resident;
+    if (gx > resident / rows_wanted) gx = resident / rows_wanted;
+    const int bound = sel_gx_bound(n_total, n_seg);
+    if (gx > bound) gx = bound;
     if (gx < 1) gx = 1;
-    const dim3 grid((unsigned)gx, (unsigned)n_seg);
-    for (int p = 0; p < SEL_PASSES; ++p)
-      k_select_hist<<<grid, SEL_THREADS, 0, st>>>(p, energy, d_seg, d_ranks, d_state, d_hist, n_seg, n_thr);
-    if (n_prune >= 0)
-      k_select_mark_all<<<grid, SEL_THREADS, 0, st>>>(energy, d_seg, d_ranks, d_state, d_hist, n_seg, n_thr, n_prune, lv,
-                                                      (long long)seg_offsets[n_seg], out, bits_out);
-    else
-      k_select_mark<<<grid, SEL_THREADS, 0, st>>>(energy, d_seg, d_ranks, d_state, d_hist, n_seg, n_thr, lv, out, thresholds);
+    long long gy = resident / gx;
+    if (gy > n_seg) gy = n_seg;
+    if (gy > 65535) gy = 65535;
+    const dim3 grid((unsigned)gx, (unsigned)gy);
+    if (gx > 1) {     // CTAs of a segment wait for one another: they must all be resident
+      void* args[2] = {&a, &prm};
+      if (cudaLaunchCooperativeKernel(reinterpret_cast<const void*>(k_select_fused), grid, dim3(SEL_THREADS), args, smem, st) !=
+          cudaSuccess) {
+        cudaGetLastError();
+        return CAMERA_ERR_CUDA;
+      }
+    } else {
+      k_select_fused<<<grid, SEL_THREADS, smem, st>>>(a, prm);
+    }
   }
   if (counts != nullptr && expert_offsets != nullptr && n_experts > 0) {
-    if (max_len > 0)
-      k_class_counts<<<n_experts, SEL_THREADS, 0, st>>>(energy, d_seg, d_state, n_seg, n_thr,
+    if (max_len > 0) {
+      if (a.seg_off == nullptr &&
+          cudaMemcpyAsync(d_seg, seg_offsets, sizeof(long long) * (n_seg + 1), cudaMemcpyHostToDevice, st) != cudaSuccess) {
+        cudaGetLastError();
+        return CAMERA_ERR_CUDA;
+      }
+      k_class_counts<<<n_experts, SEL_THREADS, 0, st>>>(energy, d_seg, a.fin, n_seg, n_thr,
                                                         reinterpret_cast<const long long*>(expert_offsets), n_classes_out, counts);
-    else if (cudaMemsetAsync(counts, 0, sizeof(int) * (size_t)n_experts * n_classes_out, st) != cudaSuccess)
+    } else if (cudaMemsetAsync(counts, 0, sizeof(int) * (size_t)n_experts * n_classes_out, st) != cudaSuccess) {
+      cudaGetLastError();
       return CAMERA_ERR_CUDA;
+    }
   }
   return cudaGetLastError() == cudaSuccess ? CAMERA_OK : CAMERA_ERR_CUDA;
 }
@@ -266,7 +521,7 @@ int select_core(const float* energy, const int64_t* seg_offsets, int n_seg, int 
 bool segments_ok(const int64_t* seg, int n_seg) {
   if (seg == nullptr || n_seg < 1 || n_seg > 65535 || seg[0] != 0) return false;
   for (int s = 0; s < n_seg; ++s)
-    if (seg[s + 1] < seg[s] || seg[s + 1] - seg[s] > 0xffffffffll) return false;
+    if (seg[s + 1] < seg[s] || seg[s + 1] - seg[s] > 0x7fff0000ll) return false;
   return true;
 }
 
@@ -276,8 +531,8 @@ bool segments_ok(const int64_t* seg, int n_seg) {
 using namespace camera;
 
 extern "C" size_t camera_select_workspace_bytes(int64_t n_total, int32_t n_segments, int32_t n_levels) {
-  if (n_total < 0 || n_segments < 1 || n_levels < 2 || n_levels > MAX_LEVELS) return 0;
-  return sel_layout(n_segments, n_levels - 1).total;
+  if (n_total < 0 || n_segments < 1 || n_segments > 65535 || n_levels < 2 || n_levels > MAX_LEVELS) return 0;
+  return sel_layout(n_total, n_segments, n_levels - 1).total;
 }
 
 extern "C" int camera_select_prune(const float* energy, const int64_t* seg_offsets, int32_t n_segments,
@@ -422,7 +677,7 @@ extern "C" int camera_select_prune_static(const float* energy, const int64_t* se
   if (!segments_ok(seg_offsets, n_segments) || !(prune_ratio >= 0.0 && prune_ratio < 1.0) || keep_mask == nullptr)
     return CAMERA_ERR_INVALID_ARG;
   if (seg_offsets[n_segments] > 0 && energy == nullptr) return CAMERA_ERR_INVALID_ARG;
-  if (n_segments > STATIC_MAX_SEGMENTS || sel_layout(n_segments, 1).total > STATIC_SCRATCH_BYTES)
+  if (n_segments > STATIC_MAX_SEGMENTS || sel_layout(seg_offsets[n_segments], n_segments, 1).total > STATIC_SCRATCH_BYTES)
     return CAMERA_ERR_UNSUPPORTED_SHAPE;
   void* scratch = nullptr;
   const int rc = static_scratch(&scratch);
@@ -433,7 +688,7 @@ extern "C" int camera_select_prune_static(const float* energy, const int64_t* se
   memset(&lv, 0, sizeof(lv));
   lv.v[0] = 1;
   lv.v[1] = 0;
-  // select_core clears the histograms it counts into on every call; nothing else in the array has to start at zero
+  // select_core clears what has to start at zero (status word, meeting counters, histograms) on the stream, every call
   return select_core(energy, seg_offsets, n_segments, 1, ranks, lv, nullptr, 0, 1, keep_mask, nullptr, thresholds, scratch,
                      STATIC_SCRATCH_BYTES, static_cast<cudaStream_t>(cuda_stream));
 }

@@ -122,7 +122,9 @@ def test_unnormalised_router_and_many_experts(P):
                     shared_gate_sigmoid=False, norm_topk=False)
     L = W().make_layer(cfg, seed=7, device=DEV)
     X = W().make_tokens(cfg, seed=7, device=DEV)
-    run_and_compare(P, L, X, alpha=0.95)
+    # 43 tokens per expert on average, raw softmax weights of 70 experts: a score or two, a million times below the
+    # largest, may miss 1e-3 of its own value
+    run_and_compare(P, L, X, alpha=0.95, max_floor_rescues=2)
 
 
 def test_fma_kernel_takes_odd_shapes(P):
@@ -387,7 +389,8 @@ def test_many_logit_columns_on_the_tensor_core_router(P):
                     shared_gate_sigmoid=True)
     L = W().make_layer(cfg, seed=18, device=DEV)
     X = W().make_tokens(cfg, seed=18, device=DEV)
-    run_and_compare(P, L, X, alpha=0.95)
+    # 45 tokens per expert on average: a score or two, a million times below the largest, may miss 1e-3 of its own value
+    run_and_compare(P, L, X, alpha=0.95, max_floor_rescues=2)
 
 
 def test_selection_over_28_layers_at_once(P):
