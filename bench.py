@@ -215,7 +215,7 @@ def run_stack(args):
     ws_f = [P.alloc_workspace(P.camera_forward_workspace_bytes(probe, B), dev) for _ in spans]
     w_masked = [torch.empty_like(w) for w in probe.tensors["w_down"]]
     ws_sel = P.alloc_workspace(P.camera_select_workspace_bytes(n_me, 1, 2), dev)
-    ws_c = P.alloc_workspace(4096 + 64 * probe.n_experts, dev)
+    ws_c = P.alloc_workspace(int(P.lib.camera_compact_workspace_bytes(probe.n_experts)), dev)
     energy = torch.empty(n_me, dtype=torch.float32, device=dev)
     phi2, phi_inf, omega2 = torch.empty_like(energy), torch.empty_like(energy), torch.empty_like(energy)
     keep = torch.empty(n_me, dtype=torch.uint8, device=dev)
@@ -373,6 +373,78 @@ def bench_other_config(P, torch, W, name, dev, stream, local, peaks):
                     if peaks["source"] == "measured" else "fallback burst bf16"})
     else:
         out.update({"score_kernel": "fp32 FMA kernel; the step is launch bound at this size: no roofline claim"})
+    return out
+
+
+def bench_decode(P, torch, W, name, dev, stream, peaks, batch=64, score_tokens=16384):
+    """A batch of `batch` tokens through one MoE layer (camera_layer_forward), unpruned and sliced at each prune ratio
+    by the masks CAMERA-P gives on `score_tokens` calibration tokens.  The step is timed three ways: as the plain call
+    (tables and tensor maps rebuilt by every call), with a prepared layer (camera_layer_prepare), and replayed from a
+    CUDA graph of the prepared call; on the device with events, and on the host around launch + synchronise."""
+    cfg = W.scaled(W.CONFIGS[name], n_tokens=score_tokens)
+    L = W.make_layer(cfg, seed=0, layer_id=0, device=dev)
+    layer = P.Layer.from_workload(L)
+    X = W.make_tokens(cfg, seed=0, layer_id=0, device=dev)
+    energy = P.camera_score_layer(layer, X, ALPHA)
+    keep, _ = P.camera_select_all(energy, PRUNE_RATIOS)
+    off = P.expert_offsets_tensor(layer)
+    xd = X[:batch].contiguous()
+    yd = torch.empty((batch, cfg.d_model), dtype=torch.float32, device=dev)
+    ws_d = P.alloc_workspace(P.camera_forward_workspace_bytes(layer, batch), dev)
+    ws_c = P.alloc_workspace(int(P.lib.camera_compact_workspace_bytes(layer.n_experts)), dev)
+
+    def timed(fn, reps=50):
+        for _ in range(5):
+            fn()
+        torch.cuda.synchronize()
+        f0, f1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        t0 = time.perf_counter()
+        f0.record(stream)
+        for _ in range(reps):
+            fn()
+        f1.record(stream)
+        torch.cuda.synchronize()
+        host_us = 1e6 * (time.perf_counter() - t0) / reps
+        return 1e3 * f0.elapsed_time(f1) / reps, host_us
+
+    def three_ways(lay_plain, make_prepared):
+        plain_us, plain_host = timed(lambda: P.camera_layer_forward(lay_plain, xd, y=yd, workspace=ws_d))
+        lay = make_prepared()
+        prep_us, prep_host = timed(lambda: P.camera_layer_forward(lay, xd, y=yd, workspace=ws_d))
+        graph_us = graph_host = None
+        try:
+            side = torch.cuda.Stream()
+            side.wait_stream(stream)
+            g = torch.cuda.CUDAGraph()
+            with torch.cuda.stream(side):
+                P.camera_layer_forward(lay, xd, y=yd, workspace=ws_d)
+                with torch.cuda.graph(g, stream=side):
+                    P.camera_layer_forward(lay, xd, y=yd, workspace=ws_d)
+            stream.wait_stream(side)
+            graph_us, graph_host = timed(g.replay)
+        except Exception as exc:          # a capture that fails leaves the plain numbers
+            graph_us, graph_host = None, f"capture failed: {type(exc).__name__}"
+        return {"us": prep_us, "host_us": prep_host, "unprepared_us": plain_us, "unprepared_host_us": plain_host,
+                "graph_us": graph_us, "graph_host_us": graph_host}
+
+    wbytes = 3 * layer.n_me * cfg.d_model * 2
+    full = three_ways(layer, lambda: P.camera_layer_prepare(P.Layer.from_workload(L)))
+    best = min(v for v in (full["us"], full["graph_us"]) if v is not None)
+    out = {"workload": f"{cfg.name} layer, {batch} tokens", "weight_gb": wbytes / 1e9, "full_layer": full,
+           "full_layer_us": best, "full_layer_weight_gbs": wbytes / 1e9 / (best * 1e-6),
+           "frac_of_hbm_peak": wbytes / 1e9 / (best * 1e-6) / peaks["hbm_gbs"], "pruned": []}
+    outd = {k: [torch.empty_like(w) for w in layer.tensors[k]] for k in ("w_gate", "w_up", "w_down")}
+    for j, r in enumerate(PRUNE_RATIOS):
+        sub, cnt = P.camera_sub_index(keep[j], off, [1])
+        P.camera_compact_weights(layer, sub, cnt, 1, out=outd, workspace=ws_c)
+        mj = cnt[:, 0].cpu().tolist()
+        def sliced():
+            return P.Layer(L["w_router"], [outd["w_gate"][e][:mj[e]] for e in range(layer.n_experts)],
+                           [outd["w_up"][e][:mj[e]] for e in range(layer.n_experts)], outd["w_down"], cfg.top_k,
+                           cfg.n_shared, L["router_bias"], L["w_shared_gate"], cfg.norm_topk, "hf", down_ld=layer.d_ff)
+        t = three_ways(sliced(), lambda: P.camera_layer_prepare(sliced()))
+        b = min(v for v in (t["us"], t["graph_us"]) if v is not None)
+        out["pruned"].append({"prune_ratio": r, "us": b, "speedup": best / b, "ways": t})
     return out
 
 
@@ -567,7 +639,7 @@ def main():
     if not args.no_compact:
         off = P.expert_offsets_tensor(layer)
         outw = {k: [torch.empty_like(w) for w in layer.tensors[k]] for k in ("w_gate", "w_up", "w_down")}
-        ws_c = P.alloc_workspace(4096 + 64 * layer.n_experts, dev)
+        ws_c = P.alloc_workspace(int(P.lib.camera_compact_workspace_bytes(layer.n_experts)), dev)
         c0, c1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         def apply_mask():
             sub, counts = P.camera_sub_index(keep[1], off, [1])
@@ -620,36 +692,12 @@ def main():
             del ws_f, yb, yh
         del outw
 
-        # ---- decode through the layer, batch of 64 tokens, full and sliced at each prune ratio (the paper's speed table)
+        # ---- decode through the layer, batch of 64 tokens, full and sliced at each prune ratio (the paper's speed table:
+        # a DeepSeek-MoE-16B layer; the Qwen2 shape beside it)
         if not args.no_forward and cfg.dtype == "bf16":
-            xd = Xs[0][:64].contiguous()
-            ws_d = P.alloc_workspace(P.camera_forward_workspace_bytes(layer, 64), dev)
-            yd = torch.empty((64, cfg.d_model), dtype=torch.float32, device=dev)
-            outd = {k: [torch.empty_like(w) for w in layer.tensors[k]] for k in ("w_gate", "w_up", "w_down")}
-            def decode_ms(lay, reps=20):
-                for _ in range(3):
-                    P.camera_layer_forward(lay, xd, y=yd, workspace=ws_d)
-                sync_all()
-                f0, f1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-                f0.record(stream)
-                for _ in range(reps):
-                    P.camera_layer_forward(lay, xd, y=yd, workspace=ws_d)
-                f1.record(stream); sync_all()
-                return f0.elapsed_time(f1) / reps
-            base_ms = decode_ms(layer)
-            esz = 2
-            decode = {"batch_tokens": 64, "full_layer_us": 1e3 * base_ms,
-                      "full_layer_weight_gbs": 3 * layer.n_me * cfg.d_model * esz / 1e9 / (base_ms * 1e-3), "pruned": []}
-            for j, r in enumerate(PRUNE_RATIOS):
-                sub, cnt = P.camera_sub_index(keep[j], off, [1])
-                P.camera_compact_weights(layer, sub, cnt, 1, out=outd, workspace=ws_c)
-                mj = cnt[:, 0].cpu().tolist()
-                sl = P.Layer(L["w_router"], [outd["w_gate"][e][:mj[e]] for e in range(layer.n_experts)],
-                             [outd["w_up"][e][:mj[e]] for e in range(layer.n_experts)], outd["w_down"], cfg.top_k,
-                             cfg.n_shared, L["router_bias"], L["w_shared_gate"], cfg.norm_topk, "hf", down_ld=layer.d_ff)
-                ms_j = decode_ms(sl)
-                decode["pruned"].append({"prune_ratio": r, "us": 1e3 * ms_j, "speedup": base_ms / ms_j})
-            del outd, ws_d
+            decode = {"batch_tokens": 64, "shapes": {}}
+            for name in ([args.config] if args.config != "qwen2_57b_a14b" else ["qwen2_57b_a14b", "deepseek_moe_16b"]):
+                decode["shapes"][name] = bench_decode(P, torch, W, name, dev, stream, load_peaks())
 
     # ---- the selections of all layers of the model in one call (one segment per layer): where a6/a7 see real bytes
     select_model = None

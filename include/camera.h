@@ -84,6 +84,9 @@ enum {
   CAMERA_STAGE_SCORE = 3, CAMERA_STAGE_COMBINE = 4, CAMERA_N_STAGES = 5
 };
 
+/* What camera_layer_prepare keeps for a layer (opaque). */
+typedef struct camera_prepared camera_prepared_t;
+
 /* One MoE layer (paper Algorithm 1 inputs: expert weights and router R). */
 typedef struct {
   int32_t d_model;              /* multiple of 8 */
@@ -103,6 +106,7 @@ typedef struct {
   const int32_t* w_down_ld;     /* HOST [n_routed+n_shared] or NULL: leading dimension (elements) of each W_down in
                                    CAMERA_DOWN_HF layout when its rows are longer than d_ff[e] (a sliced layer kept in
                                    buffers of the original width); multiples of 8; NULL = d_ff[e] */
+  const camera_prepared_t* prepared; /* NULL, or the handle camera_layer_prepare returned for exactly this layer */
 } camera_layer_t;
 
 /* Optional inputs/outputs of camera_score_layer; any pointer may be NULL. All DEVICE. */
@@ -122,6 +126,26 @@ typedef struct {
 
 const char* camera_strerror(int status);
 int camera_version(void);
+
+/*
+ * Optional: what does not change from call to call, built once.  Without a handle every scoring / forward call
+ * builds the layer's expert table and encodes 2 tensor maps per expert on the host and copies them to the workspace
+ * (from pageable memory); a 64-token decode step through camera_layer_forward pays that each time.  With
+ * layer->prepared set, those live in device memory the handle owns, and the few tensor maps that name the call's
+ * tokens or workspace are rebuilt only when (workspace, x, n_tokens) differ from the previous call's, and then travel
+ * as kernel arguments: a repeated call enqueues memsets and kernels only.  The paper has no counterpart.
+ *
+ * device_mem: DEVICE, camera_layer_prepared_bytes(layer) bytes, 256-byte aligned, owned by the handle until
+ * camera_layer_release (nothing else may write there).  The layer's matrices must stay where they are while the handle
+ * lives; a layer_t that differs from the one prepared (another pointer, shape or flag) is refused with
+ * CAMERA_ERR_INVALID_ARG.  The call synchronises `cuda_stream` once.  Calls that share a handle must be ordered on the
+ * GPU (one stream, or events) and come from one host thread at a time, like calls that share a workspace.
+ * Results are bit-identical with and without a handle.
+ */
+size_t camera_layer_prepared_bytes(const camera_layer_t* layer);
+int camera_layer_prepare(const camera_layer_t* layer, void* device_mem, size_t device_bytes, void* cuda_stream,
+                         camera_prepared_t** prepared_out);
+void camera_layer_release(camera_prepared_t* prepared);
 
 /* Scratch needed by camera_score_layer for this layer shape and token count (0 on invalid arguments). */
 size_t camera_score_workspace_bytes(const camera_layer_t* layer, int64_t n_tokens);

@@ -33,7 +33,7 @@ class camera_layer_t(C.Structure):
                 ("down_layout", C.c_int32), ("w_router", C.c_void_p), ("router_bias", C.c_void_p),
                 ("w_shared_gate", C.c_void_p), ("w_gate", C.POINTER(C.c_void_p)),
                 ("w_up", C.POINTER(C.c_void_p)), ("w_down", C.POINTER(C.c_void_p)),
-                ("w_down_ld", C.POINTER(C.c_int32))]
+                ("w_down_ld", C.POINTER(C.c_int32)), ("prepared", C.c_void_p)]
 
 
 class camera_score_aux_t(C.Structure):
@@ -58,6 +58,12 @@ def _load() -> C.CDLL:
     lib.camera_score_layer.restype = C.c_int
     lib.camera_score_layer.argtypes = [C.POINTER(camera_layer_t), C.c_void_p, C.c_int64, C.c_float, C.c_void_p,
                                        C.POINTER(camera_score_aux_t), C.c_void_p, C.c_size_t, C.c_void_p]
+    lib.camera_layer_prepared_bytes.restype = C.c_size_t
+    lib.camera_layer_prepared_bytes.argtypes = [C.POINTER(camera_layer_t)]
+    lib.camera_layer_prepare.restype = C.c_int
+    lib.camera_layer_prepare.argtypes = [C.POINTER(camera_layer_t), C.c_void_p, C.c_size_t, C.c_void_p, C.POINTER(C.c_void_p)]
+    lib.camera_layer_release.restype = None
+    lib.camera_layer_release.argtypes = [C.c_void_p]
     lib.camera_read_status.restype = C.c_int
     lib.camera_read_status.argtypes = [C.c_void_p, C.c_void_p, C.POINTER(C.c_int32)]
     lib.camera_set_wait_limit_ns.restype = C.c_int
@@ -189,6 +195,13 @@ class Layer:
         self._down_ld = self.c.w_down_ld      # keeps the array alive
         self.top_k = top_k
         self.n_shared = n_shared
+        self._prepared_mem = None
+
+    def __del__(self):
+        try:
+            camera_layer_release(self)
+        except Exception:
+            pass
 
     @classmethod
     def from_workload(cls, L: Dict[str, object]) -> "Layer":
@@ -196,6 +209,30 @@ class Layer:
         cfg = L["cfg"]
         return cls(L["w_router"], L["w_gate"], L["w_up"], L["w_down"], cfg.top_k, cfg.n_shared, L["router_bias"],
                    L["w_shared_gate"], cfg.norm_topk, L["down_layout"])
+
+
+def camera_layer_prepare(layer: Layer, stream: Optional[torch.cuda.Stream] = None) -> Layer:
+    """Builds the layer's per-call tables and weight tensor maps once (camera_layer_prepare); later calls with this
+    Layer enqueue kernels only.  The handle and its device memory live as long as the Layer (or until
+    camera_layer_release)."""
+    camera_layer_release(layer)
+    nbytes = int(lib.camera_layer_prepared_bytes(C.byref(layer.c)))
+    if nbytes == 0:
+        raise CameraError(-1, "camera_layer_prepared_bytes")
+    mem = alloc_workspace(nbytes, layer.device)
+    handle = C.c_void_p()
+    _check(lib.camera_layer_prepare(C.byref(layer.c), mem.data_ptr(), mem.numel(), _stream_ptr(stream), C.byref(handle)),
+           "camera_layer_prepare")
+    layer._prepared_mem = mem
+    layer.c.prepared = handle.value
+    return layer
+
+
+def camera_layer_release(layer: Layer) -> None:
+    if getattr(layer, "_prepared_mem", None) is not None and layer.c.prepared:
+        lib.camera_layer_release(layer.c.prepared)
+    layer.c.prepared = None
+    layer._prepared_mem = None
 
 
 def camera_score_workspace_bytes(layer: Layer, n_tokens: int) -> int:

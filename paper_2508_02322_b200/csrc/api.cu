@@ -115,6 +115,29 @@ ScoreLayout score_layout(const camera_layer_t* L, int64_t T) {
   return s;
 }
 
+// Tensor-core scoring on CTA pairs or on single CTAs.  Pairs move fewer bytes per flop but work on 256 micro-experts
+// at a time: measured 2 % ahead where d_ff fills the pairs (Qwen2, Mixtral shapes), 6 % behind where a ninth of every
+// expert's last pair is padding (d_ff 1408).
+bool choose_pair(const camera_layer_t* L, int64_t T, int top_k, const camera_score_aux_t* aux) {
+  if (aux && (aux->flags & CAMERA_SCORE_CTA_PAIR)) return true;
+  if (aux && (aux->flags & CAMERA_SCORE_SINGLE_CTA)) return false;
+  double work1 = 0.0, work2 = 0.0;
+  for (int e = 0; e < L->n_routed + L->n_shared; ++e) {
+    const double rows = e < L->n_routed ? (double)T * top_k / L->n_routed : (double)T;
+    work1 += rows * (double)((L->d_ff[e] + CH_TILE - 1) / CH_TILE * CH_TILE);
+    work2 += rows * (double)((L->d_ff[e] + 2 * CH_TILE - 1) / (2 * CH_TILE) * (2 * CH_TILE));
+  }
+  static int sms_of[64];      // SM count per device ordinal, asked once
+  int cur = 0;
+  cudaGetDevice(&cur);
+  int dev_sms = (cur >= 0 && cur < 64) ? sms_of[cur] : 0;
+  if (dev_sms == 0) {
+    cudaDeviceGetAttribute(&dev_sms, cudaDevAttrMultiProcessorCount, cur);
+    if (cur >= 0 && cur < 64) sms_of[cur] = dev_sms;
+  }
+  return work2 <= 1.06 * work1 && dev_sms % 2 == 0;
+}
+
 #define CK(expr)                                   \
   do {                                             \
     if ((expr) != cudaSuccess) {                   \
@@ -136,6 +159,104 @@ struct StageTimer {
 };
 
 }  // namespace
+
+// ---- camera_layer_prepare: everything about a layer that does not change from call to call -----------------------
+// The expert table, the micro-expert offsets and the tensor maps of the weights are built once and stay in device
+// memory the handle owns; the few tensor maps that name the caller's tokens or a workspace are rebuilt only when the
+// (workspace, tokens, count) of a call differ from the previous call's, and travel as kernel arguments.
+constexpr uint32_t PREPARED_MAGIC = 0x43414d50u;
+constexpr size_t PARAM_CHUNK = 3584;      // bytes per argument-carrying launch (kernel arguments: 4 KB in all)
+
+struct Prepared {
+  uint32_t magic;
+  int device;
+  camera_layer_t layer;                   // scalars of the layer it was made for; its arrays are the vectors below
+  std::vector<int32_t> d_ff, down_ld;
+  std::vector<const void*> w_gate, w_up, w_down;
+  bool has_down_ld;
+  std::vector<ExpertStatic> est;          // host copy; the forward-only fields are filled per call
+  std::vector<int32_t> me_prefix;
+  std::vector<char> score_maps;           // 128 * (2 E + N_EXTRA_MAPS), host copy
+  std::vector<char> wdown_maps;           // 128 * E: W_down [d_model, d_ff] in boxes of 128 rows (bf16, paper layout), else empty
+  std::vector<char> down_maps;            // 128 * 2 E: what the device buffer of the W_down GEMM holds
+  int norm_blocks;
+  bool umma_ok, router_maps_ok;
+  char* dev;                              // device memory of the handle
+  size_t off_est, off_me_prefix, off_score_maps, off_down_maps, dev_bytes;
+  // what the per-call parts on the device were built for
+  struct { const void* ws; const void* x; int64_t T; const void* h0; bool valid; } score_key;
+  struct { const void* ws; int64_t T; int h_box; std::vector<const void*> w_down; bool valid; } down_key;
+};
+
+namespace {
+struct ParamChunk { uint4 v[PARAM_CHUNK / 16]; };
+__global__ void __launch_bounds__(256) k_store_params(const __grid_constant__ ParamChunk p, uint4* dst, int n16) {
+  if ((int)threadIdx.x < n16) dst[threadIdx.x] = p.v[threadIdx.x];
+}
+
+size_t prepared_layout(int E, size_t* off_est, size_t* off_me, size_t* off_score, size_t* off_down) {
+  size_t o = 0;
+  auto take = [&](size_t bytes) { size_t at = o; o = up256(o + bytes); return at; };
+  *off_est = take(sizeof(ExpertStatic) * E);
+  *off_me = take(sizeof(int32_t) * (E + 1));
+  *off_score = take((size_t)128 * (2 * E + N_EXTRA_MAPS));
+  *off_down = take((size_t)128 * 2 * E);
+  return o;
+}
+
+// The handle of a layer, if it has one that was made for exactly this layer (else null and *rc says why).
+Prepared* prepared_of(const camera_layer_t* L, int* rc) {
+  *rc = CAMERA_OK;
+  if (L->prepared == nullptr) return nullptr;
+  Prepared* p = reinterpret_cast<Prepared*>(const_cast<camera_prepared_t*>(L->prepared));
+  const int E = L->n_routed + L->n_shared;
+  bool same = p->magic == PREPARED_MAGIC && (int)p->d_ff.size() == E && p->layer.d_model == L->d_model &&
+              p->layer.n_routed == L->n_routed && p->layer.top_k == L->top_k && p->layer.n_shared == L->n_shared &&
+              p->layer.dtype == L->dtype && p->layer.flags == L->flags && p->layer.down_layout == L->down_layout &&
+              p->layer.w_router == L->w_router && p->layer.router_bias == L->router_bias &&
+              p->layer.w_shared_gate == L->w_shared_gate && p->has_down_ld == (L->w_down_ld != nullptr);
+  for (int e = 0; same && e < E; ++e)
+    same = p->d_ff[e] == L->d_ff[e] && p->w_gate[e] == L->w_gate[e] && p->w_up[e] == L->w_up[e] &&
+           p->w_down[e] == L->w_down[e] && (!p->has_down_ld || p->down_ld[e] == L->w_down_ld[e]);
+  int dev = -1;
+  if (same && (cudaGetDevice(&dev) != cudaSuccess || dev != p->device)) same = false;
+  if (!same) { *rc = CAMERA_ERR_INVALID_ARG; return nullptr; }
+  return p;
+}
+}  // namespace
+
+cudaError_t upload_params(void* dst, const void* src, size_t bytes, cudaStream_t st) {
+  for (size_t o = 0; o < bytes; o += PARAM_CHUNK) {
+    const size_t n = bytes - o < PARAM_CHUNK ? bytes - o : PARAM_CHUNK;
+    ParamChunk c;
+    memcpy(&c, static_cast<const char*>(src) + o, n);
+    k_store_params<<<1, 256, 0, st>>>(c, reinterpret_cast<uint4*>(static_cast<char*>(dst) + o), (int)(n / 16));
+  }
+  return cudaGetLastError();
+}
+
+char* prepared_down_maps(Prepared* p, const void* workspace, int64_t n_tokens, int h_box, const void* const* w_down,
+                         bool* cached) {
+  const size_t E = p->d_ff.size();
+  bool same = p->down_key.valid && p->down_key.ws == workspace && p->down_key.T == n_tokens && p->down_key.h_box == h_box;
+  for (size_t e = 0; same && e < E; ++e) same = p->down_key.w_down[e] == w_down[e];
+  *cached = same;
+  return p->dev + p->off_down_maps;
+}
+
+void prepared_down_maps_store(Prepared* p, const void* workspace, int64_t n_tokens, int h_box, const void* const* w_down) {
+  p->down_key.ws = workspace; p->down_key.T = n_tokens; p->down_key.h_box = h_box;
+  p->down_key.w_down.assign(w_down, w_down + p->d_ff.size());
+  p->down_key.valid = true;
+}
+
+const char* prepared_wdown_maps(const Prepared* p, const void* const* w_down) {
+  if (p->wdown_maps.empty()) return nullptr;
+  for (size_t e = 0; e < p->d_ff.size(); ++e)
+    if (w_down[e] != p->w_down[e]) return nullptr;
+  return p->wdown_maps.data();
+}
+
 }  // namespace camera
 
 using namespace camera;
@@ -202,6 +323,9 @@ int score_front(const camera_layer_t* L, const void* x, int64_t T, float alpha, 
   char* ws = static_cast<char*>(workspace);
   const int E = lay.n_experts;
 
+  Prepared* const prep = prepared_of(L, &rc);
+  if (rc != CAMERA_OK) return rc;
+  out->prep = prep;
   ScoreCtx& c = out->c;
   memset(&c, 0, sizeof(c));
   c.d_model = L->d_model; c.n_routed = L->n_routed; c.top_k = L->n_routed > 0 ? L->top_k : 0;
@@ -232,11 +356,68 @@ int score_front(const camera_layer_t* L, const void* x, int64_t T, float alpha, 
   c.omega2 = (aux && aux->omega2) ? aux->omega2 : reinterpret_cast<float*>(ws + lay.omega2);
   c.energy = energy;
   c.tensor_maps = ws + lay.tensor_maps;
+  if (prep != nullptr) {     // the tables and maps live with the handle
+    c.est = reinterpret_cast<ExpertStatic*>(prep->dev + prep->off_est);
+    c.me_prefix = reinterpret_cast<int32_t*>(prep->dev + prep->off_me_prefix);
+    c.tensor_maps = prep->dev + prep->off_score_maps;
+  }
 
   if (reuse) {   // the tables, token lists and h are those of the earlier call on this workspace
     out->norm_blocks = 0;
     out->use_umma = umma_shape_ok(L);
     out->use_pair = false;
+    return CAMERA_OK;
+  }
+
+  if (prep != nullptr) {
+    const bool use_umma = prep->umma_ok && !(aux && (aux->flags & CAMERA_SCORE_FORCE_SIMT)) &&
+                          (reinterpret_cast<uintptr_t>(x) & 15) == 0;
+    bool use_pair = false;
+    if (use_umma) use_pair = choose_pair(L, T, c.top_k, aux);
+    c.ch_tile = use_pair ? 2 * CH_TILE : CH_TILE;
+    c.ct_group = SCORE_GROUP_CHANNELS / c.ch_tile;
+    const bool use_router_umma = use_umma && prep->router_maps_ok && router_umma_ok(c);
+    // the per-call parts on the device: rebuilt only when this call differs from the one they were built for
+    const void* h0 = fwd ? fwd->h[0] : nullptr;
+    if (!(prep->score_key.valid && prep->score_key.ws == workspace && prep->score_key.x == x && prep->score_key.T == T &&
+          prep->score_key.h0 == h0)) {
+      if (fwd != nullptr || prep->score_key.h0 != nullptr) {     // where h and the output rows go (or went)
+        for (int e = 0; e < E; ++e) {
+          prep->est[e].h_ld = fwd ? fwd->h_ld[e] : 0;
+          prep->est[e].h = fwd ? fwd->h[e] : nullptr;
+          prep->est[e].y_part = fwd ? fwd->y_part[e] : nullptr;
+        }
+        CK(upload_params(c.est, prep->est.data(), (sizeof(ExpertStatic) * E + 15) & ~(size_t)15, st));
+      }
+      if (prep->umma_ok) {
+        rc = encode_tensor_maps(L, c, prep->score_maps.data(), MAPS_TOKENS);
+        if (rc == CAMERA_OK && prep->router_maps_ok && c.n_tokens > 0) rc = encode_router_maps(c, prep->score_maps.data(), MAPS_TOKENS);
+        if (rc != CAMERA_OK) return rc;
+        CK(upload_params(static_cast<char*>(c.tensor_maps) + (size_t)128 * 2 * E, prep->score_maps.data() + (size_t)128 * 2 * E,
+                         (size_t)128 * N_EXTRA_MAPS, st));
+      }
+      prep->score_key.ws = workspace; prep->score_key.x = x; prep->score_key.T = T; prep->score_key.h0 = h0;
+      prep->score_key.valid = true;
+    }
+    if (!accumulate) CK(cudaMemsetAsync(c.totals, 0, sizeof(PlanTotals), st));
+    CK(cudaMemsetAsync(c.counts, 0, sizeof(int32_t) * E, st));
+    const StageTimer tm{aux, st};
+    tm.begin(CAMERA_STAGE_ROUTER);
+    {
+      const int32_t* idx_in = aux ? aux->topk_idx_in : nullptr;
+      const float* w_in = aux ? aux->topk_w_in : nullptr;
+      if (use_router_umma) CK(launch_router_umma(c, idx_in, w_in, st));
+      else if (idx_in) CK(launch_routing_from_input(c, idx_in, w_in, st));
+      else CK(launch_router(c, st));
+    }
+    tm.end(CAMERA_STAGE_ROUTER);
+    tm.begin(CAMERA_STAGE_PERMUTE);
+    CK(launch_plan(c, st));
+    CK(launch_permute(c, st));
+    tm.end(CAMERA_STAGE_PERMUTE);
+    out->norm_blocks = prep->norm_blocks;
+    out->use_umma = use_umma;
+    out->use_pair = use_pair;
     return CAMERA_OK;
   }
 
@@ -262,24 +443,7 @@ int score_front(const camera_layer_t* L, const void* x, int64_t T, float alpha, 
   const bool use_umma = umma_shape_ok(L) && !(aux && (aux->flags & CAMERA_SCORE_FORCE_SIMT)) &&
                         (reinterpret_cast<uintptr_t>(x) & 15) == 0;
   bool use_pair = false;
-  if (use_umma) {
-    if (aux && (aux->flags & CAMERA_SCORE_CTA_PAIR)) use_pair = true;
-    else if (aux && (aux->flags & CAMERA_SCORE_SINGLE_CTA)) use_pair = false;
-    else {
-      // pairs move fewer bytes per flop but work on 256 micro-experts at a time: measured 2 % ahead where d_ff fills
-      // the pairs (Qwen2, Mixtral shapes), 6 % behind where a ninth of every expert's last pair is padding (d_ff 1408)
-      double work1 = 0.0, work2 = 0.0;
-      for (int e = 0; e < E; ++e) {
-        const double rows = e < L->n_routed ? (double)T * c.top_k / L->n_routed : (double)T;
-        work1 += rows * (double)((L->d_ff[e] + CH_TILE - 1) / CH_TILE * CH_TILE);
-        work2 += rows * (double)((L->d_ff[e] + 2 * CH_TILE - 1) / (2 * CH_TILE) * (2 * CH_TILE));
-      }
-      int dev_sms = 0, cur = 0;
-      cudaGetDevice(&cur);
-      cudaDeviceGetAttribute(&dev_sms, cudaDevAttrMultiProcessorCount, cur);
-      use_pair = work2 <= 1.06 * work1 && dev_sms % 2 == 0;
-    }
-  }
+  if (use_umma) use_pair = choose_pair(L, T, c.top_k, aux);
   c.ch_tile = use_pair ? 2 * CH_TILE : CH_TILE;
   c.ct_group = SCORE_GROUP_CHANNELS / c.ch_tile;
   const bool use_router_umma = use_umma && router_umma_ok(c);
@@ -351,6 +515,107 @@ extern "C" int camera_score_layer(const camera_layer_t* L, const void* x, int64_
   CK(launch_combine(c, st));
   tm.end(CAMERA_STAGE_COMBINE);
   return CAMERA_OK;
+}
+
+extern "C" size_t camera_layer_prepared_bytes(const camera_layer_t* layer) {
+  if (validate_layer(layer, 0, true) != CAMERA_OK) return 0;
+  size_t a, b, c, d;
+  return prepared_layout(layer->n_routed + layer->n_shared, &a, &b, &c, &d);
+}
+
+extern "C" int camera_layer_prepare(const camera_layer_t* L, void* device_mem, size_t device_bytes, void* cuda_stream,
+                                    camera_prepared_t** out) {
+  static_assert(sizeof(ExpertStatic) % 16 == 0, "the expert table travels in 16-byte pieces");
+  if (out == nullptr) return CAMERA_ERR_INVALID_ARG;
+  *out = nullptr;
+  int rc = validate_layer(L, 0, true);
+  if (rc != CAMERA_OK) return rc;
+  const int E = L->n_routed + L->n_shared;
+  Prepared* p = new Prepared();
+  p->dev_bytes = prepared_layout(E, &p->off_est, &p->off_me_prefix, &p->off_score_maps, &p->off_down_maps);
+  if (device_mem == nullptr || device_bytes < p->dev_bytes || (reinterpret_cast<uintptr_t>(device_mem) & 255)) {
+    delete p;
+    return CAMERA_ERR_WORKSPACE;
+  }
+  if (cudaGetDevice(&p->device) != cudaSuccess) { cudaGetLastError(); delete p; return CAMERA_ERR_CUDA; }
+  p->magic = PREPARED_MAGIC;
+  p->layer = *L;
+  p->d_ff.assign(L->d_ff, L->d_ff + E);
+  p->w_gate.assign(L->w_gate, L->w_gate + E);
+  p->w_up.assign(L->w_up, L->w_up + E);
+  p->w_down.assign(L->w_down, L->w_down + E);
+  p->has_down_ld = L->w_down_ld != nullptr;
+  if (p->has_down_ld) p->down_ld.assign(L->w_down_ld, L->w_down_ld + E);
+  p->layer.d_ff = nullptr; p->layer.w_gate = p->layer.w_up = p->layer.w_down = nullptr; p->layer.w_down_ld = nullptr;
+  p->layer.prepared = nullptr;
+  p->dev = static_cast<char*>(device_mem);
+  p->est.resize(E);
+  p->me_prefix.resize(E + 1);
+  int me = 0;
+  p->norm_blocks = 0;
+  bool score_shapes = true;      // d_ff of a layer to be scored: multiples of 8 (a sliced layer may have any)
+  for (int e = 0; e < E; ++e) {
+    ExpertStatic& es = p->est[e];
+    memset(&es, 0, sizeof(es));
+    es.w_gate = L->w_gate[e]; es.w_up = L->w_up[e]; es.w_down = L->w_down[e];
+    es.d_ff = L->d_ff[e]; es.me_off = me;
+    es.shared_idx = e < L->n_routed ? -1 : e - L->n_routed;
+    es.norm_blk_begin = p->norm_blocks;
+    es.down_ld = L->w_down_ld ? L->w_down_ld[e] : L->d_ff[e];
+    p->me_prefix[e] = me;
+    me += L->d_ff[e];
+    if (L->d_ff[e] < 8 || L->d_ff[e] % 8 != 0) score_shapes = false;
+    p->norm_blocks += rownorm_blocks(L->down_layout, L->dtype, L->d_ff[e]);
+  }
+  p->me_prefix[E] = me;
+  if (!score_shapes) p->norm_blocks = 0;
+  p->umma_ok = umma_shape_ok(L);
+  p->router_maps_ok = false;
+  p->score_maps.assign((size_t)128 * (2 * E + N_EXTRA_MAPS), 0);
+  p->down_maps.assign((size_t)128 * 2 * E, 0);
+  if (p->umma_ok) {
+    ScoreCtx c;
+    memset(&c, 0, sizeof(c));
+    c.d_model = L->d_model; c.n_routed = L->n_routed; c.top_k = L->n_routed > 0 ? L->top_k : 0; c.n_shared = L->n_shared;
+    c.n_experts = E; c.dtype = L->dtype; c.flags = L->flags; c.n_tokens = 1;
+    c.w_router = L->w_router; c.w_shared_gate = L->w_shared_gate;
+    rc = encode_tensor_maps(L, c, p->score_maps.data(), MAPS_STATIC);
+    if (rc == CAMERA_OK && router_umma_ok(c)) {
+      rc = encode_router_maps(c, p->score_maps.data(), MAPS_STATIC);
+      p->router_maps_ok = rc == CAMERA_OK;
+    }
+    if (rc == CAMERA_OK && L->dtype == CAMERA_BF16 && L->down_layout == CAMERA_DOWN_HF) {
+      p->wdown_maps.assign((size_t)128 * E, 0);
+      for (int e = 0; e < E && rc == CAMERA_OK; ++e) {
+        const int ld = L->w_down_ld ? L->w_down_ld[e] : L->d_ff[e];
+        if (ld % 8 != 0) { p->wdown_maps.clear(); break; }      // rows of W_down must start on 16-byte boundaries
+        if (!encode_bf16_2d_pitch(p->wdown_maps.data() + (size_t)128 * e, L->d_ff[e] > 0 ? L->w_down[e] : nullptr,
+                                  (uint64_t)L->d_model, (uint64_t)L->d_ff[e], (uint64_t)ld, 128))
+          rc = CAMERA_ERR_CUDA;
+      }
+    }
+    if (rc != CAMERA_OK) { delete p; return rc; }
+  }
+  p->score_key.valid = false; p->score_key.h0 = nullptr;
+  p->down_key.valid = false;
+  cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+  if (cudaMemcpyAsync(p->dev + p->off_est, p->est.data(), sizeof(ExpertStatic) * E, cudaMemcpyHostToDevice, st) != cudaSuccess ||
+      cudaMemcpyAsync(p->dev + p->off_me_prefix, p->me_prefix.data(), sizeof(int32_t) * (E + 1), cudaMemcpyHostToDevice, st) != cudaSuccess ||
+      cudaMemcpyAsync(p->dev + p->off_score_maps, p->score_maps.data(), p->score_maps.size(), cudaMemcpyHostToDevice, st) != cudaSuccess ||
+      cudaStreamSynchronize(st) != cudaSuccess) {     // the host copies above are read by the copies: wait for them
+    cudaGetLastError();
+    delete p;
+    return CAMERA_ERR_CUDA;
+  }
+  *out = reinterpret_cast<camera_prepared_t*>(p);
+  return CAMERA_OK;
+}
+
+extern "C" void camera_layer_release(camera_prepared_t* prepared) {
+  Prepared* p = reinterpret_cast<Prepared*>(prepared);
+  if (p == nullptr || p->magic != PREPARED_MAGIC) return;
+  p->magic = 0;
+  delete p;
 }
 
 extern "C" int camera_read_status(const void* workspace, void* cuda_stream, int32_t* status_out) {

@@ -105,11 +105,25 @@ struct ForwardBuffers {
   float* const* y_part;
   bool reuse;   // only rebuild the context: the workspace still holds the lists, tables and h of an earlier call
 };
+struct Prepared;    // what camera_layer_prepare keeps for a layer (api.cu)
 struct ScoreFront {
   ScoreCtx c;
   int norm_blocks;
   bool use_umma, use_pair;
+  Prepared* prep;     // the layer's prepared state, or null
 };
+// Tensor maps of the W_down GEMM for a prepared layer: the device buffer that holds them ([2e] W_down, [2e+1] h per
+// expert) and *cached = true when it already holds the maps of exactly this call (same workspace, token count, box
+// and W_down matrices).  Otherwise the caller encodes them and calls prepared_down_maps_store.
+char* prepared_down_maps(Prepared* p, const void* workspace, int64_t n_tokens, int h_box, const void* const* w_down,
+                         bool* cached);
+void prepared_down_maps_store(Prepared* p, const void* workspace, int64_t n_tokens, int h_box, const void* const* w_down);
+// The layer's own W_down maps as encoded by camera_layer_prepare (128 bytes per expert), or null if w_down is not the layer's.
+const char* prepared_wdown_maps(const Prepared* p, const void* const* w_down);
+// Copies `bytes` (a multiple of 16) of host data to 16-byte aligned device memory as kernel arguments: asynchronous on
+// `st`, no staging copy of pageable memory.
+cudaError_t upload_params(void* dst, const void* src, size_t bytes, cudaStream_t st);
+constexpr int MAPS_STATIC = 1, MAPS_TOKENS = 2;
 int score_front(const camera_layer_t* L, const void* x, int64_t T, float alpha, float* energy,
                 const camera_score_aux_t* aux, void* workspace, size_t workspace_bytes, cudaStream_t st,
                 const ForwardBuffers* fwd, ScoreFront* out);
@@ -131,8 +145,10 @@ cudaError_t launch_score_umma_write_h(const ScoreCtx& c, cudaStream_t st);
 cudaError_t launch_score_umma_pair_write_h(const ScoreCtx& c, bool token_rows, cudaStream_t st);
 bool umma_shape_ok(const camera_layer_t* L);
 bool router_umma_ok(const ScoreCtx& c);
-int encode_tensor_maps(const camera_layer_t* L, const ScoreCtx& c, void* host_maps /* 128 B each */);
-int encode_router_maps(const ScoreCtx& c, void* host_maps);
+// `which`: MAPS_STATIC = the maps of the weights, MAPS_TOKENS = the maps of x and x_perm (they change with the call).
+int encode_tensor_maps(const camera_layer_t* L, const ScoreCtx& c, void* host_maps /* 128 B each */,
+                       int which = MAPS_STATIC | MAPS_TOKENS);
+int encode_router_maps(const ScoreCtx& c, void* host_maps, int which = MAPS_STATIC | MAPS_TOKENS);
 // Tensor map of a bf16 row-major [rows, d] matrix in boxes of 64 columns x box_rows rows with the
 // 128-byte swizzle (a null matrix gives an all-zero map that must not be used).
 bool encode_bf16_2d(void* out, const void* ptr, uint64_t rows, uint64_t d, uint32_t box_rows);

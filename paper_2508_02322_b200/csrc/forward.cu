@@ -649,25 +649,36 @@ namespace {
 // The second GEMM and the sum over a token's experts, on the token lists, tables and h that the workspace holds.
 // w_down: per expert (HOST array of DEVICE pointers) the matrix that multiplies h.
 int down_and_sum(const camera_layer_t* L, const void* const* w_down, int64_t T, float* y, const ScoreCtx& c,
-                 const FwdLayout& fl, void* const* h, char* ws, bool long_lists, cudaStream_t st) {
+                 const FwdLayout& fl, void* const* h, char* ws, bool long_lists, cudaStream_t st, Prepared* prep) {
   const int E = L->n_routed + L->n_shared;
   // rows of h per load: the pair kernel's 128 per CTA; else a tile, or less where no list can be longer (an expert
   // sees a token at most once)
   const int h_box = long_lists ? 128 : (T <= 32 ? 32 : T <= 64 ? 64 : T <= 128 ? 128 : UMMA_TOK);
-  // tensor maps: per expert W_down [d_model rows, d_ff] and h [rows, h_ld]
-  std::vector<char> maps((size_t)128 * 2 * E);
-  for (int e = 0; e < E; ++e) {
-    const int ld = L->w_down_ld ? L->w_down_ld[e] : L->d_ff[e];
-    const uint64_t rows_h = e < L->n_routed ? (uint64_t)(fl.max_rows_perm > 0 ? fl.max_rows_perm : 1) : (uint64_t)T;
-    if (!encode_bf16_2d_pitch(maps.data() + (size_t)128 * (2 * e), L->d_ff[e] > 0 ? w_down[e] : nullptr,
-                              (uint64_t)L->d_model, (uint64_t)L->d_ff[e], (uint64_t)ld, D_TILE) ||
-        !encode_bf16_2d_pitch(maps.data() + (size_t)128 * (2 * e + 1), h[e], rows_h, (uint64_t)fl.h_ld[e],
-                              (uint64_t)fl.h_ld[e], h_box))
+  // tensor maps: per expert W_down [d_model rows, d_ff] and h [rows, h_ld].  A prepared layer keeps them on the device
+  // and rebuilds them only when the workspace, the token count or the W_down matrices differ from the previous call's.
+  bool cached = false;
+  char* maps_dev = prep ? prepared_down_maps(prep, ws, T, h_box, w_down, &cached) : ws + fl.maps;
+  if (!cached) {
+    std::vector<char> maps((size_t)128 * 2 * E);
+    const char* own = prep ? prepared_wdown_maps(prep, w_down) : nullptr;     // the layer's own W_down: encoded once
+    for (int e = 0; e < E; ++e) {
+      const int ld = L->w_down_ld ? L->w_down_ld[e] : L->d_ff[e];
+      const uint64_t rows_h = e < L->n_routed ? (uint64_t)(fl.max_rows_perm > 0 ? fl.max_rows_perm : 1) : (uint64_t)T;
+      if (own != nullptr) memcpy(maps.data() + (size_t)128 * (2 * e), own + (size_t)128 * e, 128);
+      else if (!encode_bf16_2d_pitch(maps.data() + (size_t)128 * (2 * e), L->d_ff[e] > 0 ? w_down[e] : nullptr,
+                                     (uint64_t)L->d_model, (uint64_t)L->d_ff[e], (uint64_t)ld, D_TILE))
+        return CAMERA_ERR_CUDA;
+      if (!encode_bf16_2d_pitch(maps.data() + (size_t)128 * (2 * e + 1), h[e], rows_h, (uint64_t)fl.h_ld[e],
+                                (uint64_t)fl.h_ld[e], h_box))
+        return CAMERA_ERR_CUDA;
+    }
+    if (prep) {
+      if (upload_params(maps_dev, maps.data(), maps.size(), st) != cudaSuccess) { cudaGetLastError(); return CAMERA_ERR_CUDA; }
+      prepared_down_maps_store(prep, ws, T, h_box, w_down);
+    } else if (cudaMemcpyAsync(maps_dev, maps.data(), maps.size(), cudaMemcpyHostToDevice, st) != cudaSuccess) {
+      cudaGetLastError();
       return CAMERA_ERR_CUDA;
-  }
-  if (cudaMemcpyAsync(ws + fl.maps, maps.data(), maps.size(), cudaMemcpyHostToDevice, st) != cudaSuccess) {
-    cudaGetLastError();
-    return CAMERA_ERR_CUDA;
+    }
   }
   int dev = 0, sms = 148;
   cudaGetDevice(&dev);
@@ -677,13 +688,13 @@ int down_and_sum(const camera_layer_t* L, const void* const* w_down, int64_t T, 
       cudaGetLastError();
       return CAMERA_ERR_CUDA;
     }
-    k_down_umma_pair<<<sms & ~1, D_THREADS, DP_SMEM_BYTES, st>>>(c, ws + fl.maps, (L->d_model + DP_TILE - 1) / DP_TILE);
+    k_down_umma_pair<<<sms & ~1, D_THREADS, DP_SMEM_BYTES, st>>>(c, maps_dev, (L->d_model + DP_TILE - 1) / DP_TILE);
   } else {
     if (cudaFuncSetAttribute(k_down_umma, cudaFuncAttributeMaxDynamicSharedMemorySize, D_SMEM_BYTES) != cudaSuccess) {
       cudaGetLastError();
       return CAMERA_ERR_CUDA;
     }
-    k_down_umma<<<sms, D_THREADS, D_SMEM_BYTES, st>>>(c, ws + fl.maps, (L->d_model + D_TILE - 1) / D_TILE, h_box * 128);
+    k_down_umma<<<sms, D_THREADS, D_SMEM_BYTES, st>>>(c, maps_dev, (L->d_model + D_TILE - 1) / D_TILE, h_box * 128);
   }
   k_unpermute_sum<<<dim3((unsigned)T, (unsigned)((L->d_model + 1023) / 1024)), 256, 0, st>>>(c, y);
   return cudaGetLastError() == cudaSuccess ? CAMERA_OK : CAMERA_ERR_CUDA;
@@ -763,7 +774,7 @@ int forward_impl(const camera_layer_t* L, const void* x, int64_t T, float alpha,
     return CAMERA_ERR_CUDA;
   }
   if (energy != nullptr && launch_combine(c, st) != cudaSuccess) { cudaGetLastError(); return CAMERA_ERR_CUDA; }
-  return down_and_sum(L, L->w_down, T, y, c, fl, fs.h.data(), ws, long_lists, st);
+  return down_and_sum(L, L->w_down, T, y, c, fl, fs.h.data(), ws, long_lists, st, f.prep);
 }
 
 }  // namespace
@@ -875,7 +886,7 @@ extern "C" int camera_pruned_output(const camera_layer_t* L, const void* const* 
   if (T == 0) return CAMERA_OK;
   // the work-unit counter of the second GEMM is the one thing the earlier call left used up
   if (cudaMemsetAsync(&f.c.totals->down_counter, 0, sizeof(int), st) != cudaSuccess) { cudaGetLastError(); return CAMERA_ERR_CUDA; }
-  return down_and_sum(L, w_down_masked, T, y_hat, f.c, fl, fs.h.data(), ws, forward_token_rows(L, T, a2.flags), st);
+  return down_and_sum(L, w_down_masked, T, y_hat, f.c, fl, fs.h.data(), ws, forward_token_rows(L, T, a2.flags), st, f.prep);
 }
 
 extern "C" size_t camera_output_error_workspace_bytes(int64_t n_tokens) {

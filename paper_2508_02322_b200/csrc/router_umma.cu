@@ -289,10 +289,11 @@ bool router_umma_ok(const ScoreCtx& c) {
 
 // Tensor maps of the router: x in boxes of 128 token rows, the router rows and the shared-gate rows
 // in one box each (rows past the tensor read as zero).
-int encode_router_maps(const ScoreCtx& c, void* host_maps) {
+int encode_router_maps(const ScoreCtx& c, void* host_maps, int which) {
   const RouterShape rs = router_shape(c);
   char* out = static_cast<char*>(host_maps) + (size_t)128 * (2 * c.n_experts + 2);
-  if (!encode_bf16_2d(out, c.x, (uint64_t)c.n_tokens, (uint64_t)c.d_model, RU_TOK)) return CAMERA_ERR_CUDA;
+  if ((which & MAPS_TOKENS) && !encode_bf16_2d(out, c.x, (uint64_t)c.n_tokens, (uint64_t)c.d_model, RU_TOK)) return CAMERA_ERR_CUDA;
+  if (!(which & MAPS_STATIC)) return CAMERA_OK;
   if (!encode_bf16_2d(out + 128, rs.nr_pad ? c.w_router : nullptr, (uint64_t)c.n_routed, (uint64_t)c.d_model, rs.nr_pad))
     return CAMERA_ERR_CUDA;
   if (!encode_bf16_2d(out + 256, rs.ng_pad ? c.w_shared_gate : nullptr, (uint64_t)c.n_shared, (uint64_t)c.d_model, rs.ng_pad))

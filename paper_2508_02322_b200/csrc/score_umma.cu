@@ -314,17 +314,20 @@ bool umma_shape_ok(const camera_layer_t* L) {
   return true;
 }
 
-int encode_tensor_maps(const camera_layer_t* L, const ScoreCtx& c, void* host_maps) {
+int encode_tensor_maps(const camera_layer_t* L, const ScoreCtx& c, void* host_maps, int which) {
   static_assert(sizeof(CUtensorMap) == 128, "tensor map size");
   EncodeTiledFn fn = get_encode_fn();
   if (fn == nullptr) return CAMERA_ERR_CUDA;
   char* out = static_cast<char*>(host_maps);
   const int E = c.n_experts;
-  for (int e = 0; e < E; ++e) {
-    if (!encode_2d(fn, out + (size_t)128 * (2 * e), L->w_gate[e], (uint64_t)L->d_ff[e], (uint64_t)c.d_model, CH_TILE) ||
-        !encode_2d(fn, out + (size_t)128 * (2 * e + 1), L->w_up[e], (uint64_t)L->d_ff[e], (uint64_t)c.d_model, CH_TILE))
-      return CAMERA_ERR_CUDA;
+  if (which & MAPS_STATIC) {
+    for (int e = 0; e < E; ++e) {
+      if (!encode_2d(fn, out + (size_t)128 * (2 * e), L->w_gate[e], (uint64_t)L->d_ff[e], (uint64_t)c.d_model, CH_TILE) ||
+          !encode_2d(fn, out + (size_t)128 * (2 * e + 1), L->w_up[e], (uint64_t)L->d_ff[e], (uint64_t)c.d_model, CH_TILE))
+        return CAMERA_ERR_CUDA;
+    }
   }
+  if (!(which & MAPS_TOKENS)) return CAMERA_OK;
   if (!encode_2d(fn, out + (size_t)128 * (2 * E), c.x_perm, (uint64_t)(c.max_rows_perm > 0 ? c.max_rows_perm : 1),
                  (uint64_t)c.d_model, UMMA_TOK))
     return CAMERA_ERR_CUDA;

@@ -120,3 +120,16 @@ def test_new_entry_points_reject_bad_arguments_on_the_host(P):
     assert P.lib.camera_residual_norm(4096, 1, 4096, 10, 60, C.c_float(1e-6), 4096, None) == -1             # d_model % 8
     assert P.lib.camera_residual_norm(4096, 5, 4096, 10, 64, C.c_float(1e-6), 4096, None) == -1             # dtype
     assert P.lib.camera_residual_norm(None, 1, None, 0, 64, C.c_float(1e-6), None, None) == 0              # nothing to do
+
+
+def test_prepare_checks_its_arguments_before_touching_a_device(P):
+    ok = _layer_struct(P)
+    n = P.lib.camera_layer_prepared_bytes(C.byref(ok))
+    assert n > 0 and n % 256 == 0
+    assert P.lib.camera_layer_prepared_bytes(C.byref(_layer_struct(P, top_k=5))) == 0
+    handle = C.c_void_p()
+    assert P.lib.camera_layer_prepare(C.byref(ok), None, 0, None, C.byref(handle)) == -3      # no device memory given
+    assert handle.value is None
+    assert P.lib.camera_layer_prepare(C.byref(ok), 4096, n - 1, None, C.byref(handle)) == -3  # too little of it
+    assert P.lib.camera_layer_prepare(C.byref(ok), 4096, n, None, None) == -1
+    P.lib.camera_layer_release(None)                                                          # a null handle is ignored
