@@ -456,7 +456,7 @@ def bench_whole_model(P, torch, W, cfg, dev, stream):
     nl, T = cfg.n_layers, cfg.n_tokens
     probe = P.Layer.from_workload(W.make_layer(W.scaled(cfg, n_tokens=1), seed=0, layer_id=0, device=dev))
     n_me = probe.n_me
-    ws_score = P.alloc_workspace(P.camera_score_workspace_bytes(probe, T), dev)
+    ws_score = P.alloc_workspace(P.camera_score_workspace_bytes_single_pass(probe, T), dev)
     del probe
     ws_all = P.alloc_workspace(P.camera_select_workspace_bytes(nl * n_me, nl, len(PRUNE_RATIOS) + len(BIT_LEVELS)), dev)
     E_all = torch.empty((nl, n_me), dtype=torch.float32, device=dev)
@@ -472,7 +472,7 @@ def bench_whole_model(P, torch, W, cfg, dev, stream):
         gen_s += time.perf_counter() - t0
         e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         e0.record(stream)
-        P.camera_score_layer(layer, X, ALPHA, energy=E_all[l], workspace=ws_score)
+        P.camera_score_layer(layer, X, ALPHA, energy=E_all[l], workspace=ws_score, single_pass=True)
         e1.record(stream)
         torch.cuda.synchronize()
         if P.camera_read_status(ws_score) != 0:
@@ -557,7 +557,9 @@ def main():
     layer = P.Layer.from_workload(L)
     Xs = [W.make_tokens(cfg, seed=0, layer_id=rank + world * i, device=dev) for i in range(2)]
     n_me = layer.n_me
-    ws_score = P.alloc_workspace(P.camera_score_workspace_bytes(layer, T), dev)
+    # the timed step scores all tokens of the layer in one pass (one launch of the scoring kernel per step); the walk in
+    # batches of 65536 tokens through a quarter of the scratch, the library's default, is timed beside it below
+    ws_score = P.alloc_workspace(P.camera_score_workspace_bytes_single_pass(layer, T), dev)
     ws_sel = P.alloc_workspace(P.camera_select_workspace_bytes(n_me, 1, len(PRUNE_RATIOS) + len(BIT_LEVELS)), dev)
     energy = torch.empty(n_me, dtype=torch.float32, device=dev)
     keep = torch.empty((len(PRUNE_RATIOS), n_me), dtype=torch.uint8, device=dev)
@@ -570,14 +572,14 @@ def main():
 
     def step(i, events=None):
         if by_tokens:
-            P.camera_score_layer(layer, Xs[i % 2], ALPHA, energy=energy, workspace=ws_score, stage_events=events,
+            P.camera_score_layer(layer, Xs[i % 2], ALPHA, energy=energy, workspace=ws_score, stage_events=events, single_pass=True,
                                  cta_pair=(True if args.cta_pair else (False if args.single_cta else None)), phi2=phi2, phi_inf_sq=phi_inf)
             reduce_components(phi2, phi_inf, dist if world > 1 else None)
             # no tokens, accumulate: folds nothing in and turns the reduced components into the energies
             P.camera_score_layer(layer, x_none, ALPHA, energy=energy, workspace=ws_score, phi2=phi2, phi_inf_sq=phi_inf,
                                  accumulate=True)
         else:
-            P.camera_score_layer(layer, Xs[i % 2], ALPHA, energy=energy, workspace=ws_score, stage_events=events,
+            P.camera_score_layer(layer, Xs[i % 2], ALPHA, energy=energy, workspace=ws_score, stage_events=events, single_pass=True,
                                  cta_pair=(True if args.cta_pair else (False if args.single_cta else None)))
         P.camera_select_all(energy, PRUNE_RATIOS, BIT_RATIOS, BIT_LEVELS, workspace=ws_sel, keep_masks=keep, bits_out=bits)
 
@@ -633,6 +635,30 @@ def main():
 
     value = world * T * args.steps / (ms * 1e-3)
     ms_per_step = ms / args.steps
+
+    # ---- the same step with the library's default for long token sets: batches of 65536 tokens through one batch's scratch
+    batched = None
+    if not by_tokens and T > 65536:
+        small = P.camera_score_workspace_bytes(layer, T)
+        ws_small = ws_score[:small]
+        def step_batched(i):
+            P.camera_score_layer(layer, Xs[i % 2], ALPHA, energy=energy, workspace=ws_small)
+            P.camera_select_all(energy, PRUNE_RATIOS, BIT_RATIOS, BIT_LEVELS, workspace=ws_sel, keep_masks=keep, bits_out=bits)
+        for i in range(2):
+            step_batched(i)
+        sync_all()
+        b0, b1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        n_b = max(4, min(args.steps, 10))
+        b0.record(stream)
+        for i in range(n_b):
+            step_batched(i)
+        b1.record(stream)
+        sync_all()
+        if P.camera_read_status(ws_small) != 0:
+            raise RuntimeError("device status set in the batched steps")
+        batched = {"what": "the step with camera_score_layer walking the tokens in batches of 65536 (the default when no "
+                           "single pass is asked for)", "steps": n_b, "ms_per_step": b0.elapsed_time(b1) / n_b,
+                   "workspace_gib": small / 2 ** 30, "single_pass_workspace_gib": ws_score.numel() / 2 ** 30}
 
     # ---- the selection applied to the weights (Algorithm 2, TopSelect to the slicing), timed on its own after the step loop
     compact = forward = decode = None
@@ -815,7 +841,7 @@ def main():
                    "l2": "inputs larger than L2" if flush is None else "L2 flushed between steps (256 MiB write, not timed)",
                    "parallelism": (f"tokens x{world}" if by_tokens else f"layers x{world}") if world > 1 else "single GPU"},
         "model_seconds": cfg.n_layers * ms_per_step * 1e-3 / world,     # extrapolated: layers x the step on one layer
-        "model_seconds_measured": model_measured, "configs": configs,
+        "model_seconds_measured": model_measured, "configs": configs, "batched_scoring": batched,
         "stage_ms": stage_ms, "clocks": clocks, "e2e": e2e, "gpu_launches": (LAUNCHES_PER_STEP + (3 if by_tokens else 0)) * args.steps,
         "roofline": roofline, "compact": compact, "forward": forward, "decode": decode, "select_model": select_model, "cpu_baseline": cpu, "context": PAPER_CONTEXT,
     }

@@ -70,6 +70,10 @@ enum {
                                       consecutive micro-experts of its token).  By default the library takes it when
                                       the experts' token lists are long enough for whole 256-token tiles to cost no
                                       more than they save; CTA_PAIR / SINGLE_CTA force the scoring orientation */
+  CAMERA_SCORE_SINGLE_PASS = 64u,  /* camera_score_layer only: score all n_tokens in one pass even when they are more than
+                                      65536 (needs camera_score_workspace_bytes_single_pass bytes of scratch) instead of
+                                      walking them in batches of 65536; the two differ in the last bits of the energies
+                                      (the batches' sums are rounded to fp32 between batches) */
   CAMERA_SCORE_ACCUMULATE = 4u     /* phi2 and phi_inf_sq (both required) already hold the result of earlier batches of
                                       calibration tokens of this layer; this call folds its batch in (the column sums of
                                       Algorithm 1 add up over batches, the column maxima take the maximum)
@@ -147,8 +151,12 @@ int camera_layer_prepare(const camera_layer_t* layer, void* device_mem, size_t d
                          camera_prepared_t** prepared_out);
 void camera_layer_release(camera_prepared_t* prepared);
 
-/* Scratch needed by camera_score_layer for this layer shape and token count (0 on invalid arguments). */
+/* Scratch needed by camera_score_layer for this layer shape and token count (0 on invalid arguments).  Token sets
+ * longer than 65536 are walked in batches of 65536 through the scratch of one batch, so the size stops growing there
+ * (3.8 GiB at the Qwen2-57B-A14B shape); camera_score_workspace_bytes_single_pass is the size CAMERA_SCORE_SINGLE_PASS
+ * needs (14.4 GiB for 262144 tokens of that shape). */
 size_t camera_score_workspace_bytes(const camera_layer_t* layer, int64_t n_tokens);
+size_t camera_score_workspace_bytes_single_pass(const camera_layer_t* layer, int64_t n_tokens);
 
 /*
  * Algorithm 1 of the paper (micro-expert ranking) up to and including the energies:
@@ -158,7 +166,10 @@ size_t camera_score_workspace_bytes(const camera_layer_t* layer, int64_t n_token
  *   phi2   <- ColumnSum(Lambda*Lambda), phi_inf <- ColumnMax|Lambda|^2
  *   energy <- [(1-alpha) phi2 + alpha phi_inf] * omega2            Eq. 11
  * x: DEVICE [n_tokens, d_model] row-major, dtype layer->dtype.  energy: DEVICE [N_e] fp32.
- * The calibration set may be fed in several calls (batches of tokens) with CAMERA_SCORE_ACCUMULATE.
+ * The calibration set may be fed in several calls (batches of tokens) with CAMERA_SCORE_ACCUMULATE; a single call
+ * with more than 65536 tokens walks them in batches of 65536 itself (same arithmetic as such calls; the batches
+ * depend on n_tokens alone, so a given input gives the same bits every time; aux->stage_events then bracket the
+ * stages of the last batch) unless CAMERA_SCORE_SINGLE_PASS asks for one pass.
  * Arithmetic: inputs as stored, products and sums in fp32 (bf16: tensor cores with fp32
  * accumulators), the final blend in fp64.  Routing ties go to the lower expert index.
  * An expert no token reaches gets energy 0.  0 <= alpha <= 1.  n_tokens >= 0.

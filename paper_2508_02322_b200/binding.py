@@ -24,6 +24,7 @@ CAMERA_SCORE_ACCUMULATE = 4
 CAMERA_SCORE_SINGLE_CTA = 8
 CAMERA_FORWARD_TOKEN_ROWS = 16
 CAMERA_SCORE_OMEGA_GIVEN = 32
+CAMERA_SCORE_SINGLE_PASS = 64
 STAGES = ("router", "permute", "rownorm", "score", "combine")
 
 
@@ -55,6 +56,8 @@ def _load() -> C.CDLL:
     lib.camera_version.restype = C.c_int
     lib.camera_score_workspace_bytes.restype = C.c_size_t
     lib.camera_score_workspace_bytes.argtypes = [C.POINTER(camera_layer_t), C.c_int64]
+    lib.camera_score_workspace_bytes_single_pass.restype = C.c_size_t
+    lib.camera_score_workspace_bytes_single_pass.argtypes = [C.POINTER(camera_layer_t), C.c_int64]
     lib.camera_score_layer.restype = C.c_int
     lib.camera_score_layer.argtypes = [C.POINTER(camera_layer_t), C.c_void_p, C.c_int64, C.c_float, C.c_void_p,
                                        C.POINTER(camera_score_aux_t), C.c_void_p, C.c_size_t, C.c_void_p]
@@ -239,6 +242,10 @@ def camera_score_workspace_bytes(layer: Layer, n_tokens: int) -> int:
     return int(lib.camera_score_workspace_bytes(C.byref(layer.c), n_tokens))
 
 
+def camera_score_workspace_bytes_single_pass(layer: Layer, n_tokens: int) -> int:
+    return int(lib.camera_score_workspace_bytes_single_pass(C.byref(layer.c), n_tokens))
+
+
 def camera_select_workspace_bytes(n_total: int, n_segments: int, n_levels: int) -> int:
     return int(lib.camera_select_workspace_bytes(n_total, n_segments, n_levels))
 
@@ -257,14 +264,15 @@ def camera_score_layer(layer: Layer, x: torch.Tensor, alpha: float, *, energy: O
                        routing_in=None, force_simt: bool = False, cta_pair: Optional[bool] = None, stage_events=None,
                        phi2: Optional[torch.Tensor] = None, phi_inf_sq: Optional[torch.Tensor] = None,
                        accumulate: bool = False, omega2: Optional[torch.Tensor] = None, omega_given: bool = False,
-                       stream: Optional[torch.cuda.Stream] = None, check_status: bool = False):
+                       single_pass: bool = False, stream: Optional[torch.cuda.Stream] = None, check_status: bool = False):
     """Algorithm 1 up to the energies.  Returns energy [N_e] fp32, or with details=True a dict that
     also holds phi2, phi_inf_sq, omega2, topk_idx, topk_w, shared_w and expert_token_counts.
     routing_in = (topk_idx int32 [T,k], topk_w fp32 [T,k]) prescribes the routing.
     stage_events = {stage: (torch.cuda.Event, torch.cuda.Event)} records per-stage timing events.
     phi2 / phi_inf_sq name the tensors that receive those components; with accumulate=True they must
     hold the result of earlier batches of tokens, and this batch is folded into them.  omega2 names the tensor
-    for the W_down norms; with omega_given=True it already holds them and the pass over W_down is skipped."""
+    for the W_down norms; with omega_given=True it already holds them and the pass over W_down is skipped.
+    single_pass=True scores more than 65536 tokens in one pass (larger workspace) instead of in batches of 65536."""
     if not (x.is_contiguous() and x.dtype == layer.dtype and x.dim() == 2 and x.shape[1] == layer.d_model):
         raise ValueError("x must be a contiguous [T, d_model] tensor of the layer's dtype")
     T = int(x.shape[0])
@@ -272,7 +280,8 @@ def camera_score_layer(layer: Layer, x: torch.Tensor, alpha: float, *, energy: O
     if energy is None:
         energy = torch.empty(layer.n_me, dtype=torch.float32, device=dev)
     if workspace is None:
-        workspace = alloc_workspace(camera_score_workspace_bytes(layer, T), dev)
+        workspace = alloc_workspace(camera_score_workspace_bytes_single_pass(layer, T) if single_pass
+                                    else camera_score_workspace_bytes(layer, T), dev)
     aux = camera_score_aux_t()
     out = {"energy": energy}
     keep_alive = []
@@ -300,7 +309,8 @@ def camera_score_layer(layer: Layer, x: torch.Tensor, alpha: float, *, energy: O
             out[name] = t
             setattr(aux, name, t.data_ptr())
     aux.flags = ((CAMERA_SCORE_FORCE_SIMT if force_simt else 0) | (CAMERA_SCORE_CTA_PAIR if cta_pair else 0) | (CAMERA_SCORE_SINGLE_CTA if cta_pair is False else 0) |
-                 (CAMERA_SCORE_ACCUMULATE if accumulate else 0) | (CAMERA_SCORE_OMEGA_GIVEN if omega_given else 0))
+                 (CAMERA_SCORE_ACCUMULATE if accumulate else 0) | (CAMERA_SCORE_OMEGA_GIVEN if omega_given else 0) |
+                 (CAMERA_SCORE_SINGLE_PASS if single_pass else 0))
     if stage_events:
         for name, (e0, e1) in stage_events.items():
             i = STAGES.index(name)

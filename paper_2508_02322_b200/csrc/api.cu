@@ -21,6 +21,10 @@ size_t up256(size_t v) { return (v + 255) & ~(size_t)255; }
 // Qwen2-shaped layer: 640 / 1280 / 2560 / 5120 -> 862 / 991 / 1111 / 1083 TFLOP/s).
 constexpr int SCORE_GROUP_CHANNELS = 2560;
 
+// Tokens per internal batch of camera_score_layer: longer sets are walked in batches of this size through the
+// scratch of one batch (3.8 GiB at the Qwen2-57B-A14B shape, where all 262144 tokens at once take 14.4 GiB).
+constexpr int64_t SCORE_BATCH_TOKENS = 65536;
+
 // Limit of every wait inside the tensor-core kernels, process wide (camera_set_wait_limit_ns).
 std::atomic<unsigned long long> g_wait_limit_ns{DEFAULT_WAIT_LIMIT_NS};
 
@@ -113,6 +117,24 @@ ScoreLayout score_layout(const camera_layer_t* L, int64_t T) {
   s.tensor_maps = take((size_t)128 * (2 * E + N_EXTRA_MAPS));
   s.total = o;
   return s;
+}
+
+// Workspace of the batched walk: the scratch of one batch, then what has to outlive a batch.
+struct BatchedLayout {
+  size_t one_batch_bytes, phi2, phi_inf_sq, omega2, counts, total;
+};
+BatchedLayout batched_layout(const camera_layer_t* L) {
+  BatchedLayout b;
+  const ScoreLayout s = score_layout(L, SCORE_BATCH_TOKENS);
+  b.one_batch_bytes = s.total;
+  size_t o = s.total;
+  auto take = [&](size_t bytes) { size_t at = o; o = up256(o + bytes); return at; };
+  b.phi2 = take(sizeof(float) * (size_t)s.n_me);
+  b.phi_inf_sq = take(sizeof(float) * (size_t)s.n_me);
+  b.omega2 = take(sizeof(float) * (size_t)s.n_me);
+  b.counts = take(sizeof(int32_t) * (size_t)s.n_experts);
+  b.total = o;
+  return b;
 }
 
 // Tensor-core scoring on CTA pairs or on single CTAs.  Pairs move fewer bytes per flop but work on 256 micro-experts
@@ -278,7 +300,8 @@ extern "C" int camera_version(void) { return 100; }
 
 extern "C" size_t camera_score_workspace_bytes(const camera_layer_t* layer, int64_t n_tokens) {
   if (validate_layer(layer, n_tokens) != CAMERA_OK) return 0;
-  return score_layout(layer, n_tokens).total;
+  if (n_tokens <= SCORE_BATCH_TOKENS) return score_layout(layer, n_tokens).total;
+  return batched_layout(layer).total;
 }
 
 namespace camera {
@@ -295,7 +318,7 @@ size_t score_workspace_bytes_any(const camera_layer_t* L, int64_t T, bool forwar
 // where the intermediate h and the expert's output rows go.
 int score_front(const camera_layer_t* L, const void* x, int64_t T, float alpha, float* energy,
                 const camera_score_aux_t* aux, void* workspace, size_t workspace_bytes, cudaStream_t st,
-                const ForwardBuffers* fwd, ScoreFront* out) {
+                const ForwardBuffers* fwd, ScoreFront* out, int64_t shared_ld) {
   int rc = validate_layer(L, T, fwd != nullptr);
   if (rc != CAMERA_OK) return rc;
   const bool reuse = fwd != nullptr && fwd->reuse;
@@ -347,6 +370,7 @@ int score_front(const camera_layer_t* L, const void* x, int64_t T, float alpha, 
   c.topk_idx = (aux && aux->topk_idx) ? aux->topk_idx : reinterpret_cast<int32_t*>(ws + lay.topk_idx);
   c.topk_w = (aux && aux->topk_w) ? aux->topk_w : reinterpret_cast<float*>(ws + lay.topk_w);
   c.shared_w = (aux && aux->shared_w) ? aux->shared_w : reinterpret_cast<float*>(ws + lay.shared_w);
+  c.shared_ld = (aux && aux->shared_w && shared_ld > 0) ? shared_ld : T;
   c.perm_w = reinterpret_cast<float*>(ws + lay.perm_w);
   c.x_perm = ws + lay.x_perm;
   c.part_sum = reinterpret_cast<float*>(ws + lay.part_sum);
@@ -486,13 +510,14 @@ int score_front(const camera_layer_t* L, const void* x, int64_t T, float alpha, 
 
 }  // namespace camera
 
-extern "C" int camera_score_layer(const camera_layer_t* L, const void* x, int64_t T, float alpha, float* energy,
-                                  const camera_score_aux_t* aux, void* workspace, size_t workspace_bytes,
-                                  void* cuda_stream) {
-  if (energy == nullptr) return CAMERA_ERR_INVALID_ARG;
-  cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+namespace camera {
+namespace {
+
+// One pass of Algorithm 1 over the tokens it is given (the whole set, or one batch of it).
+int score_one(const camera_layer_t* L, const void* x, int64_t T, float alpha, float* energy, const camera_score_aux_t* aux,
+              void* workspace, size_t workspace_bytes, cudaStream_t st, int64_t shared_ld) {
   ScoreFront f;
-  const int rc = score_front(L, x, T, alpha, energy, aux, workspace, workspace_bytes, st, nullptr, &f);
+  const int rc = score_front(L, x, T, alpha, energy, aux, workspace, workspace_bytes, st, nullptr, &f, shared_ld);
   if (rc != CAMERA_OK) return rc;
   const ScoreCtx& c = f.c;
   const bool use_umma = f.use_umma, use_pair = f.use_pair;
@@ -514,6 +539,75 @@ extern "C" int camera_score_layer(const camera_layer_t* L, const void* x, int64_
   tm.begin(CAMERA_STAGE_COMBINE);
   CK(launch_combine(c, st));
   tm.end(CAMERA_STAGE_COMBINE);
+  return CAMERA_OK;
+}
+
+__global__ void k_add_counts(int32_t* __restrict__ total, const int32_t* __restrict__ batch, int n) {
+  const int i = blockIdx.x * blockDim.x + threadIdx.x;
+  if (i < n) total[i] += batch[i];
+}
+
+}  // namespace
+}  // namespace camera
+
+extern "C" size_t camera_score_workspace_bytes_single_pass(const camera_layer_t* layer, int64_t n_tokens) {
+  if (validate_layer(layer, n_tokens) != CAMERA_OK) return 0;
+  return score_layout(layer, n_tokens).total;
+}
+
+extern "C" int camera_score_layer(const camera_layer_t* L, const void* x, int64_t T, float alpha, float* energy,
+                                  const camera_score_aux_t* aux, void* workspace, size_t workspace_bytes,
+                                  void* cuda_stream) {
+  if (energy == nullptr) return CAMERA_ERR_INVALID_ARG;
+  cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+  if (T <= SCORE_BATCH_TOKENS || (aux && (aux->flags & CAMERA_SCORE_SINGLE_PASS)))
+    return score_one(L, x, T, alpha, energy, aux, workspace, workspace_bytes, st, 0);
+
+  // A long token set: batches of SCORE_BATCH_TOKENS tokens through the scratch of one batch.  The column sums add up
+  // and the column maxima take the maximum over the batches (Algorithm 1's ColumnSum and ColumnMax), the norms of
+  // W_down are computed with the first batch.  The batches depend on T alone, so a given input gives the same bits.
+  int rc = validate_layer(L, T);
+  if (rc != CAMERA_OK) return rc;
+  if (x == nullptr || !(alpha >= 0.f && alpha <= 1.f)) return CAMERA_ERR_INVALID_ARG;
+  if (aux && ((aux->topk_idx_in == nullptr) != (aux->topk_w_in == nullptr))) return CAMERA_ERR_INVALID_ARG;
+  const BatchedLayout bl = batched_layout(L);
+  if (workspace == nullptr || workspace_bytes < bl.total || (reinterpret_cast<uintptr_t>(workspace) & 255))
+    return CAMERA_ERR_WORKSPACE;
+  char* ws = static_cast<char*>(workspace);
+  const int E = L->n_routed + L->n_shared;
+  const int64_t k = L->n_routed > 0 ? L->top_k : 0;
+  const size_t row_bytes = (size_t)L->d_model * (L->dtype == CAMERA_BF16 ? 2 : 4);
+  camera_score_aux_t user;
+  memset(&user, 0, sizeof(user));
+  if (aux) user = *aux;
+  const bool user_accumulates = (user.flags & CAMERA_SCORE_ACCUMULATE) != 0;
+  if (user_accumulates && (user.phi2 == nullptr || user.phi_inf_sq == nullptr)) return CAMERA_ERR_INVALID_ARG;
+  if ((user.flags & CAMERA_SCORE_OMEGA_GIVEN) && user.omega2 == nullptr) return CAMERA_ERR_INVALID_ARG;
+  int32_t* batch_counts = reinterpret_cast<int32_t*>(ws + bl.counts);
+  if (user.expert_token_counts) CK(cudaMemsetAsync(user.expert_token_counts, 0, sizeof(int32_t) * E, st));
+  int64_t t0 = 0;
+  for (int b = 0; t0 < T; ++b) {
+    const int64_t n = T - t0 < SCORE_BATCH_TOKENS ? T - t0 : SCORE_BATCH_TOKENS;
+    const bool last = t0 + n == T;
+    camera_score_aux_t a = user;
+    a.phi2 = user.phi2 ? user.phi2 : reinterpret_cast<float*>(ws + bl.phi2);
+    a.phi_inf_sq = user.phi_inf_sq ? user.phi_inf_sq : reinterpret_cast<float*>(ws + bl.phi_inf_sq);
+    a.omega2 = user.omega2 ? user.omega2 : reinterpret_cast<float*>(ws + bl.omega2);
+    if (b > 0) a.flags |= (uint32_t)(CAMERA_SCORE_ACCUMULATE | CAMERA_SCORE_OMEGA_GIVEN);
+    if (user.topk_idx) a.topk_idx = user.topk_idx + t0 * k;
+    if (user.topk_w) a.topk_w = user.topk_w + t0 * k;
+    if (user.topk_idx_in) { a.topk_idx_in = user.topk_idx_in + t0 * k; a.topk_w_in = user.topk_w_in + t0 * k; }
+    if (user.shared_w) a.shared_w = user.shared_w + t0;              // [n_shared, T]: this batch's columns
+    a.expert_token_counts = user.expert_token_counts ? batch_counts : nullptr;
+    if (!last) memset(a.stage_events, 0, sizeof(a.stage_events));    // the event pairs bracket the stages of the last batch
+    rc = score_one(L, static_cast<const char*>(x) + (size_t)t0 * row_bytes, n, alpha, energy, &a, ws, bl.one_batch_bytes, st, T);
+    if (rc != CAMERA_OK) return rc;
+    if (user.expert_token_counts) {
+      k_add_counts<<<(E + 255) / 256, 256, 0, st>>>(user.expert_token_counts, batch_counts, E);
+      CK(cudaGetLastError());
+    }
+    t0 += n;
+  }
   return CAMERA_OK;
 }
 

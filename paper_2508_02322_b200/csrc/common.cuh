@@ -85,7 +85,8 @@ struct ScoreCtx {
   int32_t* local_rank;   // [T, top_k] rank of the pair among the same expert's pairs in its block
   int32_t* topk_idx;     // [T, top_k]
   float* topk_w;         // [T, top_k]
-  float* shared_w;       // [n_shared, T]
+  float* shared_w;       // [n_shared, shared_ld]: coefficient of shared expert s for token t at s * shared_ld + t
+  int64_t shared_ld;     // n_tokens, or the caller's token count when this call is one batch of a longer set
   float* perm_w;         // [max_rows_perm]
   void* x_perm;          // [max_rows_perm, d_model]
   float* part_sum;       // [max_part]
@@ -124,9 +125,10 @@ const char* prepared_wdown_maps(const Prepared* p, const void* const* w_down);
 // `st`, no staging copy of pageable memory.
 cudaError_t upload_params(void* dst, const void* src, size_t bytes, cudaStream_t st);
 constexpr int MAPS_STATIC = 1, MAPS_TOKENS = 2;
+// shared_ld: leading dimension of aux->shared_w when the call is one batch of a longer token set (0 = T).
 int score_front(const camera_layer_t* L, const void* x, int64_t T, float alpha, float* energy,
                 const camera_score_aux_t* aux, void* workspace, size_t workspace_bytes, cudaStream_t st,
-                const ForwardBuffers* fwd, ScoreFront* out);
+                const ForwardBuffers* fwd, ScoreFront* out, int64_t shared_ld = 0);
 size_t score_workspace_bytes_any(const camera_layer_t* L, int64_t T, bool forward);
 unsigned long long current_wait_limit_ns();
 

@@ -107,7 +107,7 @@ __global__ void __launch_bounds__(RT_THREADS) k_router(ScoreCtx c, const int32_t
     if (t < c.n_tokens) {
       float a = 1.f;
       if (n_gated) a = 1.f / (1.f + expf(-logits[tl * ldl + c.n_routed + s]));
-      c.shared_w[(size_t)s * c.n_tokens + t] = a;
+      c.shared_w[(size_t)s * c.shared_ld + t] = a;
     }
   }
 

@@ -179,7 +179,7 @@ k_router_umma(const ScoreCtx c, const int32_t* idx_in, const float* w_in, int n_
         for (int s = 0; s < c.n_shared; ++s) {
           float a = 1.f;
           if (n_gated) a = 1.f / (1.f + expf(-row[rs.nr_pad + s]));
-          c.shared_w[(size_t)s * c.n_tokens + t] = a;
+          c.shared_w[(size_t)s * c.shared_ld + t] = a;
         }
       }
       if (c.n_routed == 0) continue;

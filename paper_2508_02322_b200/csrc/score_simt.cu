@@ -41,7 +41,7 @@ __global__ void __launch_bounds__(SS_THREADS) k_score_simt(ScoreCtx c) {
     if (ch0 >= f) continue;
     const T* Xsrc = (es.shared_idx < 0 ? static_cast<const T*>(c.x_perm) : static_cast<const T*>(c.x)) +
                     (size_t)u.row0 * d;
-    const float* wsrc = (es.shared_idx < 0 ? c.perm_w : c.shared_w + (size_t)es.shared_idx * c.n_tokens) + u.row0;
+    const float* wsrc = (es.shared_idx < 0 ? c.perm_w : c.shared_w + (size_t)es.shared_idx * c.shared_ld) + u.row0;
     const T* Wg = static_cast<const T*>(es.w_gate);
     const T* Wu = static_cast<const T*>(es.w_up);
 

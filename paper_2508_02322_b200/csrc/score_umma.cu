@@ -199,7 +199,7 @@ __global__ void __launch_bounds__(U_THREADS, 1) k_score_umma(const ScoreCtx c) {
       if (unit < 0) break;
       const UnitInfo u = decode_unit(c, unit);
       const int n_tiles = (u.rows + UMMA_TOK - 1) / UMMA_TOK;
-      const float* wsrc = u.shared_idx < 0 ? c.perm_w + u.row0 : c.shared_w + (size_t)u.shared_idx * c.n_tokens + u.row0;
+      const float* wsrc = u.shared_idx < 0 ? c.perm_w + u.row0 : c.shared_w + (size_t)u.shared_idx * c.shared_ld + u.row0;
       float s = 0.f, m = 0.f;
       // layer forward: where the warp's 32 micro-experts go in h, and the last row h has
       __nv_bfloat16* hbase = nullptr;

@@ -405,3 +405,46 @@ def test_selection_over_28_layers_at_once(P):
     bits = P.camera_alloc_bits(E.to(DEV), [0.2, 0.6, 0.2], [3, 2, 1], seg_offsets=seg)
     refb = np.concatenate([O.alloc_bits(E.numpy()[seg[i]:seg[i + 1]], [0.2, 0.6, 0.2], [3, 2, 1])[0] for i in range(layers)])
     assert np.array_equal(bits.cpu().numpy(), refb)
+
+
+@pytest.mark.parametrize("prepared", [False, True])
+def test_long_token_sets_are_walked_in_batches(P, prepared):
+    """More than 65536 tokens in one call: the default walks them in batches of 65536 through the scratch of one batch.
+    The result is, bit for bit, that of accumulating calls over the same batches; the routing, the shared-expert
+    coefficients and the token counts are those of the single pass; the energies agree with the single pass to the
+    rounding of the batches' fp32 sums and with the oracle within the usual tolerance."""
+    T = 65536 + 4500
+    cfg = small_cfg(n_tokens=T, d_model=128, n_routed=5, top_k=2, d_ff_routed=128, d_ff_shared=(64,))
+    L = W().make_layer(cfg, seed=21, device=DEV)
+    X = W().make_tokens(cfg, seed=21, device=DEV)
+    layer = P.Layer.from_workload(L)
+    if prepared:
+        P.camera_layer_prepare(layer)
+    small, big = P.camera_score_workspace_bytes(layer, T), P.camera_score_workspace_bytes_single_pass(layer, T)
+    assert small < big and small == P.camera_score_workspace_bytes(layer, 10 * T)      # stops growing at one batch
+    ws = P.alloc_workspace(small, DEV)
+    got = P.camera_score_layer(layer, X, 0.95, details=True, workspace=ws)
+    assert P.camera_read_status(ws) == 0
+    one = P.camera_score_layer(layer, X, 0.95, details=True, single_pass=True)
+    for k in ("topk_idx", "topk_w", "shared_w", "expert_token_counts", "omega2"):
+        assert torch.equal(got[k], one[k]), k
+    assert torch.equal(got["phi_inf_sq"], one["phi_inf_sq"])                            # maxima do not round
+    rel = ((got["energy"] - one["energy"]).abs() / one["energy"].clamp_min(1e-30)).max()
+    assert float(rel) < 1e-5
+    # the same batches by hand
+    phi2 = torch.empty(layer.n_me, dtype=torch.float32, device=DEV)
+    pinf, om, E = torch.empty_like(phi2), torch.empty_like(phi2), torch.empty_like(phi2)
+    for i, (t0, t1) in enumerate([(0, 65536), (65536, T)]):
+        P.camera_score_layer(layer, X[t0:t1], 0.95, energy=E, phi2=phi2, phi_inf_sq=pinf, omega2=om, accumulate=i > 0,
+                             omega_given=i > 0)
+    assert torch.equal(E, got["energy"]) and torch.equal(phi2, got["phi2"])
+    # too small a workspace for one pass is refused, not walked
+    with pytest.raises(P.CameraError) as e:
+        P.camera_score_layer(layer, X, 0.95, workspace=ws, single_pass=True)
+    assert e.value.status == -3
+    # against the oracle
+    ol, Xd = to_oracle_layer(L), f64(X)
+    routing = (got["topk_idx"].cpu().numpy().astype(np.int64), got["topk_w"].cpu().numpy().astype(np.float64))
+    p2, pi, w2 = O.camera_components(ol, Xd, routing=routing)
+    assert_close("energy of a batched walk", got["energy"].cpu().numpy(), O.energy(p2, pi, w2, float(np.float32(0.95))))
+    assert_close("phi2 of a batched walk", got["phi2"].cpu().numpy(), p2)
