@@ -30,7 +30,7 @@ std::atomic<unsigned long long> g_wait_limit_ns{DEFAULT_WAIT_LIMIT_NS};
 
 struct ScoreLayout {
   size_t totals, est, edyn, me_prefix, unit_prefix, counts, block_hist, local_rank, topk_idx, topk_w, shared_w,
-      perm_w, x_perm, part_sum, part_max, phi2, phi_inf_sq, omega2, tensor_maps, total;
+      perm_w, x_perm, part_sum, part_max, phi2, phi_inf_sq, omega2, tensor_maps, router_part, total;
   int n_experts, n_me, n_blocks, chunk_tokens, max_rows_perm;
   long long max_part;
 };
@@ -115,6 +115,7 @@ ScoreLayout score_layout(const camera_layer_t* L, int64_t T) {
   s.phi_inf_sq = take(sizeof(float) * (size_t)n_me);
   s.omega2 = take(sizeof(float) * (size_t)n_me);
   s.tensor_maps = take((size_t)128 * (2 * E + N_EXTRA_MAPS));
+  s.router_part = take(front_small_scratch_bytes(L->d_model, T));
   s.total = o;
   return s;
 }
@@ -401,6 +402,7 @@ int score_front(const camera_layer_t* L, const void* x, int64_t T, float alpha, 
     c.ch_tile = use_pair ? 2 * CH_TILE : CH_TILE;
     c.ct_group = SCORE_GROUP_CHANNELS / c.ch_tile;
     const bool use_router_umma = use_umma && prep->router_maps_ok && router_umma_ok(c);
+    const bool small = front_small_ok(c);        // a decode-sized batch: the front end made for it
     // the per-call parts on the device: rebuilt only when this call differs from the one they were built for
     const void* h0 = fwd ? fwd->h[0] : nullptr;
     if (!(prep->score_key.valid && prep->score_key.ws == workspace && prep->score_key.x == x && prep->score_key.T == T &&
@@ -430,14 +432,18 @@ int score_front(const camera_layer_t* L, const void* x, int64_t T, float alpha, 
     {
       const int32_t* idx_in = aux ? aux->topk_idx_in : nullptr;
       const float* w_in = aux ? aux->topk_w_in : nullptr;
-      if (use_router_umma) CK(launch_router_umma(c, idx_in, w_in, st));
+      if (small) CK(launch_route_small(c, idx_in, w_in, reinterpret_cast<float*>(ws + lay.router_part), st));
+      else if (use_router_umma) CK(launch_router_umma(c, idx_in, w_in, st));
       else if (idx_in) CK(launch_routing_from_input(c, idx_in, w_in, st));
       else CK(launch_router(c, st));
     }
     tm.end(CAMERA_STAGE_ROUTER);
     tm.begin(CAMERA_STAGE_PERMUTE);
-    CK(launch_plan(c, st));
-    CK(launch_permute(c, st));
+    if (small) CK(launch_permute_small(c, st));
+    else {
+      CK(launch_plan(c, st));
+      CK(launch_permute(c, st));
+    }
     tm.end(CAMERA_STAGE_PERMUTE);
     out->norm_blocks = prep->norm_blocks;
     out->use_umma = use_umma;
@@ -471,6 +477,7 @@ int score_front(const camera_layer_t* L, const void* x, int64_t T, float alpha, 
   c.ch_tile = use_pair ? 2 * CH_TILE : CH_TILE;
   c.ct_group = SCORE_GROUP_CHANNELS / c.ch_tile;
   const bool use_router_umma = use_umma && router_umma_ok(c);
+  const bool small = front_small_ok(c);        // a decode-sized batch: the front end made for it
   std::vector<char> maps;
   if (use_umma) {
     maps.resize((size_t)128 * (2 * E + N_EXTRA_MAPS));
@@ -492,15 +499,19 @@ int score_front(const camera_layer_t* L, const void* x, int64_t T, float alpha, 
   {
     const int32_t* idx_in = aux ? aux->topk_idx_in : nullptr;
     const float* w_in = aux ? aux->topk_w_in : nullptr;
-    if (use_router_umma) CK(launch_router_umma(c, idx_in, w_in, st));
+    if (small) CK(launch_route_small(c, idx_in, w_in, reinterpret_cast<float*>(ws + lay.router_part), st));
+    else if (use_router_umma) CK(launch_router_umma(c, idx_in, w_in, st));
     else if (idx_in) CK(launch_routing_from_input(c, idx_in, w_in, st));
     else CK(launch_router(c, st));
   }
   tm.end(CAMERA_STAGE_ROUTER);
 
   tm.begin(CAMERA_STAGE_PERMUTE);
-  CK(launch_plan(c, st));
-  CK(launch_permute(c, st));
+  if (small) CK(launch_permute_small(c, st));
+  else {
+    CK(launch_plan(c, st));
+    CK(launch_permute(c, st));
+  }
   tm.end(CAMERA_STAGE_PERMUTE);
   out->norm_blocks = norm_blocks;
   out->use_umma = use_umma;

@@ -136,6 +136,12 @@ unsigned long long current_wait_limit_ns();
 cudaError_t launch_router(const ScoreCtx& c, cudaStream_t st);
 cudaError_t launch_routing_from_input(const ScoreCtx& c, const int32_t* idx_in, const float* w_in, cudaStream_t st);
 cudaError_t launch_plan(const ScoreCtx& c, cudaStream_t st);
+// Small batches (at most 128 tokens and 128 logit columns): router + counting sort + plan in two launches that spread
+// the logit sums over the GPU, and the permutation with a CTA per token.  scratch: front_small_scratch_bytes.
+bool front_small_ok(const ScoreCtx& c);
+size_t front_small_scratch_bytes(int d_model, int64_t n_tokens);
+cudaError_t launch_route_small(const ScoreCtx& c, const int32_t* idx_in, const float* w_in, float* scratch, cudaStream_t st);
+cudaError_t launch_permute_small(const ScoreCtx& c, cudaStream_t st);
 cudaError_t launch_permute(const ScoreCtx& c, cudaStream_t st);
 cudaError_t launch_rownorm(const ScoreCtx& c, int n_norm_blocks, cudaStream_t st);
 cudaError_t launch_score_simt(const ScoreCtx& c, cudaStream_t st);

@@ -317,3 +317,40 @@ def test_residual_norm(P, dtype):
     tol = 2.0 ** -8 if dtype == torch.bfloat16 else 1e-6       # one rounding to the output dtype
     assert np.abs(f64(out) - ref).max() <= tol * np.abs(ref).max()
     assert out.dtype == dtype
+
+
+@pytest.mark.parametrize("shape", ["gated_shared", "many_small_experts"])
+def test_decode_batch_full_and_sliced_layers(P, shape):
+    """A decode step: 64 tokens through the full layer and through the layer sliced at 40 % by CAMERA-P masks taken
+    on calibration tokens, each against the oracle (Eq. 1-2 on the full and on the sliced weights), with and without a
+    prepared layer."""
+    kw = dict(d_model=256, n_routed=6, top_k=2, d_ff_routed=256, d_ff_shared=(192,), shared_gate_sigmoid=True) \
+        if shape == "gated_shared" else \
+        dict(d_model=128, n_routed=16, top_k=6, d_ff_routed=64, d_ff_shared=(64, 64), shared_gate_sigmoid=False)
+    cfg = cfg_of(n_tokens=2000, **kw)
+    L = W().make_layer(cfg, seed=40, device=DEV)
+    Xcal = W().make_tokens(cfg, seed=40, device=DEV)
+    layer = P.Layer.from_workload(L)
+    keep = P.camera_select_prune(P.camera_score_layer(layer, Xcal, 0.95), 0.4)
+    X = W().make_tokens(W().scaled(cfg, n_tokens=64), seed=41, device=DEV)
+    ol, Xd = to_oracle_layer(L), f64(X)
+    rin, rout = oracle_routing(ol, Xd)
+    ref = oracle_forward(ol, Xd, rout)
+    for lay in (layer, P.camera_layer_prepare(P.Layer.from_workload(L))):
+        assert_output_close("decode batch, full layer", P.camera_layer_forward(lay, X, routing_in=rin).cpu().numpy(), ref)
+        y, (gi, gw) = P.camera_layer_forward(lay, X, want_routing=True)              # the layer's own router
+        ref_own = oracle_forward(ol, Xd, (gi.cpu().numpy().astype(np.int64), gw.cpu().numpy().astype(np.float64)))
+        assert_output_close("decode batch, own routing", y.cpu().numpy(), ref_own)
+    from _gpu import check_routing
+    check_routing(ol, Xd, gi, gw)
+    sub, counts = P.camera_sub_index(keep, P.expert_offsets_tensor(layer), [1])
+    out = P.camera_compact_weights(layer, sub, counts, 1)
+    m = counts[:, 0].cpu().numpy()
+    def sliced():
+        return P.Layer(L["w_router"], [out["w_gate"][e][:m[e]] for e in range(layer.n_experts)],
+                       [out["w_up"][e][:m[e]] for e in range(layer.n_experts)], out["w_down"], cfg.top_k, cfg.n_shared,
+                       L["router_bias"], L["w_shared_gate"], cfg.norm_topk, "hf", down_ld=layer.d_ff)
+    lists, _ = O.sub_index_lists(keep.cpu().numpy(), O.me_offsets(ol), [1])
+    ref_hat = oracle_forward(O.slice_layer(ol, lists), Xd, rout)
+    for lay in (sliced(), P.camera_layer_prepare(sliced())):
+        assert_output_close("decode batch, sliced layer", P.camera_layer_forward(lay, X, routing_in=rin).cpu().numpy(), ref_hat)

@@ -30,15 +30,16 @@ def small_layer(dtype="bf16", T=300, seed=50):
     return cfg, W.make_layer(cfg, seed=seed, device=DEV), W.make_tokens(cfg, seed=seed, device=DEV)
 
 
+@pytest.mark.parametrize("T", [300, 90])       # 90 tokens: the front end for decode-sized batches
 @pytest.mark.parametrize("router", ["tensor_core", "fma_bf16", "fma_fp32"])
-def test_non_finite_tokens_set_the_status_word_and_nothing_faults(P, router):
-    cfg, L, X = small_layer("f32" if router == "fma_fp32" else "bf16")
+def test_non_finite_tokens_set_the_status_word_and_nothing_faults(P, router, T):
+    cfg, L, X = small_layer("f32" if router == "fma_fp32" else "bf16", T=T)
     layer = P.Layer.from_workload(L)
-    bad_tokens = [5, 70, 299]
+    bad_tokens = [5, 70, T - 1]
     Xb = X.clone()
     Xb[5, 17] = float("nan")
     Xb[70, :] = float("inf")
-    Xb[299, 3] = float("-inf")
+    Xb[T - 1, 3] = float("-inf")
     ws = P.alloc_workspace(P.camera_score_workspace_bytes(layer, cfg.n_tokens), DEV)
     out = P.camera_score_layer(layer, Xb, 0.95, details=True, workspace=ws, force_simt=router != "tensor_core")
     assert P.camera_read_status(ws) == INVALID_ARG
@@ -58,9 +59,10 @@ def test_non_finite_tokens_set_the_status_word_and_nothing_faults(P, router):
     assert torch.equal(clean["energy"], fresh["energy"]) and torch.equal(clean["topk_idx"], fresh["topk_idx"])
 
 
+@pytest.mark.parametrize("T", [300, 120])
 @pytest.mark.parametrize("router", ["tensor_core", "fma_bf16"])
-def test_prescribed_routing_out_of_range_or_repeated(P, router):
-    cfg, L, X = small_layer()
+def test_prescribed_routing_out_of_range_or_repeated(P, router, T):
+    cfg, L, X = small_layer(T=T)
     layer = P.Layer.from_workload(L)
     ol, Xd = to_oracle_layer(L), f64(X)
     idx, w = O.top_and_norm(O.router_probs(ol, Xd), ol.top_k, ol.norm_topk)
@@ -68,7 +70,7 @@ def test_prescribed_routing_out_of_range_or_repeated(P, router):
     bad = idx.copy()
     bad[3, 1] = bad[3, 0]           # an expert named twice by one token
     bad[9, 2] = 99                  # past the last expert
-    bad[200, 0] = -1
+    bad[T - 100, 0] = -1
     ws = P.alloc_workspace(P.camera_score_workspace_bytes(layer, cfg.n_tokens), DEV)
     out = P.camera_score_layer(layer, X, 0.95, details=True, workspace=ws, force_simt=router != "tensor_core",
                                routing_in=(torch.from_numpy(bad.astype(np.int32)), torch.from_numpy(w32)))
@@ -77,7 +79,7 @@ def test_prescribed_routing_out_of_range_or_repeated(P, router):
     assert gi.min() >= 0 and gi.max() < cfg.n_routed
     # the three tokens count for nothing among the routed experts; everything else is scored as prescribed
     w_fixed = w32.astype(np.float64)
-    w_fixed[[3, 9, 200]] = 0.0
+    w_fixed[[3, 9, T - 100]] = 0.0
     p2, pinf, w2 = O.camera_components(ol, Xd, routing=(idx, w_fixed))
     E = O.energy(p2, pinf, w2, float(np.float32(0.95)))
     assert_close("energy with three tokens dropped", out["energy"].cpu().numpy(), E)
