@@ -138,6 +138,8 @@ k_select_fused(const __grid_constant__ SelArgs a, const __grid_constant__ SelPar
   __shared__ unsigned first_above[MAX_THR];           // local index from which such keys are at or above the threshold
   __shared__ int boundary[MAX_THR];
   __shared__ int rep[MAX_THR];
+  __shared__ unsigned lut[256];                       // by a key's last fixed digit: the thresholds it may match
+  __shared__ unsigned pre_s[MAX_THR];
   __shared__ unsigned boundary_skip[MAX_THR];
   __shared__ unsigned wtot[SEL_THREADS / 32];
   __shared__ int s_abort;
@@ -158,7 +160,7 @@ k_select_fused(const __grid_constant__ SelArgs a, const __grid_constant__ SelPar
       }
       continue;
     }
-    const long long per = (len + gx - 1) / gx;
+    const long long per = ((len + gx - 1) / gx + 3) & ~3ll;          // shares start on multiples of 4 keys
     const long long c0 = per * bx < len ? per * bx : len;
     const int n = (int)((c0 + per < len ? c0 + per : len) - c0);       // this CTA's share: [c0, c0 + n) of the segment
     const bool cached = per <= SEL_CACHE_KEYS;
@@ -187,28 +189,60 @@ k_select_fused(const __grid_constant__ SelArgs a, const __grid_constant__ SelPar
         // energies of one layer share their leading bits: a thread counts runs of equal digits in a register and
         // touches the bin once per run, not once per key
         unsigned run_digit = 0u, run_len = 0u;
-        for (int i = tid; i < n; i += SEL_THREADS) {
-          const unsigned digit = (cached ? skeys[i] : key_bits(src[i])) >> 24;
+        auto count_first = [&](unsigned b) {
+          const unsigned digit = b >> 24;
           if (digit != run_digit) {
             if (run_len) atomicAdd(&bins[0][run_digit], run_len);
             run_digit = digit;
             run_len = 0u;
           }
           ++run_len;
+        };
+        if (cached) {
+          const uint4* k4 = reinterpret_cast<const uint4*>(skeys);
+          for (int q = tid; 4 * q < n; q += SEL_THREADS) {
+            const uint4 kk = k4[q];
+            count_first(kk.x);
+            if (4 * q + 1 < n) count_first(kk.y);
+            if (4 * q + 2 < n) count_first(kk.z);
+            if (4 * q + 3 < n) count_first(kk.w);
+          }
+        } else {
+          for (int i = tid; i < n; i += SEL_THREADS) count_first(key_bits(src[i]));
         }
         if (run_len) atomicAdd(&bins[0][run_digit], run_len);
       } else {
-        // thresholds whose digits so far agree share one histogram (that of the lowest-numbered among them)
-        unsigned pre[MAX_THR];
-#pragma unroll
-        for (int j = 0; j < MAX_THR; ++j)
-          pre[j] = (j < n_thr && st[j].valid && rep[j] == j) ? (st[j].prefix >> (shift + 8)) : 0xffffffffu;
-        for (int i = tid; i < n; i += SEL_THREADS) {
-          const unsigned b = cached ? skeys[i] : key_bits(src[i]);
-          const unsigned hi = b >> (shift + 8), digit = (b >> shift) & 0xffu;
-#pragma unroll
-          for (int j = 0; j < MAX_THR; ++j)
-            if (hi == pre[j]) atomicAdd(&bins[j][digit], 1u);          // pre of an unused slot matches nothing: hi < 2^24
+        // Thresholds whose digits so far agree share one histogram (that of the lowest-numbered among them).  Most
+        // keys match none: a table on the last digit found says which thresholds a key can match at all.
+        for (int i = tid; i < 256; i += SEL_THREADS) lut[i] = 0u;
+        __syncthreads();
+        if (tid < n_thr && st[tid].valid && rep[tid] == tid) {
+          pre_s[tid] = st[tid].prefix >> (shift + 8);
+          atomicOr(&lut[pre_s[tid] & 0xffu], 1u << tid);
+        }
+        __syncthreads();
+        auto count_key = [&](unsigned b) {
+          unsigned cand = lut[(b >> (shift + 8)) & 0xffu];
+          if (cand) {
+            const unsigned hi = b >> (shift + 8), digit = (b >> shift) & 0xffu;
+            do {
+              const int j = __ffs(cand) - 1;
+              cand &= cand - 1u;
+              if (hi == pre_s[j]) atomicAdd(&bins[j][digit], 1u);
+            } while (cand);
+          }
+        };
+        if (cached) {
+          const uint4* k4 = reinterpret_cast<const uint4*>(skeys);
+          for (int q = tid; 4 * q < n; q += SEL_THREADS) {
+            const uint4 kk = k4[q];
+            count_key(kk.x);
+            if (4 * q + 1 < n) count_key(kk.y);
+            if (4 * q + 2 < n) count_key(kk.z);
+            if (4 * q + 3 < n) count_key(kk.w);
+          }
+        } else {
+          for (int i = tid; i < n; i += SEL_THREADS) count_key(key_bits(src[i]));
         }
       }
       __syncthreads();
@@ -327,26 +361,70 @@ k_select_fused(const __grid_constant__ SelArgs a, const __grid_constant__ SelPar
     }
 
     // labels
-    unsigned tau[MAX_THR], first[MAX_THR];
+    unsigned tau[MAX_THR];
+    unsigned valid_mask = 0u;
+    bool any_first = false;                            // some threshold cuts through a run of equal energies
 #pragma unroll
     for (int j = 0; j < MAX_THR; ++j) {
       const bool v = j < n_thr && st[j].valid;
       tau[j] = v ? st[j].prefix : 0xffffffffu;
-      first[j] = v ? first_above[j] : 0xffffffffu;     // (0xffffffff, 0xffffffff): no key is at or above
+      valid_mask |= (unsigned)v << j;
+      any_first = any_first || (v && first_above[j] != 0u);
     }
     const int n_prune = a.n_prune, n_bounds = n_thr - (n_prune < 0 ? 0 : n_prune);
-    for (int i = tid; i < n; i += SEL_THREADS) {
-      const unsigned b = cached ? skeys[i] : key_bits(src[i]);
-      unsigned at = 0u;                                // bit j: at or above threshold j
+    // bit j of the result: the key at local index i is at or above threshold j
+    auto at_of = [&](unsigned b, int i) {
+      unsigned at = 0u;
 #pragma unroll
-      for (int j = 0; j < MAX_THR; ++j)
-        at |= (unsigned)(b > tau[j] || (b == tau[j] && (unsigned)i >= first[j])) << j;
-      const size_t g = (size_t)(begin + c0) + i;
-      if (n_prune < 0) {
-        a.out[g] = a.lv.v[n_thr - __popc(at)];
-      } else {
-        for (int j = 0; j < n_prune; ++j) a.out[(size_t)j * a.n_total + g] = (at >> j) & 1u;
-        if (a.bits_out != nullptr) a.bits_out[g] = a.lv.v[n_bounds - __popc(at >> n_prune)];
+      for (int j = 0; j < MAX_THR; ++j) at |= (unsigned)(b >= tau[j]) << j;
+      at &= valid_mask;
+      if (any_first) {                                 // keys equal to a threshold's energy: below it before `first_above`
+#pragma unroll
+        for (int j = 0; j < MAX_THR; ++j)
+          if (b == tau[j] && (unsigned)i < first_above[j]) at &= ~(1u << j);
+      }
+      return at;
+    };
+    const size_t g0 = (size_t)(begin + c0);
+    const bool words = cached && (g0 % 4 == 0) && (a.n_total % 4 == 0) && (reinterpret_cast<uintptr_t>(a.out) % 4 == 0) &&
+                       (a.bits_out == nullptr || reinterpret_cast<uintptr_t>(a.bits_out) % 4 == 0);
+    if (words) {       // four keys per step, their labels in one 32-bit store per output
+      const uint4* k4 = reinterpret_cast<const uint4*>(skeys);
+      for (int q = tid; 4 * q < n; q += SEL_THREADS) {
+        const uint4 kk = k4[q];
+        const int i = 4 * q;
+        const unsigned at0 = at_of(kk.x, i), at1 = at_of(kk.y, i + 1), at2 = at_of(kk.z, i + 2), at3 = at_of(kk.w, i + 3);
+        const bool full = i + 3 < n;
+        const size_t g = g0 + i;
+        auto put = [&](unsigned char* base, unsigned w) {
+          if (full) *reinterpret_cast<unsigned*>(base + g) = w;
+          else
+            for (int r = 0; i + r < n; ++r) base[g + r] = (unsigned char)(w >> (8 * r));
+        };
+        if (n_prune < 0) {
+          put(a.out, (unsigned)a.lv.v[n_thr - __popc(at0)] | ((unsigned)a.lv.v[n_thr - __popc(at1)] << 8) |
+                         ((unsigned)a.lv.v[n_thr - __popc(at2)] << 16) | ((unsigned)a.lv.v[n_thr - __popc(at3)] << 24));
+        } else {
+          for (int j = 0; j < n_prune; ++j)
+            put(a.out + (size_t)j * a.n_total,
+                ((at0 >> j) & 1u) | (((at1 >> j) & 1u) << 8) | (((at2 >> j) & 1u) << 16) | (((at3 >> j) & 1u) << 24));
+          if (a.bits_out != nullptr)
+            put(a.bits_out, (unsigned)a.lv.v[n_bounds - __popc(at0 >> n_prune)] |
+                                ((unsigned)a.lv.v[n_bounds - __popc(at1 >> n_prune)] << 8) |
+                                ((unsigned)a.lv.v[n_bounds - __popc(at2 >> n_prune)] << 16) |
+                                ((unsigned)a.lv.v[n_bounds - __popc(at3 >> n_prune)] << 24));
+        }
+      }
+    } else {
+      for (int i = tid; i < n; i += SEL_THREADS) {
+        const unsigned at = at_of(cached ? skeys[i] : key_bits(src[i]), i);
+        const size_t g = g0 + i;
+        if (n_prune < 0) {
+          a.out[g] = a.lv.v[n_thr - __popc(at)];
+        } else {
+          for (int j = 0; j < n_prune; ++j) a.out[(size_t)j * a.n_total + g] = (at >> j) & 1u;
+          if (a.bits_out != nullptr) a.bits_out[g] = a.lv.v[n_bounds - __popc(at >> n_prune)];
+        }
       }
     }
     __syncthreads();       // the next segment reuses the shared arrays
