@@ -35,9 +35,9 @@ PAPER_CONTEXT = "paper: <5 min for the full Qwen2-57B-A14B analysis on one A100-
 # kernels launched by one step: score = router, block scan, plan, permute, pad, norms, scoring, combine;
 # the selections = one kernel (radix passes, tie break and labels behind one cooperative launch)
 LAUNCHES_PER_STEP = 8 + 1
-# DRAM bytes (read + write) per gate/up flop of the scoring kernel, from the committed ncu capture of a
-# 1/8 slice of the layer whose traffic grows in proportion to the flop (profiles/k_score_umma_qwen2_slice.md).
-SCORE_KERNEL_DRAM_BYTES_PER_FLOP = 4.483e9 / 1.924e13
+# DRAM bytes (read + write) of one launch of the scoring kernel on the full Qwen2-57B-A14B-shaped layer (262144 tokens,
+# single pass): the one-pass ncu capture of profiles/k_score_umma_pair_qwen2_full_dram.md.
+SCORE_KERNEL_DRAM_BYTES_FULL_LAYER = 33036971776 + 344499712
 
 
 def shard_layers(n_layers: int, world: int, rank: int):
@@ -518,6 +518,7 @@ def main():
     ap.add_argument("--no-configs", action="store_true", help="skip the other workload configs")
     ap.add_argument("--no-model", action="store_true", help="skip the measured loop over all layers of the model")
     ap.add_argument("--stack", action="store_true", help="run Algorithm 2's layer loop over a synthetic stack instead of the step benchmark")
+    ap.add_argument("--decode-only", action="store_true", help="run only the 64-token decode leg of --config and print its record")
     ap.add_argument("--stack-layers", type=int, default=0, help="layers of the stack (default: the config's)")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
@@ -525,6 +526,15 @@ def main():
         return run_reference(args)
     if args.stack:
         return run_stack(args)
+    if args.decode_only:
+        import torch
+        import paper_2508_02322_b200 as P
+        from paper_2508_02322_b200 import workloads as W
+        torch.cuda.set_device(int(os.environ.get("LOCAL_RANK", "0")))
+        dev = torch.device("cuda", int(os.environ.get("LOCAL_RANK", "0")))
+        print(json.dumps({"mode": "decode", "decode": bench_decode(P, torch, W, args.config, dev, torch.cuda.current_stream(),
+                                                                   load_peaks())}))
+        return
 
     import torch
     import torch.distributed as dist
@@ -817,8 +827,9 @@ def main():
                 "peak_source": peaks["source"] + " (cuBLAS bf16 sustained in a seconds-long loop: the kernel is timed inside "
                                                  "a multi-second step loop; the burst figure is beside it)",
                 "flop_per_launch": flop, "ms_per_launch": score_ms,
-                "traffic": SCORE_KERNEL_DRAM_BYTES_PER_FLOP * flop
-                if (args.config == "qwen2_57b_a14b" and not args.single_cta) else None}
+                "traffic": SCORE_KERNEL_DRAM_BYTES_FULL_LAYER
+                if (args.config == "qwen2_57b_a14b" and not args.single_cta and not by_tokens
+                    and not (args.tokens or args.routed or args.topk)) else None}
 
     cpu = None
     if not args.no_cpu_baseline:

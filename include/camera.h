@@ -298,7 +298,8 @@ int camera_sub_index(const uint8_t* labels, const int64_t* expert_offsets, int32
                      const int32_t* label_order, int32_t n_labels, int32_t* sub_index, int32_t* counts,
                      void* cuda_stream);
 
-/* Scratch for camera_compact_weights. */
+/* Scratch for camera_compact_weights (256-byte aligned; it starts with a status word that camera_read_status reads:
+ * the column gather waits, with the library's bounded wait, for the bulk copies that fill its tiles). */
 size_t camera_compact_workspace_bytes(int32_t n_experts);
 
 /*
