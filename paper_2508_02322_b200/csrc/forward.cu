@@ -19,14 +19,15 @@ namespace camera {
 namespace {
 
 constexpr int D_THREADS = 192;
-constexpr int D_STAGES = 4;
+constexpr int D_STAGES = 4;                       // with a full token tile per stage
+constexpr int D_MAX_STAGES = 8;                   // with the short boxes of a decode batch
 constexpr int D_TILE = 128;                       // output channels (rows of W_down) per work unit = TMEM lanes
 constexpr int D_A_BYTES = D_TILE * 128;
 constexpr int D_B_BYTES = UMMA_TOK * 128;
 constexpr int D_STAGE_BYTES = D_A_BYTES + D_B_BYTES;
 constexpr int D_TMEM_COLS = 512;
 constexpr int D_SCHED = 2;                        // ring that passes unit numbers from the producer to the other warps
-constexpr int D_SMEM_BYTES = D_STAGES * D_STAGE_BYTES + 256 + 1024;
+constexpr int D_SMEM_BYTES = D_STAGES * D_STAGE_BYTES + 256 + 1024;      // the budget every configuration stays within
 
 struct DownUnit {
   int e, rows, row0, c0, n_kb, row_limit;
@@ -58,18 +59,23 @@ __device__ __forceinline__ DownUnit decode_down_unit(const ScoreCtx& c, int unit
 
 // b_bytes: size of the box of h rows one load brings (128 bytes per row; the map's box is as many rows as a token list
 // can have, at most a tile: with a few tokens per expert a full tile's box would triple the bytes L2 has to deliver).
-__global__ void __launch_bounds__(D_THREADS, 1) k_down_umma(const ScoreCtx c, const void* maps_raw, int n_dt, int b_bytes) {
+// n_stages: depth of the operand ring; a stage is the W_down tile plus that box, so a decode batch (a box of 64 rows)
+// gets 8 stages of 24 KB where a full token tile gets 4 of 48 KB: the kernel then streams W_down from DRAM, and the
+// bytes in flight per SM are what hides the latency.
+__global__ void __launch_bounds__(D_THREADS, 1)
+k_down_umma(const ScoreCtx c, const void* maps_raw, int n_dt, int b_bytes, int n_stages) {
   extern __shared__ uint8_t smem_raw[];
   const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
   uint8_t* const base_ptr = smem_raw + (base - smem_u32(smem_raw));
-  const uint32_t bars = base + D_STAGES * D_STAGE_BYTES;
+  const int stage_bytes = D_A_BYTES + b_bytes;                 // a multiple of 1024: the swizzled tiles stay aligned
+  const uint32_t bars = base + n_stages * stage_bytes;
   auto full_bar = [&](int s) { return bars + 8u * s; };
-  auto empty_bar = [&](int s) { return bars + 8u * (D_STAGES + s); };
-  auto tfull_bar = [&](int a) { return bars + 8u * (2 * D_STAGES + a); };
-  auto tempty_bar = [&](int a) { return bars + 8u * (2 * D_STAGES + 2 + a); };
-  auto sfull_bar = [&](int q) { return bars + 8u * (2 * D_STAGES + 4 + q); };
-  auto sempty_bar = [&](int q) { return bars + 8u * (2 * D_STAGES + 4 + D_SCHED + q); };
-  uint8_t* const tail = base_ptr + D_STAGES * D_STAGE_BYTES + 8 * (2 * D_STAGES + 4 + 2 * D_SCHED);
+  auto empty_bar = [&](int s) { return bars + 8u * (D_MAX_STAGES + s); };
+  auto tfull_bar = [&](int a) { return bars + 8u * (2 * D_MAX_STAGES + a); };
+  auto tempty_bar = [&](int a) { return bars + 8u * (2 * D_MAX_STAGES + 2 + a); };
+  auto sfull_bar = [&](int q) { return bars + 8u * (2 * D_MAX_STAGES + 4 + q); };
+  auto sempty_bar = [&](int q) { return bars + 8u * (2 * D_MAX_STAGES + 4 + D_SCHED + q); };
+  uint8_t* const tail = base_ptr + n_stages * stage_bytes + 8 * (2 * D_MAX_STAGES + 4 + 2 * D_SCHED);
   volatile uint32_t* const tmem_slot = reinterpret_cast<volatile uint32_t*>(tail);
   volatile int* const abort_flag = reinterpret_cast<volatile int*>(tail + 8);
   volatile int* const sched_unit = reinterpret_cast<volatile int*>(tail + 16);
@@ -78,7 +84,7 @@ __global__ void __launch_bounds__(D_THREADS, 1) k_down_umma(const ScoreCtx c, co
   const int total_units = c.totals->total_chunks * n_dt;
 
   if (tid == 0) {
-    for (int s = 0; s < D_STAGES; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
+    for (int s = 0; s < n_stages; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
     for (int a = 0; a < 2; ++a) { mbar_init(tfull_bar(a), 1); mbar_init(tempty_bar(a), 128); }
     for (int q = 0; q < D_SCHED; ++q) { mbar_init(sfull_bar(q), 1); mbar_init(sempty_bar(q), 5); }
     wait_state_init(abort_flag, c.wait_limit_ns);
@@ -126,12 +132,12 @@ __global__ void __launch_bounds__(D_THREADS, 1) k_down_umma(const ScoreCtx c, co
           const int row = u.row0 + tt * UMMA_TOK;
           for (int kb = 0; kb < u.n_kb; ++kb) {
             if (!mbar_wait(empty_bar(stage), phase ^ 1u, abort_flag)) { ok = false; break; }
-            const uint32_t a_dst = base + stage * D_STAGE_BYTES;
+            const uint32_t a_dst = base + stage * stage_bytes;
             mbar_expect_tx(full_bar(stage), D_A_BYTES + b_bytes);
             // W_down columns past d_ff and rows past d_model, h rows past the buffer: filled with zeros
             tma_load_2d(a_dst, map_w, full_bar(stage), kb * UMMA_BK, u.c0);
             tma_load_2d(a_dst + D_A_BYTES, map_h, full_bar(stage), kb * UMMA_BK, row);
-            if (++stage == D_STAGES) { stage = 0; phase ^= 1u; }
+            if (++stage == n_stages) { stage = 0; phase ^= 1u; }
           }
         }
       }
@@ -166,14 +172,14 @@ __global__ void __launch_bounds__(D_THREADS, 1) k_down_umma(const ScoreCtx c, co
           for (int kb = 0; kb < u.n_kb; ++kb) {
             if (!mbar_wait(full_bar(stage), phase, abort_flag)) { ok = false; break; }
             tc_fence_after();
-            const uint32_t a_addr = base + stage * D_STAGE_BYTES;
+            const uint32_t a_addr = base + stage * stage_bytes;
             const unsigned long long a_desc = make_smem_desc(a_addr);
             const unsigned long long b_desc = make_smem_desc(a_addr + D_A_BYTES);
 #pragma unroll
             for (int k = 0; k < UMMA_BK / 16; ++k)
               umma_bf16(d_tmem, a_desc + 2 * k, b_desc + 2 * k, idesc, (uint32_t)((kb | k) != 0));
             umma_commit(empty_bar(stage));
-            if (++stage == D_STAGES) { stage = 0; phase ^= 1u; }
+            if (++stage == n_stages) { stage = 0; phase ^= 1u; }
           }
           if (!ok) break;
           umma_commit(tfull_bar(acc));
@@ -694,7 +700,10 @@ int down_and_sum(const camera_layer_t* L, const void* const* w_down, int64_t T, 
       cudaGetLastError();
       return CAMERA_ERR_CUDA;
     }
-    k_down_umma<<<sms, D_THREADS, D_SMEM_BYTES, st>>>(c, maps_dev, (L->d_model + D_TILE - 1) / D_TILE, h_box * 128);
+    const int stage_bytes = D_A_BYTES + h_box * 128;
+    int n_stages = (D_STAGES * D_STAGE_BYTES) / stage_bytes;
+    if (n_stages > D_MAX_STAGES) n_stages = D_MAX_STAGES;
+    k_down_umma<<<sms, D_THREADS, D_SMEM_BYTES, st>>>(c, maps_dev, (L->d_model + D_TILE - 1) / D_TILE, h_box * 128, n_stages);
   }
   k_unpermute_sum<<<dim3((unsigned)T, (unsigned)((L->d_model + 1023) / 1024)), 256, 0, st>>>(c, y);
   return cudaGetLastError() == cudaSuccess ? CAMERA_OK : CAMERA_ERR_CUDA;

@@ -20,6 +20,7 @@
 #include <math.h>
 #include <string.h>
 
+#include <atomic>
 #include <vector>
 
 #include "common.cuh"
@@ -725,24 +726,22 @@ constexpr size_t STATIC_SCRATCH_BYTES = 288 * 1024;   // room for 32 segments (c
 static __device__ __align__(256) unsigned char g_select_scratch[STATIC_SCRATCH_BYTES];
 
 constexpr int STATIC_MAX_DEVICES = 64;
-void* g_scratch_ptr[STATIC_MAX_DEVICES];     // device address of g_select_scratch, per device ordinal
-bool g_scratch_ready[STATIC_MAX_DEVICES];
+std::atomic<void*> g_scratch_ptr[STATIC_MAX_DEVICES];     // device address of g_select_scratch per device ordinal; null = not asked yet
 
 // In host code `g_select_scratch` is only a handle; the address kernels can use has to be asked for,
-// once per device, while that device is current.
+// once per device, while that device is current.  Two host threads that ask at the same time get the same answer.
 int static_scratch(void** out) {
   int dev = -1;
   if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= STATIC_MAX_DEVICES) return CAMERA_ERR_CUDA;
-  if (!g_scratch_ready[dev]) {
-    void* p = nullptr;
+  void* p = g_scratch_ptr[dev].load(std::memory_order_acquire);
+  if (p == nullptr) {
     if (cudaGetSymbolAddress(&p, g_select_scratch) != cudaSuccess || p == nullptr) {
       cudaGetLastError();
       return CAMERA_ERR_CUDA;
     }
-    g_scratch_ptr[dev] = p;
-    g_scratch_ready[dev] = true;
+    g_scratch_ptr[dev].store(p, std::memory_order_release);
   }
-  *out = g_scratch_ptr[dev];
+  *out = p;
   return CAMERA_OK;
 }
 
