@@ -133,3 +133,26 @@ def test_prepare_checks_its_arguments_before_touching_a_device(P):
     assert P.lib.camera_layer_prepare(C.byref(ok), 4096, n - 1, None, C.byref(handle)) == -3  # too little of it
     assert P.lib.camera_layer_prepare(C.byref(ok), 4096, n, None, None) == -1
     P.lib.camera_layer_release(None)                                                          # a null handle is ignored
+
+
+def test_score_scratch_stops_growing_at_one_batch(P):
+    ok = _layer_struct(P)
+    q = lambda t: P.lib.camera_score_workspace_bytes(C.byref(ok), t)
+    one = lambda t: P.lib.camera_score_workspace_bytes_single_pass(C.byref(ok), t)
+    assert q(1000) == one(1000) and q(65536) == one(65536)          # up to a batch the two are the same
+    assert q(65537) == q(10 ** 6) > q(65536)                         # beyond: one batch's scratch plus the accumulators
+    assert one(10 ** 6) > one(65537) and one(10 ** 6) > 4 * q(10 ** 6)    # a single pass keeps growing with the tokens
+    assert one(-1) == 0 and P.lib.camera_score_workspace_bytes_single_pass(None, 10) == 0
+
+
+def test_wait_limit_and_probe_check_their_arguments_on_the_host(P):
+    default = P.lib.camera_get_wait_limit_ns()
+    assert default == 4_000_000_000
+    assert P.lib.camera_set_wait_limit_ns(10) == -1                  # under a microsecond
+    assert P.lib.camera_set_wait_limit_ns(10 ** 13) == -1            # over ten minutes
+    assert P.lib.camera_get_wait_limit_ns() == default
+    assert P.lib.camera_set_wait_limit_ns(2_000_000_000) == 0 and P.lib.camera_get_wait_limit_ns() == 2_000_000_000
+    assert P.lib.camera_set_wait_limit_ns(default) == 0
+    assert P.lib.camera_wait_probe(4096, 4096, 5_000_000_000, None) == -1      # a probe may wait a second at most
+    assert P.lib.camera_wait_probe(None, 4096, 1_000_000, None) == -3          # no workspace
+    assert P.lib.camera_wait_probe(4096 + 8, 4096, 1_000_000, None) == -3      # not 256-byte aligned
