@@ -831,6 +831,15 @@ def main():
                 if (args.config == "qwen2_57b_a14b" and not args.single_cta and not by_tokens
                     and not (args.tokens or args.routed or args.topk)) else None}
 
+    # the HBM-bound stages of the step against their algorithmic bytes (X once for the router; X once in and k copies
+    # out for the permutation; W_down once for its norms) and the measured copy peak
+    esz = 2 if cfg.dtype == "bf16" else 4
+    x_bytes = T * cfg.d_model * esz
+    stage_bytes = {"router": x_bytes, "permute": (1 + cfg.top_k) * x_bytes, "rownorm": n_me * cfg.d_model * esz}
+    stage_roofline = {s: {"bound": "hbm", "algorithmic_gb": b / 1e9, "achieved_gbs": b / 1e9 / (stage_ms[s] * 1e-3),
+                          "frac": b / 1e9 / (stage_ms[s] * 1e-3) / peaks["hbm_gbs"]}
+                      for s, b in stage_bytes.items() if stage_ms[s] > 0}
+
     cpu = None
     if not args.no_cpu_baseline:
         n_s = min(args.oracle_tokens or 2048, T)
@@ -853,7 +862,7 @@ def main():
                    "parallelism": (f"tokens x{world}" if by_tokens else f"layers x{world}") if world > 1 else "single GPU"},
         "model_seconds": cfg.n_layers * ms_per_step * 1e-3 / world,     # extrapolated: layers x the step on one layer
         "model_seconds_measured": model_measured, "configs": configs, "batched_scoring": batched,
-        "stage_ms": stage_ms, "clocks": clocks, "e2e": e2e, "gpu_launches": (LAUNCHES_PER_STEP + (3 if by_tokens else 0)) * args.steps,
+        "stage_ms": stage_ms, "stage_roofline": stage_roofline, "clocks": clocks, "e2e": e2e, "gpu_launches": (LAUNCHES_PER_STEP + (3 if by_tokens else 0)) * args.steps,
         "roofline": roofline, "compact": compact, "forward": forward, "decode": decode, "select_model": select_model, "cpu_baseline": cpu, "context": PAPER_CONTEXT,
     }
     print(json.dumps(out))

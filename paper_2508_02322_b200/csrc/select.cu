@@ -568,17 +568,18 @@ int select_core(const float* energy, const int64_t* seg_offsets, int n_seg, int 
     long long gy = resident / gx;
     if (gy > n_seg) gy = n_seg;
     if (gy > 65535) gy = 65535;
-    const dim3 grid((unsigned)gx, (unsigned)gy);
+    bool launched = false;
     if (gx > 1) {     // CTAs of a segment wait for one another: they must all be resident
       void* args[2] = {&a, &prm};
-      if (cudaLaunchCooperativeKernel(reinterpret_cast<const void*>(k_select_fused), grid, dim3(SEL_THREADS), args, smem, st) !=
-          cudaSuccess) {
+      launched = cudaLaunchCooperativeKernel(reinterpret_cast<const void*>(k_select_fused), dim3((unsigned)gx, (unsigned)gy),
+                                             dim3(SEL_THREADS), args, smem, st) == cudaSuccess;
+      if (!launched) {      // a context without cooperative launches: one CTA per segment, which waits for nobody
         cudaGetLastError();
-        return CAMERA_ERR_CUDA;
+        gx = 1;
+        gy = n_seg < 65535 ? n_seg : 65535;
       }
-    } else {
-      k_select_fused<<<grid, SEL_THREADS, smem, st>>>(a, prm);
     }
+    if (!launched) k_select_fused<<<dim3((unsigned)gx, (unsigned)gy), SEL_THREADS, smem, st>>>(a, prm);
   }
   if (counts != nullptr && expert_offsets != nullptr && n_experts > 0) {
     if (max_len > 0) {
