@@ -222,15 +222,30 @@ k_select_fused(const __grid_constant__ SelArgs a, const __grid_constant__ SelPar
           atomicOr(&lut[pre_s[tid] & 0xffu], 1u << tid);
         }
         __syncthreads();
+        // the thresholds that count in this pass, in order; with one or two of them (the rule while the thresholds'
+        // leading digits still agree, when every key of a narrow energy range is a candidate) a key is compared with
+        // them directly
+        int n_act = 0, j0 = 0, j1 = 0;
+        unsigned p0 = 0xffffffffu, p1 = 0xffffffffu;
+        for (int j = 0; j < n_thr; ++j)
+          if (st[j].valid && rep[j] == j) {
+            if (n_act == 0) { j0 = j; p0 = st[j].prefix >> (shift + 8); }
+            else if (n_act == 1) { j1 = j; p1 = st[j].prefix >> (shift + 8); }
+            ++n_act;
+          }
+        const bool few = n_act <= 2;
         auto count_key = [&](unsigned b) {
-          unsigned cand = lut[(b >> (shift + 8)) & 0xffu];
-          if (cand) {
-            const unsigned hi = b >> (shift + 8), digit = (b >> shift) & 0xffu;
-            do {
-              const int j = __ffs(cand) - 1;
-              cand &= cand - 1u;
-              if (hi == pre_s[j]) atomicAdd(&bins[j][digit], 1u);
-            } while (cand);
+          const unsigned hi = b >> (shift + 8), digit = (b >> shift) & 0xffu;
+          if (few) {
+            if (hi == p0) atomicAdd(&bins[j0][digit], 1u);
+            else if (hi == p1) atomicAdd(&bins[j1][digit], 1u);
+            return;
+          }
+          unsigned cand = lut[hi & 0xffu];
+          while (cand) {
+            const int j = __ffs(cand) - 1;
+            cand &= cand - 1u;
+            if (hi == pre_s[j]) atomicAdd(&bins[j][digit], 1u);
           }
         };
         if (cached) {
@@ -390,6 +405,14 @@ k_select_fused(const __grid_constant__ SelArgs a, const __grid_constant__ SelPar
     const bool words = cached && (g0 % 4 == 0) && (a.n_total % 4 == 0) && (reinterpret_cast<uintptr_t>(a.out) % 4 == 0) &&
                        (a.bits_out == nullptr || reinterpret_cast<uintptr_t>(a.bits_out) % 4 == 0);
     if (words) {       // four keys per step, their labels in one 32-bit store per output
+      // label table by the number c of boundaries a key is at or above: byte c = lv[(boundaries) - c]
+      const int n_b = n_prune < 0 ? n_thr : n_bounds;
+      unsigned lab_lo = 0u, lab_hi = 0u;
+      for (int cnt = 0; cnt <= n_b; ++cnt) {
+        const unsigned v = a.lv.v[n_b - cnt];
+        if (cnt < 4) lab_lo |= v << (8 * cnt); else lab_hi |= v << (8 * (cnt - 4));
+      }
+      const unsigned bound_bits4 = ((1u << n_bounds) - 1u) * 0x01010101u;
       const uint4* k4 = reinterpret_cast<const uint4*>(skeys);
       for (int q = tid; 4 * q < n; q += SEL_THREADS) {
         const uint4 kk = k4[q];
@@ -402,18 +425,22 @@ k_select_fused(const __grid_constant__ SelArgs a, const __grid_constant__ SelPar
           else
             for (int r = 0; i + r < n; ++r) base[g + r] = (unsigned char)(w >> (8 * r));
         };
+        // the four keys' bits side by side, one byte per key: mask j is bit j of every byte, the class of a key the
+        // number of its boundary bits (counted in all four bytes at once), the label a byte picked from the table
+        const unsigned w4 = at0 | (at1 << 8) | (at2 << 16) | (at3 << 24);
+        auto labels_of = [&](unsigned bits4) {       // per byte: lv[(number of boundaries) - popcount(byte)]
+          unsigned x = bits4;
+          x -= (x >> 1) & 0x55555555u;
+          x = (x & 0x33333333u) + ((x >> 2) & 0x33333333u);
+          x = (x + (x >> 4)) & 0x0f0f0f0fu;
+          const unsigned sel = (x & 0xfu) | ((x >> 4) & 0xf0u) | ((x >> 8) & 0xf00u) | ((x >> 12) & 0xf000u);
+          return __byte_perm(lab_lo, lab_hi, sel);
+        };
         if (n_prune < 0) {
-          put(a.out, (unsigned)a.lv.v[n_thr - __popc(at0)] | ((unsigned)a.lv.v[n_thr - __popc(at1)] << 8) |
-                         ((unsigned)a.lv.v[n_thr - __popc(at2)] << 16) | ((unsigned)a.lv.v[n_thr - __popc(at3)] << 24));
+          put(a.out, labels_of(w4));
         } else {
-          for (int j = 0; j < n_prune; ++j)
-            put(a.out + (size_t)j * a.n_total,
-                ((at0 >> j) & 1u) | (((at1 >> j) & 1u) << 8) | (((at2 >> j) & 1u) << 16) | (((at3 >> j) & 1u) << 24));
-          if (a.bits_out != nullptr)
-            put(a.bits_out, (unsigned)a.lv.v[n_bounds - __popc(at0 >> n_prune)] |
-                                ((unsigned)a.lv.v[n_bounds - __popc(at1 >> n_prune)] << 8) |
-                                ((unsigned)a.lv.v[n_bounds - __popc(at2 >> n_prune)] << 16) |
-                                ((unsigned)a.lv.v[n_bounds - __popc(at3 >> n_prune)] << 24));
+          for (int j = 0; j < n_prune; ++j) put(a.out + (size_t)j * a.n_total, (w4 >> j) & 0x01010101u);
+          if (a.bits_out != nullptr) put(a.bits_out, labels_of((w4 >> n_prune) & bound_bits4));
         }
       }
     } else {
