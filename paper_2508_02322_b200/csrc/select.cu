@@ -294,7 +294,7 @@ k_select_fused(const __grid_constant__ SelArgs a, const __grid_constant__ SelPar
         }
       }
       __syncthreads();
-      if (tid < n_thr) {       // whose histogram threshold tid reads in the next pass
+      if (tid < n_thr && pass + 1 < SEL_PASSES) {       // whose histogram threshold tid reads in the next pass
         int r = tid;
         for (int j = tid - 1; j >= 0; --j)
           if (st[j].valid && st[tid].valid && st[j].prefix == st[tid].prefix) r = j;
@@ -309,18 +309,9 @@ k_select_fused(const __grid_constant__ SelArgs a, const __grid_constant__ SelPar
     bool ties = false;
     for (int j = 0; j < n_thr; ++j) ties = ties || (st[j].valid && st[j].rank > 0);
     if (ties) {
-      unsigned cnt[MAX_THR];
-#pragma unroll
-      for (int j = 0; j < MAX_THR; ++j) cnt[j] = 0u;
-      for (int i = tid; i < n; i += SEL_THREADS) {
-        const unsigned b = cached ? skeys[i] : key_bits(src[i]);
-#pragma unroll
-        for (int j = 0; j < MAX_THR; ++j)
-          if (j < n_thr && st[j].valid && b == st[j].prefix) ++cnt[j];
-      }
-#pragma unroll
-      for (int j = 0; j < MAX_THR; ++j)
-        if (j < n_thr && cnt[j]) atomicAdd(&eq_mine[j], cnt[j]);
+      // how many such keys this CTA holds: its own count of the threshold's last digit in the last pass (the bins still
+      // hold the CTA's counts; `rep` still says whose bins a threshold counted into)
+      if (tid < n_thr) eq_mine[tid] = st[tid].valid ? bins[rep[tid]][st[tid].prefix & 0xffu] : 0u;
       __syncthreads();
       if (tid < n_thr) a.eqcnt[((size_t)seg * n_thr + tid) * gx + bx] = eq_mine[tid];
       if (!seg_meet(bseg + SEL_PASSES, gx, a, &s_abort)) return;
@@ -338,27 +329,34 @@ k_select_fused(const __grid_constant__ SelArgs a, const __grid_constant__ SelPar
         }
       }
       __syncthreads();
-      // the one CTA that holds the boundary: the local index of its boundary_skip-th such key, by an ordered scan
+      // the one CTA that holds the boundary: the local index of its boundary_skip-th such key.  A thread counts the
+      // matches in its own run of consecutive keys, one scan over the threads orders the runs, and the thread whose
+      // run holds the key walks to it.
       for (int j = 0; j < n_thr; ++j) {
         if (!boundary[j]) continue;                    // the same for every thread
         const unsigned want = boundary_skip[j], tau = st[j].prefix;
-        unsigned run = 0;
-        for (int i0 = 0; i0 < n; i0 += SEL_THREADS) {
-          const int i = i0 + tid;
-          const bool m = i < n && (cached ? skeys[i] : key_bits(src[i])) == tau;
-          const unsigned bal = __ballot_sync(0xffffffffu, m);
-          if (lane == 0) wtot[warp] = __popc(bal);
-          __syncthreads();
-          unsigned woff = 0, total = 0;
+        const int run_len = (n + SEL_THREADS - 1) / SEL_THREADS;
+        const int i0 = min(n, tid * run_len), i1 = min(n, i0 + run_len);
+        unsigned c = 0u;
+        for (int i = i0; i < i1; ++i) c += (cached ? skeys[i] : key_bits(src[i])) == tau;
+        unsigned incl = c;
 #pragma unroll
-          for (int w = 0; w < SEL_THREADS / 32; ++w) { woff += w < warp ? wtot[w] : 0u; total += wtot[w]; }
-          if (m && run + woff + __popc(bal & ((1u << lane) - 1u)) == want) first_above[j] = (unsigned)i;
-          __syncthreads();
-          run += total;
-          if (run > want) break;                       // the same for every thread
+        for (int o = 1; o < 32; o <<= 1) {
+          const unsigned t = __shfl_up_sync(0xffffffffu, incl, o);
+          if (lane >= o) incl += t;
         }
+        if (lane == 31) wtot[warp] = incl;
+        __syncthreads();
+        unsigned before = incl - c;
+#pragma unroll
+        for (int w = 0; w < SEL_THREADS / 32; ++w) before += w < warp ? wtot[w] : 0u;
+        if (before <= want && want < before + c) {     // exactly one thread
+          unsigned seen = before;
+          for (int i = i0; i < i1; ++i)
+            if ((cached ? skeys[i] : key_bits(src[i])) == tau && seen++ == want) { first_above[j] = (unsigned)i; break; }
+        }
+        __syncthreads();
       }
-      __syncthreads();
     }
 
     // the selected keys, for the per-expert counts and the thresholds' energies
