@@ -448,3 +448,21 @@ def test_long_token_sets_are_walked_in_batches(P, prepared):
     p2, pi, w2 = O.camera_components(ol, Xd, routing=routing)
     assert_close("energy of a batched walk", got["energy"].cpu().numpy(), O.energy(p2, pi, w2, float(np.float32(0.95))))
     assert_close("phi2 of a batched walk", got["phi2"].cpu().numpy(), p2)
+
+
+@pytest.mark.parametrize("T", [1, 33, 100, 128, 129])
+@pytest.mark.parametrize("dtype", ["bf16", "f32"])
+def test_decode_sized_batches_at_the_front_end_limits(P, T, dtype):
+    """Up to 128 tokens and 128 logit columns take the front end made for decode steps: here with the most columns it
+    takes (125 routed experts + 3 gated shared experts), top-16, token counts around a counting-sort block and at the
+    limit; 129 tokens go the general way.  Routing, token counts and scores against the oracle."""
+    cfg = small_cfg(n_tokens=T, d_model=192, n_routed=125, top_k=16, d_ff_routed=64, d_ff_shared=(64, 64, 64),
+                    shared_gate_sigmoid=True, router_bias_std=1.0, dtype=dtype)
+    L = W().make_layer(cfg, seed=22, device=DEV)
+    X = W().make_tokens(cfg, seed=22, device=DEV)
+    out, _ = run_and_compare(P, L, X, alpha=0.95, max_floor_rescues=2)      # one or two tokens per expert
+    assert int(out["expert_token_counts"][:125].sum()) == T * 16
+    # a repeat on the same inputs gives the same bits (fixed summation order in the logit kernel)
+    layer = P.Layer.from_workload(L)
+    a = P.camera_score_layer(layer, X, 0.95, details=True)
+    assert torch.equal(a["energy"], out["energy"]) and torch.equal(a["topk_idx"], out["topk_idx"])
